@@ -1,0 +1,190 @@
+/*
+ * bcq.h -- C ABI of the B200 (sm_100a) library for GPTQT inference (arxiv 2407.02891).
+ *
+ * After GPTQT's two quantisation steps are merged (section "Intermediate Steps Can be
+ * Fused in Inference", Eq. fuse_step1..3), a linear layer is pure binary coding
+ *
+ *     W[n][k] = sum_{i<q} alpha[i][n][g(k)] * b_i[n][k] + z[n][g(k)],   b_i in {-1,+1}
+ *     y[n]    = sum_k W[n][k] x[k]
+ *             = sum_g ( sum_i alpha[i][n][g] * sum_{k in g} b_i[n][k] x[k] + z[n][g] * sum_{k in g} x[k] )
+ *
+ * (Eq. bcw gives the dequantisation  w = sum_i alpha_i b_i ; Eq. fuse_step3 adds the
+ * offset).  g(k) = k / group is the scaling unit along K; group == 0 means one scale per
+ * row, which is the granularity the paper states.  This library computes y at batch 1
+ * (bcq_gemv) and for 2..16 activation vectors (bcq_gemm_smallbatch), and prepares the
+ * operands (bcq_merge_linear, bcq_pack, bcq_repack).
+ *
+ * Conventions
+ *   - Every pointer named *_dev is DEVICE memory owned by the caller; *_host is host memory.
+ *     Nothing is allocated or freed by the library and no pointer is retained after a call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work; they never synchronise.  Errors found on the host return before any
+ *     launch.  The current CUDA device must be the one that owns the pointers.
+ *   - fp16 values are IEEE binary16 bit patterns in uint16_t.  Accumulation is fp32;
+ *     y is rounded to fp16 (nearest even) once, at the end.
+ *   - Device pointers must be 16-byte aligned (y: 2-byte) or BCQ_ERR_MISALIGNED is returned.
+ *   - Return value: BCQ_OK (0) or a negative bcq_status.  No exceptions, no exit().
+ *
+ * Canonical layout (BCQ_LAYOUT_CANONICAL), row-major, last index fastest:
+ *   codes   uint8  [N][K]        bit i of a code is 1  <=>  b_i = +1        (codes < 2^q)
+ *   packed  uint8  [q][N][K/8]   bit (k mod 8) of byte (k div 8), LSB = lowest k, 1 <=> b = +1
+ *   alpha   fp16   [q][N][G]     G = K / group, or 1 when group == 0
+ *   z       fp16   [N][G]
+ *   x       fp16   [B][K],   y fp16 [B][N]
+ *
+ * Tiled layout (BCQ_LAYOUT_TILED): the same bytes and the same fp16 values, permuted so
+ * that every load of the batch-1 kernel is a contiguous 512-byte warp transaction and a
+ * lane's bytes all index the lane's own shared-memory banks.  It needs K % 512 == 0,
+ * N % 8 == 0 and group in {0, 128}.  With U = N/8 row units (8 rows) and K/512 windows:
+ *   packed  tile (w,u) at byte ((w*U + u) * q) * 512; inside: [j < q][lane < 32][16 bytes];
+ *           byte p = 16 j + (byte in lane) = (r*q + i)*2 + s  holds row 8u + r, plane i,
+ *           weights k = 512 w + 16 lane + 8 s .. + 7   (bit order as canonical)
+ *   alpha   group 128: [w][u][gi < 4][i < q][r < 8] <- alpha[i][8u + r][4w + gi];  group 0: [u][i][r]
+ *   z       group 128: [w][u][gi < 4][r < 8]        <- z[8u + r][4w + gi];         group 0: [u][r]
+ * Sizes are identical in both layouts (bcq_packed_bytes, bcq_alpha_elems, bcq_offset_elems).
+ */
+#ifndef BCQ_H
+#define BCQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BCQ_VERSION 100
+
+typedef enum bcq_status {
+    BCQ_OK = 0,
+    BCQ_ERR_INVALID_ARG = -1,        /* NULL pointer, q outside 1..4, N or K <= 0, B outside 1..16, ...   */
+    BCQ_ERR_UNSUPPORTED_SHAPE = -2,  /* K % 32 != 0; group != 0 and (K % group != 0 or group % 32 != 0);   */
+                                     /* or a shape the tiled layout does not cover                        */
+    BCQ_ERR_MISALIGNED = -3,         /* a device pointer is not aligned as required                       */
+    BCQ_ERR_WORKSPACE_TOO_SMALL = -4,
+    BCQ_ERR_CUDA = -5                /* a CUDA runtime call failed; text via bcq_last_cuda_error()        */
+} bcq_status;
+
+enum { BCQ_LAYOUT_CANONICAL = 0, BCQ_LAYOUT_TILED = 1 };
+
+/* One quantised linear layer: N output rows, K inputs, q bit-planes, `group` weights per
+ * scaling unit along K (0 = one unit per row), and the memory layout of its operands. */
+typedef struct bcq_desc {
+    int32_t N;
+    int32_t K;
+    int32_t q;
+    int32_t group;
+    int32_t layout;
+} bcq_desc;
+
+/* How a product is decomposed over the GPU.  kernel: 0 = generic (one warp per row, any
+ * valid shape, either layout is NOT implied: canonical only), 1 = lookup-table kernel
+ * (tiled layout).  row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace. */
+typedef struct bcq_plan {
+    int32_t kernel;
+    int32_t row_blocks;
+    int32_t k_splits;
+    int32_t reserved;
+} bcq_plan;
+
+/* ---- sizes (pure host functions; 0 when the descriptor is invalid) -------------------- */
+size_t bcq_packed_bytes(const bcq_desc *desc);   /* q * N * K / 8                          */
+size_t bcq_alpha_elems(const bcq_desc *desc);    /* q * N * G                              */
+size_t bcq_offset_elems(const bcq_desc *desc);   /* N * G                                  */
+
+/* Validate a descriptor: BCQ_OK, BCQ_ERR_INVALID_ARG or BCQ_ERR_UNSUPPORTED_SHAPE. */
+int bcq_check_desc(const bcq_desc *desc);
+
+/* The decomposition bcq_gemv / bcq_gemm_smallbatch use by default for batch B on a GPU with
+ * `sm_count` multiprocessors (sm_count <= 0: ask the current device).  Pure host logic when
+ * sm_count > 0. */
+int bcq_plan_default(const bcq_desc *desc, int B, int sm_count, bcq_plan *plan_out);
+
+/* Bytes of workspace the plan needs (0 when k_splits == 1 and the generic kernel).  The
+ * workspace holds split-K partial sums and arrival counters.  It must be zero-filled once
+ * (bcq_workspace_init) before its first use; every call leaves the counters zero again, so
+ * it can be reused by later calls ON THE SAME STREAM.  Two products in flight at once
+ * need two workspaces. */
+size_t bcq_workspace_bytes(const bcq_desc *desc, int B, const bcq_plan *plan /* NULL = default */);
+int bcq_workspace_init(void *workspace_dev, size_t bytes, void *stream);
+
+/* ---- operand preparation (offline, once per layer) ------------------------------------ */
+
+/*
+ * Linear-int -> merged binary code (Eq. round, Eq. fuse_step1..3).
+ * w_int holds step-1 integers 0 .. 2^n_bits - 1; S and qbias ([N][G], canonical) dequantise
+ * them as S * w_int + qbias.  bit_to_plane_host[i-1] in 0..q-1 assigns step-1 bit i (weight
+ * 2^(i-2)) to a plane; every plane needs at least one bit.  Outputs, all canonical:
+ *   codes  [N][K]   code of the reachable integer nearest to w_int (ties: the smaller one)
+ *   alpha  [q][N][G] = S * sum_{i in plane j} 2^(i-2)          (rounded once to fp16)
+ *   z      [N][G]    = S * (2^n_bits - 1)/2 + qbias            (rounded once to fp16)
+ * desc->layout is ignored.  n_bits in 1..8, q <= n_bits.
+ */
+int bcq_merge_linear(const bcq_desc *desc, const uint8_t *w_int_dev, const uint16_t *S_dev,
+                     const uint16_t *qbias_dev, int n_bits, const uint8_t *bit_to_plane_host,
+                     uint8_t *codes_dev, uint16_t *alpha_dev, uint16_t *z_dev, void *stream);
+
+/*
+ * Codes + canonical scales -> packed bit-planes and scales in desc->layout.
+ * Bit-exact: only bit extraction and permutation.  alpha_in/z_in may be NULL together with
+ * alpha_out/z_out to pack the planes only.  Outputs must not overlap inputs.
+ */
+int bcq_pack(const bcq_desc *desc, const uint8_t *codes_dev, const uint16_t *alpha_in_dev,
+             const uint16_t *z_in_dev, void *packed_out_dev, uint16_t *alpha_out_dev,
+             uint16_t *z_out_dev, void *stream);
+
+/*
+ * Re-lay-out packed operands from src->layout to dst->layout (N, K, q, group must agree).
+ * Bit-exact permutation; canonical -> tiled -> canonical is the identity.  Any of the three
+ * (src, dst) pointer pairs may be NULL to skip that operand.  No in-place operation.
+ */
+int bcq_repack(const bcq_desc *src, const void *packed_src_dev, const uint16_t *alpha_src_dev,
+               const uint16_t *z_src_dev, const bcq_desc *dst, void *packed_dst_dev,
+               uint16_t *alpha_dst_dev, uint16_t *z_dst_dev, void *stream);
+
+/* ---- the products --------------------------------------------------------------------- */
+
+/*
+ * y = W x at batch 1 (the definition at the top of this file; Eq. bcw + Eq. fuse_step3).
+ * x [K], y [N] fp16.  y is overwritten.  workspace may be NULL when bcq_workspace_bytes is 0.
+ * bcq_gemv_plan is the same product with an explicit decomposition (for tuning and tests):
+ * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, and at most 64 row units
+ * (512 rows) per row block.
+ */
+int bcq_gemv(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
+             const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev,
+             void *workspace_dev, size_t workspace_bytes, void *stream);
+int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed_dev,
+                  const uint16_t *alpha_dev, const uint16_t *z_dev, const uint16_t *x_dev,
+                  uint16_t *y_dev, void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
+ * Y[b] = W X[b] for b < B, 1 <= B <= 16; X [B][K], Y [B][N] row-major fp16.  Every column is
+ * an independent product (the paper defines batch 1 only); the packed weights are read
+ * once for all columns.  B == 1 is bcq_gemv.
+ */
+int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
+                        const uint16_t *z_dev, const uint16_t *X_dev, uint16_t *Y_dev, int B,
+                        void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
+ * bcq_gemv with the activation and the result in HOST memory: enqueues x_host -> x_stage_dev,
+ * the product, y_stage_dev -> y_host on `stream` and returns without synchronising (the
+ * caller synchronises the stream before reading y_host).  Use page-locked host memory for
+ * the copies to be asynchronous.  x_stage_dev [K] and y_stage_dev [N] are caller-owned
+ * device buffers.
+ */
+int bcq_gemv_host(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
+                  const uint16_t *z_dev, const uint16_t *x_host, uint16_t *y_host,
+                  uint16_t *x_stage_dev, uint16_t *y_stage_dev,
+                  void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/* ---- misc ----------------------------------------------------------------------------- */
+const char *bcq_status_string(int status);   /* static string                              */
+const char *bcq_last_cuda_error(void);       /* text of the last CUDA error seen, "" if none */
+int bcq_version(void);                       /* BCQ_VERSION                                 */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCQ_H */

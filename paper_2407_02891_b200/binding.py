@@ -1,0 +1,245 @@
+"""ctypes binding of the C ABI in include/bcq.h -- argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory) and forwards their data pointers and
+the current torch CUDA stream to the library entry point of the same name.  There is no
+fallback: if libbcq.so is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbcq.so")
+
+LAYOUT_CANONICAL = 0
+LAYOUT_TILED = 1
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED_SHAPE = -2
+ERR_MISALIGNED = -3
+ERR_WORKSPACE_TOO_SMALL = -4
+ERR_CUDA = -5
+
+
+class Desc(ctypes.Structure):
+    """bcq_desc"""
+    _fields_ = [("N", ctypes.c_int32), ("K", ctypes.c_int32), ("q", ctypes.c_int32),
+                ("group", ctypes.c_int32), ("layout", ctypes.c_int32)]
+
+    def with_layout(self, layout: int) -> "Desc":
+        return Desc(self.N, self.K, self.q, self.group, layout)
+
+    @property
+    def G(self) -> int:
+        return 1 if self.group == 0 else self.K // self.group
+
+
+class Plan(ctypes.Structure):
+    """bcq_plan"""
+    _fields_ = [("kernel", ctypes.c_int32), ("row_blocks", ctypes.c_int32),
+                ("k_splits", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class BcqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = lib().bcq_status_string(status).decode()
+        if status == ERR_CUDA:
+            msg += ": " + lib().bcq_last_cuda_error().decode()
+        super().__init__(f"{what}: {msg} ({status})")
+
+
+_lib = None
+_vp, _sz, _i = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+_dp, _pp = ctypes.POINTER(Desc), ctypes.POINTER(Plan)
+
+SIGNATURES = {
+    "bcq_version": (_i, []),
+    "bcq_status_string": (ctypes.c_char_p, [_i]),
+    "bcq_last_cuda_error": (ctypes.c_char_p, []),
+    "bcq_check_desc": (_i, [_dp]),
+    "bcq_packed_bytes": (_sz, [_dp]),
+    "bcq_alpha_elems": (_sz, [_dp]),
+    "bcq_offset_elems": (_sz, [_dp]),
+    "bcq_plan_default": (_i, [_dp, _i, _i, _pp]),
+    "bcq_workspace_bytes": (_sz, [_dp, _i, _pp]),
+    "bcq_workspace_init": (_i, [_vp, _sz, _vp]),
+    "bcq_merge_linear": (_i, [_dp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp]),
+    "bcq_pack": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "bcq_repack": (_i, [_dp, _vp, _vp, _vp, _dp, _vp, _vp, _vp, _vp]),
+    "bcq_gemv": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_gemv_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_gemm_smallbatch": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
+    "bcq_gemv_host": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+}
+
+
+def lib() -> ctypes.CDLL:
+    """Load libbcq.so (built in-tree by paper_2407_02891_b200.build).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2407_02891_b200.build`; "
+                               "there is no fallback path")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _dev(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise ValueError("expected a CUDA tensor")
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc: int, what: str):
+    if rc != OK:
+        raise BcqError(rc, what)
+
+
+def desc(N: int, K: int, q: int, group: int, layout: int = LAYOUT_CANONICAL) -> Desc:
+    return Desc(N, K, q, group, layout)
+
+
+def check_desc(d: Desc) -> int:
+    return lib().bcq_check_desc(ctypes.byref(d))
+
+
+def packed_bytes(d: Desc) -> int:
+    return lib().bcq_packed_bytes(ctypes.byref(d))
+
+
+def alpha_elems(d: Desc) -> int:
+    return lib().bcq_alpha_elems(ctypes.byref(d))
+
+
+def offset_elems(d: Desc) -> int:
+    return lib().bcq_offset_elems(ctypes.byref(d))
+
+
+def plan_default(d: Desc, B: int = 1, sm_count: int = 0) -> Plan:
+    p = Plan()
+    _check(lib().bcq_plan_default(ctypes.byref(d), B, sm_count, ctypes.byref(p)), "bcq_plan_default")
+    return p
+
+
+def workspace_bytes(d: Desc, B: int = 1, plan: Plan | None = None) -> int:
+    return lib().bcq_workspace_bytes(ctypes.byref(d), B, ctypes.byref(plan) if plan is not None else None)
+
+
+def workspace_init(ws: torch.Tensor):
+    _dev(ws)
+    _check(lib().bcq_workspace_init(_ptr(ws), ws.numel() * ws.element_size(), _stream()), "bcq_workspace_init")
+
+
+def new_workspace(d: Desc, B: int = 1, plan: Plan | None = None, device="cuda") -> torch.Tensor | None:
+    """Allocate (torch) and zero-fill a workspace for the plan; None when none is needed."""
+    n = workspace_bytes(d, B, plan)
+    if n == 0:
+        return None
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    workspace_init(ws)
+    return ws
+
+
+def _ws_args(ws):
+    if ws is None:
+        return None, 0
+    _dev(ws)
+    return _ptr(ws), ws.numel() * ws.element_size()
+
+
+def merge_linear(d: Desc, w_int, S, qbias, n_bits: int, bit_to_plane, codes, alpha, z):
+    _dev(w_int, S, qbias, codes, alpha, z)
+    b2p = (ctypes.c_uint8 * len(bit_to_plane))(*[int(v) for v in bit_to_plane])
+    if len(bit_to_plane) != n_bits:
+        raise ValueError("bit_to_plane needs n_bits entries")
+    _check(lib().bcq_merge_linear(ctypes.byref(d), _ptr(w_int), _ptr(S), _ptr(qbias), n_bits,
+                                  ctypes.cast(b2p, ctypes.c_void_p), _ptr(codes), _ptr(alpha), _ptr(z),
+                                  _stream()), "bcq_merge_linear")
+
+
+def pack(d: Desc, codes, alpha_in, z_in, packed_out, alpha_out, z_out):
+    _dev(codes, alpha_in, z_in, packed_out, alpha_out, z_out)
+    _check(lib().bcq_pack(ctypes.byref(d), _ptr(codes), _ptr(alpha_in), _ptr(z_in), _ptr(packed_out),
+                          _ptr(alpha_out), _ptr(z_out), _stream()), "bcq_pack")
+
+
+def repack(src: Desc, packed_src, alpha_src, z_src, dst: Desc, packed_dst, alpha_dst, z_dst):
+    _dev(packed_src, alpha_src, z_src, packed_dst, alpha_dst, z_dst)
+    _check(lib().bcq_repack(ctypes.byref(src), _ptr(packed_src), _ptr(alpha_src), _ptr(z_src),
+                            ctypes.byref(dst), _ptr(packed_dst), _ptr(alpha_dst), _ptr(z_dst), _stream()),
+           "bcq_repack")
+
+
+def gemv(d: Desc, packed, alpha, z, x, y, workspace=None):
+    _dev(packed, alpha, z, x, y)
+    wp, wn = _ws_args(workspace)
+    _check(lib().bcq_gemv(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y), wp, wn,
+                          _stream()), "bcq_gemv")
+
+
+def gemv_plan(d: Desc, plan: Plan, packed, alpha, z, x, y, workspace=None):
+    _dev(packed, alpha, z, x, y)
+    wp, wn = _ws_args(workspace)
+    _check(lib().bcq_gemv_plan(ctypes.byref(d), ctypes.byref(plan), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x),
+                               _ptr(y), wp, wn, _stream()), "bcq_gemv_plan")
+
+
+def gemm_smallbatch(d: Desc, packed, alpha, z, X, Y, B: int, workspace=None):
+    _dev(packed, alpha, z, X, Y)
+    wp, wn = _ws_args(workspace)
+    _check(lib().bcq_gemm_smallbatch(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(X), _ptr(Y), B,
+                                     wp, wn, _stream()), "bcq_gemm_smallbatch")
+
+
+def gemv_host(d: Desc, packed, alpha, z, x_host, y_host, x_stage, y_stage, workspace=None):
+    """x_host / y_host are CPU tensors (pinned for asynchronous copies); the caller synchronises."""
+    _dev(packed, alpha, z, x_stage, y_stage)
+    if x_host.is_cuda or y_host.is_cuda:
+        raise ValueError("x_host and y_host must be host tensors")
+    wp, wn = _ws_args(workspace)
+    _check(lib().bcq_gemv_host(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x_host), _ptr(y_host),
+                               _ptr(x_stage), _ptr(y_stage), wp, wn, _stream()), "bcq_gemv_host")
+
+
+@dataclass
+class Layer:
+    """Device-resident operands of one packed layer (a convenience holder, no arithmetic)."""
+    d: Desc
+    packed: torch.Tensor
+    alpha: torch.Tensor
+    z: torch.Tensor
+
+
+def pack_layer(N, K, q, group, layout, codes, alpha, z) -> Layer:
+    """bcq_pack into freshly allocated torch tensors.  codes/alpha/z: canonical CUDA tensors."""
+    d = desc(N, K, q, group, layout)
+    rc = check_desc(d)
+    if rc != OK:
+        raise BcqError(rc, "bcq_check_desc")
+    packed = torch.empty(packed_bytes(d), dtype=torch.uint8, device=codes.device)
+    a = torch.empty(alpha_elems(d), dtype=torch.float16, device=codes.device)
+    zz = torch.empty(offset_elems(d), dtype=torch.float16, device=codes.device)
+    pack(d, codes, alpha, z, packed, a, zz)
+    return Layer(d, packed, a, zz)

@@ -1,0 +1,333 @@
+// The extern "C" boundary of libbcq: argument validation, the default decomposition, the
+// host-side table of the linear-int -> binary-code conversion, and dispatch to the kernels.
+#include <stdio.h>
+#include <string.h>
+
+#include "bcq_internal.cuh"
+
+using namespace bcq;
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e)
+{
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return BCQ_ERR_CUDA;
+}
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int check_desc(const bcq_desc *d)
+{
+    if (!d) return BCQ_ERR_INVALID_ARG;
+    if (d->N <= 0 || d->K <= 0 || d->q < 1 || d->q > 4 || d->group < 0) return BCQ_ERR_INVALID_ARG;
+    if (d->layout != BCQ_LAYOUT_CANONICAL && d->layout != BCQ_LAYOUT_TILED) return BCQ_ERR_INVALID_ARG;
+    if (d->K % 32 != 0) return BCQ_ERR_UNSUPPORTED_SHAPE;
+    if (d->group != 0 && (d->K % d->group != 0 || d->group % 32 != 0)) return BCQ_ERR_UNSUPPORTED_SHAPE;
+    if (d->layout == BCQ_LAYOUT_TILED) {
+        if (d->K % kWindow != 0 || d->N % kUnitRows != 0) return BCQ_ERR_UNSUPPORTED_SHAPE;
+        if (d->group != 0 && d->group != 128) return BCQ_ERR_UNSUPPORTED_SHAPE;
+    }
+    return BCQ_OK;
+}
+
+bool same_problem(const bcq_desc *a, const bcq_desc *b)
+{
+    return a->N == b->N && a->K == b->K && a->q == b->q && a->group == b->group;
+}
+
+int device_sm_count(int *out)
+{
+    int dev = 0, sm = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *out = sm;
+    return BCQ_OK;
+}
+
+bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group == 128; }
+
+// Instruction-count model of the lookup-table kernel (warp instructions on the critical warp
+// of a block); it ranks decompositions, it does not predict time.
+long long lut_cost(int U, int W, int rb, int ks, int sm)
+{
+    const long long build = 100, lookup = 200, reduce = 40, fixed = 400, finalize = 120;
+    const long long waves = (static_cast<long long>(rb) * ks + sm - 1) / sm;
+    const long long wc = (W + ks - 1) / ks;
+    const long long units = (U + rb - 1) / rb;
+    const long long upw = (units + kLutWarps - 1) / kLutWarps;
+    return waves * (fixed + wc * (build + upw * lookup) + upw * reduce + (ks > 1 ? finalize : 0));
+}
+
+int plan_lut(const bcq_desc *d, int sm, bcq_plan *out)
+{
+    const int U = d->N / kUnitRows, W = d->K / kWindow;
+    const int rb_min = (U + kMaxUnitsPerBlock - 1) / kMaxUnitsPerBlock;
+    long long best = -1;
+    for (int ks = 1; ks <= W && ks <= 64; ++ks) {
+        for (int k = 0; k <= 16; ++k) {
+            int rb = k == 0 ? rb_min : (k * sm) / ks;
+            if (rb < rb_min || rb > U || rb > kMaxRowBlocks) continue;
+            const long long c = lut_cost(U, W, rb, ks, sm);
+            if (best < 0 || c < best) {
+                best = c;
+                out->kernel = 1;
+                out->row_blocks = rb;
+                out->k_splits = ks;
+                out->reserved = 0;
+            }
+        }
+    }
+    return best < 0 ? BCQ_ERR_UNSUPPORTED_SHAPE : BCQ_OK;
+}
+
+int check_plan(const bcq_desc *d, const bcq_plan *p)
+{
+    if (p->kernel == 0) return BCQ_OK;
+    if (p->kernel != 1 || !lut_kernel_covers(d)) return BCQ_ERR_INVALID_ARG;
+    const int U = d->N / kUnitRows, W = d->K / kWindow;
+    if (p->row_blocks < 1 || p->row_blocks > U || p->row_blocks > kMaxRowBlocks) return BCQ_ERR_INVALID_ARG;
+    if (p->k_splits < 1 || p->k_splits > W) return BCQ_ERR_INVALID_ARG;
+    if ((U + p->row_blocks - 1) / p->row_blocks > kMaxUnitsPerBlock) return BCQ_ERR_INVALID_ARG;
+    return BCQ_OK;
+}
+
+size_t plan_workspace(const bcq_desc *d, const bcq_plan *p)
+{
+    if (p->kernel == 1 && p->k_splits > 1) return kCounterBytes + size_t(p->k_splits) * d->N * sizeof(float);
+    return 0;
+}
+
+int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, const uint16_t *alpha, const uint16_t *z,
+             const uint16_t *x, uint16_t *y, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!packed || !alpha || !z || !x || !y) return BCQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 16) || !aligned(alpha, 16) || !aligned(z, 16) || !aligned(x, 16) || !aligned(y, 2))
+        return BCQ_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (plan->kernel == 0) {
+        e = launch_generic(*desc, packed, alpha, z, x, y, 1, st);
+    } else {
+        const size_t need = plan_workspace(desc, plan);
+        if (need > 0) {
+            if (!ws) return BCQ_ERR_INVALID_ARG;
+            if (!aligned(ws, 16)) return BCQ_ERR_MISALIGNED;
+            if (ws_bytes < need) return BCQ_ERR_WORKSPACE_TOO_SMALL;
+        }
+        e = launch_lut_gemv(*desc, *plan, packed, alpha, z, x, y, need ? ws : nullptr, st);
+    }
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int bcq_version(void) { return BCQ_VERSION; }
+
+const char *bcq_last_cuda_error(void) { return g_cuda_error; }
+
+const char *bcq_status_string(int s)
+{
+    switch (s) {
+        case BCQ_OK: return "ok";
+        case BCQ_ERR_INVALID_ARG: return "invalid argument";
+        case BCQ_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case BCQ_ERR_MISALIGNED: return "misaligned pointer";
+        case BCQ_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case BCQ_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+int bcq_check_desc(const bcq_desc *desc) { return check_desc(desc); }
+
+size_t bcq_packed_bytes(const bcq_desc *d)
+{
+    return check_desc(d) == BCQ_OK ? size_t(d->q) * d->N * (d->K / 8) : 0;
+}
+size_t bcq_alpha_elems(const bcq_desc *d) { return check_desc(d) == BCQ_OK ? size_t(d->q) * d->N * n_groups(*d) : 0; }
+size_t bcq_offset_elems(const bcq_desc *d) { return check_desc(d) == BCQ_OK ? size_t(d->N) * n_groups(*d) : 0; }
+
+int bcq_plan_default(const bcq_desc *desc, int B, int sm_count, bcq_plan *out)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!out || B < 1 || B > 16) return BCQ_ERR_INVALID_ARG;
+    out->kernel = 0;
+    out->row_blocks = (desc->N + 7) / 8;
+    out->k_splits = 1;
+    out->reserved = 0;
+    if (B == 1 && lut_kernel_covers(desc)) {
+        if (sm_count <= 0) {
+            rc = device_sm_count(&sm_count);
+            if (rc != BCQ_OK) return rc;
+        }
+        return plan_lut(desc, sm_count, out);
+    }
+    return BCQ_OK;
+}
+
+size_t bcq_workspace_bytes(const bcq_desc *desc, int B, const bcq_plan *plan)
+{
+    bcq_plan def;
+    if (check_desc(desc) != BCQ_OK) return 0;
+    if (!plan) {
+        if (bcq_plan_default(desc, B, 0, &def) != BCQ_OK) return 0;
+        plan = &def;
+    }
+    return plan_workspace(desc, plan);
+}
+
+int bcq_workspace_init(void *ws, size_t bytes, void *stream)
+{
+    if (bytes == 0) return BCQ_OK;
+    if (!ws) return BCQ_ERR_INVALID_ARG;
+    cudaError_t e = cudaMemsetAsync(ws, 0, bytes, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_merge_linear(const bcq_desc *desc, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias, int n_bits,
+                     const uint8_t *bit_to_plane, uint8_t *codes, uint16_t *alpha, uint16_t *z, void *stream)
+{
+    bcq_desc d;
+    if (!desc) return BCQ_ERR_INVALID_ARG;
+    d = *desc;
+    d.layout = BCQ_LAYOUT_CANONICAL;
+    int rc = check_desc(&d);
+    if (rc != BCQ_OK) return rc;
+    if (!w_int || !S || !qbias || !bit_to_plane || !codes || !alpha || !z) return BCQ_ERR_INVALID_ARG;
+    if (n_bits < 1 || n_bits > 8 || d.q > n_bits) return BCQ_ERR_INVALID_ARG;
+    if (!aligned(w_int, 16) || !aligned(codes, 16) || !aligned(S, 2) || !aligned(qbias, 2) || !aligned(alpha, 2) ||
+        !aligned(z, 2))
+        return BCQ_ERR_MISALIGNED;
+
+    // A sign pattern (code) drives all step-1 bits of a plane together, so the integers it can
+    // reach are those whose binary digit (i-1) equals the code's bit for the plane of step-1 bit i.
+    double weight[4] = {0, 0, 0, 0};
+    for (int i = 0; i < n_bits; ++i) {
+        if (bit_to_plane[i] >= d.q) return BCQ_ERR_INVALID_ARG;
+        weight[bit_to_plane[i]] += double(1u << i) * 0.5;  // step-1 bit i+1 weighs 2^(i-1)
+    }
+    for (int j = 0; j < d.q; ++j)
+        if (weight[j] == 0.0) return BCQ_ERR_INVALID_ARG;
+    int reach[16];
+    for (int c = 0; c < (1 << d.q); ++c) {
+        int v = 0;
+        for (int i = 0; i < n_bits; ++i) v |= ((c >> bit_to_plane[i]) & 1) << i;
+        reach[c] = v;
+    }
+    uint8_t code_of_int[256];
+    for (int t = 0; t < 256; ++t) {
+        int best = 0;
+        for (int c = 1; c < (1 << d.q); ++c) {
+            const int dc = abs(t - reach[c]), db = abs(t - reach[best]);
+            if (dc < db || (dc == db && reach[c] < reach[best])) best = c;
+        }
+        code_of_int[t] = uint8_t(best);
+    }
+    cudaError_t e = launch_merge(d, w_int, S, qbias, n_bits, code_of_int, weight, codes, alpha, z,
+                                 static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_pack(const bcq_desc *desc, const uint8_t *codes, const uint16_t *alpha_in, const uint16_t *z_in, void *packed,
+             uint16_t *alpha_out, uint16_t *z_out, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!codes || !packed) return BCQ_ERR_INVALID_ARG;
+    const bool scales = alpha_in || z_in || alpha_out || z_out;
+    if (scales && !(alpha_in && z_in && alpha_out && z_out)) return BCQ_ERR_INVALID_ARG;
+    if (!aligned(codes, 16) || !aligned(packed, 16) || !aligned(alpha_in, 2) || !aligned(z_in, 2) ||
+        !aligned(alpha_out, 2) || !aligned(z_out, 2))
+        return BCQ_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_pack(*desc, codes, packed, st);
+    if (e == cudaSuccess && scales) {
+        bcq_desc src = *desc;
+        src.layout = BCQ_LAYOUT_CANONICAL;
+        e = launch_permute_scales(src, alpha_in, z_in, *desc, alpha_out, z_out, st);
+    }
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_repack(const bcq_desc *src, const void *packed_src, const uint16_t *alpha_src, const uint16_t *z_src,
+               const bcq_desc *dst, void *packed_dst, uint16_t *alpha_dst, uint16_t *z_dst, void *stream)
+{
+    int rc = check_desc(src);
+    if (rc != BCQ_OK) return rc;
+    rc = check_desc(dst);
+    if (rc != BCQ_OK) return rc;
+    if (!same_problem(src, dst)) return BCQ_ERR_INVALID_ARG;
+    if ((packed_src == nullptr) != (packed_dst == nullptr) || (alpha_src == nullptr) != (alpha_dst == nullptr) ||
+        (z_src == nullptr) != (z_dst == nullptr))
+        return BCQ_ERR_INVALID_ARG;
+    if ((packed_src && packed_src == packed_dst) || (alpha_src && alpha_src == alpha_dst) || (z_src && z_src == z_dst))
+        return BCQ_ERR_INVALID_ARG;
+    if (!aligned(packed_src, 16) || !aligned(packed_dst, 16) || !aligned(alpha_src, 2) || !aligned(alpha_dst, 2) ||
+        !aligned(z_src, 2) || !aligned(z_dst, 2))
+        return BCQ_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaSuccess;
+    if (packed_src) e = launch_permute_planes(*src, packed_src, *dst, packed_dst, st);
+    if (e == cudaSuccess && (alpha_src || z_src))
+        e = launch_permute_scales(*src, alpha_src, z_src, *dst, alpha_dst, z_dst, st);
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed, const uint16_t *alpha,
+                  const uint16_t *z, const uint16_t *x, uint16_t *y, void *ws, size_t ws_bytes, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!plan) return BCQ_ERR_INVALID_ARG;
+    rc = check_plan(desc, plan);
+    if (rc != BCQ_OK) return rc;
+    return run_gemv(desc, plan, packed, alpha, z, x, y, ws, ws_bytes, stream);
+}
+
+int bcq_gemv(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z, const uint16_t *x,
+             uint16_t *y, void *ws, size_t ws_bytes, void *stream)
+{
+    bcq_plan plan;
+    int rc = bcq_plan_default(desc, 1, 0, &plan);
+    if (rc != BCQ_OK) return rc;
+    return run_gemv(desc, &plan, packed, alpha, z, x, y, ws, ws_bytes, stream);
+}
+
+int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z,
+                        const uint16_t *X, uint16_t *Y, int B, void *ws, size_t ws_bytes, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (B < 1 || B > 16) return BCQ_ERR_INVALID_ARG;
+    if (B == 1) return bcq_gemv(desc, packed, alpha, z, X, Y, ws, ws_bytes, stream);
+    if (!packed || !alpha || !z || !X || !Y) return BCQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 16) || !aligned(alpha, 16) || !aligned(z, 16) || !aligned(X, 16) || !aligned(Y, 2))
+        return BCQ_ERR_MISALIGNED;
+    cudaError_t e = launch_generic(*desc, packed, alpha, z, X, Y, B, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_gemv_host(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z,
+                  const uint16_t *x_host, uint16_t *y_host, uint16_t *x_stage, uint16_t *y_stage, void *ws,
+                  size_t ws_bytes, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!x_host || !y_host || !x_stage || !y_stage) return BCQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(x_stage, x_host, size_t(desc->K) * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    rc = bcq_gemv(desc, packed, alpha, z, x_stage, y_stage, ws, ws_bytes, stream);
+    if (rc != BCQ_OK) return rc;
+    e = cudaMemcpyAsync(y_host, y_stage, size_t(desc->N) * 2, cudaMemcpyDeviceToHost, st);
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+}  // extern "C"

@@ -1,0 +1,55 @@
+"""Shared test helpers: synthetic layers as numpy arrays, and the tiled layout restated from
+the documentation in include/bcq.h (numpy index arithmetic, independent of the library)."""
+import numpy as np
+
+from paper_2407_02891_b200 import synth
+
+TOL = 5e-3   # max|y_gpu - y_ref| <= TOL * max|y_ref|  (fp16 I/O, fp32 accumulation)
+
+
+def make_layer(name, N, K, q, group, B=1):
+    """Canonical numpy operands of a synthetic layer: planes, codes, alpha, z, x."""
+    p = synth.planes(name, N, K, q)
+    alpha, z = synth.scale_rows(name, N, K, q, group)
+    x = synth.activations(name, B, K)
+    return p, synth.codes_from_planes(p), alpha, z, x
+
+
+def tiled_planes(planes):
+    """canonical uint8 [q,N,K/8] -> tiled byte stream, per the layout comment of include/bcq.h."""
+    q, N, KB = planes.shape
+    U, W = N // 8, KB // 64
+    out = np.empty(q * N * KB, np.uint8)
+    i, n, kb = np.meshgrid(np.arange(q), np.arange(N), np.arange(KB), indexing="ij")
+    w, c = kb // 64, kb % 64
+    lane, s = c // 2, c % 2
+    u, r = n // 8, n % 8
+    p = (r * q + i) * 2 + s
+    off = ((w * U + u) * q + p // 16) * 512 + lane * 16 + p % 16
+    out[off.ravel()] = planes.ravel()
+    return out
+
+
+def tiled_scales(alpha, z, group):
+    """canonical alpha [q,N,G], z [N,G] -> tiled element streams."""
+    q, N, G = alpha.shape
+    U = N // 8
+    i, n, g = np.meshgrid(np.arange(q), np.arange(N), np.arange(G), indexing="ij")
+    u, r = n // 8, n % 8
+    if group == 0:
+        a_off = (u * q + i) * 8 + r
+        z_off = (u[0] * 8 + r[0])
+    else:
+        w, gi = g // 4, g % 4
+        a_off = (((w * U + u) * 4 + gi) * q + i) * 8 + r
+        z_off = ((w[0] * U + u[0]) * 4 + gi[0]) * 8 + r[0]
+    a_out = np.empty(alpha.size, alpha.dtype)
+    z_out = np.empty(z.size, z.dtype)
+    a_out[a_off.ravel()] = alpha.ravel()
+    z_out[z_off.ravel()] = z.ravel()
+    return a_out, z_out
+
+
+def rel_err(y_gpu, y_ref):
+    y_ref = np.asarray(y_ref, np.float64)
+    return float(np.abs(np.asarray(y_gpu, np.float64) - y_ref).max() / np.abs(y_ref).max())

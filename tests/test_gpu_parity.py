@@ -1,0 +1,283 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Integer / byte work must be bit-exact; products must satisfy
+max|y_gpu - y_ref| <= 5e-3 * max|y_ref|."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import TOL, make_layer, rel_err, tiled_planes, tiled_scales
+from paper_2407_02891_b200 import binding as bq
+from paper_2407_02891_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+
+
+def gpu_layer(N, K, q, group, layout, codes, alpha, z):
+    return bq.pack_layer(N, K, q, group, layout, dev(codes), dev(alpha), dev(z))
+
+
+def run_gemv(layer, x, plan=None):
+    y = torch.full((layer.d.N,), float("nan"), dtype=torch.float16, device=DEV)
+    xd = dev(x.reshape(-1))
+    if plan is None:
+        ws = bq.new_workspace(layer.d, 1)
+        bq.gemv(layer.d, layer.packed, layer.alpha, layer.z, xd, y, ws)
+    else:
+        ws = bq.new_workspace(layer.d, 1, plan)
+        bq.gemv_plan(layer.d, plan, layer.packed, layer.alpha, layer.z, xd, y, ws)
+    torch.cuda.synchronize()
+    return y.cpu().numpy().astype(np.float64)
+
+
+# ---------------------------------------------------------------------------------------
+# packing / repacking: bit-exact
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("N,K,q,group", [(16, 32, 3, 32), (16, 32, 3, 0), (40, 1024, 3, 128), (24, 512, 2, 128),
+                                         (8, 1536, 4, 128), (72, 512, 1, 0), (13, 96, 3, 32)])
+def test_pack_canonical_bit_exact(N, K, q, group):
+    p, codes, alpha, z, _ = make_layer(f"pack/{N}x{K}", N, K, q, group)
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_CANONICAL, codes, alpha, z)
+    assert np.array_equal(L.packed.cpu().numpy(), oracle.pack_canonical(codes, q).ravel())
+    assert np.array_equal(L.alpha.cpu().numpy().view(np.uint16), alpha.ravel().view(np.uint16))
+    assert np.array_equal(L.z.cpu().numpy().view(np.uint16), z.ravel().view(np.uint16))
+
+
+@pytest.mark.parametrize("N,K,q,group", [(40, 1024, 3, 128), (24, 512, 2, 128), (8, 1536, 4, 128), (72, 512, 1, 0),
+                                         (296, 2048, 3, 128), (64, 1024, 2, 0)])
+def test_pack_tiled_and_repack_bit_exact(N, K, q, group):
+    p, codes, alpha, z, _ = make_layer(f"tile/{N}x{K}", N, K, q, group)
+    canon = oracle.pack_canonical(codes, q)
+    want_p = tiled_planes(canon)
+    want_a, want_z = tiled_scales(alpha, z, group)
+    T = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    assert np.array_equal(T.packed.cpu().numpy(), want_p)
+    assert np.array_equal(T.alpha.cpu().numpy().view(np.uint16), want_a.view(np.uint16))
+    assert np.array_equal(T.z.cpu().numpy().view(np.uint16), want_z.view(np.uint16))
+    # canonical -> tiled via repack gives the same bytes; tiled -> canonical is the inverse
+    C = gpu_layer(N, K, q, group, bq.LAYOUT_CANONICAL, codes, alpha, z)
+    p2, a2, z2 = torch.zeros_like(C.packed), torch.zeros_like(C.alpha), torch.zeros_like(C.z)
+    bq.repack(C.d, C.packed, C.alpha, C.z, T.d, p2, a2, z2)
+    assert torch.equal(p2, T.packed) and torch.equal(a2.view(torch.int16), T.alpha.view(torch.int16))
+    assert torch.equal(z2.view(torch.int16), T.z.view(torch.int16))
+    p3, a3, z3 = torch.zeros_like(C.packed), torch.zeros_like(C.alpha), torch.zeros_like(C.z)
+    bq.repack(T.d, p2, a2, z2, C.d, p3, a3, z3)
+    assert np.array_equal(p3.cpu().numpy(), canon.ravel())
+    assert np.array_equal(a3.cpu().numpy().view(np.uint16), alpha.ravel().view(np.uint16))
+    assert np.array_equal(z3.cpu().numpy().view(np.uint16), z.ravel().view(np.uint16))
+
+
+# ---------------------------------------------------------------------------------------
+# linear-int -> merged binary code: bit-exact codes, alpha, z
+# ---------------------------------------------------------------------------------------
+
+def _partitions(n, q):
+    out = []
+
+    def rec(i, assign, used):
+        if i == n:
+            if used == q:
+                out.append(list(assign))
+            return
+        for j in range(min(used + 1, q)):
+            rec(i + 1, assign + [j], max(used, j + 1))
+
+    rec(0, [], 0)
+    return out
+
+
+@pytest.mark.parametrize("N,K,group,n,q", [(16, 32, 32, 4, 3), (16, 32, 0, 4, 3), (16, 32, 32, 5, 3),
+                                           (64, 512, 128, 5, 2), (16, 32, 32, 3, 2), (24, 256, 64, 4, 4)])
+def test_merge_linear_bit_exact(N, K, group, n, q):
+    w, S, qbias = synth.linear_int_case(f"merge/n{n}", N, K, group, n)
+    d = bq.desc(N, K, q, group)
+    G = d.G
+    for b2p in _partitions(n, q):
+        codes = torch.zeros((N, K), dtype=torch.uint8, device=DEV)
+        alpha = torch.zeros((q, N, G), dtype=torch.float16, device=DEV)
+        z = torch.zeros((N, G), dtype=torch.float16, device=DEV)
+        bq.merge_linear(d, dev(w), dev(S), dev(qbias), n, b2p, codes, alpha, z)
+        rc, ra, rz = oracle.merge_linear(w, S, qbias, group, n, b2p)
+        assert np.array_equal(codes.cpu().numpy(), rc)
+        assert np.array_equal(alpha.cpu().numpy().view(np.uint16), ra.view(np.uint16))
+        assert np.array_equal(z.cpu().numpy().view(np.uint16), rz.view(np.uint16))
+
+
+def test_merge_linear_rounds_general_scales_like_the_oracle():
+    """S, qbias with full 11-bit significands: alpha and z need a real rounding to fp16."""
+    N, K, group, n, q = 32, 256, 64, 5, 3
+    w, _, _ = synth.linear_int_case("merge/general", N, K, group, n)
+    G = K // group
+    S = (0.002 + 0.03 * synth.uniform("merge/general/S", 0, N * G)).astype(np.float16).reshape(N, G)
+    qbias = (synth.normal("merge/general/b", 0, N * G) * 0.1).astype(np.float16).reshape(N, G)
+    d = bq.desc(N, K, q, group)
+    b2p = [0, 1, 1, 2, 2]
+    codes = torch.zeros((N, K), dtype=torch.uint8, device=DEV)
+    alpha = torch.zeros((q, N, G), dtype=torch.float16, device=DEV)
+    z = torch.zeros((N, G), dtype=torch.float16, device=DEV)
+    bq.merge_linear(d, dev(w), dev(S), dev(qbias), n, b2p, codes, alpha, z)
+    rc, ra, rz = oracle.merge_linear(w, S, qbias, group, n, b2p)
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    assert np.array_equal(alpha.cpu().numpy().view(np.uint16), ra.view(np.uint16))
+    assert np.array_equal(z.cpu().numpy().view(np.uint16), rz.view(np.uint16))
+
+
+def test_tiny_case_end_to_end():
+    """16 x 32, 4-bit linear codes -> 3 planes -> pack -> product, against the oracle chain."""
+    N, K, group, n, q = 16, 32, 32, 4, 3
+    w, S, qbias = synth.linear_int_case("tiny/e2e", N, K, group, n)
+    x = synth.activations("tiny/e2e", 1, K)
+    d = bq.desc(N, K, q, group)
+    for b2p in _partitions(n, q):
+        codes = torch.zeros((N, K), dtype=torch.uint8, device=DEV)
+        alpha = torch.zeros((q, N, 1), dtype=torch.float16, device=DEV)
+        z = torch.zeros((N, 1), dtype=torch.float16, device=DEV)
+        bq.merge_linear(d, dev(w), dev(S), dev(qbias), n, b2p, codes, alpha, z)
+        L = bq.pack_layer(N, K, q, group, bq.LAYOUT_CANONICAL, codes, alpha, z)
+        y = run_gemv(L, x)
+        rc, ra, rz = oracle.merge_linear(w, S, qbias, group, n, b2p)
+        ref = oracle.forward_dequant(rc, ra, rz, x, group)[0]
+        assert rel_err(y, ref) <= TOL
+
+
+# ---------------------------------------------------------------------------------------
+# products
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("N,K,q,group", [(16, 32, 3, 32), (13, 96, 3, 32), (50, 256, 2, 64), (33, 1024, 4, 0),
+                                         (1024, 1024, 3, 128), (7, 2048, 1, 128)])
+def test_gemv_generic_kernel(N, K, q, group):
+    p, codes, alpha, z, x = make_layer(f"gen/{N}x{K}", N, K, q, group)
+    ref = oracle.forward_planes(p, alpha, z, x, group)[0]
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_CANONICAL, codes, alpha, z)
+    assert rel_err(run_gemv(L, x), ref) <= TOL
+
+
+LUT_SHAPES = [(1024, 1024, 3, 128), (8, 512, 3, 128), (296, 2048, 3, 128), (1000, 1536, 2, 128),
+              (520, 3584, 3, 128), (64, 1024, 1, 128), (136, 1024, 4, 128), (4096, 4096, 3, 128)]
+
+
+@pytest.mark.parametrize("N,K,q,group", LUT_SHAPES)
+def test_gemv_lut_kernel_default_plan(N, K, q, group):
+    p, codes, alpha, z, x = make_layer(f"lut/{N}x{K}", N, K, q, group)
+    ref = oracle.forward_planes(p, alpha, z, x, group)[0]
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    assert bq.plan_default(L.d).kernel == 1
+    assert rel_err(run_gemv(L, x), ref) <= TOL
+
+
+@pytest.mark.parametrize("N,K,q,rb,ks", [(520, 3584, 3, 2, 1), (520, 3584, 3, 2, 7), (520, 3584, 3, 3, 2),
+                                         (520, 3584, 3, 65, 3), (520, 3584, 3, 5, 4), (512, 1024, 2, 1, 1),
+                                         (512, 1024, 2, 1, 2), (1000, 1536, 2, 125, 3), (1000, 1536, 2, 2, 1)])
+def test_gemv_lut_kernel_explicit_plans(N, K, q, rb, ks):
+    """Ragged row blocks, one and several windows per block, with and without split-K."""
+    p, codes, alpha, z, x = make_layer(f"lutp/{N}x{K}", N, K, q, 128)
+    ref = oracle.forward_planes(p, alpha, z, x, 128)[0]
+    L = gpu_layer(N, K, q, 128, bq.LAYOUT_TILED, codes, alpha, z)
+    assert rel_err(run_gemv(L, x, bq.Plan(1, rb, ks, 0)), ref) <= TOL
+
+
+def test_gemv_workspace_is_reusable_and_result_deterministic():
+    N, K, q = 520, 3584, 3
+    p, codes, alpha, z, x = make_layer("lut/reuse", N, K, q, 128)
+    L = gpu_layer(N, K, q, 128, bq.LAYOUT_TILED, codes, alpha, z)
+    plan = bq.Plan(1, 3, 7, 0)
+    ws = bq.new_workspace(L.d, 1, plan)
+    xd = dev(x.reshape(-1))
+    ys = []
+    for _ in range(3):
+        y = torch.zeros(N, dtype=torch.float16, device=DEV)
+        bq.gemv_plan(L.d, plan, L.packed, L.alpha, L.z, xd, y, ws)
+        ys.append(y)
+    torch.cuda.synchronize()
+    assert torch.equal(ys[0].view(torch.int16), ys[1].view(torch.int16))
+    assert torch.equal(ys[0].view(torch.int16), ys[2].view(torch.int16))
+    ref = oracle.forward_planes(p, alpha, z, x, 128)[0]
+    assert rel_err(ys[2].cpu().numpy(), ref) <= TOL
+
+
+@pytest.mark.parametrize("layout", [bq.LAYOUT_CANONICAL, bq.LAYOUT_TILED])
+def test_gemv_structured_inputs(layout):
+    N, K, q, group = 64, 1024, 3, 128
+    p, codes, alpha, z, x = make_layer("struct", N, K, q, group)
+    W = oracle.dequant(codes, alpha, z, group)
+    L = gpu_layer(N, K, q, group, layout, codes, alpha, z)
+    # unit vectors return columns of the dequantised matrix (rounded to fp16 once)
+    for k in (0, 7, 8, 15, 16, 127, 128, 511, 512, 1023):
+        e = np.zeros((1, K), np.float16)
+        e[0, k] = 1.0
+        y = run_gemv(L, e)
+        assert np.abs(y - W[:, k]).max() <= 2.0 ** -10 * np.abs(W[:, k]).max() + 1e-7
+    # all planes +1
+    ones = np.full_like(codes, (1 << q) - 1)
+    L1 = gpu_layer(N, K, q, group, layout, ones, alpha, z)
+    ref = oracle.forward_dequant(ones, alpha, z, x, group)[0]
+    assert rel_err(run_gemv(L1, x), ref) <= TOL
+    # alpha = 0: only the offsets remain
+    L0 = gpu_layer(N, K, q, group, layout, codes, np.zeros_like(alpha), z)
+    ref = oracle.forward_dequant(codes, np.zeros_like(alpha), z, x, group)[0]
+    assert rel_err(run_gemv(L0, x), ref) <= TOL
+    # a single non-zero group
+    xg = np.zeros((1, K), np.float16)
+    xg[0, 384:512] = x[0, 384:512]
+    ref = oracle.forward_dequant(codes, alpha, z, xg, group)[0]
+    assert rel_err(run_gemv(L, xg), ref) <= TOL
+    # negative and zero scales are legal
+    a2 = alpha.copy()
+    a2[1] = -a2[1]
+    a2[2, ::2] = 0
+    L2 = gpu_layer(N, K, q, group, layout, codes, a2, z)
+    ref = oracle.forward_dequant(codes, a2, z, x, group)[0]
+    assert rel_err(run_gemv(L2, x), ref) <= TOL
+
+
+@pytest.mark.parametrize("layout,N,K,q,group", [(bq.LAYOUT_CANONICAL, 50, 256, 3, 64), (bq.LAYOUT_TILED, 264, 1024, 3, 128),
+                                                (bq.LAYOUT_CANONICAL, 16, 32, 3, 32), (bq.LAYOUT_TILED, 64, 512, 2, 0)])
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 8, 16])
+def test_gemm_smallbatch(layout, N, K, q, group, B):
+    p, codes, alpha, z, X = make_layer(f"sb/{N}x{K}", N, K, q, group, B)
+    ref = oracle.forward_planes(p, alpha, z, X, group)
+    L = gpu_layer(N, K, q, group, layout, codes, alpha, z)
+    Y = torch.full((B, N), float("nan"), dtype=torch.float16, device=DEV)
+    ws = bq.new_workspace(L.d, B)
+    bq.gemm_smallbatch(L.d, L.packed, L.alpha, L.z, dev(X), Y, B, ws)
+    torch.cuda.synchronize()
+    Yh = Y.cpu().numpy()
+    assert rel_err(Yh, ref) <= TOL
+    if B > 1:
+        # permuting the batch permutes the result bit for bit
+        perm = np.roll(np.arange(B), 1)
+        Y2 = torch.zeros_like(Y)
+        bq.gemm_smallbatch(L.d, L.packed, L.alpha, L.z, dev(X[perm]), Y2, B, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(Y2.cpu().numpy().view(np.uint16), Yh[perm].view(np.uint16))
+
+
+def test_gemv_host_buffers():
+    N, K, q, group = 520, 3584, 3, 128
+    p, codes, alpha, z, x = make_layer("host", N, K, q, group)
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    xh = torch.from_numpy(x.reshape(-1).copy()).pin_memory()
+    yh = torch.zeros(N, dtype=torch.float16).pin_memory()
+    xs = torch.zeros(K, dtype=torch.float16, device=DEV)
+    ys = torch.zeros(N, dtype=torch.float16, device=DEV)
+    ws = bq.new_workspace(L.d, 1)
+    bq.gemv_host(L.d, L.packed, L.alpha, L.z, xh, yh, xs, ys, ws)
+    torch.cuda.synchronize()
+    ref = oracle.forward_planes(p, alpha, z, x, group)[0]
+    assert rel_err(yh.numpy(), ref) <= TOL
+
+
+def test_device_errors_are_reported_not_raised_as_faults():
+    """Bad arguments come back as status codes through the binding, with the GPU untouched."""
+    d = bq.desc(64, 1000, 3, 128)
+    t = torch.zeros(64, dtype=torch.float16, device=DEV)
+    with pytest.raises(bq.BcqError) as e:
+        bq.gemv(d, t, t, t, t, t)
+    assert e.value.status == bq.ERR_UNSUPPORTED_SHAPE

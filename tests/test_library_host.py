@@ -1,0 +1,132 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, validates arguments before any launch, and plans decompositions."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2407_02891_b200 import binding as bq
+from paper_2407_02891_b200 import build as bq_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    bq_build.build()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "bcq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bcq_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert len(names) >= 15
+    L = ctypes.CDLL(bq.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(names) == set(bq.SIGNATURES), "binding and header disagree"
+    assert bq.lib().bcq_version() == 100
+
+
+def test_status_strings():
+    for s in (0, -1, -2, -3, -4, -5):
+        assert bq.lib().bcq_status_string(s)
+    assert bq.lib().bcq_status_string(-99) == b"unknown status"
+
+
+def test_desc_validation_and_sizes():
+    d = bq.desc(7168, 7168, 3, 128, bq.LAYOUT_TILED)
+    assert bq.check_desc(d) == bq.OK
+    assert bq.packed_bytes(d) == 3 * 7168 * 7168 // 8
+    assert bq.alpha_elems(d) == 3 * 7168 * 56 and bq.offset_elems(d) == 7168 * 56
+    assert bq.offset_elems(bq.desc(16, 32, 3, 0)) == 16
+    bad = [(0, 32, 3, 32, 0, bq.ERR_INVALID_ARG), (16, 32, 0, 32, 0, bq.ERR_INVALID_ARG),
+           (16, 32, 5, 32, 0, bq.ERR_INVALID_ARG), (16, 32, 3, 32, 7, bq.ERR_INVALID_ARG),
+           (16, 40, 3, 0, 0, bq.ERR_UNSUPPORTED_SHAPE), (16, 96, 3, 64, 0, bq.ERR_UNSUPPORTED_SHAPE),
+           (16, 96, 3, 48, 0, bq.ERR_UNSUPPORTED_SHAPE), (16, 256, 3, 128, 1, bq.ERR_UNSUPPORTED_SHAPE),
+           (12, 512, 3, 128, 1, bq.ERR_UNSUPPORTED_SHAPE), (16, 512, 3, 64, 1, bq.ERR_UNSUPPORTED_SHAPE)]
+    for N, K, q, g, lay, want in bad:
+        d = bq.desc(N, K, q, g, lay)
+        assert bq.check_desc(d) == want, (N, K, q, g, lay)
+        assert bq.packed_bytes(d) == 0 and bq.alpha_elems(d) == 0 and bq.offset_elems(d) == 0
+
+
+def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
+    L = bq.lib()
+    d = bq.desc(64, 512, 3, 128, bq.LAYOUT_CANONICAL)
+    plan = bq.Plan(0, 8, 1, 0)
+    ok = ctypes.c_void_p(0x10000)   # never dereferenced: every call below fails validation first
+    odd = ctypes.c_void_p(0x10004)
+    call = lambda *ptrs: L.bcq_gemv_plan(ctypes.byref(d), ctypes.byref(plan), *ptrs, None, 0, None)
+    assert call(None, ok, ok, ok, ok) == bq.ERR_INVALID_ARG
+    assert call(ok, ok, ok, ok, None) == bq.ERR_INVALID_ARG
+    assert call(odd, ok, ok, ok, ok) == bq.ERR_MISALIGNED
+    assert call(ok, ok, ok, odd, ok) == bq.ERR_MISALIGNED
+    assert L.bcq_gemv_plan(ctypes.byref(d), None, ok, ok, ok, ok, ok, None, 0, None) == bq.ERR_INVALID_ARG
+    # a lookup-table plan on a canonical descriptor is invalid
+    lut = bq.Plan(1, 1, 1, 0)
+    assert L.bcq_gemv_plan(ctypes.byref(d), ctypes.byref(lut), ok, ok, ok, ok, ok, None, 0, None) == bq.ERR_INVALID_ARG
+    # split-K without (enough) workspace
+    dt = bq.desc(64, 1024, 3, 128, bq.LAYOUT_TILED)
+    split = bq.Plan(1, 1, 2, 0)
+    need = bq.workspace_bytes(dt, 1, split)
+    assert need == 4096 * 4 + 2 * 64 * 4
+    args = (ctypes.byref(dt), ctypes.byref(split), ok, ok, ok, ok, ok)
+    assert L.bcq_gemv_plan(*args, None, 0, None) == bq.ERR_INVALID_ARG
+    assert L.bcq_gemv_plan(*args, ok, need - 1, None) == bq.ERR_WORKSPACE_TOO_SMALL
+    assert L.bcq_gemv_plan(*args, odd, need, None) == bq.ERR_MISALIGNED
+    # plans that break the limits
+    for p in (bq.Plan(1, 0, 1, 0), bq.Plan(1, 9, 1, 0), bq.Plan(1, 1, 3, 0), bq.Plan(2, 1, 1, 0)):
+        assert L.bcq_gemv_plan(ctypes.byref(dt), ctypes.byref(p), ok, ok, ok, ok, ok, ok, 1 << 20, None) == bq.ERR_INVALID_ARG
+    big = bq.desc(1024, 512, 3, 128, bq.LAYOUT_TILED)     # 128 units in one row block > 64
+    p = bq.Plan(1, 1, 1, 0)
+    assert L.bcq_gemv_plan(ctypes.byref(big), ctypes.byref(p), ok, ok, ok, ok, ok, None, 0, None) == bq.ERR_INVALID_ARG
+    # batch limits
+    assert L.bcq_gemm_smallbatch(ctypes.byref(d), ok, ok, ok, ok, ok, 17, None, 0, None) == bq.ERR_INVALID_ARG
+    assert L.bcq_gemm_smallbatch(ctypes.byref(d), ok, ok, ok, ok, ok, 0, None, 0, None) == bq.ERR_INVALID_ARG
+    assert L.bcq_gemm_smallbatch(ctypes.byref(d), ok, ok, ok, odd, ok, 2, None, 0, None) == bq.ERR_MISALIGNED
+
+
+def test_merge_and_pack_argument_checks():
+    L = bq.lib()
+    d = bq.desc(16, 32, 3, 32)
+    ok = ctypes.c_void_p(0x10000)
+    b2p = (ctypes.c_uint8 * 4)(0, 1, 2, 2)
+    bp = ctypes.cast(b2p, ctypes.c_void_p)
+    m = lambda dd, n_bits, table: L.bcq_merge_linear(ctypes.byref(dd), ok, ok, ok, n_bits, table, ok, ok, ok, None)
+    assert m(d, 9, bp) == bq.ERR_INVALID_ARG
+    assert m(d, 2, bp) == bq.ERR_INVALID_ARG                       # q > n_bits
+    assert m(d, 4, None) == bq.ERR_INVALID_ARG
+    unused = (ctypes.c_uint8 * 4)(0, 0, 2, 2)                      # plane 1 has no bit
+    assert m(d, 4, ctypes.cast(unused, ctypes.c_void_p)) == bq.ERR_INVALID_ARG
+    toobig = (ctypes.c_uint8 * 4)(0, 1, 2, 3)
+    assert m(d, 4, ctypes.cast(toobig, ctypes.c_void_p)) == bq.ERR_INVALID_ARG
+    assert L.bcq_pack(ctypes.byref(d), None, None, None, ok, None, None, None) == bq.ERR_INVALID_ARG
+    assert L.bcq_pack(ctypes.byref(d), ok, ok, None, ok, ok, ok, None) == bq.ERR_INVALID_ARG
+    d2 = bq.desc(16, 64, 3, 32)
+    assert L.bcq_repack(ctypes.byref(d), ok, None, None, ctypes.byref(d2), ok, None, None, None) == bq.ERR_INVALID_ARG
+    assert L.bcq_repack(ctypes.byref(d), ok, None, None, ctypes.byref(d), ok, None, None, None) == bq.ERR_INVALID_ARG  # in place
+
+
+@pytest.mark.parametrize("N,K", [(7168, 7168), (28672, 7168), (7168, 28672), (1024, 1024), (4096, 4096),
+                                 (16384, 4096), (4096, 16384), (9216, 9216), (36864, 9216), (9216, 36864),
+                                 (8192, 8192), (2048, 8192), (28672, 8192), (8192, 28672), (8, 512)])
+def test_default_plan_is_valid_and_fills_the_gpu(N, K):
+    d = bq.desc(N, K, 3, 128, bq.LAYOUT_TILED)
+    p = bq.plan_default(d, 1, 148)
+    assert p.kernel == 1
+    U, W = N // 8, K // 512
+    assert 1 <= p.row_blocks <= U and 1 <= p.k_splits <= W
+    assert -(-U // p.row_blocks) <= 64
+    blocks = p.row_blocks * p.k_splits
+    if U * W >= 148 * 8:
+        assert blocks >= 0.75 * 148
+    assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * N * 4)
+    # canonical descriptors and batches > 1 use the generic kernel
+    assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
+    assert bq.plan_default(d, 4, 148).kernel == 0
