@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the BCQ GEMV hot path: per-token time of all linear layers of a decoder stack.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one token at batch 1: every linear layer of the stack (6 per decoder layer) once,
+each with its own packed weights resident in HBM (the stack is far larger than L2, so every
+launch streams its weights from DRAM).  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2407_02891_b200 import synth
+
+# name -> (hidden, ffn, layers, q, group, description)
+WORKLOADS = {
+    "opt30b_q3_g128": dict(hidden=7168, ffn=28672, layers=48, q=3, group=128),
+    "opt30b_q2_g128": dict(hidden=7168, ffn=28672, layers=48, q=2, group=128),
+    "opt6.7b_q3_g128": dict(hidden=4096, ffn=16384, layers=32, q=3, group=128),
+    "opt66b_q2_g128": dict(hidden=9216, ffn=36864, layers=64, q=2, group=128),
+    "opt66b_q2_row": dict(hidden=9216, ffn=36864, layers=64, q=2, group=0),
+}
+DEFAULT_WORKLOAD = "opt30b_q3_g128"
+METRIC = "BCQ GEMV us/token (sum of all linear layers of the decoder stack, bs=1)"
+UNIT = "us/token"
+
+
+def layer_shapes(w):
+    """(name, N, K) of the six linear layers of one OPT decoder layer."""
+    h, f = w["hidden"], w["ffn"]
+    return [("q", h, h), ("k", h, h), ("v", h, h), ("out", h, h), ("fc1", f, h), ("fc2", h, f)]
+
+
+def algorithmic_bytes(N, K, q, group, B=1):
+    """Packed planes + fp16 alphas + fp16 offsets + x + y."""
+    G = 1 if group == 0 else K // group
+    return q * N * K // 8 + 2 * q * N * G + 2 * N * G + 2 * B * K + 2 * B * N
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int, period=0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+        self.period = period
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                mask = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# ---------------------------------------------------------------------------------------------
+# the stack on the device
+# ---------------------------------------------------------------------------------------------
+
+class Stack:
+    """All packed layers of the workload, resident on one GPU, plus per-shape x and per-layer y."""
+
+    def __init__(self, wname, device):
+        import torch
+        from paper_2407_02891_b200 import binding as bq
+
+        self.bq, self.torch, self.device = bq, torch, device
+        w = WORKLOADS[wname]
+        self.w, self.wname = w, wname
+        q, group = w["q"], w["group"]
+        self.items = []       # (desc, packed, alpha, z, x, y, ws)
+        self.bytes = 0
+        scales, xs, wss = {}, {}, {}
+        for (pname, N, K) in layer_shapes(w):
+            if (N, K) in scales:
+                continue
+            a, z = synth.scale_rows(f"{wname}/{N}x{K}", N, K, q, group)
+            dc = bq.desc(N, K, q, group, bq.LAYOUT_CANONICAL)
+            dt = dc.with_layout(bq.LAYOUT_TILED)
+            ad, zd = torch.from_numpy(a).to(device), torch.from_numpy(z).to(device)
+            at, zt = torch.empty_like(ad).view(-1), torch.empty_like(zd).view(-1)
+            bq.repack(dc, None, ad, zd, dt, None, at, zt)
+            scales[(N, K)] = (at, zt)
+            xs[(N, K)] = torch.from_numpy(synth.activations(f"{wname}/{N}x{K}", 1, K).reshape(-1)).to(device)
+            wss[(N, K)] = bq.new_workspace(dt, 1, device=device)
+        self.x_host = {k: v.cpu() for k, v in xs.items()}
+        for layer in range(w["layers"]):
+            for (pname, N, K) in layer_shapes(w):
+                dc = bq.desc(N, K, q, group, bq.LAYOUT_CANONICAL)
+                dt = dc.with_layout(bq.LAYOUT_TILED)
+                canon = synth.planes_device(f"{wname}/L{layer}/{pname}", N, K, q, device).reshape(-1)
+                packed = torch.empty_like(canon)
+                bq.repack(dc, canon, None, None, dt, packed, None, None)
+                at, zt = scales[(N, K)]
+                y = torch.zeros(N, dtype=torch.float16, device=device)
+                self.items.append((dt, packed, at.clone(), zt.clone(), xs[(N, K)], y, wss[(N, K)], (N, K)))
+                self.bytes += algorithmic_bytes(N, K, q, group)
+            torch.cuda.synchronize(device)
+        self.graph = None
+
+    def launch_all(self):
+        bq = self.bq
+        for (d, packed, a, z, x, y, ws, _) in self.items:
+            bq.gemv(d, packed, a, z, x, y, ws)
+
+    def capture(self):
+        torch = self.torch
+        self.launch_all()                      # first launches configure the kernels before capture
+        torch.cuda.synchronize(self.device)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.launch_all()
+        self.graph = g
+
+    def step(self):
+        self.graph.replay()
+
+    def time_steps(self, steps):
+        """Device time of `steps` graph replays, in ms (CUDA events on the launching stream)."""
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            self.graph.replay()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1)
+
+    def per_shape_us(self, reps=3):
+        """Mean device time per launch of each distinct shape, every launch on different weights."""
+        torch = self.torch
+        out = {}
+        shapes = sorted({it[7] for it in self.items})
+        for s in shapes:
+            its = [it for it in self.items if it[7] == s]
+            best = None
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for (d, packed, a, z, x, y, ws, _) in its:
+                    self.bq.gemv(d, packed, a, z, x, y, ws)
+                e1.record()
+                e1.synchronize()
+                t = e0.elapsed_time(e1) * 1e3 / len(its)
+                best = t if best is None else min(best, t)
+            N, K = s
+            b = algorithmic_bytes(N, K, self.w["q"], self.w["group"])
+            out[f"{N}x{K}"] = {"us": round(best, 3), "gbs": round(b / best * 1e-3, 1), "launches": len(its)}
+        return out
+
+    def e2e_steps(self, steps):
+        """The same token through bcq_gemv_host: x from pinned host memory, y back to host, per layer."""
+        torch, bq = self.torch, self.bq
+        xh = {k: v.pin_memory() for k, v in self.x_host.items()}
+        yh = {k: torch.zeros(k[0], dtype=torch.float16).pin_memory() for k in xh}
+        xs = {k: torch.zeros(k[1], dtype=torch.float16, device=self.device) for k in xh}
+        h2d = sum(2 * it[7][1] for it in self.items)
+        d2h = sum(2 * it[7][0] for it in self.items)
+
+        def one():
+            for (d, packed, a, z, x, y, ws, s) in self.items:
+                bq.gemv_host(d, packed, a, z, xh[s], yh[s], xs[s], y, ws)
+            torch.cuda.current_stream().synchronize()
+
+        for _ in range(2):
+            one()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(self.device)
+        e0.record()
+        for _ in range(steps):
+            one()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1) / steps, h2d, d2h
+
+
+# ---------------------------------------------------------------------------------------------
+# the oracle, timed on the host cores (CPU baseline / reference arm)
+# ---------------------------------------------------------------------------------------------
+
+class OracleSample:
+    """One decoder layer of the workload (6 products) for the CPU oracle, generated once on the host."""
+
+    def __init__(self, wname):
+        import oracle
+
+        self.oracle, self.wname, self.w = oracle, wname, WORKLOADS[wname]
+        q, group = self.w["q"], self.w["group"]
+        self.data = []
+        for (pname, N, K) in layer_shapes(self.w):
+            p = synth.planes(f"{wname}/L0/{pname}", N, K, q)
+            a, z = synth.scale_rows(f"{wname}/{N}x{K}", N, K, q, group)
+            x = synth.activations(f"{wname}/{N}x{K}", 1, K)
+            self.data.append((p, a, z, x))
+        self.cores = oracle.num_threads()
+
+    def layer_seconds(self):
+        t0 = time.perf_counter()
+        for (p, a, z, x) in self.data:
+            self.oracle.forward_planes(p, a, z, x, self.w["group"])
+        return time.perf_counter() - t0
+
+    def us_per_token(self, budget_s=12.0, max_reps=48):
+        """Time the oracle on the layer as often as fits the budget; scale the median to the stack."""
+        times, t_start = [], time.perf_counter()
+        while len(times) < max_reps:
+            times.append(self.layer_seconds())
+            if time.perf_counter() - t_start + times[-1] > budget_s:
+                break
+        sample = (f"{len(times)} x one decoder layer (6 products) of {self.wname}, fp64 bit-plane form, "
+                  f"median x {self.w['layers']} layers")
+        return float(np.median(times)) * self.w["layers"] * 1e6, sample
+
+
+# ---------------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w = WORKLOADS[args.workload]
+    config = {"workload": args.workload, "shapes": "4x(h x h), ffn x h, h x ffn per layer", "hidden": w["hidden"],
+              "ffn": w["ffn"], "layers": w["layers"], "q": w["q"], "group": w["group"], "batch": 1,
+              "cache": "inputs larger than L2 (every launch reads its own weights)", "parallelism": "replicas only"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        # each step is one decoder layer of the stack (a bounded sample), scaled to the whole stack
+        smp = OracleSample(args.workload)
+        steps, warmup = min(args.steps, 20), min(args.warmup, 2)
+        for _ in range(warmup):
+            smp.layer_seconds()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            smp.layer_seconds()
+        v = (time.perf_counter() - t0) / steps * w["layers"] * 1e6
+        cores = smp.cores
+        sample = (f"one decoder layer (6 products) of {args.workload} per step, {steps} steps timed, "
+                  f"scaled x {w['layers']} layers")
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": v / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "each step: " + sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}))
+        return
+
+    import torch
+
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    from paper_2407_02891_b200 import binding as bq
+    bq.lib()   # fail loudly if the CUDA library is missing
+
+    stack = Stack(args.workload, device)
+    stack.capture()
+    for _ in range(max(3, args.warmup)):
+        stack.step()
+    torch.cuda.synchronize(device)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    with ClockSampler(physical_gpu_index(local)) as clocks:
+        ms = stack.time_steps(args.steps)
+        torch.cuda.synchronize(device)
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    launches_per_step = len(stack.items)
+
+    per_shape = stack.per_shape_us()
+    e2e = None
+    if not args.no_e2e:
+        e_ms, h2d, d2h = stack.e2e_steps(max(3, min(args.steps, 20)))
+        if world > 1:
+            t = torch.tensor([e_ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": e_ms * 1e3 / world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "api": "bcq_gemv_host per layer, pinned host x and y, one stream sync per token"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak_gbs()
+    achieved = stack.bytes / (ms_per_step * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": ms_per_step * 1e3 / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+        "tokens_per_s": world * 1e3 / ms_per_step,
+        "clocks": clocks.summary(),
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "frac_of_nominal_8000": round(achieved / 8000.0, 4),
+                     "peak_kind": peak_kind, "traffic": None, "kernel": f"lut_gemv_kernel<{w['q']}>",
+                     "algorithmic_bytes_per_launch": stack.bytes // launches_per_step,
+                     "launches_per_step": launches_per_step},
+        "per_shape": per_shape,
+        "e2e": e2e,
+    }
+    if not args.no_cpu_baseline:
+        smp = OracleSample(args.workload)
+        v, sample = smp.us_per_token()
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": sample}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -352,11 +352,18 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 template <int Q>
 static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
 {
-    static bool configured = false;  // per process; the attribute is per function, set on every device on demand
+    // The opt-in to more than 48 KB of dynamic shared memory is per function and per device:
+    // done on the first launch on each device, remembered afterwards.
+    static bool configured[64] = {};
     constexpr int smem = LutSmem<Q>::kTotal;
-    cudaError_t e = cudaFuncSetAttribute(lut_gemv_kernel<Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    (void)configured;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(lut_gemv_kernel<Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
     lut_gemv_kernel<Q><<<prm.row_blocks * prm.k_splits, kLutThreads, smem, st>>>(prm);
     return cudaGetLastError();
 }
