@@ -62,7 +62,8 @@ typedef enum bcq_status {
                                      /* or a shape the tiled layout does not cover                        */
     BCQ_ERR_MISALIGNED = -3,         /* a device pointer is not aligned as required                       */
     BCQ_ERR_WORKSPACE_TOO_SMALL = -4,
-    BCQ_ERR_CUDA = -5                /* a CUDA runtime call failed; text via bcq_last_cuda_error()        */
+    BCQ_ERR_CUDA = -5,               /* a CUDA runtime call failed; text via bcq_last_cuda_error()        */
+    BCQ_ERR_SCRATCH_LIMIT = -6       /* bcq_gemv_noalloc: the product needs more than the built-in scratch */
 } bcq_status;
 
 enum { BCQ_LAYOUT_CANONICAL = 0, BCQ_LAYOUT_TILED = 1 };
@@ -178,6 +179,36 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed_dev, const uint16_t *
                   const uint16_t *z_dev, const uint16_t *x_host, uint16_t *y_host,
                   uint16_t *x_stage_dev, uint16_t *y_stage_dev,
                   void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
+ * bcq_gemv without a workspace argument and without any allocation.  (The paper has no
+ * counterpart; this entry point exists for the library's users.)
+ *
+ * Who it is for: callers that must not, or cannot, obtain device memory at the point where
+ * they need the product -- a plugin running inside a host application that owns all device
+ * memory and hands none out, a serving loop where an allocation would stall the whole device,
+ * a process whose memory budget is already fully committed.  Such callers cannot create the
+ * workspace bcq_gemv wants for its split-K partial sums.
+ *
+ * Here the scratch is a fixed array of BCQ_NOALLOC_SCRATCH_BYTES inside the library image.
+ * Consequences to know about:
+ *   - every GPU on which this library is loaded gives up that much memory until the process
+ *     exits, whether or not this function is ever called;
+ *   - a product whose default decomposition needs more scratch (k_splits * N * 4 bytes plus
+ *     16 KiB of counters) is refused with BCQ_ERR_SCRATCH_LIMIT and nothing is launched;
+ *   - the first call on each device looks up the array's device address (a host-side runtime
+ *     query, done with that device current).  Make that first call during start-up, before
+ *     any stream capture is begun;
+ *   - all calls on a device share the one array.  Calls on the same stream are ordered and
+ *     safe; calls whose kernels can overlap on the GPU (different streams, no dependency)
+ *     race on it and give wrong results.  The array keeps the previous call's contents; the
+ *     function clears the part that has to start at zero on every call.
+ * Neither this function nor anything it calls uses cudaMalloc, cudaFree or an allocating
+ * library routine.  Result and error behaviour are otherwise those of bcq_gemv.
+ */
+#define BCQ_NOALLOC_SCRATCH_BYTES (2u << 20)
+int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
+                     const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev, void *stream);
 
 /* ---- misc ----------------------------------------------------------------------------- */
 const char *bcq_status_string(int status);   /* static string                              */

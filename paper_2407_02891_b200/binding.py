@@ -24,6 +24,8 @@ ERR_UNSUPPORTED_SHAPE = -2
 ERR_MISALIGNED = -3
 ERR_WORKSPACE_TOO_SMALL = -4
 ERR_CUDA = -5
+ERR_SCRATCH_LIMIT = -6
+NOALLOC_SCRATCH_BYTES = 2 << 20
 
 
 class Desc(ctypes.Structure):
@@ -76,6 +78,7 @@ SIGNATURES = {
     "bcq_gemv_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemm_smallbatch": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "bcq_gemv_host": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_gemv_noalloc": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
 }
 
 
@@ -221,6 +224,17 @@ def gemv_host(d: Desc, packed, alpha, z, x_host, y_host, x_stage, y_stage, works
     wp, wn = _ws_args(workspace)
     _check(lib().bcq_gemv_host(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x_host), _ptr(y_host),
                                _ptr(x_stage), _ptr(y_stage), wp, wn, _stream()), "bcq_gemv_host")
+
+
+def gemv_noalloc(d: Desc, packed, alpha, z, x, y):
+    """bcq_gemv_noalloc: no workspace argument; the library's built-in scratch array is used.
+
+    For callers that cannot allocate device memory.  All calls on a device share that array, so
+    only issue them on one stream (or otherwise ordered); see include/bcq.h for the limits.
+    """
+    _dev(packed, alpha, z, x, y)
+    _check(lib().bcq_gemv_noalloc(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y),
+                                  _stream()), "bcq_gemv_noalloc")
 
 
 @dataclass

@@ -140,6 +140,7 @@ const char *bcq_status_string(int s)
         case BCQ_ERR_MISALIGNED: return "misaligned pointer";
         case BCQ_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case BCQ_ERR_CUDA: return "CUDA error";
+        case BCQ_ERR_SCRATCH_LIMIT: return "product needs more scratch than bcq_gemv_noalloc has built in";
     }
     return "unknown status";
 }
