@@ -124,12 +124,11 @@ def physical_gpu_index(local: int) -> int:
 class Stack:
     """All packed layers of the workload, resident on one GPU, plus per-shape x and per-layer y."""
 
-    def __init__(self, wname, device):
+    def __init__(self, wname, w, device):
         import torch
         from paper_2407_02891_b200 import binding as bq
 
         self.bq, self.torch, self.device = bq, torch, device
-        w = WORKLOADS[wname]
         self.w, self.wname = w, wname
         q, group = w["q"], w["group"]
         self.items = []       # (desc, packed, alpha, z, x, y, ws)
@@ -245,10 +244,10 @@ class Stack:
 class OracleSample:
     """One decoder layer of the workload (6 products) for the CPU oracle, generated once on the host."""
 
-    def __init__(self, wname):
+    def __init__(self, wname, w):
         import oracle
 
-        self.oracle, self.wname, self.w = oracle, wname, WORKLOADS[wname]
+        self.oracle, self.wname, self.w = oracle, wname, w
         q, group = self.w["q"], self.w["group"]
         self.data = []
         for (pname, N, K) in layer_shapes(self.w):
@@ -287,12 +286,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of decoder layers (profiling)")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under ncu: plain launches instead of a CUDA graph, warm-up as given, "
+                         "no per-shape, e2e or CPU legs; the printed number is not a benchmark value")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    w = WORKLOADS[args.workload]
+    w = dict(WORKLOADS[args.workload])
+    if args.layers > 0:
+        w["layers"] = args.layers
     config = {"workload": args.workload, "shapes": "4x(h x h), ffn x h, h x ffn per layer", "hidden": w["hidden"],
               "ffn": w["ffn"], "layers": w["layers"], "q": w["q"], "group": w["group"], "batch": 1,
               "cache": "inputs larger than L2 (every launch reads its own weights)", "parallelism": "replicas only"}
@@ -301,7 +306,7 @@ def main():
         if rank != 0:
             return
         # each step is one decoder layer of the stack (a bounded sample), scaled to the whole stack
-        smp = OracleSample(args.workload)
+        smp = OracleSample(args.workload, w)
         steps, warmup = min(args.steps, 20), min(args.warmup, 2)
         for _ in range(warmup):
             smp.layer_seconds()
@@ -332,7 +337,20 @@ def main():
     from paper_2407_02891_b200 import binding as bq
     bq.lib()   # fail loudly if the CUDA library is missing
 
-    stack = Stack(args.workload, device)
+    stack = Stack(args.workload, w, device)
+    if args.profile:
+        for _ in range(args.warmup):
+            stack.launch_all()
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            stack.launch_all()
+        e1.record()
+        e1.synchronize()
+        print(json.dumps({"profile_run": True, "config": config, "launches": len(stack.items) * args.steps,
+                          "ms_per_step_not_a_bench_value": e0.elapsed_time(e1) / args.steps}))
+        return
     stack.capture()
     for _ in range(max(3, args.warmup)):
         stack.step()
@@ -385,7 +403,7 @@ def main():
         "e2e": e2e,
     }
     if not args.no_cpu_baseline:
-        smp = OracleSample(args.workload)
+        smp = OracleSample(args.workload, w)
         v, sample = smp.us_per_token()
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": sample}
     print(json.dumps(out))

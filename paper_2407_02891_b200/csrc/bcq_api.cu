@@ -67,7 +67,7 @@ int plan_lut(const bcq_desc *d, int sm, bcq_plan *out)
     const int U = d->N / kUnitRows, W = d->K / kWindow;
     const int rb_min = (U + kMaxUnitsPerBlock - 1) / kMaxUnitsPerBlock;
     long long best = -1;
-    for (int ks = 1; ks <= W && ks <= 64; ++ks) {
+    for (int ks = (W + kMaxWindowsPerBlock - 1) / kMaxWindowsPerBlock; ks <= W && ks <= 64; ++ks) {
         for (int k = 0; k <= 16; ++k) {
             int rb = k == 0 ? rb_min : (k * sm) / ks;
             if (rb < rb_min || rb > U || rb > kMaxRowBlocks) continue;
@@ -91,6 +91,7 @@ int check_plan(const bcq_desc *d, const bcq_plan *p)
     const int U = d->N / kUnitRows, W = d->K / kWindow;
     if (p->row_blocks < 1 || p->row_blocks > U || p->row_blocks > kMaxRowBlocks) return BCQ_ERR_INVALID_ARG;
     if (p->k_splits < 1 || p->k_splits > W) return BCQ_ERR_INVALID_ARG;
+    if ((W + p->k_splits - 1) / p->k_splits > kMaxWindowsPerBlock) return BCQ_ERR_INVALID_ARG;
     if ((U + p->row_blocks - 1) / p->row_blocks > kMaxUnitsPerBlock) return BCQ_ERR_INVALID_ARG;
     return BCQ_OK;
 }

@@ -16,6 +16,7 @@ constexpr int kGroupsPerWindow = 4; // 128-weight groups in a window
 constexpr int kLutWarps = 16;       // warps per block of the lookup-table kernel
 constexpr int kLutUnitsPerWarp = 4; // row units a warp keeps accumulators for
 constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
+constexpr int kMaxWindowsPerBlock = 14; // windows of x a block keeps in shared memory
 constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace
 constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);
 
