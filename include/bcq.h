@@ -63,7 +63,8 @@ typedef enum bcq_status {
     BCQ_ERR_MISALIGNED = -3,         /* a device pointer is not aligned as required                       */
     BCQ_ERR_WORKSPACE_TOO_SMALL = -4,
     BCQ_ERR_CUDA = -5,               /* a CUDA runtime call failed; text via bcq_last_cuda_error()        */
-    BCQ_ERR_SCRATCH_LIMIT = -6       /* bcq_gemv_noalloc: the product needs more than the built-in scratch */
+    BCQ_ERR_SCRATCH_LIMIT = -6,      /* bcq_gemv_noalloc: the product needs more than the built-in scratch */
+    BCQ_ERR_TIMEOUT = -7             /* bcq_poll_status: a bounded wait inside a kernel ran out           */
 } bcq_status;
 
 enum { BCQ_LAYOUT_CANONICAL = 0, BCQ_LAYOUT_TILED = 1 };
@@ -209,6 +210,15 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed_dev, const uint16_t *
 #define BCQ_NOALLOC_SCRATCH_BYTES (2u << 20)
 int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
                      const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev, void *stream);
+
+/*
+ * Every wait inside the kernels (on an mbarrier fed by an asynchronous copy or by other warps)
+ * is bounded.  If one ever runs out, the block stops waiting, lets its outstanding copies land,
+ * returns without a fault, and records the event in a device status word; y is then undefined.
+ * bcq_poll_status synchronises with the device, returns BCQ_ERR_TIMEOUT if that happened since
+ * the last poll (detail via bcq_last_cuda_error) and clears the word; BCQ_OK otherwise.
+ */
+int bcq_poll_status(void);
 
 /* ---- misc ----------------------------------------------------------------------------- */
 const char *bcq_status_string(int status);   /* static string                              */

@@ -25,6 +25,7 @@ ERR_MISALIGNED = -3
 ERR_WORKSPACE_TOO_SMALL = -4
 ERR_CUDA = -5
 ERR_SCRATCH_LIMIT = -6
+ERR_TIMEOUT = -7
 NOALLOC_SCRATCH_BYTES = 2 << 20
 
 
@@ -79,6 +80,7 @@ SIGNATURES = {
     "bcq_gemm_smallbatch": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "bcq_gemv_host": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_noalloc": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "bcq_poll_status": (_i, []),
 }
 
 
@@ -224,6 +226,11 @@ def gemv_host(d: Desc, packed, alpha, z, x_host, y_host, x_stage, y_stage, works
     wp, wn = _ws_args(workspace)
     _check(lib().bcq_gemv_host(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x_host), _ptr(y_host),
                                _ptr(x_stage), _ptr(y_stage), wp, wn, _stream()), "bcq_gemv_host")
+
+
+def poll_status():
+    """bcq_poll_status: synchronise and raise if a bounded device-side wait ran out since the last poll."""
+    _check(lib().bcq_poll_status(), "bcq_poll_status")
 
 
 def gemv_noalloc(d: Desc, packed, alpha, z, x, y):

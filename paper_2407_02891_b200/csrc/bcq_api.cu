@@ -142,8 +142,21 @@ const char *bcq_status_string(int s)
         case BCQ_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case BCQ_ERR_CUDA: return "CUDA error";
         case BCQ_ERR_SCRATCH_LIMIT: return "product needs more scratch than bcq_gemv_noalloc has built in";
+        case BCQ_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     }
     return "unknown status";
+}
+
+int bcq_poll_status(void)
+{
+    int v = 0;
+    cudaError_t e = lut_status_take(&v);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (v != 0) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "lut_gemv_kernel: bounded wait %d ran out", v);
+        return BCQ_ERR_TIMEOUT;
+    }
+    return BCQ_OK;
 }
 
 int bcq_check_desc(const bcq_desc *desc) { return check_desc(desc); }

@@ -73,4 +73,6 @@ cudaError_t launch_generic(const bcq_desc &d, const void *packed, const uint16_t
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st);
 
+cudaError_t lut_status_take(int *status);
+
 }  // namespace bcq

@@ -1,0 +1,533 @@
+// Lookup-table BCQ GEMV (batch 1, tiled layout, group 128) for sm_100a.
+//
+//   y = sum_g ( sum_i alpha_i (B_i x)_g + z (sum x)_g )          (Eq. bcw + Eq. fuse_step3)
+//
+// Per 512-wide window of K the block builds, in shared memory, all 2^8 signed sums of every
+// 8-activation chunk; packed weight bytes index those tables directly.  One block per SM, three
+// kinds of warps:
+//
+//   builders  (warps 0-2)   convert the block's slice of x to fp32 and build the window tables,
+//                           one window ahead of the consumers (two 64 KB tables, double buffered);
+//   producer  (warp 3)      one thread feeds a ring of shared-memory slots with bulk async copies
+//                           (cp.async.bulk, completion on an mbarrier): per (window, row unit) one
+//                           slot = q*512 B of plane bytes + the unit's alphas and offsets;
+//   consumers (warps 4-19)  copy a filled slot into registers, hand the slot back, look every
+//                           weight byte up in the window table and accumulate in fp32.
+//
+// Table layout: word address of (entry e, chunk c) = e*64 + (c&1)*32 + (c>>1).  Lane l of a
+// consumer warp only ever looks up chunks 2l and 2l+1, so a warp's lookups always hit 32 distinct
+// banks whatever the weight bytes are.  The tables sit at shared-window addresses that are
+// multiples of 64 KB and an entry is 256 B apart from the next, so ONE byte-permute builds the
+// complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + 4*lane): a lookup is
+// PRMT + LDS.  The memory before and after the tables (99 KB together) holds x, the barriers and
+// the slot ring.
+//
+// Every wait on an mbarrier is bounded; if one runs out the block sets an abort flag and a
+// device status word, stops waiting, drains its own copies and returns (see lut_status_take).
+#include <type_traits>
+
+#include "bcq_internal.cuh"
+
+namespace bcq {
+
+constexpr int kBuilderWarps = 3;
+constexpr int kBuilderThreads = kBuilderWarps * 32;
+constexpr int kProducerWarp = kBuilderWarps;
+constexpr int kFirstConsumerWarp = kBuilderWarps + 1;
+constexpr int kConsumerThreads = kLutWarps * 32;
+constexpr int kLutThreads = (kBuilderWarps + 1 + kLutWarps) * 32;  // 640
+constexpr int kTableBytes = 256 * 64 * 4;                          // 65536
+constexpr int kLutSmemBytes = 232448;                              // 227 KB: the per-block opt-in maximum
+constexpr int kMaxSlots = 48;
+constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
+constexpr int kXBytes = kMaxWindowsPerBlock * kWindow * 4;
+constexpr int kBarrierBytes = 1024;
+constexpr int kFixedBytes = kXBytes + kBarrierBytes;
+constexpr int kSpinLimit = 1 << 20;   // tries per wait (each try blocks for a short, hardware-defined time)
+
+static_assert(2 * kFixedBytes <= kLutSmemBytes - 2 * kTableBytes, "x + barriers must fit before or after the tables");
+
+__device__ int g_lut_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
+
+template <int Q>
+struct Slot {
+    static constexpr int kPlaneBytes = Q * 512;
+    static constexpr int kAlphaBytes = Q * 64;
+    static constexpr int kOffsetBytes = 64;
+    static constexpr int kBytes = kPlaneBytes + kAlphaBytes + kOffsetBytes;
+};
+
+struct LutParams {
+    const uint8_t *planes;
+    const uint8_t *alpha;  // tiled
+    const uint8_t *z;      // tiled
+    const __half *x;
+    __half *y;
+    float *partial;  // [k_splits][N] when k_splits > 1
+    int *counters;   // [row_blocks]
+    int N, K, U, W;
+    int row_blocks, k_splits;
+};
+
+template <int I, int N, class F>
+__device__ __forceinline__ void static_for(F &&f)
+{
+    if constexpr (I < N) {
+        f(std::integral_constant<int, I>{});
+        static_for<I + 1, N>(f);
+    }
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
+
+// ---- mbarrier / bulk-copy primitives ------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the block is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code)
+{
+    for (int it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63) == 63 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicExch(&g_lut_status, code);
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void named_barrier(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// table lookup: the address register already holds the complete shared-window address
+template <int OFF>
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(OFF));
+    return v;
+}
+
+// two fp32 lanes in one 64-bit register
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ float2 unpack2(f32x2 v)
+{
+    float2 r;
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
+{
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// Index, inside a window's 512 staged activations, of activation j of chunk c = 2*(4*lq + k) + s:
+// [j][quad = 8s + lq][k], so that one 128-bit load gives activation j of the four chunks of a build
+// item and the 16 quads a warp reads at once are 256 contiguous bytes (no bank conflicts).
+__device__ __forceinline__ int xs_index(int kk)
+{
+    const int l = kk >> 4, s = (kk >> 3) & 1, j = kk & 7;
+    return ((j * 16 + s * 8 + (l >> 2)) << 2) + (l & 3);
+}
+
+// One build item = 8 table entries (entry bits 3..7 = item >> 4) of the four chunks of quad
+// item & 15 (slot s = quad >> 3, lanes 4*(quad&7) .. +3).  The 8 entries are walked in Gray-code
+// order: one packed FMA per entry and chunk pair, one 128-bit conflict-free store per entry.
+__device__ __forceinline__ void build_item(unsigned char *table, const float *xs_w, int item)
+{
+    const int quad = item & 15;
+    const int hi = item >> 4;
+    const float4 *xq = reinterpret_cast<const float4 *>(xs_w) + quad;  // xq[16 j] = activation j of the 4 chunks
+    f32x2 c01 = pack2(0.f, 0.f), c23 = c01;
+#pragma unroll
+    for (int j = 3; j < 8; ++j) {
+        const float4 v = xq[16 * j];
+        const float sg = ((hi >> (j - 3)) & 1) ? 1.f : -1.f;
+        const f32x2 s2 = pack2(sg, sg);
+        c01 = fma2(s2, pack2(v.x, v.y), c01);
+        c23 = fma2(s2, pack2(v.z, v.w), c23);
+    }
+    f32x2 x01[3], x23[3];
+    const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        const float4 v = xq[16 * j];
+        x01[j] = pack2(v.x, v.y);
+        x23[j] = pack2(v.z, v.w);
+        c01 = fma2(m1, x01[j], c01);
+        c23 = fma2(m1, x23[j], c23);
+    }
+    unsigned char *dst = table + quad * 16 + hi * (8 * 256);
+    static_for<0, 8>([&](auto step_c) {
+        constexpr int step = decltype(step_c)::value;
+        constexpr int gray = step ^ (step >> 1);
+        if constexpr (step > 0) {
+            constexpr int bit = (step & 1) ? 0 : ((step & 2) ? 1 : 2);  // lowest set bit of step
+            constexpr bool on = (gray >> bit) & 1;
+            c01 = fma2(on ? p2 : m2, x01[bit], c01);
+            c23 = fma2(on ? p2 : m2, x23[bit], c23);
+        }
+        const float2 a = unpack2(c01), b = unpack2(c23);
+        *reinterpret_cast<float4 *>(dst + gray * 256) = make_float4(a.x, a.y, b.x, b.y);
+    });
+}
+
+enum { kWaitEmpty = 1, kWaitFull = 2, kWaitTableReady = 3, kWaitTableFree = 4, kWaitDrain = 5, kTooFewSlots = 6 };
+
+template <int Q>
+__global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    using SL = Slot<Q>;
+    constexpr int UMAX = kLutUnitsPerWarp;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    const int rbi = blockIdx.x % p.row_blocks, ks = blockIdx.x / p.row_blocks;
+    const int u0 = int((long long)rbi * p.U / p.row_blocks), u1 = int((long long)(rbi + 1) * p.U / p.row_blocks);
+    const int w0 = int((long long)ks * p.W / p.k_splits), w1 = int((long long)(ks + 1) * p.W / p.k_splits);
+    const int V = u1 - u0;       // row units of this block
+    const int nwin = w1 - w0;    // windows of this block
+
+    // ---- carve shared memory: [front | table 0 | table 1 | back] --------------------------------
+    const uint32_t base = smem_u32(smem);
+    const uint32_t tab0 = (base + 0xFFFFu) & ~0xFFFFu;  // shared-window address of table 0
+    const int front = int(tab0 - base), back = kLutSmemBytes - front - 2 * kTableBytes;
+    unsigned char *tables = smem + front;
+    unsigned char *after = tables + 2 * kTableBytes;
+    const bool fixed_in_back = back >= kFixedBytes;
+    unsigned char *fixed = fixed_in_back ? after : smem;
+    unsigned char *ring_a = fixed_in_back ? smem : smem + kFixedBytes;
+    unsigned char *ring_b = fixed_in_back ? after + kFixedBytes : after;
+    const int n_a = (fixed_in_back ? front : front - kFixedBytes) / SL::kBytes;
+    const int n_b = (fixed_in_back ? back - kFixedBytes : back) / SL::kBytes;
+    const int NS = min(n_a + n_b, kMaxSlots);
+    const int D = min(NS / kLutWarps, 3);   // ring slots per consumer warp
+    auto slot_ptr = [&](int s) -> unsigned char * { return s < n_a ? ring_a + s * SL::kBytes : ring_b + (s - n_a) * SL::kBytes; };
+
+    float *xs = reinterpret_cast<float *>(fixed);
+    const uint32_t bars = smem_u32(fixed + kXBytes);
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kMaxSlots;
+    const uint32_t bar_tab_ready = bars + 16 * kMaxSlots, bar_tab_free = bar_tab_ready + 16;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + kXBytes + 16 * kMaxSlots + 32);
+    int *s_last = const_cast<int *>(abort_flag) + 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < kMaxSlots; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_tab_ready + 8 * b, kBuilderThreads);
+            mbar_init(bar_tab_free + 8 * b, kLutWarps);
+        }
+        *abort_flag = (NS < kMinSlots) ? 1 : 0;
+        if (NS < kMinSlots) atomicExch(&g_lut_status, int(kTooFewSlots));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    // =============================================================================================
+    if (warp < kBuilderWarps) {
+        // ---- builders: x slice fp16 -> fp32 (permuted for the build), then one table per window ----
+        const __half *xg = p.x + size_t(w0) * kWindow;
+        for (int e = tid; e < nwin * kWindow; e += kBuilderThreads)
+            xs[(e & ~(kWindow - 1)) + xs_index(e & (kWindow - 1))] = __half2float(xg[e]);
+        named_barrier(1, kBuilderThreads);
+        for (int wi = 0; wi < nwin; ++wi) {
+            const int b = wi & 1, use = wi >> 1;
+            if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree)) break;
+            unsigned char *table = tables + b * kTableBytes;
+            for (int item = tid; item < 512; item += kBuilderThreads) build_item(table, xs + wi * kWindow, item);
+            mbar_arrive(bar_tab_ready + 8 * b);
+        }
+        return;
+    }
+
+    if (warp == kProducerWarp) {
+        // ---- producer: one thread keeps the slot ring full ---------------------------------------
+        // Lane c feeds consumer warp c: slots c and c + 16 (+ 32) belong to that warp alone, so a
+        // slot's fills are consumed by one warp, in order, and a wait can never be satisfied by
+        // an older phase of the barrier.
+        if (lane < kLutWarps && !*abort_flag) {
+            const int c = lane;
+            const int mine = (V - c + kLutWarps - 1) / kLutWarps;  // units of warp c per window
+            int d = 0, k = 0, last_s = -1, last_par = 0, prev_s = -1, prev_par = 0, pprev_s = -1, pprev_par = 0;
+            bool ok = true;
+            for (int wi = 0; wi < nwin && ok; ++wi) {
+                size_t tile = size_t(w0 + wi) * p.U + u0 + c;
+                for (int t = 0; t < mine; ++t, tile += kLutWarps) {
+                    const int s = c + kLutWarps * d;
+                    if (k > 0 && !mbar_wait(bar_empty + 8 * s, (k - 1) & 1, abort_flag, kWaitEmpty)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t dst = smem_u32(slot_ptr(s)), full = bar_full + 8 * s;
+                    mbar_expect_tx(full, SL::kBytes);
+                    bulk_g2s(dst, p.planes + tile * SL::kPlaneBytes, SL::kPlaneBytes, full);
+                    bulk_g2s(dst + SL::kPlaneBytes, p.alpha + tile * SL::kAlphaBytes, SL::kAlphaBytes, full);
+                    bulk_g2s(dst + SL::kPlaneBytes + SL::kAlphaBytes, p.z + tile * SL::kOffsetBytes, SL::kOffsetBytes, full);
+                    pprev_s = prev_s, pprev_par = prev_par, prev_s = last_s, prev_par = last_par;
+                    last_s = s, last_par = k & 1;
+                    if (++d == D) {
+                        d = 0;
+                        ++k;
+                    }
+                }
+            }
+            // See the last fill of each of this lane's (at most 3) slots land, with a bounded wait,
+            // before the warp leaves: the block's shared memory must not be handed to another block
+            // while copies into it are in flight, also when the consumers gave up.
+            const int ss[3] = {last_s, prev_s, pprev_s}, pp[3] = {last_par, prev_par, pprev_par};
+#pragma unroll
+            for (int q3 = 0; q3 < 3; ++q3) {
+                if (ss[q3] < 0 || q3 >= D) continue;
+                bool landed = false;
+                for (int it = 0; it < kSpinLimit && !landed; ++it) landed = mbar_try_wait(bar_full + 8 * ss[q3], uint32_t(pp[q3]));
+                if (!landed) atomicExch(&g_lut_status, int(kWaitDrain));
+            }
+        }
+        return;
+    }
+
+    // =============================================================================================
+    // ---- consumers ---------------------------------------------------------------------------------
+    const int cw = warp - kFirstConsumerWarp;   // 0..15
+    const int ctid = tid - kFirstConsumerWarp * 32;
+    f32x2 acc[UMAX][4];
+    float zacc[UMAX];
+#pragma unroll
+    for (int t = 0; t < UMAX; ++t) {
+        zacc[t] = 0.f;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc[t][r] = pack2(0.f, 0.f);
+    }
+    bool alive = !*abort_flag;
+    int d = 0, k = 0;   // this warp's ring position: slot cw + 16 d, fill number k
+
+    for (int wi = 0; wi < nwin && alive; ++wi) {
+        const int b = wi & 1;
+        if (!mbar_wait(bar_tab_ready + 8 * b, (wi >> 1) & 1, abort_flag, kWaitTableReady)) {
+            alive = false;
+            break;
+        }
+        const uint32_t lane_off = tab0 + uint32_t(b * kTableBytes + lane * 4);
+        // sum of this lane's 16 activations (the all-ones entries of its two chunks), then of its group
+        float xsum = lds_f32<255 * 256>(lane_off) + lds_f32<255 * 256 + 128>(lane_off);
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+        xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
+
+        static_for<0, UMAX>([&](auto T) {
+            constexpr int t = decltype(T)::value;
+            if (alive && cw + kLutWarps * t < V) {
+                const int s = cw + kLutWarps * d;
+                if (!mbar_wait(bar_full + 8 * s, k & 1, abort_flag, kWaitFull)) {
+                    alive = false;
+                } else {
+                    // slot -> registers, then hand the slot back to the producer
+                    const unsigned char *slot = slot_ptr(s);
+                    uint32_t wbuf[4 * Q];
+                    uint4 araw[Q];
+#pragma unroll
+                    for (int j = 0; j < Q; ++j) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(slot + j * 512 + lane * 16);
+                        wbuf[4 * j + 0] = v.x;
+                        wbuf[4 * j + 1] = v.y;
+                        wbuf[4 * j + 2] = v.z;
+                        wbuf[4 * j + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int i = 0; i < Q; ++i)
+                        araw[i] = *reinterpret_cast<const uint4 *>(slot + SL::kPlaneBytes + (lane >> 3) * (Q * 16) + i * 16);
+                    const __half zh = *reinterpret_cast<const __half *>(slot + SL::kPlaneBytes + SL::kAlphaBytes + lane * 2);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+
+                    // offsets: lane (g, j) adds z[g][row j] * (sum of x over group g)
+                    zacc[t] = fmaf(__half2float(zh), xsum, zacc[t]);
+                    static_for<0, 4>([&](auto PR) {
+                        constexpr int pr = decltype(PR)::value;  // rows 2pr and 2pr+1
+                        f32x2 a2 = acc[t][pr];
+                        static_for<0, Q>([&](auto I) {
+                            constexpr int i = decltype(I)::value;
+                            constexpr int b0 = ((2 * pr) * Q + i) * 2, b1 = ((2 * pr + 1) * Q + i) * 2;
+                            const uint32_t word0 = wbuf[b0 >> 2], word1 = wbuf[b1 >> 2];
+                            const float v00 = lds_f32<0>(__byte_perm(word0, lane_off, 0x7604 | ((b0 & 3) << 4)));
+                            const float v01 = lds_f32<128>(__byte_perm(word0, lane_off, 0x7604 | (((b0 + 1) & 3) << 4)));
+                            const float v10 = lds_f32<0>(__byte_perm(word1, lane_off, 0x7604 | ((b1 & 3) << 4)));
+                            const float v11 = lds_f32<128>(__byte_perm(word1, lane_off, 0x7604 | (((b1 + 1) & 3) << 4)));
+                            const f32x2 s2 = add2(pack2(v00, v10), pack2(v01, v11));
+                            const uint32_t aw = reinterpret_cast<const uint32_t *>(&araw[i])[pr];
+                            const float2 af = __half22float2(*reinterpret_cast<const __half2 *>(&aw));
+                            a2 = fma2(pack2(af.x, af.y), s2, a2);
+                        });
+                        acc[t][pr] = a2;
+                    });
+                }
+                if (++d == D) {
+                    d = 0;
+                    ++k;
+                }
+            }
+        });
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tab_free + 8 * b);
+    }
+
+    // ---- reduce each unit's 8 row sums over the 32 lanes: lane l ends with row l & 7 -------------
+    float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * p.N : nullptr;
+    static_for<0, UMAX>([&](auto T) {
+        constexpr int t = decltype(T)::value;
+        if (cw + kLutWarps * t < V) {
+            float v4[4], v2[2], v1;
+#pragma unroll
+            for (int pr = 0; pr < 4; ++pr) {  // lane bit 0 picks the row of the pair
+                const float2 a = unpack2(acc[t][pr]);
+                const bool odd = lane & 1;
+                v4[pr] = (odd ? a.y : a.x) + __shfl_xor_sync(0xffffffffu, odd ? a.x : a.y, 1);
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {  // lane bit 1 picks the pair inside a half
+                const bool up = lane & 2;
+                v2[h] = (up ? v4[2 * h + 1] : v4[2 * h]) + __shfl_xor_sync(0xffffffffu, up ? v4[2 * h] : v4[2 * h + 1], 2);
+            }
+            {
+                const bool up = lane & 4;  // lane bit 2 picks the half
+                v1 = (up ? v2[1] : v2[0]) + __shfl_xor_sync(0xffffffffu, up ? v2[0] : v2[1], 4);
+            }
+            v1 += zacc[t];  // lane (g, j) holds group g's offset term of row j = l & 7
+            v1 += __shfl_xor_sync(0xffffffffu, v1, 8);
+            v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
+            if (lane < 8) {
+                const int n = (u0 + cw + kLutWarps * t) * kUnitRows + lane;
+                if (partial)
+                    partial[n] = v1;
+                else
+                    p.y[n] = __float2half_rn(v1);
+            }
+        }
+    });
+
+    // ---- split-K: the last block to arrive for this row block adds the partials in fixed order --
+    if (p.k_splits > 1) {
+        __threadfence();
+        named_barrier(2, kConsumerThreads);
+        if (ctid == 0) {
+            const int old = atomicAdd(p.counters + rbi, 1);
+            *s_last = (old == p.k_splits - 1);
+        }
+        named_barrier(2, kConsumerThreads);
+        if (*s_last) {
+            __threadfence();
+            for (int n = u0 * kUnitRows + ctid; n < u1 * kUnitRows; n += kConsumerThreads) {
+                float v = 0.f;
+                for (int k = 0; k < p.k_splits; ++k) v += __ldcg(p.partial + size_t(k) * p.N + n);
+                p.y[n] = __float2half_rn(v);
+            }
+            if (ctid == 0) p.counters[rbi] = 0;
+        }
+    }
+}
+
+template <int Q>
+static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
+{
+    // The opt-in to more than 48 KB of dynamic shared memory is per function and per device:
+    // done on the first launch on each device, remembered afterwards.
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(lut_gemv_kernel<Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    lut_gemv_kernel<Q><<<prm.row_blocks * prm.k_splits, kLutThreads, kLutSmemBytes, st>>>(prm);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
+                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st)
+{
+    LutParams prm;
+    prm.planes = static_cast<const uint8_t *>(packed);
+    prm.alpha = reinterpret_cast<const uint8_t *>(alpha);
+    prm.z = reinterpret_cast<const uint8_t *>(z);
+    prm.x = reinterpret_cast<const __half *>(x);
+    prm.y = reinterpret_cast<__half *>(y);
+    prm.counters = static_cast<int *>(workspace);
+    prm.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + kCounterBytes) : nullptr;
+    prm.N = d.N;
+    prm.K = d.K;
+    prm.U = d.N / kUnitRows;
+    prm.W = d.K / kWindow;
+    prm.row_blocks = plan.row_blocks;
+    prm.k_splits = plan.k_splits;
+    switch (d.q) {
+        case 1: return launch_lut_q<1>(prm, st);
+        case 2: return launch_lut_q<2>(prm, st);
+        case 3: return launch_lut_q<3>(prm, st);
+        case 4: return launch_lut_q<4>(prm, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// Read and clear the device status word (synchronises with the device).
+cudaError_t lut_status_take(int *status)
+{
+    int v = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&v, g_lut_status, sizeof(int));
+    if (e != cudaSuccess) return e;
+    if (v != 0) {
+        const int zero = 0;
+        e = cudaMemcpyToSymbol(g_lut_status, &zero, sizeof(int));
+    }
+    *status = v;
+    return e;
+}
+
+}  // namespace bcq
