@@ -138,12 +138,8 @@ class Stack:
             if (N, K) in scales:
                 continue
             a, z = synth.scale_rows(f"{wname}/{N}x{K}", N, K, q, group)
-            dc = bq.desc(N, K, q, group, bq.LAYOUT_CANONICAL)
-            dt = dc.with_layout(bq.LAYOUT_TILED)
-            ad, zd = torch.from_numpy(a).to(device), torch.from_numpy(z).to(device)
-            at, zt = torch.empty_like(ad).view(-1), torch.empty_like(zd).view(-1)
-            bq.repack(dc, None, ad, zd, dt, None, at, zt)
-            scales[(N, K)] = (at, zt)
+            dt = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
+            scales[(N, K)] = (torch.from_numpy(a).to(device), torch.from_numpy(z).to(device))
             xs[(N, K)] = torch.from_numpy(synth.activations(f"{wname}/{N}x{K}", 1, K).reshape(-1)).to(device)
             wss[(N, K)] = bq.new_workspace(dt, 1, device=device)
         self.x_host = {k: v.cpu() for k, v in xs.items()}
@@ -152,11 +148,11 @@ class Stack:
                 dc = bq.desc(N, K, q, group, bq.LAYOUT_CANONICAL)
                 dt = dc.with_layout(bq.LAYOUT_TILED)
                 canon = synth.planes_device(f"{wname}/L{layer}/{pname}", N, K, q, device).reshape(-1)
-                packed = torch.empty_like(canon)
-                bq.repack(dc, canon, None, None, dt, packed, None, None)
-                at, zt = scales[(N, K)]
+                ad, zd = scales[(N, K)]
+                packed, at, zt = bq.empty_operands(dt, device)      # every layer owns its operands
+                bq.repack(dc, canon, ad, zd, dt, packed, at, zt)
                 y = torch.zeros(N, dtype=torch.float16, device=device)
-                self.items.append((dt, packed, at.clone(), zt.clone(), xs[(N, K)], y, wss[(N, K)], (N, K)))
+                self.items.append((dt, packed, at, zt, xs[(N, K)], y, wss[(N, K)], (N, K)))
                 self.bytes += algorithmic_bytes(N, K, q, group)
             torch.cuda.synchronize(device)
         self.graph = None

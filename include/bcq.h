@@ -32,16 +32,23 @@
  *   z       fp16   [N][G]
  *   x       fp16   [B][K],   y fp16 [B][N]
  *
- * Tiled layout (BCQ_LAYOUT_TILED): the same bytes and the same fp16 values, permuted so
- * that every load of the batch-1 kernel is a contiguous 512-byte warp transaction and a
- * lane's bytes all index the lane's own shared-memory banks.  It needs K % 512 == 0,
- * N % 8 == 0 and group in {0, 128}.  With U = N/8 row units (8 rows) and K/512 windows:
- *   packed  tile (w,u) at byte ((w*U + u) * q) * 512; inside: [j < q][lane < 32][16 bytes];
- *           byte p = 16 j + (byte in lane) = (r*q + i)*2 + s  holds row 8u + r, plane i,
- *           weights k = 512 w + 16 lane + 8 s .. + 7   (bit order as canonical)
- *   alpha   group 128: [w][u][gi < 4][i < q][r < 8] <- alpha[i][8u + r][4w + gi];  group 0: [u][i][r]
- *   z       group 128: [w][u][gi < 4][r < 8]        <- z[8u + r][4w + gi];         group 0: [u][r]
- * Sizes are identical in both layouts (bcq_packed_bytes, bcq_alpha_elems, bcq_offset_elems).
+ * Tiled layout (BCQ_LAYOUT_TILED): the same bytes and the same fp16 values, permuted so that
+ * the batch-1 kernel fetches everything it needs for 8 rows x 512 weights with ONE contiguous
+ * bulk copy and a lane's bytes all index the lane's own shared-memory banks.  It needs
+ * K % 512 == 0, N % 8 == 0 and group in {0, 128}.  With U = N/8 row units and K/512 windows,
+ * `packed` is a sequence of tiles, tile (w, u) at byte (w*U + u) * T:
+ *   bytes [0, q*512)      planes as [j < q][lane < 32][16 bytes]; byte p = 16 j + (byte in lane)
+ *                         = (r*q + i)*2 + s  holds row 8u + r, plane i, weights
+ *                         k = 512 w + 16 lane + 8 s .. + 7   (bit order as canonical)
+ *   group 128, T = q*576 + 64: the tile continues with the scales of its four groups,
+ *     bytes [q*512, q*576)   alpha fp16 [gi < 4][i < q][r < 8]  <- alpha[i][8u + r][4w + gi]
+ *     bytes [q*576, T)       z     fp16 [gi < 4][r < 8]         <- z[8u + r][4w + gi]
+ *     and the alpha / z arguments of every call are ignored for this layout (pass NULL);
+ *   group 0 (one scale per row), T = q*512: alpha and z stay in arrays of their own,
+ *     alpha [u][i][r], z [u][r].
+ * bcq_packed_bytes gives the size of `packed` for the descriptor's layout (it includes the
+ * scales exactly when they live in the tiles); bcq_alpha_elems and bcq_offset_elems give the
+ * element counts of separate alpha / z arrays (the canonical counts).
  */
 #ifndef BCQ_H
 #define BCQ_H
@@ -79,9 +86,9 @@ typedef struct bcq_desc {
     int32_t layout;
 } bcq_desc;
 
-/* How a product is decomposed over the GPU.  kernel: 0 = generic (one warp per row, any
- * valid shape, either layout is NOT implied: canonical only), 1 = lookup-table kernel
- * (tiled layout).  row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace. */
+/* How a product is decomposed over the GPU.  kernel: 0 = generic (one warp per row; any valid
+ * shape, either layout), 1 = lookup-table kernel (tiled layout, group 128) launched as
+ * row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace. */
 typedef struct bcq_plan {
     int32_t kernel;
     int32_t row_blocks;
@@ -90,7 +97,7 @@ typedef struct bcq_plan {
 } bcq_plan;
 
 /* ---- sizes (pure host functions; 0 when the descriptor is invalid) -------------------- */
-size_t bcq_packed_bytes(const bcq_desc *desc);   /* q * N * K / 8                          */
+size_t bcq_packed_bytes(const bcq_desc *desc);   /* q*N*K/8, plus 2*(q+1)*N*G when tiled with group 128 */
 size_t bcq_alpha_elems(const bcq_desc *desc);    /* q * N * G                              */
 size_t bcq_offset_elems(const bcq_desc *desc);   /* N * G                                  */
 
@@ -128,8 +135,10 @@ int bcq_merge_linear(const bcq_desc *desc, const uint8_t *w_int_dev, const uint1
 
 /*
  * Codes + canonical scales -> packed bit-planes and scales in desc->layout.
- * Bit-exact: only bit extraction and permutation.  alpha_in/z_in may be NULL together with
- * alpha_out/z_out to pack the planes only.  Outputs must not overlap inputs.
+ * Bit-exact: only bit extraction and permutation.  Canonical, or tiled with group 0:
+ * alpha_in/z_in may be NULL together with alpha_out/z_out to pack the planes only.  Tiled with
+ * group 128: alpha_in and z_in are required (they go into the tiles); alpha_out/z_out are
+ * ignored.  Outputs must not overlap inputs.
  */
 int bcq_pack(const bcq_desc *desc, const uint8_t *codes_dev, const uint16_t *alpha_in_dev,
              const uint16_t *z_in_dev, void *packed_out_dev, uint16_t *alpha_out_dev,
@@ -137,8 +146,11 @@ int bcq_pack(const bcq_desc *desc, const uint8_t *codes_dev, const uint16_t *alp
 
 /*
  * Re-lay-out packed operands from src->layout to dst->layout (N, K, q, group must agree).
- * Bit-exact permutation; canonical -> tiled -> canonical is the identity.  Any of the three
- * (src, dst) pointer pairs may be NULL to skip that operand.  No in-place operation.
+ * Bit-exact permutation; canonical -> tiled -> canonical is the identity.  The packed pointers
+ * are required.  Scales move when the source has them (inside its tiles, or alpha_src and z_src
+ * given) and the destination takes them (inside its tiles, or alpha_dst and z_dst given); a
+ * destination that keeps its scales in the tiles cannot be made without them.  Scale pointers of
+ * a side whose scales live in the tiles are ignored.  No in-place operation.
  */
 int bcq_repack(const bcq_desc *src, const void *packed_src_dev, const uint16_t *alpha_src_dev,
                const uint16_t *z_src_dev, const bcq_desc *dst, void *packed_dst_dev,
@@ -150,8 +162,8 @@ int bcq_repack(const bcq_desc *src, const void *packed_src_dev, const uint16_t *
  * y = W x at batch 1 (the definition at the top of this file; Eq. bcw + Eq. fuse_step3).
  * x [K], y [N] fp16.  y is overwritten.  workspace may be NULL when bcq_workspace_bytes is 0.
  * bcq_gemv_plan is the same product with an explicit decomposition (for tuning and tests):
- * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, and at most 64 row units
- * (512 rows) per row block.
+ * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 64 row units (512 rows)
+ * per row block and at most 7 windows (3584 weights along K) per K split.
  */
 int bcq_gemv(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
              const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev,

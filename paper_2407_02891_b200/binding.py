@@ -249,18 +249,31 @@ class Layer:
     """Device-resident operands of one packed layer (a convenience holder, no arithmetic)."""
     d: Desc
     packed: torch.Tensor
-    alpha: torch.Tensor
-    z: torch.Tensor
+    alpha: torch.Tensor | None
+    z: torch.Tensor | None
+
+
+def scales_in_tiles(d: Desc) -> bool:
+    """True when the layout keeps alpha and z inside `packed` (tiled, group 128)."""
+    return d.layout == LAYOUT_TILED and d.group != 0
+
+
+def empty_operands(d: Desc, device):
+    """Uninitialised torch tensors for (packed, alpha, z) of a descriptor; alpha/z are None when
+    the scales live inside `packed`."""
+    rc = check_desc(d)
+    if rc != OK:
+        raise BcqError(rc, "bcq_check_desc")
+    packed = torch.empty(packed_bytes(d), dtype=torch.uint8, device=device)
+    if scales_in_tiles(d):
+        return packed, None, None
+    return (packed, torch.empty(alpha_elems(d), dtype=torch.float16, device=device),
+            torch.empty(offset_elems(d), dtype=torch.float16, device=device))
 
 
 def pack_layer(N, K, q, group, layout, codes, alpha, z) -> Layer:
     """bcq_pack into freshly allocated torch tensors.  codes/alpha/z: canonical CUDA tensors."""
     d = desc(N, K, q, group, layout)
-    rc = check_desc(d)
-    if rc != OK:
-        raise BcqError(rc, "bcq_check_desc")
-    packed = torch.empty(packed_bytes(d), dtype=torch.uint8, device=codes.device)
-    a = torch.empty(alpha_elems(d), dtype=torch.float16, device=codes.device)
-    zz = torch.empty(offset_elems(d), dtype=torch.float16, device=codes.device)
+    packed, a, zz = empty_operands(d, codes.device)
     pack(d, codes, alpha, z, packed, a, zz)
     return Layer(d, packed, a, zz)

@@ -50,6 +50,9 @@ int device_sm_count(int *out)
 
 bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group == 128; }
 
+// tiled layout with grouped scales: alpha and z live inside `packed`
+bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group != 0; }
+
 // Instruction-count model of the lookup-table kernel (warp instructions on the critical warp
 // of a block); it ranks decompositions, it does not predict time.
 long long lut_cost(int U, int W, int rb, int ks, int sm)
@@ -105,7 +108,11 @@ size_t plan_workspace(const bcq_desc *d, const bcq_plan *p)
 int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, const uint16_t *alpha, const uint16_t *z,
              const uint16_t *x, uint16_t *y, void *ws, size_t ws_bytes, void *stream)
 {
-    if (!packed || !alpha || !z || !x || !y) return BCQ_ERR_INVALID_ARG;
+    if (!packed || !x || !y) return BCQ_ERR_INVALID_ARG;
+    if (interleaved(desc))
+        alpha = z = nullptr;
+    else if (!alpha || !z)
+        return BCQ_ERR_INVALID_ARG;
     if (!aligned(packed, 16) || !aligned(alpha, 16) || !aligned(z, 16) || !aligned(x, 16) || !aligned(y, 2))
         return BCQ_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -163,7 +170,10 @@ int bcq_check_desc(const bcq_desc *desc) { return check_desc(desc); }
 
 size_t bcq_packed_bytes(const bcq_desc *d)
 {
-    return check_desc(d) == BCQ_OK ? size_t(d->q) * d->N * (d->K / 8) : 0;
+    if (check_desc(d) != BCQ_OK) return 0;
+    size_t bytes = size_t(d->q) * d->N * (d->K / 8);
+    if (interleaved(d)) bytes += (size_t(d->q) + 1) * d->N * n_groups(*d) * sizeof(uint16_t);
+    return bytes;
 }
 size_t bcq_alpha_elems(const bcq_desc *d) { return check_desc(d) == BCQ_OK ? size_t(d->q) * d->N * n_groups(*d) : 0; }
 size_t bcq_offset_elems(const bcq_desc *d) { return check_desc(d) == BCQ_OK ? size_t(d->N) * n_groups(*d) : 0; }
@@ -256,17 +266,25 @@ int bcq_pack(const bcq_desc *desc, const uint8_t *codes, const uint16_t *alpha_i
     int rc = check_desc(desc);
     if (rc != BCQ_OK) return rc;
     if (!codes || !packed) return BCQ_ERR_INVALID_ARG;
-    const bool scales = alpha_in || z_in || alpha_out || z_out;
-    if (scales && !(alpha_in && z_in && alpha_out && z_out)) return BCQ_ERR_INVALID_ARG;
+    bool scales;
+    if (interleaved(desc)) {
+        if (!alpha_in || !z_in) return BCQ_ERR_INVALID_ARG;  // the tiles carry the scales
+        alpha_out = z_out = nullptr;
+        scales = true;
+    } else {
+        scales = alpha_in || z_in || alpha_out || z_out;
+        if (scales && !(alpha_in && z_in && alpha_out && z_out)) return BCQ_ERR_INVALID_ARG;
+    }
     if (!aligned(codes, 16) || !aligned(packed, 16) || !aligned(alpha_in, 2) || !aligned(z_in, 2) ||
         !aligned(alpha_out, 2) || !aligned(z_out, 2))
         return BCQ_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_pack(*desc, codes, packed, st);
+    const View dst = make_view(*desc, packed, alpha_out, z_out);
+    cudaError_t e = launch_pack(codes, dst, st);
     if (e == cudaSuccess && scales) {
-        bcq_desc src = *desc;
-        src.layout = BCQ_LAYOUT_CANONICAL;
-        e = launch_permute_scales(src, alpha_in, z_in, *desc, alpha_out, z_out, st);
+        bcq_desc canon = *desc;
+        canon.layout = BCQ_LAYOUT_CANONICAL;
+        e = launch_permute_scales(make_view(canon, nullptr, alpha_in, z_in), dst, st);
     }
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
@@ -279,19 +297,21 @@ int bcq_repack(const bcq_desc *src, const void *packed_src, const uint16_t *alph
     rc = check_desc(dst);
     if (rc != BCQ_OK) return rc;
     if (!same_problem(src, dst)) return BCQ_ERR_INVALID_ARG;
-    if ((packed_src == nullptr) != (packed_dst == nullptr) || (alpha_src == nullptr) != (alpha_dst == nullptr) ||
-        (z_src == nullptr) != (z_dst == nullptr))
-        return BCQ_ERR_INVALID_ARG;
-    if ((packed_src && packed_src == packed_dst) || (alpha_src && alpha_src == alpha_dst) || (z_src && z_src == z_dst))
-        return BCQ_ERR_INVALID_ARG;
+    if (!packed_src || !packed_dst || packed_src == packed_dst) return BCQ_ERR_INVALID_ARG;
+    if (interleaved(src)) alpha_src = z_src = nullptr;
+    if (interleaved(dst)) alpha_dst = z_dst = nullptr;
+    if ((alpha_src == nullptr) != (z_src == nullptr) || (alpha_dst == nullptr) != (z_dst == nullptr)) return BCQ_ERR_INVALID_ARG;
+    const bool have_scales = interleaved(src) || alpha_src;
+    const bool want_scales = interleaved(dst) || alpha_dst;
+    if (interleaved(dst) && !have_scales) return BCQ_ERR_INVALID_ARG;  // a tiled operand cannot exist without its scales
+    if ((alpha_src && alpha_src == alpha_dst) || (z_src && z_src == z_dst)) return BCQ_ERR_INVALID_ARG;
     if (!aligned(packed_src, 16) || !aligned(packed_dst, 16) || !aligned(alpha_src, 2) || !aligned(alpha_dst, 2) ||
         !aligned(z_src, 2) || !aligned(z_dst, 2))
         return BCQ_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaSuccess;
-    if (packed_src) e = launch_permute_planes(*src, packed_src, *dst, packed_dst, st);
-    if (e == cudaSuccess && (alpha_src || z_src))
-        e = launch_permute_scales(*src, alpha_src, z_src, *dst, alpha_dst, z_dst, st);
+    const View vs = make_view(*src, packed_src, alpha_src, z_src), vd = make_view(*dst, packed_dst, alpha_dst, z_dst);
+    cudaError_t e = launch_permute_planes(vs, vd, st);
+    if (e == cudaSuccess && have_scales && want_scales) e = launch_permute_scales(vs, vd, st);
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
 
@@ -322,7 +342,11 @@ int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed, const uint16_t
     if (rc != BCQ_OK) return rc;
     if (B < 1 || B > 16) return BCQ_ERR_INVALID_ARG;
     if (B == 1) return bcq_gemv(desc, packed, alpha, z, X, Y, ws, ws_bytes, stream);
-    if (!packed || !alpha || !z || !X || !Y) return BCQ_ERR_INVALID_ARG;
+    if (!packed || !X || !Y) return BCQ_ERR_INVALID_ARG;
+    if (interleaved(desc))
+        alpha = z = nullptr;
+    else if (!alpha || !z)
+        return BCQ_ERR_INVALID_ARG;
     if (!aligned(packed, 16) || !aligned(alpha, 16) || !aligned(z, 16) || !aligned(X, 16) || !aligned(Y, 2))
         return BCQ_ERR_MISALIGNED;
     cudaError_t e = launch_generic(*desc, packed, alpha, z, X, Y, B, static_cast<cudaStream_t>(stream));

@@ -10,16 +10,12 @@ namespace bcq {
 // =============================================================================================
 
 template <int BMAX>
-__global__ void __launch_bounds__(256) generic_kernel(const uint8_t *__restrict__ packed,
-                                                       const __half *__restrict__ alpha,
-                                                       const __half *__restrict__ z, const __half *__restrict__ X,
-                                                       __half *__restrict__ Y, int N, int K, int q, int group,
-                                                       int layout, int B)
+__global__ void __launch_bounds__(256) generic_kernel(const View v, const __half *__restrict__ X, __half *__restrict__ Y, int B)
 {
+    const int N = v.N, K = v.K, q = v.q, group = v.group;
     const int lane = threadIdx.x & 31;
     const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (n >= N) return;
-    const int G = group == 0 ? 1 : K / group;
     const int L = group == 0 ? K : group;
     float acc[BMAX];
 #pragma unroll
@@ -27,12 +23,12 @@ __global__ void __launch_bounds__(256) generic_kernel(const uint8_t *__restrict_
 
     for (int kb = lane; kb < K / 8; kb += 32) {
         const int g = (kb * 8) / L;
-        const float zz = __half2float(z[offset_elem_offset(layout, N, G, group, n, g)]);
+        const float zz = __half2float(*reinterpret_cast<const __half *>(v.z_elem(n, g)));
         float a[4];
         uint32_t bits[4];
         for (int i = 0; i < q; ++i) {
-            a[i] = __half2float(alpha[alpha_elem_offset(layout, N, G, q, group, i, n, g)]);
-            bits[i] = packed[plane_byte_offset(layout, N, K, q, i, n, kb)];
+            a[i] = __half2float(*reinterpret_cast<const __half *>(v.alpha_elem(i, n, g)));
+            bits[i] = *v.plane_byte(i, n, kb);
         }
 #pragma unroll
         for (int b = 0; b < BMAX; ++b) {
@@ -65,17 +61,15 @@ cudaError_t launch_generic(const bcq_desc &d, const void *packed, const uint16_t
 {
     const int warps = 8;
     dim3 grid((d.N + warps - 1) / warps), block(32 * warps);
-    auto p = static_cast<const uint8_t *>(packed);
-    auto a = reinterpret_cast<const __half *>(alpha);
-    auto zz = reinterpret_cast<const __half *>(z);
+    const View v = make_view(d, packed, alpha, z);
     auto x = reinterpret_cast<const __half *>(X);
     auto y = reinterpret_cast<__half *>(Y);
     if (B == 1)
-        generic_kernel<1><<<grid, block, 0, st>>>(p, a, zz, x, y, d.N, d.K, d.q, d.group, d.layout, B);
+        generic_kernel<1><<<grid, block, 0, st>>>(v, x, y, B);
     else if (B <= 4)
-        generic_kernel<4><<<grid, block, 0, st>>>(p, a, zz, x, y, d.N, d.K, d.q, d.group, d.layout, B);
+        generic_kernel<4><<<grid, block, 0, st>>>(v, x, y, B);
     else
-        generic_kernel<16><<<grid, block, 0, st>>>(p, a, zz, x, y, d.N, d.K, d.q, d.group, d.layout, B);
+        generic_kernel<16><<<grid, block, 0, st>>>(v, x, y, B);
     return cudaGetLastError();
 }
 

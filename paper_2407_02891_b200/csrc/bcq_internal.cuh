@@ -16,46 +16,68 @@ constexpr int kGroupsPerWindow = 4; // 128-weight groups in a window
 constexpr int kLutWarps = 16;       // warps per block of the lookup-table kernel
 constexpr int kLutUnitsPerWarp = 4; // row units a warp keeps accumulators for
 constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
-constexpr int kMaxWindowsPerBlock = 14; // windows of x a block keeps in shared memory
+constexpr int kMaxWindowsPerBlock = 7;  // windows of x a block keeps in shared memory
 constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace
 constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);
 
 inline int n_groups(const bcq_desc &d) { return d.group == 0 ? 1 : d.K / d.group; }
 
-// ---- layout index arithmetic (host and device) ------------------------------------------
+// ---- where the operands of one layer live (host and device) ---------------------------------
+//
+// Canonical: packed[i][n][k/8], alpha[i][n][g], z[n][g] in three arrays.
+// Tiled: tile (w, u) of `packed` covers window w (512 weights) of row unit u (8 rows):
+//   q*512 bytes of planes as [j < q][lane < 32][16 B], byte p = (r*q + i)*2 + s of a lane's 16q
+//   bytes = row 8u + r, plane i, chunk 2*lane + s;
+//   group 128 only: followed, in the same tile, by alpha [gi < 4][i < q][r < 8] and z [gi < 4][r < 8]
+//   (fp16) -- the tile is one contiguous piece of memory, fetched by one bulk copy;
+//   group 0 (per row): alpha [u][i][r] and z [u][r] stay in their own arrays.
+struct View {
+    int layout, N, K, q, group;
+    unsigned char *packed;
+    uint16_t *alpha;
+    uint16_t *z;
 
-// Byte offset of the byte holding weights k = 8*kb .. 8*kb+7 of (plane i, row n).
-__host__ __device__ inline size_t plane_byte_offset(int layout, int N, int K, int q, int i, int n, int kb)
-{
-    if (layout == BCQ_LAYOUT_CANONICAL) return (size_t(i) * N + n) * size_t(K / 8) + kb;
-    const int U = N / kUnitRows;
-    const int w = kb / (kWindow / 8), c = kb % (kWindow / 8);
-    const int lane = c >> 1, s = c & 1;
-    const int u = n / kUnitRows, r = n % kUnitRows;
-    const int p = (r * q + i) * 2 + s;
-    return ((size_t(w) * U + u) * q + (p >> 4)) * 512 + size_t(lane) * 16 + (p & 15);
-}
+    __host__ __device__ int G() const { return group == 0 ? 1 : K / group; }
+    __host__ __device__ bool interleaved() const { return layout == BCQ_LAYOUT_TILED && group != 0; }
+    __host__ __device__ size_t tile_bytes() const { return size_t(q) * 512 + (interleaved() ? size_t(q) * 64 + 64 : 0); }
+    __host__ __device__ size_t tile_base(int w, int u) const { return (size_t(w) * (N / kUnitRows) + u) * tile_bytes(); }
 
-// Element offset of alpha[i][n][g].
-__host__ __device__ inline size_t alpha_elem_offset(int layout, int N, int G, int q, int group, int i, int n, int g)
-{
-    if (layout == BCQ_LAYOUT_CANONICAL) return (size_t(i) * N + n) * G + g;
-    const int U = N / kUnitRows;
-    const int u = n / kUnitRows, r = n % kUnitRows;
-    if (group == 0) return (size_t(u) * q + i) * kUnitRows + r;
-    const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
-    return (((size_t(w) * U + u) * kGroupsPerWindow + gi) * q + i) * kUnitRows + r;
-}
+    // the byte holding weights k = 8*kb .. 8*kb+7 of (plane i, row n)
+    __host__ __device__ unsigned char *plane_byte(int i, int n, int kb) const
+    {
+        if (layout == BCQ_LAYOUT_CANONICAL) return packed + (size_t(i) * N + n) * size_t(K / 8) + kb;
+        const int w = kb / (kWindow / 8), c = kb % (kWindow / 8);
+        const int lane = c >> 1, s = c & 1;
+        const int u = n / kUnitRows, r = n % kUnitRows;
+        const int p = (r * q + i) * 2 + s;
+        return packed + tile_base(w, u) + size_t(p >> 4) * 512 + size_t(lane) * 16 + (p & 15);
+    }
+    __host__ __device__ uint16_t *alpha_elem(int i, int n, int g) const
+    {
+        if (layout == BCQ_LAYOUT_CANONICAL) return alpha + (size_t(i) * N + n) * G() + g;
+        const int u = n / kUnitRows, r = n % kUnitRows;
+        if (group == 0) return alpha + (size_t(u) * q + i) * kUnitRows + r;
+        const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
+        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + (gi * q + i) * kUnitRows + r;
+    }
+    __host__ __device__ uint16_t *z_elem(int n, int g) const
+    {
+        if (layout == BCQ_LAYOUT_CANONICAL) return z + size_t(n) * G() + g;
+        const int u = n / kUnitRows, r = n % kUnitRows;
+        if (group == 0) return z + size_t(u) * kUnitRows + r;
+        const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
+        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 576) + gi * kUnitRows + r;
+    }
+};
 
-// Element offset of z[n][g].
-__host__ __device__ inline size_t offset_elem_offset(int layout, int N, int G, int group, int n, int g)
+inline View make_view(const bcq_desc &d, const void *packed, const uint16_t *alpha, const uint16_t *z)
 {
-    if (layout == BCQ_LAYOUT_CANONICAL) return size_t(n) * G + g;
-    const int U = N / kUnitRows;
-    const int u = n / kUnitRows, r = n % kUnitRows;
-    if (group == 0) return size_t(u) * kUnitRows + r;
-    const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
-    return ((size_t(w) * U + u) * kGroupsPerWindow + gi) * kUnitRows + r;
+    View v;
+    v.layout = d.layout, v.N = d.N, v.K = d.K, v.q = d.q, v.group = d.group;
+    v.packed = static_cast<unsigned char *>(const_cast<void *>(packed));
+    v.alpha = const_cast<uint16_t *>(alpha);
+    v.z = const_cast<uint16_t *>(z);
+    return v;
 }
 
 // ---- launchers (each returns the cudaError_t of its launch) ------------------------------
@@ -63,10 +85,9 @@ __host__ __device__ inline size_t offset_elem_offset(int layout, int N, int G, i
 cudaError_t launch_merge(const bcq_desc &d, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias,
                          int n_bits, const uint8_t *code_of_int /*[256]*/, const double *plane_weight /*[q]*/,
                          uint8_t *codes, uint16_t *alpha, uint16_t *z, cudaStream_t st);
-cudaError_t launch_pack(const bcq_desc &d, const uint8_t *codes, void *packed, cudaStream_t st);
-cudaError_t launch_permute_planes(const bcq_desc &src, const void *in, const bcq_desc &dst, void *out, cudaStream_t st);
-cudaError_t launch_permute_scales(const bcq_desc &src, const uint16_t *alpha_in, const uint16_t *z_in,
-                                  const bcq_desc &dst, uint16_t *alpha_out, uint16_t *z_out, cudaStream_t st);
+cudaError_t launch_pack(const uint8_t *codes, const View &dst, cudaStream_t st);
+cudaError_t launch_permute_planes(const View &src, const View &dst, cudaStream_t st);
+cudaError_t launch_permute_scales(const View &src, const View &dst, cudaStream_t st);
 
 cudaError_t launch_generic(const bcq_desc &d, const void *packed, const uint16_t *alpha, const uint16_t *z,
                            const uint16_t *X, uint16_t *Y, int B, cudaStream_t st);

@@ -10,7 +10,7 @@
 //                           one window ahead of the consumers (two 64 KB tables, double buffered);
 //   producer  (warp 3)      one thread feeds a ring of shared-memory slots with bulk async copies
 //                           (cp.async.bulk, completion on an mbarrier): per (window, row unit) one
-//                           slot = q*512 B of plane bytes + the unit's alphas and offsets;
+//                           slot = one tile = q*512 B of plane bytes + the unit's alphas and offsets;
 //   consumers (warps 4-19)  copy a filled slot into registers, hand the slot back, look every
 //                           weight byte up in the window table and accumulate in fp32.
 //
@@ -43,11 +43,28 @@ constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
 constexpr int kXBytes = kMaxWindowsPerBlock * kWindow * 4;
 constexpr int kBarrierBytes = 1024;
 constexpr int kFixedBytes = kXBytes + kBarrierBytes;
-constexpr int kSpinLimit = 1 << 20;   // tries per wait (each try blocks for a short, hardware-defined time)
+constexpr int kProducerIdleLimit = 1 << 24;   // polling rounds without progress before the producer gives up
+constexpr int kSpinLimit = 1 << 24;   // tries per wait (each try blocks for a short, hardware-defined time)
 
 static_assert(2 * kFixedBytes <= kLutSmemBytes - 2 * kTableBytes, "x + barriers must fit before or after the tables");
 
 __device__ int g_lut_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
+
+#ifdef BCQ_TRACE
+// Development aid (not compiled into the product): per-block event times in ns.
+__device__ unsigned long long g_trace[1024][16];
+__device__ __forceinline__ unsigned long long gtime()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define TRACE(slot) do { if (blockIdx.x < 1024) g_trace[blockIdx.x][slot] = gtime(); } while (0)
+#define TRACE_ADD(slot, v) do { if (blockIdx.x < 1024) g_trace[blockIdx.x][slot] += (v); } while (0)
+#else
+#define TRACE(slot) do { } while (0)
+#define TRACE_ADD(slot, v) do { } while (0)
+#endif
 
 template <int Q>
 struct Slot {
@@ -58,9 +75,7 @@ struct Slot {
 };
 
 struct LutParams {
-    const uint8_t *planes;
-    const uint8_t *alpha;  // tiled
-    const uint8_t *z;      // tiled
+    const uint8_t *tiles;  // tiled operand: per (window, unit) planes, alphas, offsets
     const __half *x;
     __half *y;
     float *partial;  // [k_splits][N] when k_splits > 1
@@ -105,12 +120,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)   // never blocks
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false if the block is aborting (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code)
 {
     for (int it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63) == 63 && *abort_flag) return false;
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((it & 1023) == 1023 && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicExch(&g_lut_status, code);
@@ -254,6 +281,10 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     int *s_last = const_cast<int *>(abort_flag) + 1;
 
     if (tid == 0) {
+        TRACE(0);
+#ifdef BCQ_TRACE
+        g_trace[blockIdx.x % 1024][13] = 0; g_trace[blockIdx.x % 1024][14] = 0;
+#endif
         for (int s = 0; s < kMaxSlots; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
@@ -268,15 +299,28 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    if (tid == 0) TRACE(1);
 
     // =============================================================================================
-    if (warp < kBuilderWarps) {
-        // ---- builders: x slice fp16 -> fp32 (permuted for the build), then one table per window ----
+    if (warp != kProducerWarp) {
+        // ---- start-up, all warps but the producer: x slice fp16 -> fp32 (permuted for the build)
+        //      and the first window's table ----------------------------------------------------------
+        constexpr int kStartThreads = kLutThreads - 32;
+        const int sid = warp < kProducerWarp ? tid : tid - 32;
         const __half *xg = p.x + size_t(w0) * kWindow;
-        for (int e = tid; e < nwin * kWindow; e += kBuilderThreads)
+        for (int e = sid; e < nwin * kWindow; e += kStartThreads)
             xs[(e & ~(kWindow - 1)) + xs_index(e & (kWindow - 1))] = __half2float(xg[e]);
-        named_barrier(1, kBuilderThreads);
-        for (int wi = 0; wi < nwin; ++wi) {
+        named_barrier(1, kStartThreads);
+        if (sid == 0) TRACE(2);
+        if (sid < 512) build_item(tables, xs, sid);
+        named_barrier(1, kStartThreads);
+        if (sid == 0) TRACE(3);
+    }
+
+    if (warp < kBuilderWarps) {
+        // ---- builders: one table per window, one window ahead of the consumers ----------------------
+        mbar_arrive(bar_tab_ready);   // window 0 was built by everybody above
+        for (int wi = 1; wi < nwin; ++wi) {
             const int b = wi & 1, use = wi >> 1;
             if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree)) break;
             unsigned char *table = tables + b * kTableBytes;
@@ -294,32 +338,50 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         if (lane < kLutWarps && !*abort_flag) {
             const int c = lane;
             const int mine = (V - c + kLutWarps - 1) / kLutWarps;  // units of warp c per window
+            int remaining = mine * nwin, t_in_win = 0, wi = 0, idle = 0;
+            size_t tile = size_t(w0) * p.U + u0 + c;
             int d = 0, k = 0, last_s = -1, last_par = 0, prev_s = -1, prev_par = 0, pprev_s = -1, pprev_par = 0;
-            bool ok = true;
-            for (int wi = 0; wi < nwin && ok; ++wi) {
-                size_t tile = size_t(w0 + wi) * p.U + u0 + c;
-                for (int t = 0; t < mine; ++t, tile += kLutWarps) {
+            // The 16 lanes stay together in one polling loop and never block on a barrier, so
+            // each refills its warp's slot as soon as that slot is handed back.
+            while (true) {
+                bool issued = false;
+                if (remaining > 0) {
                     const int s = c + kLutWarps * d;
-                    if (k > 0 && !mbar_wait(bar_empty + 8 * s, (k - 1) & 1, abort_flag, kWaitEmpty)) {
-                        ok = false;
-                        break;
+                    if (k == 0 || mbar_test_wait(bar_empty + 8 * s, (k - 1) & 1)) {
+                        const uint32_t dst = smem_u32(slot_ptr(s)), full = bar_full + 8 * s;
+                        mbar_expect_tx(full, SL::kBytes);
+                        bulk_g2s(dst, p.tiles + tile * SL::kBytes, SL::kBytes, full);   // planes + alphas + offsets
+                        pprev_s = prev_s, pprev_par = prev_par, prev_s = last_s, prev_par = last_par;
+                        last_s = s, last_par = k & 1;
+                        if (++d == D) {
+                            d = 0;
+                            ++k;
+                        }
+                        tile += kLutWarps;
+                        if (++t_in_win == mine) {
+                            t_in_win = 0;
+                            ++wi;
+                            tile = size_t(w0 + wi) * p.U + u0 + c;
+                        }
+                        --remaining;
+                        issued = true;
                     }
-                    const uint32_t dst = smem_u32(slot_ptr(s)), full = bar_full + 8 * s;
-                    mbar_expect_tx(full, SL::kBytes);
-                    bulk_g2s(dst, p.planes + tile * SL::kPlaneBytes, SL::kPlaneBytes, full);
-                    bulk_g2s(dst + SL::kPlaneBytes, p.alpha + tile * SL::kAlphaBytes, SL::kAlphaBytes, full);
-                    bulk_g2s(dst + SL::kPlaneBytes + SL::kAlphaBytes, p.z + tile * SL::kOffsetBytes, SL::kOffsetBytes, full);
-                    pprev_s = prev_s, pprev_par = prev_par, prev_s = last_s, prev_par = last_par;
-                    last_s = s, last_par = k & 1;
-                    if (++d == D) {
-                        d = 0;
-                        ++k;
+                }
+                if (__ballot_sync(0xFFFFu, remaining > 0) == 0) break;
+                if (__any_sync(0xFFFFu, issued)) {
+                    idle = 0;
+                } else if (++idle > kProducerIdleLimit || *abort_flag) {
+                    if (idle > kProducerIdleLimit) {
+                        *abort_flag = 1;
+                        atomicExch(&g_lut_status, int(kWaitEmpty));
                     }
+                    break;
                 }
             }
             // See the last fill of each of this lane's (at most 3) slots land, with a bounded wait,
             // before the warp leaves: the block's shared memory must not be handed to another block
             // while copies into it are in flight, also when the consumers gave up.
+            if (lane == 0) TRACE(12);
             const int ss[3] = {last_s, prev_s, pprev_s}, pp[3] = {last_par, prev_par, pprev_par};
 #pragma unroll
             for (int q3 = 0; q3 < 3; ++q3) {
@@ -353,6 +415,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             alive = false;
             break;
         }
+        if (ctid == 0 && wi == 0) TRACE(4);
         const uint32_t lane_off = tab0 + uint32_t(b * kTableBytes + lane * 4);
         // sum of this lane's 16 activations (the all-ones entries of its two chunks), then of its group
         float xsum = lds_f32<255 * 256>(lane_off) + lds_f32<255 * 256 + 128>(lane_off);
@@ -364,7 +427,14 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             constexpr int t = decltype(T)::value;
             if (alive && cw + kLutWarps * t < V) {
                 const int s = cw + kLutWarps * d;
-                if (!mbar_wait(bar_full + 8 * s, k & 1, abort_flag, kWaitFull)) {
+#ifdef BCQ_TRACE
+                const unsigned long long tw0 = gtime();
+#endif
+                const bool got = mbar_wait(bar_full + 8 * s, k & 1, abort_flag, kWaitFull);
+#ifdef BCQ_TRACE
+                if (ctid == 0) { TRACE_ADD(13, gtime() - tw0); TRACE_ADD(14, 1); if (wi == 0 && t == 0) TRACE(5); }
+#endif
+                if (!got) {
                     alive = false;
                 } else {
                     // slot -> registers, then hand the slot back to the producer
@@ -415,6 +485,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         });
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tab_free + 8 * b);
+        if (ctid == 0 && wi < 4) TRACE(6 + wi);
     }
 
     // ---- reduce each unit's 8 row sums over the 32 lanes: lane l ends with row l & 7 -------------
@@ -451,6 +522,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         }
     });
 
+    if (ctid == 0) TRACE(10);
     // ---- split-K: the last block to arrive for this row block adds the partials in fixed order --
     if (p.k_splits > 1) {
         __threadfence();
@@ -470,6 +542,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             if (ctid == 0) p.counters[rbi] = 0;
         }
     }
+    if (ctid == 0) TRACE(11);
 }
 
 template <int Q>
@@ -494,9 +567,9 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
                             const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st)
 {
     LutParams prm;
-    prm.planes = static_cast<const uint8_t *>(packed);
-    prm.alpha = reinterpret_cast<const uint8_t *>(alpha);
-    prm.z = reinterpret_cast<const uint8_t *>(z);
+    prm.tiles = static_cast<const uint8_t *>(packed);
+    (void)alpha;
+    (void)z;
     prm.x = reinterpret_cast<const __half *>(x);
     prm.y = reinterpret_cast<__half *>(y);
     prm.counters = static_cast<int *>(workspace);
@@ -515,6 +588,13 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
     }
     return cudaErrorInvalidValue;
 }
+
+#ifdef BCQ_TRACE
+extern "C" int bcq_debug_read_trace(unsigned long long *host, int blocks)
+{
+    return int(cudaMemcpyFromSymbol(host, g_trace, size_t(blocks) * 16 * sizeof(unsigned long long)));
+}
+#endif
 
 // Read and clear the device status word (synchronises with the device).
 cudaError_t lut_status_take(int *status)

@@ -58,77 +58,66 @@ cudaError_t launch_merge(const bcq_desc &d, const uint8_t *w_int, const uint16_t
 
 // ---- pack: one thread per (row, 8-weight chunk) ---------------------------------------------
 
-__global__ void pack_kernel(const uint8_t *__restrict__ codes, uint8_t *__restrict__ packed, int N, int K, int q,
-                            int layout)
+__global__ void pack_kernel(const uint8_t *__restrict__ codes, const View dst)
 {
-    const int kbytes = K / 8;
+    const int kbytes = dst.K / 8;
     size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (t >= size_t(N) * kbytes) return;
+    if (t >= size_t(dst.N) * kbytes) return;
     const int n = int(t / kbytes), kb = int(t % kbytes);
-    const uint2 c8 = *reinterpret_cast<const uint2 *>(codes + size_t(n) * K + size_t(kb) * 8);
+    const uint2 c8 = *reinterpret_cast<const uint2 *>(codes + size_t(n) * dst.K + size_t(kb) * 8);
     const uint32_t lo = c8.x, hi = c8.y;
-    for (int i = 0; i < q; ++i) {
+    for (int i = 0; i < dst.q; ++i) {
         uint32_t byte = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             byte |= ((lo >> (8 * j + i)) & 1u) << j;
             byte |= ((hi >> (8 * j + i)) & 1u) << (4 + j);
         }
-        packed[plane_byte_offset(layout, N, K, q, i, n, kb)] = uint8_t(byte);
+        *dst.plane_byte(i, n, kb) = uint8_t(byte);
     }
 }
 
-cudaError_t launch_pack(const bcq_desc &d, const uint8_t *codes, void *packed, cudaStream_t st)
+cudaError_t launch_pack(const uint8_t *codes, const View &dst, cudaStream_t st)
 {
-    size_t count = size_t(d.N) * (d.K / 8);
-    pack_kernel<<<unsigned((count + 255) / 256), 256, 0, st>>>(codes, static_cast<uint8_t *>(packed), d.N, d.K, d.q,
-                                                              d.layout);
+    size_t count = size_t(dst.N) * (dst.K / 8);
+    pack_kernel<<<unsigned((count + 255) / 256), 256, 0, st>>>(codes, dst);
     return cudaGetLastError();
 }
 
 // ---- permutations between layouts -----------------------------------------------------------
 
-__global__ void permute_planes_kernel(const uint8_t *__restrict__ in, uint8_t *__restrict__ out, int N, int K, int q,
-                                      int src_layout, int dst_layout)
+__global__ void permute_planes_kernel(const View src, const View dst)
 {
-    const int kbytes = K / 8;
+    const int kbytes = src.K / 8;
     size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (t >= size_t(q) * N * kbytes) return;
+    if (t >= size_t(src.q) * src.N * kbytes) return;
     const int kb = int(t % kbytes);
-    const int n = int((t / kbytes) % N);
-    const int i = int(t / (size_t(kbytes) * N));
-    out[plane_byte_offset(dst_layout, N, K, q, i, n, kb)] = in[plane_byte_offset(src_layout, N, K, q, i, n, kb)];
+    const int n = int((t / kbytes) % src.N);
+    const int i = int(t / (size_t(kbytes) * src.N));
+    *dst.plane_byte(i, n, kb) = *src.plane_byte(i, n, kb);
 }
 
-__global__ void permute_scales_kernel(const uint16_t *__restrict__ alpha_in, const uint16_t *__restrict__ z_in,
-                                      uint16_t *__restrict__ alpha_out, uint16_t *__restrict__ z_out, int N, int G,
-                                      int q, int group, int src_layout, int dst_layout)
+__global__ void permute_scales_kernel(const View src, const View dst)
 {
+    const int G = src.G();
     size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (t >= size_t(N) * G) return;
+    if (t >= size_t(src.N) * G) return;
     const int n = int(t / G), g = int(t % G);
-    if (alpha_in)
-        for (int i = 0; i < q; ++i)
-            alpha_out[alpha_elem_offset(dst_layout, N, G, q, group, i, n, g)] =
-                alpha_in[alpha_elem_offset(src_layout, N, G, q, group, i, n, g)];
-    if (z_in) z_out[offset_elem_offset(dst_layout, N, G, group, n, g)] = z_in[offset_elem_offset(src_layout, N, G, group, n, g)];
+    for (int i = 0; i < src.q; ++i) *dst.alpha_elem(i, n, g) = *src.alpha_elem(i, n, g);
+    *dst.z_elem(n, g) = *src.z_elem(n, g);
 }
 
-cudaError_t launch_permute_planes(const bcq_desc &src, const void *in, const bcq_desc &dst, void *out, cudaStream_t st)
+cudaError_t launch_permute_planes(const View &src, const View &dst, cudaStream_t st)
 {
     size_t count = size_t(src.q) * src.N * (src.K / 8);
-    permute_planes_kernel<<<unsigned((count + 255) / 256), 256, 0, st>>>(
-        static_cast<const uint8_t *>(in), static_cast<uint8_t *>(out), src.N, src.K, src.q, src.layout, dst.layout);
+    permute_planes_kernel<<<unsigned((count + 255) / 256), 256, 0, st>>>(src, dst);
     return cudaGetLastError();
 }
 
-cudaError_t launch_permute_scales(const bcq_desc &src, const uint16_t *alpha_in, const uint16_t *z_in,
-                                  const bcq_desc &dst, uint16_t *alpha_out, uint16_t *z_out, cudaStream_t st)
+cudaError_t launch_permute_scales(const View &src, const View &dst, cudaStream_t st)
 {
-    size_t count = size_t(src.N) * n_groups(src);
-    permute_scales_kernel<<<unsigned((count + 255) / 256), 256, 0, st>>>(alpha_in, z_in, alpha_out, z_out, src.N,
-                                                                        n_groups(src), src.q, src.group, src.layout,
-                                                                        dst.layout);
+    size_t count = size_t(src.N) * src.G();
+    permute_scales_kernel<<<unsigned((count + 255) / 256), 256, 0, st>>>(src, dst);
     return cudaGetLastError();
 }
 

@@ -15,39 +15,39 @@ def make_layer(name, N, K, q, group, B=1):
     return p, synth.codes_from_planes(p), alpha, z, x
 
 
-def tiled_planes(planes):
-    """canonical uint8 [q,N,K/8] -> tiled byte stream, per the layout comment of include/bcq.h."""
+def tiled_operands(planes, alpha, z, group):
+    """canonical planes uint8 [q,N,K/8], alpha f16 [q,N,G], z f16 [N,G] -> (packed bytes, alpha, z) of
+    the tiled layout, per the layout comment of include/bcq.h.  alpha and z come back as None when
+    the scales live inside the tiles (group 128)."""
     q, N, KB = planes.shape
     U, W = N // 8, KB // 64
-    out = np.empty(q * N * KB, np.uint8)
+    T = q * 512 + (q * 64 + 64 if group else 0)
+    out = np.zeros(U * W * T, np.uint8)
     i, n, kb = np.meshgrid(np.arange(q), np.arange(N), np.arange(KB), indexing="ij")
     w, c = kb // 64, kb % 64
     lane, s = c // 2, c % 2
     u, r = n // 8, n % 8
     p = (r * q + i) * 2 + s
-    off = ((w * U + u) * q + p // 16) * 512 + lane * 16 + p % 16
+    off = (w * U + u) * T + (p // 16) * 512 + lane * 16 + p % 16
     out[off.ravel()] = planes.ravel()
-    return out
-
-
-def tiled_scales(alpha, z, group):
-    """canonical alpha [q,N,G], z [N,G] -> tiled element streams."""
-    q, N, G = alpha.shape
-    U = N // 8
+    G = alpha.shape[2]
     i, n, g = np.meshgrid(np.arange(q), np.arange(N), np.arange(G), indexing="ij")
     u, r = n // 8, n % 8
     if group == 0:
-        a_off = (u * q + i) * 8 + r
-        z_off = (u[0] * 8 + r[0])
-    else:
-        w, gi = g // 4, g % 4
-        a_off = (((w * U + u) * 4 + gi) * q + i) * 8 + r
-        z_off = ((w[0] * U + u[0]) * 4 + gi[0]) * 8 + r[0]
-    a_out = np.empty(alpha.size, alpha.dtype)
-    z_out = np.empty(z.size, z.dtype)
-    a_out[a_off.ravel()] = alpha.ravel()
-    z_out[z_off.ravel()] = z.ravel()
-    return a_out, z_out
+        a_out = np.empty(alpha.size, alpha.dtype)
+        z_out = np.empty(z.size, z.dtype)
+        a_out[((u * q + i) * 8 + r).ravel()] = alpha.ravel()
+        z_out[(u[0] * 8 + r[0]).ravel()] = z.ravel()
+        return out, a_out, z_out
+    w, gi = g // 4, g % 4
+    a_off = (w * U + u) * T + q * 512 + 2 * ((gi * q + i) * 8 + r)
+    z_off = (w[0] * U + u[0]) * T + q * 576 + 2 * (gi[0] * 8 + r[0])
+    ab = alpha.view(np.uint8).reshape(q, N, G, 2)
+    zb = z.view(np.uint8).reshape(N, G, 2)
+    for byte in range(2):
+        out[(a_off + byte).ravel()] = ab[..., byte].ravel()
+        out[(z_off + byte).ravel()] = zb[..., byte].ravel()
+    return out, None, None
 
 
 def rel_err(y_gpu, y_ref):

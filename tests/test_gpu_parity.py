@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import TOL, make_layer, rel_err, tiled_planes, tiled_scales
+from helpers import TOL, make_layer, rel_err, tiled_operands
 from paper_2407_02891_b200 import binding as bq
 from paper_2407_02891_b200 import synth
 
@@ -54,18 +54,24 @@ def test_pack_canonical_bit_exact(N, K, q, group):
 def test_pack_tiled_and_repack_bit_exact(N, K, q, group):
     p, codes, alpha, z, _ = make_layer(f"tile/{N}x{K}", N, K, q, group)
     canon = oracle.pack_canonical(codes, q)
-    want_p = tiled_planes(canon)
-    want_a, want_z = tiled_scales(alpha, z, group)
+    want_p, want_a, want_z = tiled_operands(canon, alpha, z, group)
     T = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    assert T.packed.numel() == want_p.size == bq.packed_bytes(T.d)
     assert np.array_equal(T.packed.cpu().numpy(), want_p)
-    assert np.array_equal(T.alpha.cpu().numpy().view(np.uint16), want_a.view(np.uint16))
-    assert np.array_equal(T.z.cpu().numpy().view(np.uint16), want_z.view(np.uint16))
+    if group == 0:
+        assert np.array_equal(T.alpha.cpu().numpy().view(np.uint16), want_a.view(np.uint16))
+        assert np.array_equal(T.z.cpu().numpy().view(np.uint16), want_z.view(np.uint16))
+    else:
+        assert T.alpha is None and T.z is None
     # canonical -> tiled via repack gives the same bytes; tiled -> canonical is the inverse
     C = gpu_layer(N, K, q, group, bq.LAYOUT_CANONICAL, codes, alpha, z)
-    p2, a2, z2 = torch.zeros_like(C.packed), torch.zeros_like(C.alpha), torch.zeros_like(C.z)
+    p2, a2, z2 = bq.empty_operands(T.d, DEV)
+    p2.zero_()
     bq.repack(C.d, C.packed, C.alpha, C.z, T.d, p2, a2, z2)
-    assert torch.equal(p2, T.packed) and torch.equal(a2.view(torch.int16), T.alpha.view(torch.int16))
-    assert torch.equal(z2.view(torch.int16), T.z.view(torch.int16))
+    assert torch.equal(p2, T.packed)
+    if group == 0:
+        assert torch.equal(a2.view(torch.int16), T.alpha.view(torch.int16))
+        assert torch.equal(z2.view(torch.int16), T.z.view(torch.int16))
     p3, a3, z3 = torch.zeros_like(C.packed), torch.zeros_like(C.alpha), torch.zeros_like(C.z)
     bq.repack(T.d, p2, a2, z2, C.d, p3, a3, z3)
     assert np.array_equal(p3.cpu().numpy(), canon.ravel())
@@ -281,3 +287,4 @@ def test_device_errors_are_reported_not_raised_as_faults():
     with pytest.raises(bq.BcqError) as e:
         bq.gemv(d, t, t, t, t, t)
     assert e.value.status == bq.ERR_UNSUPPORTED_SHAPE
+    bq.poll_status()        # no bounded wait ran out in any kernel launched so far

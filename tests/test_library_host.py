@@ -42,7 +42,9 @@ def test_status_strings():
 def test_desc_validation_and_sizes():
     d = bq.desc(7168, 7168, 3, 128, bq.LAYOUT_TILED)
     assert bq.check_desc(d) == bq.OK
-    assert bq.packed_bytes(d) == 3 * 7168 * 7168 // 8
+    assert bq.packed_bytes(d) == 3 * 7168 * 7168 // 8 + 2 * 4 * 7168 * 56     # tiles carry the scales
+    assert bq.packed_bytes(d.with_layout(bq.LAYOUT_CANONICAL)) == 3 * 7168 * 7168 // 8
+    assert bq.packed_bytes(bq.desc(64, 1024, 2, 0, bq.LAYOUT_TILED)) == 2 * 64 * 1024 // 8
     assert bq.alpha_elems(d) == 3 * 7168 * 56 and bq.offset_elems(d) == 7168 * 56
     assert bq.offset_elems(bq.desc(16, 32, 3, 0)) == 16
     bad = [(0, 32, 3, 32, 0, bq.ERR_INVALID_ARG), (16, 32, 0, 32, 0, bq.ERR_INVALID_ARG),
@@ -64,6 +66,7 @@ def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
     odd = ctypes.c_void_p(0x10004)
     call = lambda *ptrs: L.bcq_gemv_plan(ctypes.byref(d), ctypes.byref(plan), *ptrs, None, 0, None)
     assert call(None, ok, ok, ok, ok) == bq.ERR_INVALID_ARG
+    assert call(ok, None, ok, ok, ok) == bq.ERR_INVALID_ARG      # canonical operands need alpha and z
     assert call(ok, ok, ok, ok, None) == bq.ERR_INVALID_ARG
     assert call(odd, ok, ok, ok, ok) == bq.ERR_MISALIGNED
     assert call(ok, ok, ok, odd, ok) == bq.ERR_MISALIGNED
@@ -111,6 +114,11 @@ def test_merge_and_pack_argument_checks():
     d2 = bq.desc(16, 64, 3, 32)
     assert L.bcq_repack(ctypes.byref(d), ok, None, None, ctypes.byref(d2), ok, None, None, None) == bq.ERR_INVALID_ARG
     assert L.bcq_repack(ctypes.byref(d), ok, None, None, ctypes.byref(d), ok, None, None, None) == bq.ERR_INVALID_ARG  # in place
+    dc, dtl = bq.desc(64, 512, 3, 128), bq.desc(64, 512, 3, 128, bq.LAYOUT_TILED)
+    ok2 = ctypes.c_void_p(0x20000)
+    # a tiled operand cannot be made without its scales; bcq_pack needs them too
+    assert L.bcq_repack(ctypes.byref(dc), ok, None, None, ctypes.byref(dtl), ok2, None, None, None) == bq.ERR_INVALID_ARG
+    assert L.bcq_pack(ctypes.byref(dtl), ok, None, None, ok2, None, None, None) == bq.ERR_INVALID_ARG
 
 
 @pytest.mark.parametrize("N,K", [(7168, 7168), (28672, 7168), (7168, 28672), (1024, 1024), (4096, 4096),
