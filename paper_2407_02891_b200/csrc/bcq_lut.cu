@@ -43,8 +43,8 @@ constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
 constexpr int kXBytes = kMaxWindowsPerBlock * kWindow * 4;
 constexpr int kBarrierBytes = 1024;
 constexpr int kFixedBytes = kXBytes + kBarrierBytes;
-constexpr int kProducerIdleLimit = 1 << 24;   // polling rounds without progress before the producer gives up
-constexpr int kSpinLimit = 1 << 24;   // tries per wait (each try blocks for a short, hardware-defined time)
+constexpr int kProducerIdleLimit = 1 << 21;   // polling rounds without progress before the producer gives up
+constexpr int kSpinLimit = 1 << 20;   // tries per wait (each try blocks for a short, hardware-defined time)
 
 static_assert(2 * kFixedBytes <= kLutSmemBytes - 2 * kTableBytes, "x + barriers must fit before or after the tables");
 
@@ -136,8 +136,8 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)   
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code)
 {
     for (int it = 0; it < kSpinLimit; ++it) {
-        if (mbar_test_wait(bar, parity)) return true;
-        if ((it & 1023) == 1023 && *abort_flag) return false;
+        if (mbar_try_wait(bar, parity)) return true;   // sleeps in hardware until the phase completes or a short time-out
+        if ((it & 15) == 15 && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicExch(&g_lut_status, code);
@@ -199,46 +199,50 @@ __device__ __forceinline__ int xs_index(int kk)
     return ((j * 16 + s * 8 + (l >> 2)) << 2) + (l & 3);
 }
 
-// One build item = 8 table entries (entry bits 3..7 = item >> 4) of the four chunks of quad
-// item & 15 (slot s = quad >> 3, lanes 4*(quad&7) .. +3).  The 8 entries are walked in Gray-code
-// order: one packed FMA per entry and chunk pair, one 128-bit conflict-free store per entry.
-__device__ __forceinline__ void build_item(unsigned char *table, const float *xs_w, int item)
+// Table build.  A thread owns one quad of chunks (slot s = quad >> 3, lanes 4*(quad&7) .. +3): it
+// reads the quad's 8 x 4 activations once, then for each of its values of the entry bits 3..7
+// (hi = hi0, hi0 + hi_step, ... < 32) walks the 8 entries sharing those bits in Gray-code order:
+// one packed FMA per entry and chunk pair, one 128-bit conflict-free store per entry.
+__device__ __forceinline__ void build_quad(unsigned char *table, const float *xs_w, int quad, int hi0, int hi_step)
 {
-    const int quad = item & 15;
-    const int hi = item >> 4;
     const float4 *xq = reinterpret_cast<const float4 *>(xs_w) + quad;  // xq[16 j] = activation j of the 4 chunks
-    f32x2 c01 = pack2(0.f, 0.f), c23 = c01;
+    f32x2 x01[8], x23[8];
 #pragma unroll
-    for (int j = 3; j < 8; ++j) {
-        const float4 v = xq[16 * j];
-        const float sg = ((hi >> (j - 3)) & 1) ? 1.f : -1.f;
-        const f32x2 s2 = pack2(sg, sg);
-        c01 = fma2(s2, pack2(v.x, v.y), c01);
-        c23 = fma2(s2, pack2(v.z, v.w), c23);
-    }
-    f32x2 x01[3], x23[3];
-    const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
+    for (int j = 0; j < 8; ++j) {
         const float4 v = xq[16 * j];
         x01[j] = pack2(v.x, v.y);
         x23[j] = pack2(v.z, v.w);
-        c01 = fma2(m1, x01[j], c01);
-        c23 = fma2(m1, x23[j], c23);
     }
-    unsigned char *dst = table + quad * 16 + hi * (8 * 256);
-    static_for<0, 8>([&](auto step_c) {
-        constexpr int step = decltype(step_c)::value;
-        constexpr int gray = step ^ (step >> 1);
-        if constexpr (step > 0) {
-            constexpr int bit = (step & 1) ? 0 : ((step & 2) ? 1 : 2);  // lowest set bit of step
-            constexpr bool on = (gray >> bit) & 1;
-            c01 = fma2(on ? p2 : m2, x01[bit], c01);
-            c23 = fma2(on ? p2 : m2, x23[bit], c23);
+    const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
+    f32x2 low01 = pack2(0.f, 0.f), low23 = low01;   // -(x0 + x1 + x2): entry bits 0..2 clear
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        low01 = fma2(m1, x01[j], low01);
+        low23 = fma2(m1, x23[j], low23);
+    }
+    for (int hi = hi0; hi < 32; hi += hi_step) {
+        f32x2 c01 = low01, c23 = low23;
+#pragma unroll
+        for (int j = 3; j < 8; ++j) {
+            const float sg = ((hi >> (j - 3)) & 1) ? 1.f : -1.f;
+            const f32x2 s2 = pack2(sg, sg);
+            c01 = fma2(s2, x01[j], c01);
+            c23 = fma2(s2, x23[j], c23);
         }
-        const float2 a = unpack2(c01), b = unpack2(c23);
-        *reinterpret_cast<float4 *>(dst + gray * 256) = make_float4(a.x, a.y, b.x, b.y);
-    });
+        unsigned char *dst = table + quad * 16 + hi * (8 * 256);
+        static_for<0, 8>([&](auto step_c) {
+            constexpr int step = decltype(step_c)::value;
+            constexpr int gray = step ^ (step >> 1);
+            if constexpr (step > 0) {
+                constexpr int bit = (step & 1) ? 0 : ((step & 2) ? 1 : 2);  // lowest set bit of step
+                constexpr bool on = (gray >> bit) & 1;
+                c01 = fma2(on ? p2 : m2, x01[bit], c01);
+                c23 = fma2(on ? p2 : m2, x23[bit], c23);
+            }
+            const float2 a = unpack2(c01), b = unpack2(c23);
+            *reinterpret_cast<float4 *>(dst + gray * 256) = make_float4(a.x, a.y, b.x, b.y);
+        });
+    }
 }
 
 enum { kWaitEmpty = 1, kWaitFull = 2, kWaitTableReady = 3, kWaitTableFree = 4, kWaitDrain = 5, kTooFewSlots = 6 };
@@ -307,12 +311,17 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         //      and the first window's table ----------------------------------------------------------
         constexpr int kStartThreads = kLutThreads - 32;
         const int sid = warp < kProducerWarp ? tid : tid - 32;
-        const __half *xg = p.x + size_t(w0) * kWindow;
-        for (int e = sid; e < nwin * kWindow; e += kStartThreads)
-            xs[(e & ~(kWindow - 1)) + xs_index(e & (kWindow - 1))] = __half2float(xg[e]);
+        static_assert(kMaxWindowsPerBlock * (kWindow / 8) <= kStartThreads, "one 8-activation chunk per thread");
+        if (sid < nwin * (kWindow / 8)) {   // one chunk of 8 activations per thread, one 128-bit load
+            const uint4 raw = *reinterpret_cast<const uint4 *>(p.x + size_t(w0) * kWindow + size_t(sid) * 8);
+            const __half *h = reinterpret_cast<const __half *>(&raw);
+            float *dst = xs + (sid >> 6) * kWindow + xs_index((sid & 63) * 8);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) dst[j * 64] = __half2float(h[j]);   // xs_index advances by 64 per activation
+        }
         named_barrier(1, kStartThreads);
         if (sid == 0) TRACE(2);
-        if (sid < 512) build_item(tables, xs, sid);
+        if (sid < 512) build_quad(tables, xs, sid & 15, sid >> 4, 32);
         named_barrier(1, kStartThreads);
         if (sid == 0) TRACE(3);
     }
@@ -324,7 +333,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             const int b = wi & 1, use = wi >> 1;
             if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree)) break;
             unsigned char *table = tables + b * kTableBytes;
-            for (int item = tid; item < 512; item += kBuilderThreads) build_item(table, xs + wi * kWindow, item);
+            build_quad(table, xs + wi * kWindow, tid & 15, tid >> 4, kBuilderThreads / 16);
             mbar_arrive(bar_tab_ready + 8 * b);
         }
         return;
@@ -370,7 +379,10 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                 if (__ballot_sync(0xFFFFu, remaining > 0) == 0) break;
                 if (__any_sync(0xFFFFu, issued)) {
                     idle = 0;
-                } else if (++idle > kProducerIdleLimit || *abort_flag) {
+                    continue;
+                }
+                __nanosleep(100);   // nothing to refill: leave the issue slots to the consumers
+                if (++idle > kProducerIdleLimit || *abort_flag) {
                     if (idle > kProducerIdleLimit) {
                         *abort_flag = 1;
                         atomicExch(&g_lut_status, int(kWaitEmpty));
@@ -398,13 +410,13 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     // ---- consumers ---------------------------------------------------------------------------------
     const int cw = warp - kFirstConsumerWarp;   // 0..15
     const int ctid = tid - kFirstConsumerWarp * 32;
-    f32x2 acc[UMAX][4];
+    float acc[UMAX][8];
     float zacc[UMAX];
 #pragma unroll
     for (int t = 0; t < UMAX; ++t) {
         zacc[t] = 0.f;
 #pragma unroll
-        for (int r = 0; r < 4; ++r) acc[t][r] = pack2(0.f, 0.f);
+        for (int r = 0; r < 8; ++r) acc[t][r] = 0.f;
     }
     bool alive = !*abort_flag;
     int d = 0, k = 0;   // this warp's ring position: slot cw + 16 d, fill number k
@@ -458,23 +470,20 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
                     // offsets: lane (g, j) adds z[g][row j] * (sum of x over group g)
                     zacc[t] = fmaf(__half2float(zh), xsum, zacc[t]);
-                    static_for<0, 4>([&](auto PR) {
-                        constexpr int pr = decltype(PR)::value;  // rows 2pr and 2pr+1
-                        f32x2 a2 = acc[t][pr];
+                    static_for<0, 8>([&](auto R) {
+                        constexpr int r = decltype(R)::value;
+                        float a = acc[t][r];
                         static_for<0, Q>([&](auto I) {
                             constexpr int i = decltype(I)::value;
-                            constexpr int b0 = ((2 * pr) * Q + i) * 2, b1 = ((2 * pr + 1) * Q + i) * 2;
-                            const uint32_t word0 = wbuf[b0 >> 2], word1 = wbuf[b1 >> 2];
-                            const float v00 = lds_f32<0>(__byte_perm(word0, lane_off, 0x7604 | ((b0 & 3) << 4)));
-                            const float v01 = lds_f32<128>(__byte_perm(word0, lane_off, 0x7604 | (((b0 + 1) & 3) << 4)));
-                            const float v10 = lds_f32<0>(__byte_perm(word1, lane_off, 0x7604 | ((b1 & 3) << 4)));
-                            const float v11 = lds_f32<128>(__byte_perm(word1, lane_off, 0x7604 | (((b1 + 1) & 3) << 4)));
-                            const f32x2 s2 = add2(pack2(v00, v10), pack2(v01, v11));
-                            const uint32_t aw = reinterpret_cast<const uint32_t *>(&araw[i])[pr];
-                            const float2 af = __half22float2(*reinterpret_cast<const __half2 *>(&aw));
-                            a2 = fma2(pack2(af.x, af.y), s2, a2);
+                            constexpr int b0 = (r * Q + i) * 2;   // byte of chunk 2*lane; chunk 2*lane+1 is the next byte
+                            const uint32_t word = wbuf[b0 >> 2];
+                            const float v0 = lds_f32<0>(__byte_perm(word, lane_off, 0x7604 | ((b0 & 3) << 4)));
+                            const float v1 = lds_f32<128>(__byte_perm(word, lane_off, 0x7604 | (((b0 + 1) & 3) << 4)));
+                            const float al = __half2float(reinterpret_cast<const __half *>(&araw[i])[r]);
+                            a = fmaf(al, v0, a);
+                            a = fmaf(al, v1, a);
                         });
-                        acc[t][pr] = a2;
+                        acc[t][r] = a;
                     });
                 }
                 if (++d == D) {
@@ -496,9 +505,9 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             float v4[4], v2[2], v1;
 #pragma unroll
             for (int pr = 0; pr < 4; ++pr) {  // lane bit 0 picks the row of the pair
-                const float2 a = unpack2(acc[t][pr]);
+                const float ax = acc[t][2 * pr], ay = acc[t][2 * pr + 1];
                 const bool odd = lane & 1;
-                v4[pr] = (odd ? a.y : a.x) + __shfl_xor_sync(0xffffffffu, odd ? a.x : a.y, 1);
+                v4[pr] = (odd ? ay : ax) + __shfl_xor_sync(0xffffffffu, odd ? ax : ay, 1);
             }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {  // lane bit 1 picks the pair inside a half
