@@ -34,15 +34,17 @@
  *
  * Tiled layout (BCQ_LAYOUT_TILED): the same bytes and the same fp16 values, permuted so that
  * the batch-1 kernel fetches everything it needs for 8 rows x 512 weights with ONE contiguous
- * bulk copy and a lane's bytes all index the lane's own shared-memory banks.  It needs
- * K % 512 == 0, N % 8 == 0 and group in {0, 128}.  With U = N/8 row units and K/512 windows,
- * `packed` is a sequence of tiles, tile (w, u) at byte (w*U + u) * T:
- *   bytes [0, q*512)      planes as [j < q][lane < 32][16 bytes]; byte p = 16 j + (byte in lane)
- *                         = (r*q + i)*2 + s  holds row 8u + r, plane i, weights
- *                         k = 512 w + 16 lane + 8 s .. + 7   (bit order as canonical)
- *   group 128, T = q*576 + 64: the tile continues with the scales of its four groups,
- *     bytes [q*512, q*576)   alpha fp16 [gi < 4][i < q][r < 8]  <- alpha[i][8u + r][4w + gi]
- *     bytes [q*576, T)       z     fp16 [gi < 4][r < 8]         <- z[8u + r][4w + gi]
+ * bulk copy, and so that the 32 lanes of a warp always look up 32 different shared-memory
+ * banks.  It needs K % 512 == 0, N % 8 == 0 and group in {0, 128}.  With U = N/8 row units and
+ * K/512 windows, `packed` is a sequence of tiles, tile (w, u) at byte (w*U + u) * T.  Inside a
+ * tile, lane l = 8 g + j (g < 4, j < 8) stands for row 8u + j and the g-th group of 128 weights
+ * of window w:
+ *   bytes [0, q*512)      planes as [jq < q][lane < 32][16 bytes]; byte p = 16 jq + (byte in lane)
+ *                         = s*q + i  (s < 16) holds plane i of the 8 weights
+ *                         k = 512 w + 128 g + 8 ((s + 2 j) mod 16) .. + 7   (bit order as canonical)
+ *   group 128, T = q*576 + 64: the tile continues with the lanes' scales,
+ *     bytes [q*512, T)    fp16 [lane < 32][alpha_0 .. alpha_{q-1}, z]
+ *                         <- alpha[i][8u + j][4w + g], z[8u + j][4w + g]
  *     and the alpha / z arguments of every call are ignored for this layout (pass NULL);
  *   group 0 (one scale per row), T = q*512: alpha and z stay in arrays of their own,
  *     alpha [u][i][r], z [u][r].
@@ -162,7 +164,7 @@ int bcq_repack(const bcq_desc *src, const void *packed_src_dev, const uint16_t *
  * y = W x at batch 1 (the definition at the top of this file; Eq. bcw + Eq. fuse_step3).
  * x [K], y [N] fp16.  y is overwritten.  workspace may be NULL when bcq_workspace_bytes is 0.
  * bcq_gemv_plan is the same product with an explicit decomposition (for tuning and tests):
- * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 64 row units (512 rows)
+ * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 128 row units (1024 rows)
  * per row block and at most 7 windows (3584 weights along K) per K split.
  */
 int bcq_gemv(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,

@@ -53,16 +53,19 @@ bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED
 // tiled layout with grouped scales: alpha and z live inside `packed`
 bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group != 0; }
 
-// Instruction-count model of the lookup-table kernel (warp instructions on the critical warp
-// of a block); it ranks decompositions, it does not predict time.
+// Time model of the lookup-table kernel in nanoseconds, fitted to traces on B200: a fixed
+// start-up + tail, one "round" per 16 row units of a block per window (each consumer warp does one
+// unit), a floor of one round per window (the table build), and a split-K combine that grows with
+// the number of splits.  It ranks decompositions; it does not predict time exactly.
 long long lut_cost(int U, int W, int rb, int ks, int sm)
 {
-    const long long build = 100, lookup = 200, reduce = 40, fixed = 400, finalize = 120;
+    const long long fixed = 4000, round = 890, per_split = 150;
     const long long waves = (static_cast<long long>(rb) * ks + sm - 1) / sm;
     const long long wc = (W + ks - 1) / ks;
     const long long units = (U + rb - 1) / rb;
-    const long long upw = (units + kLutWarps - 1) / kLutWarps;
-    return waves * (fixed + wc * (build + upw * lookup) + upw * reduce + (ks > 1 ? finalize : 0));
+    long long upw = (units + kLutWarps - 1) / kLutWarps;
+    if (upw < 1) upw = 1;
+    return waves * (fixed + wc * upw * round + (ks > 1 ? per_split * ks : 0));
 }
 
 int plan_lut(const bcq_desc *d, int sm, bcq_plan *out)

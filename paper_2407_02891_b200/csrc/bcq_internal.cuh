@@ -14,7 +14,7 @@ constexpr int kWindow = 512;        // weights along K covered by one lookup-tab
 constexpr int kUnitRows = 8;        // rows of one row unit
 constexpr int kGroupsPerWindow = 4; // 128-weight groups in a window
 constexpr int kLutWarps = 16;       // warps per block of the lookup-table kernel
-constexpr int kLutUnitsPerWarp = 4; // row units a warp keeps accumulators for
+constexpr int kLutUnitsPerWarp = 8; // row units a warp keeps accumulators for
 constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
 constexpr int kMaxWindowsPerBlock = 7;  // windows of x a block keeps in shared memory
 constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace
@@ -25,10 +25,13 @@ inline int n_groups(const bcq_desc &d) { return d.group == 0 ? 1 : d.K / d.group
 // ---- where the operands of one layer live (host and device) ---------------------------------
 //
 // Canonical: packed[i][n][k/8], alpha[i][n][g], z[n][g] in three arrays.
-// Tiled: tile (w, u) of `packed` covers window w (512 weights) of row unit u (8 rows):
-//   q*512 bytes of planes as [j < q][lane < 32][16 B], byte p = (r*q + i)*2 + s of a lane's 16q
-//   bytes = row 8u + r, plane i, chunk 2*lane + s;
-//   group 128 only: followed, in the same tile, by alpha [gi < 4][i < q][r < 8] and z [gi < 4][r < 8]
+// Tiled: tile (w, u) of `packed` covers window w (512 weights = 64 chunks of 8 = 4 groups of 128)
+// of row unit u (8 rows).  Lane l = 8 g + j of a warp owns row 8u + j and group g of the window:
+//   q*512 bytes of planes as [jq < q][lane < 32][16 B]; byte p = s*q + i of a lane's 16q bytes is
+//   plane i of chunk 16 g + ((s + 2 j) mod 16): the 8 lanes of a group walk the group's 16 chunks
+//   skewed by two chunks per row, so that at every step the 32 lanes of a warp look up 32
+//   different chunk columns of the table (32 different shared-memory banks);
+//   group 128 only: followed, in the same tile, by the lanes' scales [lane < 32][alpha_0 .. alpha_{q-1}, z]
 //   (fp16) -- the tile is one contiguous piece of memory, fetched by one bulk copy;
 //   group 0 (per row): alpha [u][i][r] and z [u][r] stay in their own arrays.
 struct View {
@@ -47,9 +50,10 @@ struct View {
     {
         if (layout == BCQ_LAYOUT_CANONICAL) return packed + (size_t(i) * N + n) * size_t(K / 8) + kb;
         const int w = kb / (kWindow / 8), c = kb % (kWindow / 8);
-        const int lane = c >> 1, s = c & 1;
-        const int u = n / kUnitRows, r = n % kUnitRows;
-        const int p = (r * q + i) * 2 + s;
+        const int g = c >> 4, u = n / kUnitRows, j = n % kUnitRows;
+        const int s = ((c & 15) - 2 * j) & 15;   // step at which lane 8g + j reaches chunk c
+        const int lane = 8 * g + j;
+        const int p = s * q + i;
         return packed + tile_base(w, u) + size_t(p >> 4) * 512 + size_t(lane) * 16 + (p & 15);
     }
     __host__ __device__ uint16_t *alpha_elem(int i, int n, int g) const
@@ -58,7 +62,7 @@ struct View {
         const int u = n / kUnitRows, r = n % kUnitRows;
         if (group == 0) return alpha + (size_t(u) * q + i) * kUnitRows + r;
         const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
-        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + (gi * q + i) * kUnitRows + r;
+        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + (gi * kUnitRows + r) * (q + 1) + i;
     }
     __host__ __device__ uint16_t *z_elem(int n, int g) const
     {
@@ -66,7 +70,7 @@ struct View {
         const int u = n / kUnitRows, r = n % kUnitRows;
         if (group == 0) return z + size_t(u) * kUnitRows + r;
         const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
-        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 576) + gi * kUnitRows + r;
+        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + (gi * kUnitRows + r) * (q + 1) + q;
     }
 };
 

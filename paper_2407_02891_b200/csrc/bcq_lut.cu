@@ -14,11 +14,13 @@
 //   consumers (warps 4-19)  copy a filled slot into registers, hand the slot back, look every
 //                           weight byte up in the window table and accumulate in fp32.
 //
-// Table layout: word address of (entry e, chunk c) = e*64 + (c&1)*32 + (c>>1).  Lane l of a
-// consumer warp only ever looks up chunks 2l and 2l+1, so a warp's lookups always hit 32 distinct
-// banks whatever the weight bytes are.  The tables sit at shared-window addresses that are
+// Table layout: word address of (entry e, chunk c) = e*64 + (c&1)*32 + (c>>1).  Lane l = 8 g + j
+// of a consumer warp handles row j of a unit and the g-th group of 128 weights of the window; it
+// walks the group's 16 chunks skewed by 2 j, so at every step the 32 lanes look up 32 different
+// chunk columns -- 32 distinct banks whatever the weight bytes are -- and a lane needs only its
+// own (row, group) scales.  The tables sit at shared-window addresses that are
 // multiples of 64 KB and an entry is 256 B apart from the next, so ONE byte-permute builds the
-// complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + 4*lane): a lookup is
+// complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + 4*bank): a lookup is
 // PRMT + LDS.  The memory before and after the tables (99 KB together) holds x, the barriers and
 // the slot ring.
 //
@@ -408,16 +410,15 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     // =============================================================================================
     // ---- consumers ---------------------------------------------------------------------------------
+    // Lane l = 8 g + j owns row 8u + j of every unit and the g-th group of 128 weights of every
+    // window: its 16q bytes of a tile are the group's 16 chunks (skewed by 2 j, see the layout), so
+    // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
     const int cw = warp - kFirstConsumerWarp;   // 0..15
     const int ctid = tid - kFirstConsumerWarp * 32;
-    float acc[UMAX][8];
-    float zacc[UMAX];
+    const int g4 = lane >> 3, jr = lane & 7;
+    float acc[UMAX];
 #pragma unroll
-    for (int t = 0; t < UMAX; ++t) {
-        zacc[t] = 0.f;
-#pragma unroll
-        for (int r = 0; r < 8; ++r) acc[t][r] = 0.f;
-    }
+    for (int t = 0; t < UMAX; ++t) acc[t] = 0.f;
     bool alive = !*abort_flag;
     int d = 0, k = 0;   // this warp's ring position: slot cw + 16 d, fill number k
 
@@ -428,9 +429,13 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             break;
         }
         if (ctid == 0 && wi == 0) TRACE(4);
-        const uint32_t lane_off = tab0 + uint32_t(b * kTableBytes + lane * 4);
-        // sum of this lane's 16 activations (the all-ones entries of its two chunks), then of its group
-        float xsum = lds_f32<255 * 256>(lane_off) + lds_f32<255 * 256 + 128>(lane_off);
+        // Table address part of the lookups of step pair h: chunk 16 g + ((2h + 2j) mod 16) and the
+        // next one share bank 8 g + ((h + j) mod 8); the odd chunk sits 128 bytes further.
+        uint32_t off[8];
+#pragma unroll
+        for (int h = 0; h < 8; ++h) off[h] = tab0 + uint32_t(b * kTableBytes + 4 * (8 * g4 + ((h + jr) & 7)));
+        // sum of x over this lane's group: the all-ones entries of the group's 16 chunks
+        float xsum = lds_f32<255 * 256>(off[0]) + lds_f32<255 * 256 + 128>(off[0]);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
@@ -452,7 +457,6 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                     // slot -> registers, then hand the slot back to the producer
                     const unsigned char *slot = slot_ptr(s);
                     uint32_t wbuf[4 * Q];
-                    uint4 araw[Q];
 #pragma unroll
                     for (int j = 0; j < Q; ++j) {
                         const uint4 v = *reinterpret_cast<const uint4 *>(slot + j * 512 + lane * 16);
@@ -461,30 +465,35 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                         wbuf[4 * j + 2] = v.z;
                         wbuf[4 * j + 3] = v.w;
                     }
+                    __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
+                    const unsigned char *sp = slot + SL::kPlaneBytes + lane * (2 * (Q + 1));
+                    if constexpr (Q == 3) {
+                        *reinterpret_cast<uint2 *>(sc) = *reinterpret_cast<const uint2 *>(sp);
+                    } else if constexpr (Q == 1) {
+                        *reinterpret_cast<uint32_t *>(sc) = *reinterpret_cast<const uint32_t *>(sp);
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < Q; ++i)
-                        araw[i] = *reinterpret_cast<const uint4 *>(slot + SL::kPlaneBytes + (lane >> 3) * (Q * 16) + i * 16);
-                    const __half zh = *reinterpret_cast<const __half *>(slot + SL::kPlaneBytes + SL::kAlphaBytes + lane * 2);
+                        for (int i = 0; i <= Q; ++i) sc[i] = reinterpret_cast<const __half *>(sp)[i];
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_empty + 8 * s);
 
-                    // offsets: lane (g, j) adds z[g][row j] * (sum of x over group g)
-                    zacc[t] = fmaf(__half2float(zh), xsum, zacc[t]);
-                    static_for<0, 8>([&](auto R) {
-                        constexpr int r = decltype(R)::value;
-                        float a = acc[t][r];
+                    float sum[Q][2];
+#pragma unroll
+                    for (int i = 0; i < Q; ++i) sum[i][0] = sum[i][1] = 0.f;
+                    static_for<0, 16>([&](auto S) {
+                        constexpr int st = decltype(S)::value;
                         static_for<0, Q>([&](auto I) {
                             constexpr int i = decltype(I)::value;
-                            constexpr int b0 = (r * Q + i) * 2;   // byte of chunk 2*lane; chunk 2*lane+1 is the next byte
-                            const uint32_t word = wbuf[b0 >> 2];
-                            const float v0 = lds_f32<0>(__byte_perm(word, lane_off, 0x7604 | ((b0 & 3) << 4)));
-                            const float v1 = lds_f32<128>(__byte_perm(word, lane_off, 0x7604 | (((b0 + 1) & 3) << 4)));
-                            const float al = __half2float(reinterpret_cast<const __half *>(&araw[i])[r]);
-                            a = fmaf(al, v0, a);
-                            a = fmaf(al, v1, a);
+                            constexpr int pb = st * Q + i;
+                            const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
+                            sum[i][st & 1] += (st & 1) ? lds_f32<128>(addr) : lds_f32<0>(addr);
                         });
-                        acc[t][r] = a;
                     });
+                    float a = fmaf(__half2float(sc[Q]), xsum, acc[t]);
+#pragma unroll
+                    for (int i = 0; i < Q; ++i) a = fmaf(__half2float(sc[i]), sum[i][0] + sum[i][1], a);
+                    acc[t] = a;
                 }
                 if (++d == D) {
                     d = 0;
@@ -497,39 +506,21 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         if (ctid == 0 && wi < 4) TRACE(6 + wi);
     }
 
-    // ---- reduce each unit's 8 row sums over the 32 lanes: lane l ends with row l & 7 -------------
+    // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up, lanes 0..7 store ---------
     float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * p.N : nullptr;
-    static_for<0, UMAX>([&](auto T) {
-        constexpr int t = decltype(T)::value;
-        if (cw + kLutWarps * t < V) {
-            float v4[4], v2[2], v1;
 #pragma unroll
-            for (int pr = 0; pr < 4; ++pr) {  // lane bit 0 picks the row of the pair
-                const float ax = acc[t][2 * pr], ay = acc[t][2 * pr + 1];
-                const bool odd = lane & 1;
-                v4[pr] = (odd ? ay : ax) + __shfl_xor_sync(0xffffffffu, odd ? ax : ay, 1);
-            }
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {  // lane bit 1 picks the pair inside a half
-                const bool up = lane & 2;
-                v2[h] = (up ? v4[2 * h + 1] : v4[2 * h]) + __shfl_xor_sync(0xffffffffu, up ? v4[2 * h] : v4[2 * h + 1], 2);
-            }
-            {
-                const bool up = lane & 4;  // lane bit 2 picks the half
-                v1 = (up ? v2[1] : v2[0]) + __shfl_xor_sync(0xffffffffu, up ? v2[0] : v2[1], 4);
-            }
-            v1 += zacc[t];  // lane (g, j) holds group g's offset term of row j = l & 7
-            v1 += __shfl_xor_sync(0xffffffffu, v1, 8);
-            v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
-            if (lane < 8) {
-                const int n = (u0 + cw + kLutWarps * t) * kUnitRows + lane;
-                if (partial)
-                    partial[n] = v1;
-                else
-                    p.y[n] = __float2half_rn(v1);
-            }
+    for (int t = 0; t < UMAX; ++t) {
+        float v = acc[t];
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        if (lane < 8 && cw + kLutWarps * t < V) {
+            const int n = (u0 + cw + kLutWarps * t) * kUnitRows + lane;
+            if (partial)
+                partial[n] = v;
+            else
+                p.y[n] = __float2half_rn(v);
         }
-    });
+    }
 
     if (ctid == 0) TRACE(10);
     // ---- split-K: the last block to arrive for this row block adds the partials in fixed order --
@@ -543,9 +534,17 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         named_barrier(2, kConsumerThreads);
         if (*s_last) {
             __threadfence();
+            // fixed summation order (deterministic); the loads of 8 splits are issued together
             for (int n = u0 * kUnitRows + ctid; n < u1 * kUnitRows; n += kConsumerThreads) {
                 float v = 0.f;
-                for (int k = 0; k < p.k_splits; ++k) v += __ldcg(p.partial + size_t(k) * p.N + n);
+                for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
+                    float part[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        part[k] = (k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * p.N + n) : 0.f;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) v += part[k];
+                }
                 p.y[n] = __float2half_rn(v);
             }
             if (ctid == 0) p.counters[rbi] = 0;

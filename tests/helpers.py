@@ -25,9 +25,11 @@ def tiled_operands(planes, alpha, z, group):
     out = np.zeros(U * W * T, np.uint8)
     i, n, kb = np.meshgrid(np.arange(q), np.arange(N), np.arange(KB), indexing="ij")
     w, c = kb // 64, kb % 64
-    lane, s = c // 2, c % 2
-    u, r = n // 8, n % 8
-    p = (r * q + i) * 2 + s
+    g, cc = c // 16, c % 16
+    u, j = n // 8, n % 8
+    s = (cc - 2 * j) % 16
+    lane = 8 * g + j
+    p = s * q + i
     off = (w * U + u) * T + (p // 16) * 512 + lane * 16 + p % 16
     out[off.ravel()] = planes.ravel()
     G = alpha.shape[2]
@@ -40,8 +42,9 @@ def tiled_operands(planes, alpha, z, group):
         z_out[(u[0] * 8 + r[0]).ravel()] = z.ravel()
         return out, a_out, z_out
     w, gi = g // 4, g % 4
-    a_off = (w * U + u) * T + q * 512 + 2 * ((gi * q + i) * 8 + r)
-    z_off = (w[0] * U + u[0]) * T + q * 576 + 2 * (gi[0] * 8 + r[0])
+    lane = 8 * gi + r
+    a_off = (w * U + u) * T + q * 512 + 2 * (lane * (q + 1) + i)
+    z_off = (w[0] * U + u[0]) * T + q * 512 + 2 * (lane[0] * (q + 1) + q)
     ab = alpha.view(np.uint8).reshape(q, N, G, 2)
     zb = z.view(np.uint8).reshape(N, G, 2)
     for byte in range(2):

@@ -86,7 +86,7 @@ def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
     # plans that break the limits
     for p in (bq.Plan(1, 0, 1, 0), bq.Plan(1, 9, 1, 0), bq.Plan(1, 1, 3, 0), bq.Plan(2, 1, 1, 0)):
         assert L.bcq_gemv_plan(ctypes.byref(dt), ctypes.byref(p), ok, ok, ok, ok, ok, ok, 1 << 20, None) == bq.ERR_INVALID_ARG
-    big = bq.desc(1024, 512, 3, 128, bq.LAYOUT_TILED)     # 128 units in one row block > 64
+    big = bq.desc(2048, 512, 3, 128, bq.LAYOUT_TILED)     # 256 units in one row block > 128
     p = bq.Plan(1, 1, 1, 0)
     assert L.bcq_gemv_plan(ctypes.byref(big), ctypes.byref(p), ok, ok, ok, ok, ok, None, 0, None) == bq.ERR_INVALID_ARG
     # batch limits
@@ -130,7 +130,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert p.kernel == 1
     U, W = N // 8, K // 512
     assert 1 <= p.row_blocks <= U and 1 <= p.k_splits <= W
-    assert -(-U // p.row_blocks) <= 64
+    assert -(-U // p.row_blocks) <= 128 and -(-W // p.k_splits) <= 7
     blocks = p.row_blocks * p.k_splits
     if U * W >= 148 * 8:
         assert blocks >= 0.75 * 148
