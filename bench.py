@@ -33,6 +33,9 @@ WORKLOADS = {
     "opt66b_q2_row": dict(hidden=9216, ffn=36864, layers=64, q=2, group=0),
 }
 DEFAULT_WORKLOAD = "opt30b_q3_g128"
+# DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
+# profiles/lut_gemv_kernel_opt30b_q3_g128.md; valid only for the library revision it was taken on.
+NCU_TRAFFIC = {"lib_version": 101, "workload": "opt30b_q3_g128", "bytes_per_launch": 46.3e6}
 METRIC = "BCQ GEMV us/token (sum of all linear layers of the decoder stack, bs=1)"
 UNIT = "us/token"
 
@@ -392,7 +395,10 @@ def main():
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "frac_of_nominal_8000": round(achieved / 8000.0, 4),
-                     "peak_kind": peak_kind, "traffic": None, "kernel": f"lut_gemv_kernel<{w['q']}>",
+                     "peak_kind": peak_kind,
+                     "traffic": (NCU_TRAFFIC["bytes_per_launch"]
+                                 if bq.lib().bcq_version() == NCU_TRAFFIC["lib_version"]
+                                 and args.workload == NCU_TRAFFIC["workload"] and args.layers == 0 else None), "kernel": f"lut_gemv_kernel<{w['q']}>",
                      "algorithmic_bytes_per_launch": stack.bytes // launches_per_step,
                      "launches_per_step": launches_per_step},
         "per_shape": per_shape,

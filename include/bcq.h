@@ -62,7 +62,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 100
+#define BCQ_VERSION 101
 
 typedef enum bcq_status {
     BCQ_OK = 0,
