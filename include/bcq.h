@@ -21,7 +21,8 @@
  *     enqueue work; they never synchronise.  Errors found on the host return before any
  *     launch.  The current CUDA device must be the one that owns the pointers.
  *   - fp16 values are IEEE binary16 bit patterns in uint16_t.  Accumulation is fp32;
- *     y is rounded to fp16 (nearest even) once, at the end.
+ *     y is rounded to fp16 (nearest even) once, at the end.  (The lookup-table kernel keeps
+ *     its table of 8-activation partial sums in fp16: each is computed in fp32 and rounded once.)
  *   - Device pointers must be 16-byte aligned (y: 2-byte) or BCQ_ERR_MISALIGNED is returned.
  *   - Return value: BCQ_OK (0) or a negative bcq_status.  No exceptions, no exit().
  *
@@ -62,7 +63,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 101
+#define BCQ_VERSION 102
 
 typedef enum bcq_status {
     BCQ_OK = 0,
@@ -165,7 +166,7 @@ int bcq_repack(const bcq_desc *src, const void *packed_src_dev, const uint16_t *
  * x [K], y [N] fp16.  y is overwritten.  workspace may be NULL when bcq_workspace_bytes is 0.
  * bcq_gemv_plan is the same product with an explicit decomposition (for tuning and tests):
  * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 128 row units (1024 rows)
- * per row block and at most 7 windows (3584 weights along K) per K split.
+ * per row block and at most 32 windows (16384 weights along K) per K split.
  */
 int bcq_gemv(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
              const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev,

@@ -16,7 +16,7 @@ constexpr int kGroupsPerWindow = 4; // 128-weight groups in a window
 constexpr int kLutWarps = 16;       // warps per block of the lookup-table kernel
 constexpr int kLutUnitsPerWarp = 8; // row units a warp keeps accumulators for
 constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
-constexpr int kMaxWindowsPerBlock = 7;  // windows of x a block keeps in shared memory
+constexpr int kMaxWindowsPerBlock = 32; // windows one block may walk (bounds the planner's search)
 constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace
 constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);
 

@@ -6,23 +6,25 @@
 // 8-activation chunk; packed weight bytes index those tables directly.  One block per SM, three
 // kinds of warps:
 //
-//   builders  (warps 0-2)   convert the block's slice of x to fp32 and build the window tables,
-//                           one window ahead of the consumers (two 64 KB tables, double buffered);
-//   producer  (warp 3)      one thread feeds a ring of shared-memory slots with bulk async copies
+//   builders  (warps 0-2)   build the window tables from x, one window ahead of the consumers
+//                           (two tables, double buffered);
+//   producer  (warp 3)      16 lanes feed a ring of shared-memory slots with bulk async copies
 //                           (cp.async.bulk, completion on an mbarrier): per (window, row unit) one
 //                           slot = one tile = q*512 B of plane bytes + the unit's alphas and offsets;
 //   consumers (warps 4-19)  copy a filled slot into registers, hand the slot back, look every
 //                           weight byte up in the window table and accumulate in fp32.
 //
-// Table layout: word address of (entry e, chunk c) = e*64 + (c&1)*32 + (c>>1).  Lane l = 8 g + j
+// Tables.  The sums are computed in fp32 and stored as fp16 (one rounding, relative 2^-11; the
+// accumulation of the looked-up values stays fp32).  Halving the tables to 32 KB each is what
+// leaves 140 KB of shared memory for tiles in flight -- the stream is otherwise bound by the DRAM
+// latency.  Both tables share one 64 KB region at a shared-window address that is a multiple of
+// 64 KB: entry e of table b, chunk c at byte  e*256 + b*128 + (c>>1)*4 + (c&1)*2.  Lane l = 8 g + j
 // of a consumer warp handles row j of a unit and the g-th group of 128 weights of the window; it
-// walks the group's 16 chunks skewed by 2 j, so at every step the 32 lanes look up 32 different
-// chunk columns -- 32 distinct banks whatever the weight bytes are -- and a lane needs only its
-// own (row, group) scales.  The tables sit at shared-window addresses that are
-// multiples of 64 KB and an entry is 256 B apart from the next, so ONE byte-permute builds the
-// complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + 4*bank): a lookup is
-// PRMT + LDS.  The memory before and after the tables (99 KB together) holds x, the barriers and
-// the slot ring.
+// walks the group's 16 chunks skewed by 2 j, so at every step the 32 lanes address 32 different
+// 4-byte columns -- 32 distinct banks whatever the weight bytes are -- and a lane needs only its
+// own (row, group) scales.  With the 256-byte entry stride and the 64 KB alignment ONE byte-permute
+// builds the complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + column): a
+// lookup is PRMT + LDS.U16 + one mixed-precision add (fp32 += fp16).
 //
 // Every wait on an mbarrier is bounded; if one runs out the block sets an abort flag and a
 // device status word, stops waiting, drains its own copies and returns (see lut_status_take).
@@ -38,17 +40,17 @@ constexpr int kProducerWarp = kBuilderWarps;
 constexpr int kFirstConsumerWarp = kBuilderWarps + 1;
 constexpr int kConsumerThreads = kLutWarps * 32;
 constexpr int kLutThreads = (kBuilderWarps + 1 + kLutWarps) * 32;  // 640
-constexpr int kTableBytes = 256 * 64 * 4;                          // 65536
+constexpr int kTablesBytes = 256 * 256;                            // both fp16 tables, entry stride 256 B
 constexpr int kLutSmemBytes = 232448;                              // 227 KB: the per-block opt-in maximum
-constexpr int kMaxSlots = 48;
+constexpr int kMaxSlotsPerWarp = 5;
+constexpr int kMaxSlots = kLutWarps * kMaxSlotsPerWarp;
 constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
-constexpr int kXBytes = kMaxWindowsPerBlock * kWindow * 4;
-constexpr int kBarrierBytes = 1024;
-constexpr int kFixedBytes = kXBytes + kBarrierBytes;
+constexpr int kFixedBytes = 2048;      // barriers and flags
 constexpr int kProducerIdleLimit = 1 << 21;   // polling rounds without progress before the producer gives up
 constexpr int kSpinLimit = 1 << 20;   // tries per wait (each try blocks for a short, hardware-defined time)
 
-static_assert(2 * kFixedBytes <= kLutSmemBytes - 2 * kTableBytes, "x + barriers must fit before or after the tables");
+static_assert(16 * kMaxSlots + 64 <= kFixedBytes, "barrier area");
+static_assert(2 * kFixedBytes <= kLutSmemBytes - kTablesBytes, "barriers must fit before or after the tables");
 
 __device__ int g_lut_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
 
@@ -156,12 +158,23 @@ __device__ __forceinline__ void named_barrier(int id, int threads)
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-// table lookup: the address register already holds the complete shared-window address
+// table lookup + accumulate: the address register already holds the complete shared-window
+// address of an fp16 entry; acc (fp32) += entry, in one mixed-precision add
 template <int OFF>
-__device__ __forceinline__ float lds_f32(uint32_t addr)
+__device__ __forceinline__ void lut_add(float &acc, uint32_t addr)
 {
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(OFF));
+    asm volatile(
+        "{\n\t.reg .b16 h;\n\t"
+        "ld.shared.b16 h, [%1+%2];\n\t"
+        "add.rn.f32.f16 %0, h, %0;\n\t}"
+        : "+f"(acc)
+        : "r"(addr), "n"(OFF));
+}
+template <int OFF>
+__device__ __forceinline__ uint32_t lds_b32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(OFF));
     return v;
 }
 
@@ -192,28 +205,33 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
     return d;
 }
 
-// Index, inside a window's 512 staged activations, of activation j of chunk c = 2*(4*lq + k) + s:
-// [j][quad = 8s + lq][k], so that one 128-bit load gives activation j of the four chunks of a build
-// item and the 16 quads a warp reads at once are 256 contiguous bytes (no bank conflicts).
-__device__ __forceinline__ int xs_index(int kk)
+// Table build.  A thread owns four consecutive chunks (quad cq: chunks 4cq .. 4cq+3, i.e. 32
+// activations read straight from x): it converts them once, then for each of its values of the
+// entry bits 3..7 (hi = hi0, hi0 + hi_step, ... < 32) walks the 8 entries sharing those bits in
+// Gray-code order: one packed fp32 FMA per entry and chunk pair, the four sums rounded to fp16 and
+// stored with one 64-bit store (16 quads = 128 contiguous bytes per entry: no bank conflicts).
+// `table` points at entry 0 of the buffer being built.
+__device__ __forceinline__ void build_quad(unsigned char *table, const __half *xw, int cq, int hi0, int hi_step)
 {
-    const int l = kk >> 4, s = (kk >> 3) & 1, j = kk & 7;
-    return ((j * 16 + s * 8 + (l >> 2)) << 2) + (l & 3);
-}
-
-// Table build.  A thread owns one quad of chunks (slot s = quad >> 3, lanes 4*(quad&7) .. +3): it
-// reads the quad's 8 x 4 activations once, then for each of its values of the entry bits 3..7
-// (hi = hi0, hi0 + hi_step, ... < 32) walks the 8 entries sharing those bits in Gray-code order:
-// one packed FMA per entry and chunk pair, one 128-bit conflict-free store per entry.
-__device__ __forceinline__ void build_quad(unsigned char *table, const float *xs_w, int quad, int hi0, int hi_step)
-{
-    const float4 *xq = reinterpret_cast<const float4 *>(xs_w) + quad;  // xq[16 j] = activation j of the 4 chunks
     f32x2 x01[8], x23[8];
+    {
+        float xf[4][8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const float4 v = xq[16 * j];
-        x01[j] = pack2(v.x, v.y);
-        x23[j] = pack2(v.z, v.w);
+        for (int k = 0; k < 4; ++k) {
+            const uint4 raw = *reinterpret_cast<const uint4 *>(xw + 32 * cq + 8 * k);
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 f = __half22float2(h2[j]);
+                xf[k][2 * j] = f.x;
+                xf[k][2 * j + 1] = f.y;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            x01[j] = pack2(xf[0][j], xf[1][j]);
+            x23[j] = pack2(xf[2][j], xf[3][j]);
+        }
     }
     const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
     f32x2 low01 = pack2(0.f, 0.f), low23 = low01;   // -(x0 + x1 + x2): entry bits 0..2 clear
@@ -231,7 +249,7 @@ __device__ __forceinline__ void build_quad(unsigned char *table, const float *xs
             c01 = fma2(s2, x01[j], c01);
             c23 = fma2(s2, x23[j], c23);
         }
-        unsigned char *dst = table + quad * 16 + hi * (8 * 256);
+        unsigned char *dst = table + cq * 8 + hi * (8 * 256);
         static_for<0, 8>([&](auto step_c) {
             constexpr int step = decltype(step_c)::value;
             constexpr int gray = step ^ (step >> 1);
@@ -242,7 +260,11 @@ __device__ __forceinline__ void build_quad(unsigned char *table, const float *xs
                 c23 = fma2(on ? p2 : m2, x23[bit], c23);
             }
             const float2 a = unpack2(c01), b = unpack2(c23);
-            *reinterpret_cast<float4 *>(dst + gray * 256) = make_float4(a.x, a.y, b.x, b.y);
+            const __half2 h01 = __floats2half2_rn(a.x, a.y), h23 = __floats2half2_rn(b.x, b.y);
+            uint2 out;
+            out.x = *reinterpret_cast<const uint32_t *>(&h01);
+            out.y = *reinterpret_cast<const uint32_t *>(&h23);
+            *reinterpret_cast<uint2 *>(dst + gray * 256) = out;
         });
     }
 }
@@ -263,12 +285,12 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     const int V = u1 - u0;       // row units of this block
     const int nwin = w1 - w0;    // windows of this block
 
-    // ---- carve shared memory: [front | table 0 | table 1 | back] --------------------------------
+    // ---- carve shared memory: [front | tables (64 KB, 64 KB aligned) | back] ----------------------
     const uint32_t base = smem_u32(smem);
-    const uint32_t tab0 = (base + 0xFFFFu) & ~0xFFFFu;  // shared-window address of table 0
-    const int front = int(tab0 - base), back = kLutSmemBytes - front - 2 * kTableBytes;
+    const uint32_t tab0 = (base + 0xFFFFu) & ~0xFFFFu;  // shared-window address of the tables
+    const int front = int(tab0 - base), back = kLutSmemBytes - front - kTablesBytes;
     unsigned char *tables = smem + front;
-    unsigned char *after = tables + 2 * kTableBytes;
+    unsigned char *after = tables + kTablesBytes;
     const bool fixed_in_back = back >= kFixedBytes;
     unsigned char *fixed = fixed_in_back ? after : smem;
     unsigned char *ring_a = fixed_in_back ? smem : smem + kFixedBytes;
@@ -276,14 +298,13 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     const int n_a = (fixed_in_back ? front : front - kFixedBytes) / SL::kBytes;
     const int n_b = (fixed_in_back ? back - kFixedBytes : back) / SL::kBytes;
     const int NS = min(n_a + n_b, kMaxSlots);
-    const int D = min(NS / kLutWarps, 3);   // ring slots per consumer warp
+    const int D = min(NS / kLutWarps, kMaxSlotsPerWarp);   // ring slots per consumer warp
     auto slot_ptr = [&](int s) -> unsigned char * { return s < n_a ? ring_a + s * SL::kBytes : ring_b + (s - n_a) * SL::kBytes; };
 
-    float *xs = reinterpret_cast<float *>(fixed);
-    const uint32_t bars = smem_u32(fixed + kXBytes);
+    const uint32_t bars = smem_u32(fixed);
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kMaxSlots;
     const uint32_t bar_tab_ready = bars + 16 * kMaxSlots, bar_tab_free = bar_tab_ready + 16;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + kXBytes + 16 * kMaxSlots + 32);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 16 * kMaxSlots + 32);
     int *s_last = const_cast<int *>(abort_flag) + 1;
 
     if (tid == 0) {
@@ -308,22 +329,12 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     if (tid == 0) TRACE(1);
 
     // =============================================================================================
+    const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
     if (warp != kProducerWarp) {
-        // ---- start-up, all warps but the producer: x slice fp16 -> fp32 (permuted for the build)
-        //      and the first window's table ----------------------------------------------------------
+        // ---- start-up: all warps but the producer build the first window's table ----------------
         constexpr int kStartThreads = kLutThreads - 32;
         const int sid = warp < kProducerWarp ? tid : tid - 32;
-        static_assert(kMaxWindowsPerBlock * (kWindow / 8) <= kStartThreads, "one 8-activation chunk per thread");
-        if (sid < nwin * (kWindow / 8)) {   // one chunk of 8 activations per thread, one 128-bit load
-            const uint4 raw = *reinterpret_cast<const uint4 *>(p.x + size_t(w0) * kWindow + size_t(sid) * 8);
-            const __half *h = reinterpret_cast<const __half *>(&raw);
-            float *dst = xs + (sid >> 6) * kWindow + xs_index((sid & 63) * 8);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) dst[j * 64] = __half2float(h[j]);   // xs_index advances by 64 per activation
-        }
-        named_barrier(1, kStartThreads);
-        if (sid == 0) TRACE(2);
-        if (sid < 512) build_quad(tables, xs, sid & 15, sid >> 4, 32);
+        if (sid < 512) build_quad(tables, xblk, sid & 15, sid >> 4, 32);
         named_barrier(1, kStartThreads);
         if (sid == 0) TRACE(3);
     }
@@ -334,8 +345,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         for (int wi = 1; wi < nwin; ++wi) {
             const int b = wi & 1, use = wi >> 1;
             if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree)) break;
-            unsigned char *table = tables + b * kTableBytes;
-            build_quad(table, xs + wi * kWindow, tid & 15, tid >> 4, kBuilderThreads / 16);
+            build_quad(tables + b * 128, xblk + wi * kWindow, tid & 15, tid >> 4, kBuilderThreads / 16);
             mbar_arrive(bar_tab_ready + 8 * b);
         }
         return;
@@ -351,7 +361,10 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             const int mine = (V - c + kLutWarps - 1) / kLutWarps;  // units of warp c per window
             int remaining = mine * nwin, t_in_win = 0, wi = 0, idle = 0;
             size_t tile = size_t(w0) * p.U + u0 + c;
-            int d = 0, k = 0, last_s = -1, last_par = 0, prev_s = -1, prev_par = 0, pprev_s = -1, pprev_par = 0;
+            int d = 0, k = 0;
+            int last_par[kMaxSlotsPerWarp];   // parity of the last fill of each of this lane's slots, -1 = never filled
+#pragma unroll
+            for (int q5 = 0; q5 < kMaxSlotsPerWarp; ++q5) last_par[q5] = -1;
             // The 16 lanes stay together in one polling loop and never block on a barrier, so
             // each refills its warp's slot as soon as that slot is handed back.
             while (true) {
@@ -362,8 +375,9 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                         const uint32_t dst = smem_u32(slot_ptr(s)), full = bar_full + 8 * s;
                         mbar_expect_tx(full, SL::kBytes);
                         bulk_g2s(dst, p.tiles + tile * SL::kBytes, SL::kBytes, full);   // planes + alphas + offsets
-                        pprev_s = prev_s, pprev_par = prev_par, prev_s = last_s, prev_par = last_par;
-                        last_s = s, last_par = k & 1;
+#pragma unroll
+                        for (int q5 = 0; q5 < kMaxSlotsPerWarp; ++q5)
+                            if (q5 == d) last_par[q5] = k & 1;
                         if (++d == D) {
                             d = 0;
                             ++k;
@@ -392,16 +406,16 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                     break;
                 }
             }
-            // See the last fill of each of this lane's (at most 3) slots land, with a bounded wait,
-            // before the warp leaves: the block's shared memory must not be handed to another block
-            // while copies into it are in flight, also when the consumers gave up.
+            // See the last fill of each of this lane's slots land, with a bounded wait, before the
+            // warp leaves: the block's shared memory must not be handed to another block while copies
+            // into it are in flight, also when the consumers gave up.
             if (lane == 0) TRACE(12);
-            const int ss[3] = {last_s, prev_s, pprev_s}, pp[3] = {last_par, prev_par, pprev_par};
 #pragma unroll
-            for (int q3 = 0; q3 < 3; ++q3) {
-                if (ss[q3] < 0 || q3 >= D) continue;
+            for (int q5 = 0; q5 < kMaxSlotsPerWarp; ++q5) {
+                if (q5 >= D || last_par[q5] < 0) continue;
                 bool landed = false;
-                for (int it = 0; it < kSpinLimit && !landed; ++it) landed = mbar_try_wait(bar_full + 8 * ss[q3], uint32_t(pp[q3]));
+                for (int it = 0; it < kSpinLimit && !landed; ++it)
+                    landed = mbar_try_wait(bar_full + 8 * (c + kLutWarps * q5), uint32_t(last_par[q5]));
                 if (!landed) atomicExch(&g_lut_status, int(kWaitDrain));
             }
         }
@@ -430,12 +444,14 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         }
         if (ctid == 0 && wi == 0) TRACE(4);
         // Table address part of the lookups of step pair h: chunk 16 g + ((2h + 2j) mod 16) and the
-        // next one share bank 8 g + ((h + j) mod 8); the odd chunk sits 128 bytes further.
+        // next one share the 4-byte column 8 g + ((h + j) mod 8); the odd chunk is its upper half.
         uint32_t off[8];
 #pragma unroll
-        for (int h = 0; h < 8; ++h) off[h] = tab0 + uint32_t(b * kTableBytes + 4 * (8 * g4 + ((h + jr) & 7)));
-        // sum of x over this lane's group: the all-ones entries of the group's 16 chunks
-        float xsum = lds_f32<255 * 256>(off[0]) + lds_f32<255 * 256 + 128>(off[0]);
+        for (int h = 0; h < 8; ++h) off[h] = tab0 + uint32_t(b * 128 + 4 * (8 * g4 + ((h + jr) & 7)));
+        // sum of x over this lane's group: the all-ones entries of the group's 16 chunks (two per lane)
+        const uint32_t ones = lds_b32<255 * 256>(off[0]);
+        const float2 ones_f = __half22float2(*reinterpret_cast<const __half2 *>(&ones));
+        float xsum = ones_f.x + ones_f.y;
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
@@ -487,7 +503,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                             constexpr int i = decltype(I)::value;
                             constexpr int pb = st * Q + i;
                             const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
-                            sum[i][st & 1] += (st & 1) ? lds_f32<128>(addr) : lds_f32<0>(addr);
+                            lut_add<(st & 1) * 2>(sum[i][st & 1], addr);
                         });
                     });
                     float a = fmaf(__half2float(sc[Q]), xsum, acc[t]);
