@@ -13,7 +13,7 @@ namespace bcq {
 constexpr int kWindow = 512;        // weights along K covered by one lookup-table build
 constexpr int kUnitRows = 8;        // rows of one row unit
 constexpr int kGroupsPerWindow = 4; // 128-weight groups in a window
-constexpr int kLutWarps = 16;       // warps per block of the lookup-table kernel
+constexpr int kLutWarps = 24;       // warps per block of the lookup-table kernel
 constexpr int kLutUnitsPerWarp = 8; // row units a warp keeps accumulators for
 constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
 constexpr int kMaxWindowsPerBlock = 32; // windows one block may walk (bounds the planner's search)

@@ -45,6 +45,7 @@ constexpr int kLutSmemBytes = 232448;                              // 227 KB: th
 constexpr int kMaxSlotsPerWarp = 5;
 constexpr int kMaxSlots = kLutWarps * kMaxSlotsPerWarp;
 constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
+constexpr unsigned kProducerMask = (1u << kLutWarps) - 1u;   // producer lanes: one per consumer warp
 constexpr int kFixedBytes = 2048;      // barriers and flags
 constexpr int kProducerIdleLimit = 1 << 21;   // polling rounds without progress before the producer gives up
 constexpr int kSpinLimit = 1 << 20;   // tries per wait (each try blocks for a short, hardware-defined time)
@@ -392,8 +393,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                         issued = true;
                     }
                 }
-                if (__ballot_sync(0xFFFFu, remaining > 0) == 0) break;
-                if (__any_sync(0xFFFFu, issued)) {
+                if (__ballot_sync(kProducerMask, remaining > 0) == 0) break;
+                if (__any_sync(kProducerMask, issued)) {
                     idle = 0;
                     continue;
                 }
