@@ -3,16 +3,19 @@
 //   y = sum_g ( sum_i alpha_i (B_i x)_g + z (sum x)_g )          (Eq. bcw + Eq. fuse_step3)
 //
 // Per 512-wide window of K the block builds, in shared memory, all 2^8 signed sums of every
-// 8-activation chunk; packed weight bytes index those tables directly.  One block per SM, three
+// 8-activation chunk; packed weight bytes index those tables directly.  One block per SM, two
 // kinds of warps:
 //
-//   builders  (warps 0-2)   build the window tables from x, one window ahead of the consumers
+//   builders  (warps 0-3)   build the window tables from x, one window ahead of the consumers
 //                           (two tables, double buffered);
-//   producer  (warp 3)      16 lanes feed a ring of shared-memory slots with bulk async copies
-//                           (cp.async.bulk, completion on an mbarrier): per (window, row unit) one
-//                           slot = one tile = q*512 B of plane bytes + the unit's alphas and offsets;
-//   consumers (warps 4-19)  copy a filled slot into registers, hand the slot back, look every
-//                           weight byte up in the window table and accumulate in fp32.
+//   consumers (warps 4-27)  each owns a few shared-memory slots that it keeps filled with bulk
+//                           async copies (cp.async.bulk, completion on an mbarrier), one slot =
+//                           one tile = q*512 B of plane bytes + the unit's alphas and offsets of
+//                           one (window, row unit).  A consumer waits for its next tile, copies
+//                           it into registers, immediately re-uses the slot for the tile that
+//                           many jobs ahead, then looks every weight byte up in the window table
+//                           and accumulates in fp32.  (One warp can start only about 18 bulk
+//                           copies per microsecond: the copies have to be issued by many warps.)
 //
 // Tables.  The sums are computed in fp32 and stored as fp16 (one rounding, relative 2^-11; the
 // accumulation of the looked-up values stays fp32).  Halving the tables to 32 KB each is what
@@ -34,23 +37,20 @@
 
 namespace bcq {
 
-constexpr int kBuilderWarps = 3;
+constexpr int kBuilderWarps = 4;
 constexpr int kBuilderThreads = kBuilderWarps * 32;
-constexpr int kProducerWarp = kBuilderWarps;
-constexpr int kFirstConsumerWarp = kBuilderWarps + 1;
+constexpr int kFirstConsumerWarp = kBuilderWarps;
 constexpr int kConsumerThreads = kLutWarps * 32;
-constexpr int kLutThreads = (kBuilderWarps + 1 + kLutWarps) * 32;  // 640
+constexpr int kLutThreads = (kBuilderWarps + kLutWarps) * 32;      // 896
 constexpr int kTablesBytes = 256 * 256;                            // both fp16 tables, entry stride 256 B
 constexpr int kLutSmemBytes = 232448;                              // 227 KB: the per-block opt-in maximum
 constexpr int kMaxSlotsPerWarp = 5;
 constexpr int kMaxSlots = kLutWarps * kMaxSlotsPerWarp;
 constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
-constexpr unsigned kProducerMask = (1u << kLutWarps) - 1u;   // producer lanes: one per consumer warp
 constexpr int kFixedBytes = 2048;      // barriers and flags
-constexpr int kProducerIdleLimit = 1 << 21;   // polling rounds without progress before the producer gives up
 constexpr int kSpinLimit = 1 << 20;   // tries per wait (each try blocks for a short, hardware-defined time)
 
-static_assert(16 * kMaxSlots + 64 <= kFixedBytes, "barrier area");
+static_assert(8 * kMaxSlots + 64 <= kFixedBytes, "barrier area");
 static_assert(2 * kFixedBytes <= kLutSmemBytes - kTablesBytes, "barriers must fit before or after the tables");
 
 __device__ int g_lut_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
@@ -303,9 +303,9 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     auto slot_ptr = [&](int s) -> unsigned char * { return s < n_a ? ring_a + s * SL::kBytes : ring_b + (s - n_a) * SL::kBytes; };
 
     const uint32_t bars = smem_u32(fixed);
-    const uint32_t bar_full = bars, bar_empty = bars + 8 * kMaxSlots;
-    const uint32_t bar_tab_ready = bars + 16 * kMaxSlots, bar_tab_free = bar_tab_ready + 16;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 16 * kMaxSlots + 32);
+    const uint32_t bar_full = bars;
+    const uint32_t bar_tab_ready = bars + 8 * kMaxSlots, bar_tab_free = bar_tab_ready + 16;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 8 * kMaxSlots + 32);
     int *s_last = const_cast<int *>(abort_flag) + 1;
 
     if (tid == 0) {
@@ -315,7 +315,6 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 #endif
         for (int s = 0; s < kMaxSlots; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_tab_ready + 8 * b, kBuilderThreads);
@@ -331,14 +330,10 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     // =============================================================================================
     const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
-    if (warp != kProducerWarp) {
-        // ---- start-up: all warps but the producer build the first window's table ----------------
-        constexpr int kStartThreads = kLutThreads - 32;
-        const int sid = warp < kProducerWarp ? tid : tid - 32;
-        if (sid < 512) build_quad(tables, xblk, sid & 15, sid >> 4, 32);
-        named_barrier(1, kStartThreads);
-        if (sid == 0) TRACE(3);
-    }
+    // ---- start-up: everybody builds the first window's table -------------------------------------
+    if (tid < 512) build_quad(tables, xblk, tid & 15, tid >> 4, 32);
+    __syncthreads();
+    if (tid == 0) TRACE(3);
 
     if (warp < kBuilderWarps) {
         // ---- builders: one table per window, one window ahead of the consumers ----------------------
@@ -352,90 +347,41 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         return;
     }
 
-    if (warp == kProducerWarp) {
-        // ---- producer: one thread keeps the slot ring full ---------------------------------------
-        // Lane c feeds consumer warp c: slots c and c + 16 (+ 32) belong to that warp alone, so a
-        // slot's fills are consumed by one warp, in order, and a wait can never be satisfied by
-        // an older phase of the barrier.
-        if (lane < kLutWarps && !*abort_flag) {
-            const int c = lane;
-            const int mine = (V - c + kLutWarps - 1) / kLutWarps;  // units of warp c per window
-            int remaining = mine * nwin, t_in_win = 0, wi = 0, idle = 0;
-            size_t tile = size_t(w0) * p.U + u0 + c;
-            int d = 0, k = 0;
-            int last_par[kMaxSlotsPerWarp];   // parity of the last fill of each of this lane's slots, -1 = never filled
-#pragma unroll
-            for (int q5 = 0; q5 < kMaxSlotsPerWarp; ++q5) last_par[q5] = -1;
-            // The 16 lanes stay together in one polling loop and never block on a barrier, so
-            // each refills its warp's slot as soon as that slot is handed back.
-            while (true) {
-                bool issued = false;
-                if (remaining > 0) {
-                    const int s = c + kLutWarps * d;
-                    if (k == 0 || mbar_test_wait(bar_empty + 8 * s, (k - 1) & 1)) {
-                        const uint32_t dst = smem_u32(slot_ptr(s)), full = bar_full + 8 * s;
-                        mbar_expect_tx(full, SL::kBytes);
-                        bulk_g2s(dst, p.tiles + tile * SL::kBytes, SL::kBytes, full);   // planes + alphas + offsets
-#pragma unroll
-                        for (int q5 = 0; q5 < kMaxSlotsPerWarp; ++q5)
-                            if (q5 == d) last_par[q5] = k & 1;
-                        if (++d == D) {
-                            d = 0;
-                            ++k;
-                        }
-                        tile += kLutWarps;
-                        if (++t_in_win == mine) {
-                            t_in_win = 0;
-                            ++wi;
-                            tile = size_t(w0 + wi) * p.U + u0 + c;
-                        }
-                        --remaining;
-                        issued = true;
-                    }
-                }
-                if (__ballot_sync(kProducerMask, remaining > 0) == 0) break;
-                if (__any_sync(kProducerMask, issued)) {
-                    idle = 0;
-                    continue;
-                }
-                __nanosleep(100);   // nothing to refill: leave the issue slots to the consumers
-                if (++idle > kProducerIdleLimit || *abort_flag) {
-                    if (idle > kProducerIdleLimit) {
-                        *abort_flag = 1;
-                        atomicExch(&g_lut_status, int(kWaitEmpty));
-                    }
-                    break;
-                }
-            }
-            // See the last fill of each of this lane's slots land, with a bounded wait, before the
-            // warp leaves: the block's shared memory must not be handed to another block while copies
-            // into it are in flight, also when the consumers gave up.
-            if (lane == 0) TRACE(12);
-#pragma unroll
-            for (int q5 = 0; q5 < kMaxSlotsPerWarp; ++q5) {
-                if (q5 >= D || last_par[q5] < 0) continue;
-                bool landed = false;
-                for (int it = 0; it < kSpinLimit && !landed; ++it)
-                    landed = mbar_try_wait(bar_full + 8 * (c + kLutWarps * q5), uint32_t(last_par[q5]));
-                if (!landed) atomicExch(&g_lut_status, int(kWaitDrain));
-            }
-        }
-        return;
-    }
-
     // =============================================================================================
     // ---- consumers ---------------------------------------------------------------------------------
     // Lane l = 8 g + j owns row 8u + j of every unit and the g-th group of 128 weights of every
     // window: its 16q bytes of a tile are the group's 16 chunks (skewed by 2 j, see the layout), so
     // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
-    const int cw = warp - kFirstConsumerWarp;   // 0..15
+    const int cw = warp - kFirstConsumerWarp;   // 0 .. kLutWarps-1
     const int ctid = tid - kFirstConsumerWarp * 32;
     const int g4 = lane >> 3, jr = lane & 7;
     float acc[UMAX];
 #pragma unroll
     for (int t = 0; t < UMAX; ++t) acc[t] = 0.f;
     bool alive = !*abort_flag;
-    int d = 0, k = 0;   // this warp's ring position: slot cw + 16 d, fill number k
+    int d = 0, k = 0;   // this warp's ring position: slot cw + kLutWarps * d, fill number k
+
+    // This warp's jobs, in the order it consumes them: windows outermost, its units innermost.
+    // Lane 0 keeps D of them in flight; the issue cursor (iw, it) runs D jobs ahead.
+    const int mine = V > cw ? (V - cw + kLutWarps - 1) / kLutWarps : 0;   // units of this warp per window
+    const int total_jobs = mine * nwin;
+    int issued = 0, consumed = 0, iw = 0, it = 0;
+    auto issue_next = [&](int slot_d) {   // lane 0 only
+        if (issued < total_jobs) {
+            const size_t tile = size_t(w0 + iw) * p.U + u0 + cw + kLutWarps * it;
+            const int s = cw + kLutWarps * slot_d;
+            const uint32_t full = bar_full + 8 * s;
+            mbar_expect_tx(full, SL::kBytes);
+            bulk_g2s(smem_u32(slot_ptr(s)), p.tiles + tile * SL::kBytes, SL::kBytes, full);   // planes + alphas + offsets
+            ++issued;
+            if (++it == mine) {
+                it = 0;
+                ++iw;
+            }
+        }
+    };
+    if (lane == 0 && alive)
+        for (int q5 = 0; q5 < D; ++q5) issue_next(q5);
 
     for (int wi = 0; wi < nwin && alive; ++wi) {
         const int b = wi & 1;
@@ -471,6 +417,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                 if (!got) {
                     alive = false;
                 } else {
+                    ++consumed;
                     // slot -> registers, then hand the slot back to the producer
                     const unsigned char *slot = slot_ptr(s);
                     uint32_t wbuf[4 * Q];
@@ -492,8 +439,11 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 #pragma unroll
                         for (int i = 0; i <= Q; ++i) sc[i] = reinterpret_cast<const __half *>(sp)[i];
                     }
+                    // The tile is in registers: order those reads before the next copy into the slot
+                    // (generic-proxy reads, then an async-proxy write), then refill the slot.
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+                    if (lane == 0) issue_next(d);
 
                     float sum[Q][2];
 #pragma unroll
@@ -521,6 +471,17 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tab_free + 8 * b);
         if (ctid == 0 && wi < 4) TRACE(6 + wi);
+    }
+
+    // Gave up on a wait: copies this warp started may still be in flight.  See them land (bounded)
+    // before the block's shared memory can be handed to another block.
+    if (!alive && lane == 0) {
+        for (int m = consumed; m < issued; ++m) {
+            bool landed = false;
+            for (int itr = 0; itr < kSpinLimit && !landed; ++itr)
+                landed = mbar_try_wait(bar_full + 8 * (cw + kLutWarps * (m % D)), uint32_t((m / D) & 1));
+            if (!landed) atomicExch(&g_lut_status, int(kWaitDrain));
+        }
     }
 
     // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up, lanes 0..7 store ---------
