@@ -165,7 +165,7 @@ int bcq_repack(const bcq_desc *src, const void *packed_src_dev, const uint16_t *
  * y = W x at batch 1 (the definition at the top of this file; Eq. bcw + Eq. fuse_step3).
  * x [K], y [N] fp16.  y is overwritten.  workspace may be NULL when bcq_workspace_bytes is 0.
  * bcq_gemv_plan is the same product with an explicit decomposition (for tuning and tests):
- * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 128 row units (1024 rows)
+ * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 192 row units (1536 rows)
  * per row block and at most 32 windows (16384 weights along K) per K split.
  */
 int bcq_gemv(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,

@@ -211,10 +211,10 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
 // entry bits 3..7 (hi = hi0, hi0 + hi_step, ... < 32) walks the 8 entries sharing those bits in
 // Gray-code order: one packed fp32 FMA per entry and chunk pair, the four sums rounded to fp16 and
 // stored with one 64-bit store (16 quads = 128 contiguous bytes per entry: no bank conflicts).
-// `table` points at entry 0 of the buffer being built.
-__device__ __forceinline__ void build_quad(unsigned char *table, const __half *xw, int cq, int hi0, int hi_step)
+// `table` points at entry 0 of the buffer being built.  Loading (load_quad) and building are separate
+// so that a builder can have the next window's activations on their way while it waits for the buffer.
+__device__ __forceinline__ void load_quad(const __half *xw, int cq, f32x2 (&x01)[8], f32x2 (&x23)[8])
 {
-    f32x2 x01[8], x23[8];
     {
         float xf[4][8];
 #pragma unroll
@@ -234,6 +234,10 @@ __device__ __forceinline__ void build_quad(unsigned char *table, const __half *x
             x23[j] = pack2(xf[2][j], xf[3][j]);
         }
     }
+}
+__device__ __forceinline__ void build_quad(unsigned char *table, const f32x2 (&x01)[8], const f32x2 (&x23)[8], int cq, int hi0,
+                                           int hi_step)
+{
     const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
     f32x2 low01 = pack2(0.f, 0.f), low23 = low01;   // -(x0 + x1 + x2): entry bits 0..2 clear
 #pragma unroll
@@ -330,43 +334,14 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     // =============================================================================================
     const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
-    // ---- start-up: everybody builds the first window's table -------------------------------------
-    if (tid < 512) build_quad(tables, xblk, tid & 15, tid >> 4, 32);
-    __syncthreads();
-    if (tid == 0) TRACE(3);
-
-    if (warp < kBuilderWarps) {
-        // ---- builders: one table per window, one window ahead of the consumers ----------------------
-        mbar_arrive(bar_tab_ready);   // window 0 was built by everybody above
-        for (int wi = 1; wi < nwin; ++wi) {
-            const int b = wi & 1, use = wi >> 1;
-            if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree)) break;
-            build_quad(tables + b * 128, xblk + wi * kWindow, tid & 15, tid >> 4, kBuilderThreads / 16);
-            mbar_arrive(bar_tab_ready + 8 * b);
-        }
-        return;
-    }
-
-    // =============================================================================================
-    // ---- consumers ---------------------------------------------------------------------------------
-    // Lane l = 8 g + j owns row 8u + j of every unit and the g-th group of 128 weights of every
-    // window: its 16q bytes of a tile are the group's 16 chunks (skewed by 2 j, see the layout), so
-    // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
-    const int cw = warp - kFirstConsumerWarp;   // 0 .. kLutWarps-1
-    const int ctid = tid - kFirstConsumerWarp * 32;
-    const int g4 = lane >> 3, jr = lane & 7;
-    float acc[UMAX];
-#pragma unroll
-    for (int t = 0; t < UMAX; ++t) acc[t] = 0.f;
-    bool alive = !*abort_flag;
-    int d = 0, k = 0;   // this warp's ring position: slot cw + kLutWarps * d, fill number k
-
-    // This warp's jobs, in the order it consumes them: windows outermost, its units innermost.
-    // Lane 0 keeps D of them in flight; the issue cursor (iw, it) runs D jobs ahead.
-    const int mine = V > cw ? (V - cw + kLutWarps - 1) / kLutWarps : 0;   // units of this warp per window
+    // ---- consumer warps: job bookkeeping, and the first D tiles of each warp on their way -----------
+    // A warp's jobs, in the order it consumes them: windows outermost, its units innermost.  Lane 0
+    // keeps D of them in flight; the issue cursor (iw, it) runs D jobs ahead of the consumption.
+    const int cw = warp - kFirstConsumerWarp;   // 0 .. kLutWarps-1 for consumers, negative for builders
+    const int mine = (cw >= 0 && V > cw) ? (V - cw + kLutWarps - 1) / kLutWarps : 0;   // units of this warp per window
     const int total_jobs = mine * nwin;
     int issued = 0, consumed = 0, iw = 0, it = 0;
-    auto issue_next = [&](int slot_d) {   // lane 0 only
+    auto issue_next = [&](int slot_d) {   // lane 0 of a consumer warp only
         if (issued < total_jobs) {
             const size_t tile = size_t(w0 + iw) * p.U + u0 + cw + kLutWarps * it;
             const int s = cw + kLutWarps * slot_d;
@@ -380,8 +355,45 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             }
         }
     };
-    if (lane == 0 && alive)
+    if (cw >= 0 && lane == 0 && !*abort_flag)
         for (int q5 = 0; q5 < D; ++q5) issue_next(q5);
+
+    // ---- start-up: everybody builds the first window's table -------------------------------------
+    if (tid < 512) {
+        f32x2 x01[8], x23[8];
+        load_quad(xblk, tid & 15, x01, x23);
+        build_quad(tables, x01, x23, tid & 15, tid >> 4, 32);
+    }
+    __syncthreads();
+    if (tid == 0) TRACE(3);
+
+    if (warp < kBuilderWarps) {
+        // ---- builders: one table per window, one window ahead of the consumers ----------------------
+        mbar_arrive(bar_tab_ready);   // window 0 was built by everybody above
+        for (int wi = 1; wi < nwin; ++wi) {
+            const int b = wi & 1, use = wi >> 1;
+            f32x2 x01[8], x23[8];
+            load_quad(xblk + wi * kWindow, tid & 15, x01, x23);   // in flight while waiting for the buffer
+            if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree)) break;
+            build_quad(tables + b * 128, x01, x23, tid & 15, tid >> 4, kBuilderThreads / 16);
+            mbar_arrive(bar_tab_ready + 8 * b);
+        }
+        return;
+    }
+
+    // =============================================================================================
+    // ---- consumers ---------------------------------------------------------------------------------
+    // Lane l = 8 g + j owns row 8u + j of every unit and the g-th group of 128 weights of every
+    // window: its 16q bytes of a tile are the group's 16 chunks (skewed by 2 j, see the layout), so
+    // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
+    const int ctid = tid - kFirstConsumerWarp * 32;
+    const int g4 = lane >> 3, jr = lane & 7;
+    float acc[UMAX];
+#pragma unroll
+    for (int t = 0; t < UMAX; ++t) acc[t] = 0.f;
+    bool alive = !*abort_flag;
+    int d = 0, k = 0;   // this warp's ring position: slot cw + kLutWarps * d, fill number k
+
 
     for (int wi = 0; wi < nwin && alive; ++wi) {
         const int b = wi & 1;

@@ -130,7 +130,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert p.kernel == 1
     U, W = N // 8, K // 512
     assert 1 <= p.row_blocks <= U and 1 <= p.k_splits <= W
-    assert -(-U // p.row_blocks) <= 128 and -(-W // p.k_splits) <= 32
+    assert -(-U // p.row_blocks) <= 192 and -(-W // p.k_splits) <= 32
     blocks = p.row_blocks * p.k_splits
     if U * W >= 148 * 8:
         assert blocks >= 0.75 * 148
