@@ -48,7 +48,7 @@ constexpr int kMaxSlotsPerWarp = 5;
 constexpr int kMaxSlots = kLutWarps * kMaxSlotsPerWarp;
 constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
 constexpr int kFixedBytes = 2048;      // barriers and flags
-constexpr int kSpinLimit = 1 << 20;   // tries per wait (each try blocks for a short, hardware-defined time)
+constexpr int kSpinLimit = 1 << 22;   // polls per wait, about 32 ns apart: a wait gives up after roughly 0.2 s
 
 static_assert(8 * kMaxSlots + 64 <= kFixedBytes, "barrier area");
 static_assert(2 * kFixedBytes <= kLutSmemBytes - kTablesBytes, "barriers must fit before or after the tables");
@@ -140,9 +140,12 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)   
 // Bounded wait.  Returns false if the block is aborting (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code)
 {
+    // Poll without blocking and nap briefly in between: a warp suspended inside a blocking
+    // try_wait was seen to resume only about a microsecond after the phase had completed.
     for (int it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;   // sleeps in hardware until the phase completes or a short time-out
-        if ((it & 15) == 15 && *abort_flag) return false;
+        if (mbar_test_wait(bar, parity)) return true;
+        __nanosleep(32);
+        if ((it & 255) == 255 && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicExch(&g_lut_status, code);
@@ -369,7 +372,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     if (warp < kBuilderWarps) {
         // ---- builders: one table per window, one window ahead of the consumers ----------------------
-        mbar_arrive(bar_tab_ready);   // window 0 was built by everybody above
+        // Window 0 was built by everybody above (published by __syncthreads); the builders' fills of
+        // buffer 0 are windows 2, 4, ... and of buffer 1 windows 1, 3, ...
         for (int wi = 1; wi < nwin; ++wi) {
             const int b = wi & 1, use = wi >> 1;
             f32x2 x01[8], x23[8];
@@ -397,7 +401,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     for (int wi = 0; wi < nwin && alive; ++wi) {
         const int b = wi & 1;
-        if (!mbar_wait(bar_tab_ready + 8 * b, (wi >> 1) & 1, abort_flag, kWaitTableReady)) {
+        if (wi > 0 && !mbar_wait(bar_tab_ready + 8 * b, ((wi >> 1) - (b == 0 ? 1 : 0)) & 1, abort_flag, kWaitTableReady)) {
             alive = false;
             break;
         }
