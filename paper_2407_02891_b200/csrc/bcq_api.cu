@@ -54,18 +54,18 @@ bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED
 bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group != 0; }
 
 // Time model of the lookup-table kernel in nanoseconds, fitted to traces on B200: a fixed
-// start-up + tail, one "round" per 16 row units of a block per window (each consumer warp does one
-// unit), a floor of one round per window (the table build), and a split-K combine that grows with
-// the number of splits.  It ranks decompositions; it does not predict time exactly.
+// start-up + tail, a per-window overhead, one "round" per kLutWarps row units of a block per window
+// (each consumer warp does one tile), and a split-K combine that grows with the number of splits.
+// It ranks decompositions; it does not predict time exactly.
 long long lut_cost(int U, int W, int rb, int ks, int sm)
 {
-    const long long fixed = 4000, round = 890, per_split = 150;
+    const long long fixed = 4500, per_window = 700, round = 1200, per_split = 150;
     const long long waves = (static_cast<long long>(rb) * ks + sm - 1) / sm;
     const long long wc = (W + ks - 1) / ks;
     const long long units = (U + rb - 1) / rb;
     long long upw = (units + kLutWarps - 1) / kLutWarps;
     if (upw < 1) upw = 1;
-    return waves * (fixed + wc * upw * round + (ks > 1 ? per_split * ks : 0));
+    return waves * (fixed + wc * (per_window + upw * round) + (ks > 1 ? per_split * ks : 0));
 }
 
 int plan_lut(const bcq_desc *d, int sm, bcq_plan *out)

@@ -318,7 +318,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     if (tid == 0) {
         TRACE(0);
 #ifdef BCQ_TRACE
-        g_trace[blockIdx.x % 1024][13] = 0; g_trace[blockIdx.x % 1024][14] = 0;
+        g_trace[blockIdx.x % 1024][13] = 0; g_trace[blockIdx.x % 1024][14] = 0; g_trace[blockIdx.x % 1024][15] = 0;
 #endif
         for (int s = 0; s < kMaxSlots; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -401,10 +401,17 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     for (int wi = 0; wi < nwin && alive; ++wi) {
         const int b = wi & 1;
+#ifdef BCQ_TRACE
+        const unsigned long long tt0 = gtime();
+#endif
         if (wi > 0 && !mbar_wait(bar_tab_ready + 8 * b, ((wi >> 1) - (b == 0 ? 1 : 0)) & 1, abort_flag, kWaitTableReady)) {
             alive = false;
             break;
         }
+#ifdef BCQ_TRACE
+        if (ctid == 0) TRACE_ADD(15, gtime() - tt0);
+        if (ctid == 0 && wi == 0) TRACE(2);
+#endif
         if (ctid == 0 && wi == 0) TRACE(4);
         // Table address part of the lookups of step pair h: chunk 16 g + ((2h + 2j) mod 16) and the
         // next one share the 4-byte column 8 g + ((h + j) mod 8); the odd chunk is its upper half.
