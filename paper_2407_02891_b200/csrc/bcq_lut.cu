@@ -334,6 +334,10 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     }
     __syncthreads();
     if (tid == 0) TRACE(1);
+    // Programmatic dependent launch: the next kernel in the stream may start taking SMs as soon as
+    // this kernel's blocks leave them (it still waits, below, for its predecessor to finish before
+    // it reads x or writes anything).  Without the launch attribute both instructions do nothing.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // =============================================================================================
     const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
@@ -360,6 +364,10 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     };
     if (cw >= 0 && lane == 0 && !*abort_flag)
         for (int q5 = 0; q5 < D; ++q5) issue_next(q5);
+
+    // The weights above are constants; everything from here on (x, partial sums, counters, y) may
+    // depend on the previous kernel in the stream: wait for it to be complete and visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- start-up: everybody builds the first window's table -------------------------------------
     if (tid < 512) {
@@ -568,8 +576,17 @@ static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    lut_gemv_kernel<Q><<<prm.row_blocks * prm.k_splits, kLutThreads, kLutSmemBytes, st>>>(prm);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(prm.row_blocks * prm.k_splits);
+    cfg.blockDim = dim3(kLutThreads);
+    cfg.dynamicSmemBytes = kLutSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q>, prm);
 }
 
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
