@@ -63,7 +63,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 102
+#define BCQ_VERSION 103
 
 typedef enum bcq_status {
     BCQ_OK = 0,
