@@ -90,7 +90,7 @@ typedef struct bcq_desc {
 } bcq_desc;
 
 /* How a product is decomposed over the GPU.  kernel: 0 = generic (one warp per row; any valid
- * shape, either layout), 1 = lookup-table kernel (tiled layout, group 128) launched as
+ * shape, either layout), 1 = lookup-table kernel (tiled layout) launched as
  * row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace. */
 typedef struct bcq_plan {
     int32_t kernel;

@@ -48,7 +48,7 @@ int device_sm_count(int *out)
     return BCQ_OK;
 }
 
-bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group == 128; }
+bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED; }   // group 128 or one scale per row
 
 // tiled layout with grouped scales: alpha and z live inside `packed`
 bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group != 0; }

@@ -71,16 +71,18 @@ __device__ __forceinline__ unsigned long long gtime()
 #define TRACE_ADD(slot, v) do { } while (0)
 #endif
 
-template <int Q>
+// One tile = one ring slot.  GROUPED (group 128): planes + the tile's alphas and offsets;
+// otherwise (one scale per row) the planes only, alphas and offsets live in their own arrays.
+template <int Q, bool GROUPED>
 struct Slot {
     static constexpr int kPlaneBytes = Q * 512;
-    static constexpr int kAlphaBytes = Q * 64;
-    static constexpr int kOffsetBytes = 64;
-    static constexpr int kBytes = kPlaneBytes + kAlphaBytes + kOffsetBytes;
+    static constexpr int kBytes = kPlaneBytes + (GROUPED ? Q * 64 + 64 : 0);
 };
 
 struct LutParams {
-    const uint8_t *tiles;  // tiled operand: per (window, unit) planes, alphas, offsets
+    const uint8_t *tiles;  // tiled operand: per (window, unit) planes (+ alphas, offsets when grouped)
+    const __half *alpha;   // per-row scales only: [u][i][r]
+    const __half *z;       // per-row scales only: [u][r]
     const __half *x;
     __half *y;
     float *partial;  // [k_splits][N] when k_splits > 1
@@ -279,11 +281,12 @@ __device__ __forceinline__ void build_quad(unsigned char *table, const f32x2 (&x
 
 enum { kWaitEmpty = 1, kWaitFull = 2, kWaitTableReady = 3, kWaitTableFree = 4, kWaitDrain = 5, kTooFewSlots = 6 };
 
-template <int Q>
+template <int Q, bool GROUPED>
 __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    using SL = Slot<Q>;
+    using SL = Slot<Q, GROUPED>;
+    constexpr int NACC = GROUPED ? 1 : Q;   // accumulators per unit and lane: the row's sum, or one per plane
     constexpr int UMAX = kLutUnitsPerWarp;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -400,9 +403,12 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
     const int ctid = tid - kFirstConsumerWarp * 32;
     const int g4 = lane >> 3, jr = lane & 7;
-    float acc[UMAX];
+    float acc[UMAX][NACC];
+    float xacc = 0.f;   // per-row scales: sum of x over this lane's groups of all windows
 #pragma unroll
-    for (int t = 0; t < UMAX; ++t) acc[t] = 0.f;
+    for (int t = 0; t < UMAX; ++t)
+#pragma unroll
+        for (int i = 0; i < NACC; ++i) acc[t][i] = 0.f;
     bool alive = !*abort_flag;
     int d = 0, k = 0;   // this warp's ring position: slot cw + kLutWarps * d, fill number k
 
@@ -433,6 +439,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
+        xacc += xsum;
 
         static_for<0, UMAX>([&](auto T) {
             constexpr int t = decltype(T)::value;
@@ -461,14 +468,16 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                         wbuf[4 * j + 3] = v.w;
                     }
                     __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
-                    const unsigned char *sp = slot + SL::kPlaneBytes + lane * (2 * (Q + 1));
-                    if constexpr (Q == 3) {
-                        *reinterpret_cast<uint2 *>(sc) = *reinterpret_cast<const uint2 *>(sp);
-                    } else if constexpr (Q == 1) {
-                        *reinterpret_cast<uint32_t *>(sc) = *reinterpret_cast<const uint32_t *>(sp);
-                    } else {
+                    if constexpr (GROUPED) {
+                        const unsigned char *sp = slot + SL::kPlaneBytes + lane * (2 * (Q + 1));
+                        if constexpr (Q == 3) {
+                            *reinterpret_cast<uint2 *>(sc) = *reinterpret_cast<const uint2 *>(sp);
+                        } else if constexpr (Q == 1) {
+                            *reinterpret_cast<uint32_t *>(sc) = *reinterpret_cast<const uint32_t *>(sp);
+                        } else {
 #pragma unroll
-                        for (int i = 0; i <= Q; ++i) sc[i] = reinterpret_cast<const __half *>(sp)[i];
+                            for (int i = 0; i <= Q; ++i) sc[i] = reinterpret_cast<const __half *>(sp)[i];
+                        }
                     }
                     // The tile is in registers: order those reads before the next copy into the slot
                     // (generic-proxy reads, then an async-proxy write), then refill the slot.
@@ -488,10 +497,15 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                             lut_add<(st & 1) * 2>(sum[i][st & 1], addr);
                         });
                     });
-                    float a = fmaf(__half2float(sc[Q]), xsum, acc[t]);
+                    if constexpr (GROUPED) {
+                        float a = fmaf(__half2float(sc[Q]), xsum, acc[t][0]);
 #pragma unroll
-                    for (int i = 0; i < Q; ++i) a = fmaf(__half2float(sc[i]), sum[i][0] + sum[i][1], a);
-                    acc[t] = a;
+                        for (int i = 0; i < Q; ++i) a = fmaf(__half2float(sc[i]), sum[i][0] + sum[i][1], a);
+                        acc[t][0] = a;
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < Q; ++i) acc[t][i % NACC] += sum[i][0] + sum[i][1];
+                    }
                 }
                 if (++d == D) {
                     d = 0;
@@ -519,7 +533,17 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * p.N : nullptr;
 #pragma unroll
     for (int t = 0; t < UMAX; ++t) {
-        float v = acc[t];
+        float v = acc[t][0];
+        if constexpr (!GROUPED) {
+            // one scale per row: apply the row's alphas and offset to the sums over this block's K range
+            const int u = u0 + cw + kLutWarps * t;
+            v = 0.f;
+            if (u < u1) {
+#pragma unroll
+                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(p.alpha[(size_t(u) * Q + i) * kUnitRows + jr]), acc[t][i % NACC], v);
+                v = fmaf(__half2float(p.z[size_t(u) * kUnitRows + jr]), xacc, v);
+            }
+        }
         v += __shfl_xor_sync(0xffffffffu, v, 8);
         v += __shfl_xor_sync(0xffffffffu, v, 16);
         if (lane < 8 && cw + kLutWarps * t < V) {
@@ -562,7 +586,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     if (ctid == 0) TRACE(11);
 }
 
-template <int Q>
+template <int Q, bool GROUPED>
 static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
 {
     // The opt-in to more than 48 KB of dynamic shared memory is per function and per device:
@@ -572,7 +596,7 @@ static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(lut_gemv_kernel<Q>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
+        e = cudaFuncSetAttribute(lut_gemv_kernel<Q, GROUPED>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
@@ -586,7 +610,7 @@ static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q>, prm);
+    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, GROUPED>, prm);
 }
 
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
@@ -594,8 +618,8 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
 {
     LutParams prm;
     prm.tiles = static_cast<const uint8_t *>(packed);
-    (void)alpha;
-    (void)z;
+    prm.alpha = reinterpret_cast<const __half *>(alpha);   // used with per-row scales only
+    prm.z = reinterpret_cast<const __half *>(z);
     prm.x = reinterpret_cast<const __half *>(x);
     prm.y = reinterpret_cast<__half *>(y);
     prm.counters = static_cast<int *>(workspace);
@@ -606,11 +630,12 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
     prm.W = d.K / kWindow;
     prm.row_blocks = plan.row_blocks;
     prm.k_splits = plan.k_splits;
+    const bool grouped = d.group != 0;
     switch (d.q) {
-        case 1: return launch_lut_q<1>(prm, st);
-        case 2: return launch_lut_q<2>(prm, st);
-        case 3: return launch_lut_q<3>(prm, st);
-        case 4: return launch_lut_q<4>(prm, st);
+        case 1: return grouped ? launch_lut_q<1, true>(prm, st) : launch_lut_q<1, false>(prm, st);
+        case 2: return grouped ? launch_lut_q<2, true>(prm, st) : launch_lut_q<2, false>(prm, st);
+        case 3: return grouped ? launch_lut_q<3, true>(prm, st) : launch_lut_q<3, false>(prm, st);
+        case 4: return grouped ? launch_lut_q<4, true>(prm, st) : launch_lut_q<4, false>(prm, st);
     }
     return cudaErrorInvalidValue;
 }

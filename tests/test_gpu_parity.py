@@ -166,7 +166,10 @@ def test_gemv_generic_kernel(N, K, q, group):
 
 
 LUT_SHAPES = [(1024, 1024, 3, 128), (8, 512, 3, 128), (296, 2048, 3, 128), (1000, 1536, 2, 128),
-              (520, 3584, 3, 128), (64, 1024, 1, 128), (136, 1024, 4, 128), (4096, 4096, 3, 128)]
+              (520, 3584, 3, 128), (64, 1024, 1, 128), (136, 1024, 4, 128), (4096, 4096, 3, 128),
+              # one scale per row (the paper's granularity)
+              (1024, 1024, 2, 0), (8, 512, 3, 0), (296, 2048, 2, 0), (520, 3584, 3, 0), (136, 1024, 4, 0),
+              (64, 1024, 1, 0), (2304, 9216, 2, 0)]
 
 
 @pytest.mark.parametrize("N,K,q,group", LUT_SHAPES)
@@ -178,14 +181,16 @@ def test_gemv_lut_kernel_default_plan(N, K, q, group):
     assert rel_err(run_gemv(L, x), ref) <= TOL
 
 
+@pytest.mark.parametrize("group", [128, 0])
 @pytest.mark.parametrize("N,K,q,rb,ks", [(520, 3584, 3, 2, 1), (520, 3584, 3, 2, 7), (520, 3584, 3, 3, 2),
                                          (520, 3584, 3, 65, 3), (520, 3584, 3, 5, 4), (512, 1024, 2, 1, 1),
-                                         (512, 1024, 2, 1, 2), (1000, 1536, 2, 125, 3), (1000, 1536, 2, 2, 1)])
-def test_gemv_lut_kernel_explicit_plans(N, K, q, rb, ks):
+                                         (512, 1024, 2, 1, 2), (1000, 1536, 2, 125, 3), (1000, 1536, 2, 2, 1),
+                                         (1600, 1024, 3, 1, 2), (4000, 512, 2, 3, 1)])
+def test_gemv_lut_kernel_explicit_plans(N, K, q, rb, ks, group):
     """Ragged row blocks, one and several windows per block, with and without split-K."""
-    p, codes, alpha, z, x = make_layer(f"lutp/{N}x{K}", N, K, q, 128)
-    ref = oracle.forward_planes(p, alpha, z, x, 128)[0]
-    L = gpu_layer(N, K, q, 128, bq.LAYOUT_TILED, codes, alpha, z)
+    p, codes, alpha, z, x = make_layer(f"lutp/{N}x{K}", N, K, q, group)
+    ref = oracle.forward_planes(p, alpha, z, x, group)[0]
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
     assert rel_err(run_gemv(L, x, bq.Plan(1, rb, ks, 0)), ref) <= TOL
 
 

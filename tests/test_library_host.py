@@ -138,3 +138,4 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
     assert bq.plan_default(d, 4, 148).kernel == 0
+    assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
