@@ -185,7 +185,7 @@ def test_gemv_lut_kernel_default_plan(N, K, q, group):
 @pytest.mark.parametrize("N,K,q,rb,ks", [(520, 3584, 3, 2, 1), (520, 3584, 3, 2, 7), (520, 3584, 3, 3, 2),
                                          (520, 3584, 3, 65, 3), (520, 3584, 3, 5, 4), (512, 1024, 2, 1, 1),
                                          (512, 1024, 2, 1, 2), (1000, 1536, 2, 125, 3), (1000, 1536, 2, 2, 1),
-                                         (1600, 1024, 3, 1, 2), (4000, 512, 2, 3, 1)])
+                                         (1536, 1024, 3, 1, 2), (4000, 512, 2, 3, 1)])
 def test_gemv_lut_kernel_explicit_plans(N, K, q, rb, ks, group):
     """Ragged row blocks, one and several windows per block, with and without split-K."""
     p, codes, alpha, z, x = make_layer(f"lutp/{N}x{K}", N, K, q, group)
