@@ -31,6 +31,9 @@ WORKLOADS = {
     "opt6.7b_q3_g128": dict(hidden=4096, ffn=16384, layers=32, q=3, group=128),
     "opt66b_q2_g128": dict(hidden=9216, ffn=36864, layers=64, q=2, group=128),
     "opt66b_q2_row": dict(hidden=9216, ffn=36864, layers=64, q=2, group=0),
+    # Llama-2-70B-shaped layers (GQA: fused k/v of 2 x 1024 rows, gated FFN); 8 of them so that the
+    # operands (3 GB) are far larger than L2.  Use --batch 1|2|4|8|16 for the small-batch sweep.
+    "llama70b_q3_g128": dict(family="llama", hidden=8192, ffn=28672, kv=2048, layers=8, q=3, group=128),
 }
 DEFAULT_WORKLOAD = "opt30b_q3_g128"
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
@@ -41,8 +44,10 @@ UNIT = "us/token"
 
 
 def layer_shapes(w):
-    """(name, N, K) of the six linear layers of one OPT decoder layer."""
+    """(name, N, K) of the six linear layers of one decoder layer (OPT, or Llama-2 with GQA)."""
     h, f = w["hidden"], w["ffn"]
+    if w.get("family") == "llama":
+        return [("q", h, h), ("kv", w["kv"], h), ("o", h, h), ("gate", f, h), ("up", f, h), ("down", h, f)]
     return [("q", h, h), ("k", h, h), ("v", h, h), ("out", h, h), ("fc1", f, h), ("fc2", h, f)]
 
 
@@ -127,12 +132,12 @@ def physical_gpu_index(local: int) -> int:
 class Stack:
     """All packed layers of the workload, resident on one GPU, plus per-shape x and per-layer y."""
 
-    def __init__(self, wname, w, device):
+    def __init__(self, wname, w, device, B=1):
         import torch
         from paper_2407_02891_b200 import binding as bq
 
         self.bq, self.torch, self.device = bq, torch, device
-        self.w, self.wname = w, wname
+        self.w, self.wname, self.B = w, wname, B
         q, group = w["q"], w["group"]
         self.items = []       # (desc, packed, alpha, z, x, y, ws)
         self.bytes = 0
@@ -143,7 +148,7 @@ class Stack:
             a, z = synth.scale_rows(f"{wname}/{N}x{K}", N, K, q, group)
             dt = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
             scales[(N, K)] = (torch.from_numpy(a).to(device), torch.from_numpy(z).to(device))
-            xs[(N, K)] = torch.from_numpy(synth.activations(f"{wname}/{N}x{K}", 1, K).reshape(-1)).to(device)
+            xs[(N, K)] = torch.from_numpy(synth.activations(f"{wname}/{N}x{K}", B, K).reshape(-1)).to(device)
             wss[(N, K)] = bq.new_workspace(dt, 1, device=device)
         self.x_host = {k: v.cpu() for k, v in xs.items()}
         for layer in range(w["layers"]):
@@ -154,16 +159,22 @@ class Stack:
                 ad, zd = scales[(N, K)]
                 packed, at, zt = bq.empty_operands(dt, device)      # every layer owns its operands
                 bq.repack(dc, canon, ad, zd, dt, packed, at, zt)
-                y = torch.zeros(N, dtype=torch.float16, device=device)
+                y = torch.zeros(B * N, dtype=torch.float16, device=device)
                 self.items.append((dt, packed, at, zt, xs[(N, K)], y, wss[(N, K)], (N, K)))
-                self.bytes += algorithmic_bytes(N, K, q, group)
+                self.bytes += algorithmic_bytes(N, K, q, group, B)
             torch.cuda.synchronize(device)
         self.graph = None
 
+    def launch_one(self, it):
+        (d, packed, a, z, x, y, ws, _) = it
+        if self.B == 1:
+            self.bq.gemv(d, packed, a, z, x, y, ws)
+        else:
+            self.bq.gemm_smallbatch(d, packed, a, z, x, y, self.B, ws)
+
     def launch_all(self):
-        bq = self.bq
-        for (d, packed, a, z, x, y, ws, _) in self.items:
-            bq.gemv(d, packed, a, z, x, y, ws)
+        for it in self.items:
+            self.launch_one(it)
 
     def capture(self):
         torch = self.torch
@@ -199,14 +210,14 @@ class Stack:
             for _ in range(reps):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                for (d, packed, a, z, x, y, ws, _) in its:
-                    self.bq.gemv(d, packed, a, z, x, y, ws)
+                for it in its:
+                    self.launch_one(it)
                 e1.record()
                 e1.synchronize()
                 t = e0.elapsed_time(e1) * 1e3 / len(its)
                 best = t if best is None else min(best, t)
             N, K = s
-            b = algorithmic_bytes(N, K, self.w["q"], self.w["group"])
+            b = algorithmic_bytes(N, K, self.w["q"], self.w["group"], self.B)
             out[f"{N}x{K}"] = {"us": round(best, 3), "gbs": round(b / best * 1e-3, 1), "launches": len(its)}
         return out
 
@@ -285,6 +296,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--batch", type=int, default=1, help="activation vectors per product (1..16)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of decoder layers (profiling)")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: plain launches instead of a CUDA graph, warm-up as given, "
@@ -297,8 +309,10 @@ def main():
     w = dict(WORKLOADS[args.workload])
     if args.layers > 0:
         w["layers"] = args.layers
-    config = {"workload": args.workload, "shapes": "4x(h x h), ffn x h, h x ffn per layer", "hidden": w["hidden"],
-              "ffn": w["ffn"], "layers": w["layers"], "q": w["q"], "group": w["group"], "batch": 1,
+    config = {"workload": args.workload,
+              "shapes": ", ".join(f"{n}:{N}x{K}" for (n, N, K) in layer_shapes(w)) + " per layer",
+              "hidden": w["hidden"], "ffn": w["ffn"], "layers": w["layers"], "q": w["q"], "group": w["group"],
+              "batch": args.batch,
               "cache": "inputs larger than L2 (every launch reads its own weights)", "parallelism": "replicas only"}
 
     if args.impl == "reference":
@@ -336,7 +350,7 @@ def main():
     from paper_2407_02891_b200 import binding as bq
     bq.lib()   # fail loudly if the CUDA library is missing
 
-    stack = Stack(args.workload, w, device)
+    stack = Stack(args.workload, w, device, args.batch)
     if args.profile:
         for _ in range(args.warmup):
             stack.launch_all()
@@ -370,7 +384,7 @@ def main():
 
     per_shape = stack.per_shape_us()
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and args.batch == 1:
         e_ms, h2d, d2h = stack.e2e_steps(max(3, min(args.steps, 20)))
         if world > 1:
             t = torch.tensor([e_ms], device=device)
@@ -398,13 +412,15 @@ def main():
                      "peak_kind": peak_kind,
                      "traffic": (NCU_TRAFFIC["bytes_per_launch"]
                                  if bq.lib().bcq_version() == NCU_TRAFFIC["lib_version"]
-                                 and args.workload == NCU_TRAFFIC["workload"] and args.layers == 0 else None), "kernel": f"lut_gemv_kernel<{w['q']}>",
+                                 and args.workload == NCU_TRAFFIC["workload"] and args.layers == 0
+                                 and args.batch == 1 else None),
+                     "kernel": f"lut_gemv_kernel<{w['q']}>" if args.batch == 1 else "bcq_gemm_smallbatch kernels",
                      "algorithmic_bytes_per_launch": stack.bytes // launches_per_step,
                      "launches_per_step": launches_per_step},
         "per_shape": per_shape,
         "e2e": e2e,
     }
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and args.batch == 1:
         smp = OracleSample(args.workload, w)
         v, sample = smp.us_per_token()
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": sample}
