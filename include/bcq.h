@@ -177,8 +177,10 @@ int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed
 
 /*
  * Y[b] = W X[b] for b < B, 1 <= B <= 16; X [B][K], Y [B][N] row-major fp16.  Every column is
- * an independent product (the paper defines batch 1 only); the packed weights are read
- * once for all columns.  B == 1 is bcq_gemv.
+ * an independent product (the paper defines batch 1 only), bit-identical to bcq_gemv on that
+ * column.  B == 1 is bcq_gemv.  Tiled layout: the lookup-table kernel runs once per column
+ * (B passes over the packed weights; workspace as for bcq_gemv, X rows must be 16-byte
+ * aligned, i.e. K % 8 == 0).  Canonical layout: one pass of the generic kernel for all columns.
  */
 int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
                         const uint16_t *z_dev, const uint16_t *X_dev, uint16_t *Y_dev, int B,

@@ -190,7 +190,7 @@ int bcq_plan_default(const bcq_desc *desc, int B, int sm_count, bcq_plan *out)
     out->row_blocks = (desc->N + 7) / 8;
     out->k_splits = 1;
     out->reserved = 0;
-    if (B == 1 && lut_kernel_covers(desc)) {
+    if (lut_kernel_covers(desc)) {   // batches run the batch-1 kernel column by column
         if (sm_count <= 0) {
             rc = device_sm_count(&sm_count);
             if (rc != BCQ_OK) return rc;
@@ -352,6 +352,19 @@ int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed, const uint16_t
         return BCQ_ERR_INVALID_ARG;
     if (!aligned(packed, 16) || !aligned(alpha, 16) || !aligned(z, 16) || !aligned(X, 16) || !aligned(Y, 2))
         return BCQ_ERR_MISALIGNED;
+    if (lut_kernel_covers(desc)) {
+        // The lookup-table kernel once per column: B passes over the weights, each at the batch-1
+        // rate, which is far ahead of the generic kernel's direct sign arithmetic.
+        bcq_plan plan;
+        rc = bcq_plan_default(desc, 1, 0, &plan);
+        if (rc != BCQ_OK) return rc;
+        for (int b = 0; b < B; ++b) {
+            rc = run_gemv(desc, &plan, packed, alpha, z, X + size_t(b) * desc->K, Y + size_t(b) * desc->N, ws, ws_bytes,
+                          stream);
+            if (rc != BCQ_OK) return rc;
+        }
+        return BCQ_OK;
+    }
     cudaError_t e = launch_generic(*desc, packed, alpha, z, X, Y, B, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }

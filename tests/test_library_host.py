@@ -137,5 +137,5 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * N * 4)
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
-    assert bq.plan_default(d, 4, 148).kernel == 0
+    assert bq.plan_default(d, 4, 148).kernel == 1         # batches run the same kernel per column
     assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
