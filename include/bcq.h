@@ -40,8 +40,8 @@
  * K/512 windows, `packed` is a sequence of tiles, tile (w, u) at byte (w*U + u) * T.  Inside a
  * tile, lane l = 8 g + j (g < 4, j < 8) stands for row 8u + j and the g-th group of 128 weights
  * of window w:
- *   bytes [0, q*512)      planes as [jq < q][lane < 32][16 bytes]; byte p = 16 jq + (byte in lane)
- *                         = s*q + i  (s < 16) holds plane i of the 8 weights
+ *   bytes [0, q*512)      planes as [i < q][lane < 32][s < 16]: byte s of lane l in plane i holds
+ *                         plane i of the 8 weights
  *                         k = 512 w + 128 g + 8 ((s + 2 j) mod 16) .. + 7   (bit order as canonical)
  *   group 128, T = q*576 + 64: the tile continues with the lanes' scales,
  *     bytes [q*512, T)    fp16 [lane < 32][alpha_0 .. alpha_{q-1}, z]
@@ -63,7 +63,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 103
+#define BCQ_VERSION 104
 
 typedef enum bcq_status {
     BCQ_OK = 0,
@@ -90,8 +90,11 @@ typedef struct bcq_desc {
 } bcq_desc;
 
 /* How a product is decomposed over the GPU.  kernel: 0 = generic (one warp per row; any valid
- * shape, either layout), 1 = lookup-table kernel (tiled layout) launched as
- * row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace. */
+ * shape, either layout), 1 = lookup-table kernel (tiled layout, one column per launch),
+ * 2 = tensor-core small-batch kernel (tiled layout, 2..16 columns per launch); kernels 1 and 2
+ * are launched as row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace.
+ * Limits: at most 192 (kernel 1) or 176 (kernel 2) row units of 8 rows per block, at most 32
+ * windows of 512 weights per K split. */
 typedef struct bcq_plan {
     int32_t kernel;
     int32_t row_blocks;
@@ -177,14 +180,22 @@ int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed
 
 /*
  * Y[b] = W X[b] for b < B, 1 <= B <= 16; X [B][K], Y [B][N] row-major fp16.  Every column is
- * an independent product (the paper defines batch 1 only), bit-identical to bcq_gemv on that
- * column.  B == 1 is bcq_gemv.  Tiled layout: the lookup-table kernel runs once per column
- * (B passes over the packed weights; workspace as for bcq_gemv, X rows must be 16-byte
- * aligned, i.e. K % 8 == 0).  Canonical layout: one pass of the generic kernel for all columns.
+ * an independent product (the paper defines batch 1 only; Eq. bcw + Eq. fuse_step3 per column).
+ * B == 1 is bcq_gemv.  Tiled layout, B >= 2: ONE pass over the packed weights for all columns
+ * (tensor-core kernel: a weight bit becomes the fp16 value +-alpha of its row and group, the
+ * products with x are exact, all sums fp32; the offset term uses the fp32 group sums of x,
+ * kept to 22 bits).  The workspace depends on B: bcq_workspace_bytes(desc, B, plan).
+ * Canonical layout: one pass of the generic kernel for all columns.
+ * bcq_gemm_smallbatch_plan takes the decomposition from the caller; a plan with kernel 1 runs
+ * the lookup-table kernel once per column (B passes, workspace as for bcq_gemv).
  */
 int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
                         const uint16_t *z_dev, const uint16_t *X_dev, uint16_t *Y_dev, int B,
                         void *workspace_dev, size_t workspace_bytes, void *stream);
+int bcq_gemm_smallbatch_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed_dev,
+                             const uint16_t *alpha_dev, const uint16_t *z_dev, const uint16_t *X_dev,
+                             uint16_t *Y_dev, int B, void *workspace_dev, size_t workspace_bytes,
+                             void *stream);
 
 /*
  * bcq_gemv with the activation and the result in HOST memory: enqueues x_host -> x_stage_dev,

@@ -78,6 +78,7 @@ SIGNATURES = {
     "bcq_gemv": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemm_smallbatch": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
+    "bcq_gemm_smallbatch_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "bcq_gemv_host": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_noalloc": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bcq_poll_status": (_i, []),
@@ -216,6 +217,13 @@ def gemm_smallbatch(d: Desc, packed, alpha, z, X, Y, B: int, workspace=None):
     wp, wn = _ws_args(workspace)
     _check(lib().bcq_gemm_smallbatch(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(X), _ptr(Y), B,
                                      wp, wn, _stream()), "bcq_gemm_smallbatch")
+
+
+def gemm_smallbatch_plan(d: Desc, plan: Plan, packed, alpha, z, X, Y, B: int, workspace=None):
+    _dev(packed, alpha, z, X, Y)
+    wp, wn = _ws_args(workspace)
+    _check(lib().bcq_gemm_smallbatch_plan(ctypes.byref(d), ctypes.byref(plan), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(X),
+                                          _ptr(Y), B, wp, wn, _stream()), "bcq_gemm_smallbatch_plan")
 
 
 def gemv_host(d: Desc, packed, alpha, z, x_host, y_host, x_stage, y_stage, workspace=None):

@@ -48,6 +48,8 @@ int device_sm_count(int *out)
     return BCQ_OK;
 }
 
+constexpr int kSmallBatchMin = 2;   // from this many columns on the default plan is the tensor-core kernel
+
 bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED; }   // group 128 or one scale per row
 
 // tiled layout with grouped scales: alpha and z live inside `packed`
@@ -90,21 +92,61 @@ int plan_lut(const bcq_desc *d, int sm, bcq_plan *out)
     return best < 0 ? BCQ_ERR_UNSUPPORTED_SHAPE : BCQ_OK;
 }
 
-int check_plan(const bcq_desc *d, const bcq_plan *p)
+// The same kind of model for the small-batch kernel: a round is one pair of row units per consumer
+// warp (kMmaWarps pairs per block and window).
+long long mma_cost(int U, int W, int rb, int ks, int sm, int B)
+{
+    const long long fixed = 5000, per_window = 400, round = B > 8 ? 5200 : 3600, per_split = 150LL * (B > 4 ? 2 : 1);
+    const long long waves = (static_cast<long long>(rb) * ks + sm - 1) / sm;
+    const long long wc = (W + ks - 1) / ks;
+    const long long pairs = ((U + rb - 1) / rb + 1) / 2;
+    long long rounds = (pairs + kMmaWarps - 1) / kMmaWarps;
+    if (rounds < 1) rounds = 1;
+    return waves * (fixed + wc * (per_window + rounds * round) + (ks > 1 ? per_split * ks : 0));
+}
+
+int plan_mma(const bcq_desc *d, int sm, int B, bcq_plan *out)
+{
+    const int U = d->N / kUnitRows, W = d->K / kWindow;
+    const int rb_min = (U + kMmaMaxUnitsPerBlock - 1) / kMmaMaxUnitsPerBlock;
+    long long best = -1;
+    for (int ks = (W + kMaxWindowsPerBlock - 1) / kMaxWindowsPerBlock; ks <= W && ks <= 64; ++ks) {
+        for (int k = 0; k <= 16; ++k) {
+            int rb = k == 0 ? rb_min : (k * sm) / ks;
+            if (rb < rb_min || rb > U || rb > kMaxRowBlocks) continue;
+            const long long c = mma_cost(U, W, rb, ks, sm, B);
+            if (best < 0 || c < best) {
+                best = c;
+                out->kernel = 2;
+                out->row_blocks = rb;
+                out->k_splits = ks;
+                out->reserved = 0;
+            }
+        }
+    }
+    return best < 0 ? BCQ_ERR_UNSUPPORTED_SHAPE : BCQ_OK;
+}
+
+// B: the number of columns the plan is for (kernel 1 handles one column per launch, kernel 2 needs 2..16)
+int check_plan(const bcq_desc *d, const bcq_plan *p, int B)
 {
     if (p->kernel == 0) return BCQ_OK;
-    if (p->kernel != 1 || !lut_kernel_covers(d)) return BCQ_ERR_INVALID_ARG;
+    if ((p->kernel != 1 && p->kernel != 2) || !lut_kernel_covers(d)) return BCQ_ERR_INVALID_ARG;
+    if (p->kernel == 2 && B < 2) return BCQ_ERR_INVALID_ARG;
     const int U = d->N / kUnitRows, W = d->K / kWindow;
+    const int max_units = p->kernel == 1 ? kMaxUnitsPerBlock : kMmaMaxUnitsPerBlock;
     if (p->row_blocks < 1 || p->row_blocks > U || p->row_blocks > kMaxRowBlocks) return BCQ_ERR_INVALID_ARG;
     if (p->k_splits < 1 || p->k_splits > W) return BCQ_ERR_INVALID_ARG;
     if ((W + p->k_splits - 1) / p->k_splits > kMaxWindowsPerBlock) return BCQ_ERR_INVALID_ARG;
-    if ((U + p->row_blocks - 1) / p->row_blocks > kMaxUnitsPerBlock) return BCQ_ERR_INVALID_ARG;
+    if ((U + p->row_blocks - 1) / p->row_blocks > max_units) return BCQ_ERR_INVALID_ARG;
     return BCQ_OK;
 }
 
-size_t plan_workspace(const bcq_desc *d, const bcq_plan *p)
+size_t plan_workspace(const bcq_desc *d, const bcq_plan *p, int B)
 {
-    if (p->kernel == 1 && p->k_splits > 1) return kCounterBytes + size_t(p->k_splits) * d->N * sizeof(float);
+    if (p->k_splits <= 1) return 0;
+    if (p->kernel == 1) return kCounterBytes + size_t(p->k_splits) * d->N * sizeof(float);
+    if (p->kernel == 2) return kCounterBytes + size_t(p->k_splits) * B * d->N * sizeof(float);
     return 0;
 }
 
@@ -123,7 +165,7 @@ int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, con
     if (plan->kernel == 0) {
         e = launch_generic(*desc, packed, alpha, z, x, y, 1, st);
     } else {
-        const size_t need = plan_workspace(desc, plan);
+        const size_t need = plan_workspace(desc, plan, 1);
         if (need > 0) {
             if (!ws) return BCQ_ERR_INVALID_ARG;
             if (!aligned(ws, 16)) return BCQ_ERR_MISALIGNED;
@@ -160,10 +202,13 @@ const char *bcq_status_string(int s)
 int bcq_poll_status(void)
 {
     int v = 0;
+    int w = 0;
     cudaError_t e = lut_status_take(&v);
+    if (e == cudaSuccess) e = mma_status_take(&w);
     if (e != cudaSuccess) return cuda_fail(e);
-    if (v != 0) {
-        snprintf(g_cuda_error, sizeof(g_cuda_error), "lut_gemv_kernel: bounded wait %d ran out", v);
+    if (v != 0 || w != 0) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: bounded wait %d ran out", v ? "lut_gemv_kernel" : "mma_gemm_kernel",
+                 v ? v : w);
         return BCQ_ERR_TIMEOUT;
     }
     return BCQ_OK;
@@ -190,12 +235,12 @@ int bcq_plan_default(const bcq_desc *desc, int B, int sm_count, bcq_plan *out)
     out->row_blocks = (desc->N + 7) / 8;
     out->k_splits = 1;
     out->reserved = 0;
-    if (lut_kernel_covers(desc)) {   // batches run the batch-1 kernel column by column
+    if (lut_kernel_covers(desc)) {
         if (sm_count <= 0) {
             rc = device_sm_count(&sm_count);
             if (rc != BCQ_OK) return rc;
         }
-        return plan_lut(desc, sm_count, out);
+        return B < kSmallBatchMin ? plan_lut(desc, sm_count, out) : plan_mma(desc, sm_count, B, out);
     }
     return BCQ_OK;
 }
@@ -208,7 +253,8 @@ size_t bcq_workspace_bytes(const bcq_desc *desc, int B, const bcq_plan *plan)
         if (bcq_plan_default(desc, B, 0, &def) != BCQ_OK) return 0;
         plan = &def;
     }
-    return plan_workspace(desc, plan);
+    if (B < 1 || B > 16 || check_plan(desc, plan, B) != BCQ_OK) return 0;
+    return plan_workspace(desc, plan, B);
 }
 
 int bcq_workspace_init(void *ws, size_t bytes, void *stream)
@@ -324,7 +370,7 @@ int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed
     int rc = check_desc(desc);
     if (rc != BCQ_OK) return rc;
     if (!plan) return BCQ_ERR_INVALID_ARG;
-    rc = check_plan(desc, plan);
+    rc = check_plan(desc, plan, 1);
     if (rc != BCQ_OK) return rc;
     return run_gemv(desc, plan, packed, alpha, z, x, y, ws, ws_bytes, stream);
 }
@@ -338,13 +384,15 @@ int bcq_gemv(const bcq_desc *desc, const void *packed, const uint16_t *alpha, co
     return run_gemv(desc, &plan, packed, alpha, z, x, y, ws, ws_bytes, stream);
 }
 
-int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z,
-                        const uint16_t *X, uint16_t *Y, int B, void *ws, size_t ws_bytes, void *stream)
+int bcq_gemm_smallbatch_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed, const uint16_t *alpha,
+                             const uint16_t *z, const uint16_t *X, uint16_t *Y, int B, void *ws, size_t ws_bytes,
+                             void *stream)
 {
     int rc = check_desc(desc);
     if (rc != BCQ_OK) return rc;
-    if (B < 1 || B > 16) return BCQ_ERR_INVALID_ARG;
-    if (B == 1) return bcq_gemv(desc, packed, alpha, z, X, Y, ws, ws_bytes, stream);
+    if (!plan || B < 1 || B > 16) return BCQ_ERR_INVALID_ARG;
+    rc = check_plan(desc, plan, B);
+    if (rc != BCQ_OK) return rc;
     if (!packed || !X || !Y) return BCQ_ERR_INVALID_ARG;
     if (interleaved(desc))
         alpha = z = nullptr;
@@ -352,21 +400,37 @@ int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed, const uint16_t
         return BCQ_ERR_INVALID_ARG;
     if (!aligned(packed, 16) || !aligned(alpha, 16) || !aligned(z, 16) || !aligned(X, 16) || !aligned(Y, 2))
         return BCQ_ERR_MISALIGNED;
-    if (lut_kernel_covers(desc)) {
-        // The lookup-table kernel once per column: B passes over the weights, each at the batch-1
-        // rate, which is far ahead of the generic kernel's direct sign arithmetic.
-        bcq_plan plan;
-        rc = bcq_plan_default(desc, 1, 0, &plan);
-        if (rc != BCQ_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (plan->kernel == 1) {
+        // The lookup-table kernel once per column: B passes over the weights, each at the batch-1 rate.
         for (int b = 0; b < B; ++b) {
-            rc = run_gemv(desc, &plan, packed, alpha, z, X + size_t(b) * desc->K, Y + size_t(b) * desc->N, ws, ws_bytes,
-                          stream);
+            rc = run_gemv(desc, plan, packed, alpha, z, X + size_t(b) * desc->K, Y + size_t(b) * desc->N, ws, ws_bytes, stream);
             if (rc != BCQ_OK) return rc;
         }
         return BCQ_OK;
     }
-    cudaError_t e = launch_generic(*desc, packed, alpha, z, X, Y, B, static_cast<cudaStream_t>(stream));
+    cudaError_t e;
+    if (plan->kernel == 2) {
+        const size_t need = plan_workspace(desc, plan, B);
+        if (need > 0) {
+            if (!ws) return BCQ_ERR_INVALID_ARG;
+            if (!aligned(ws, 16)) return BCQ_ERR_MISALIGNED;
+            if (ws_bytes < need) return BCQ_ERR_WORKSPACE_TOO_SMALL;
+        }
+        e = launch_mma_gemm(*desc, *plan, packed, alpha, z, X, Y, B, need ? ws : nullptr, st);
+    } else {
+        e = launch_generic(*desc, packed, alpha, z, X, Y, B, st);
+    }
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z,
+                        const uint16_t *X, uint16_t *Y, int B, void *ws, size_t ws_bytes, void *stream)
+{
+    bcq_plan plan;
+    int rc = bcq_plan_default(desc, B, 0, &plan);
+    if (rc != BCQ_OK) return rc;
+    return bcq_gemm_smallbatch_plan(desc, &plan, packed, alpha, z, X, Y, B, ws, ws_bytes, stream);
 }
 
 int bcq_gemv_host(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z,

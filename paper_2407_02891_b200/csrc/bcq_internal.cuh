@@ -17,6 +17,9 @@ constexpr int kLutWarps = 24;       // warps per block of the lookup-table kerne
 constexpr int kLutUnitsPerWarp = 8; // row units a warp keeps accumulators for
 constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
 constexpr int kMaxWindowsPerBlock = 32; // windows one block may walk (bounds the planner's search)
+constexpr int kMmaWarps = 22;        // consumer warps per block of the small-batch kernel
+constexpr int kMmaPairsPerWarp = 4;  // pairs of row units a warp keeps accumulators for
+constexpr int kMmaMaxUnitsPerBlock = 2 * kMmaWarps * kMmaPairsPerWarp;
 constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace
 constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);
 
@@ -27,7 +30,7 @@ inline int n_groups(const bcq_desc &d) { return d.group == 0 ? 1 : d.K / d.group
 // Canonical: packed[i][n][k/8], alpha[i][n][g], z[n][g] in three arrays.
 // Tiled: tile (w, u) of `packed` covers window w (512 weights = 64 chunks of 8 = 4 groups of 128)
 // of row unit u (8 rows).  Lane l = 8 g + j of a warp owns row 8u + j and group g of the window:
-//   q*512 bytes of planes as [jq < q][lane < 32][16 B]; byte p = s*q + i of a lane's 16q bytes is
+//   q*512 bytes of planes as [i < q][lane < 32][s < 16]; byte s of a lane in plane i is
 //   plane i of chunk 16 g + ((s + 2 j) mod 16): the 8 lanes of a group walk the group's 16 chunks
 //   skewed by two chunks per row, so that at every step the 32 lanes of a warp look up 32
 //   different chunk columns of the table (32 different shared-memory banks);
@@ -53,8 +56,7 @@ struct View {
         const int g = c >> 4, u = n / kUnitRows, j = n % kUnitRows;
         const int s = ((c & 15) - 2 * j) & 15;   // step at which lane 8g + j reaches chunk c
         const int lane = 8 * g + j;
-        const int p = s * q + i;
-        return packed + tile_base(w, u) + size_t(p >> 4) * 512 + size_t(lane) * 16 + (p & 15);
+        return packed + tile_base(w, u) + size_t(i) * 512 + size_t(lane) * 16 + s;
     }
     __host__ __device__ uint16_t *alpha_elem(int i, int n, int g) const
     {
@@ -98,6 +100,10 @@ cudaError_t launch_generic(const bcq_desc &d, const void *packed, const uint16_t
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st);
 
+cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
+                            const uint16_t *z, const uint16_t *X, uint16_t *Y, int B, void *workspace, cudaStream_t st);
+
 cudaError_t lut_status_take(int *status);
+cudaError_t mma_status_take(int *status);
 
 }  // namespace bcq

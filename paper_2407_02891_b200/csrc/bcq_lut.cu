@@ -31,8 +31,7 @@
 //
 // Every wait on an mbarrier is bounded; if one runs out the block sets an abort flag and a
 // device status word, stops waiting, drains its own copies and returns (see lut_status_take).
-#include <type_traits>
-
+#include "bcq_async.cuh"
 #include "bcq_internal.cuh"
 
 namespace bcq {
@@ -48,7 +47,6 @@ constexpr int kMaxSlotsPerWarp = 5;
 constexpr int kMaxSlots = kLutWarps * kMaxSlotsPerWarp;
 constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
 constexpr int kFixedBytes = 2048;      // barriers and flags
-constexpr int kSpinLimit = 1 << 22;   // polls per wait, about 32 ns apart: a wait gives up after roughly 0.2 s
 
 static_assert(8 * kMaxSlots + 64 <= kFixedBytes, "barrier area");
 static_assert(2 * kFixedBytes <= kLutSmemBytes - kTablesBytes, "barriers must fit before or after the tables");
@@ -90,79 +88,6 @@ struct LutParams {
     int N, K, U, W;
     int row_blocks, k_splits;
 };
-
-template <int I, int N, class F>
-__device__ __forceinline__ void static_for(F &&f)
-{
-    if constexpr (I < N) {
-        f(std::integral_constant<int, I>{});
-        static_for<I + 1, N>(f);
-    }
-}
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return uint32_t(__cvta_generic_to_shared(p)); }
-
-// ---- mbarrier / bulk-copy primitives ------------------------------------------------------------
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)   // never blocks
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if the block is aborting (this wait or another one ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code)
-{
-    // Poll without blocking and nap briefly in between: a warp suspended inside a blocking
-    // try_wait was seen to resume only about a microsecond after the phase had completed.
-    for (int it = 0; it < kSpinLimit; ++it) {
-        if (mbar_test_wait(bar, parity)) return true;
-        __nanosleep(32);
-        if ((it & 255) == 255 && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    atomicExch(&g_lut_status, code);
-    return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void named_barrier(int id, int threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 
 // table lookup + accumulate: the address register already holds the complete shared-window
 // address of an fp16 entry; acc (fp32) += entry, in one mixed-precision add
@@ -389,7 +314,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             const int b = wi & 1, use = wi >> 1;
             f32x2 x01[8], x23[8];
             load_quad(xblk + wi * kWindow, tid & 15, x01, x23);   // in flight while waiting for the buffer
-            if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree)) break;
+            if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, &g_lut_status)) break;
             build_quad(tables + b * 128, x01, x23, tid & 15, tid >> 4, kBuilderThreads / 16);
             mbar_arrive(bar_tab_ready + 8 * b);
         }
@@ -418,7 +343,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 #ifdef BCQ_TRACE
         const unsigned long long tt0 = gtime();
 #endif
-        if (wi > 0 && !mbar_wait(bar_tab_ready + 8 * b, ((wi >> 1) - (b == 0 ? 1 : 0)) & 1, abort_flag, kWaitTableReady)) {
+        if (wi > 0 && !mbar_wait(bar_tab_ready + 8 * b, ((wi >> 1) - (b == 0 ? 1 : 0)) & 1, abort_flag, kWaitTableReady, &g_lut_status)) {
             alive = false;
             break;
         }
@@ -448,7 +373,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 #ifdef BCQ_TRACE
                 const unsigned long long tw0 = gtime();
 #endif
-                const bool got = mbar_wait(bar_full + 8 * s, k & 1, abort_flag, kWaitFull);
+                const bool got = mbar_wait(bar_full + 8 * s, k & 1, abort_flag, kWaitFull, &g_lut_status);
 #ifdef BCQ_TRACE
                 if (ctid == 0) { TRACE_ADD(13, gtime() - tw0); TRACE_ADD(14, 1); if (wi == 0 && t == 0) TRACE(5); }
 #endif
@@ -492,7 +417,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                         constexpr int st = decltype(S)::value;
                         static_for<0, Q>([&](auto I) {
                             constexpr int i = decltype(I)::value;
-                            constexpr int pb = st * Q + i;
+                            constexpr int pb = i * 16 + st;
                             const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
                             lut_add<(st & 1) * 2>(sum[i][st & 1], addr);
                         });

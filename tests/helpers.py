@@ -29,8 +29,7 @@ def tiled_operands(planes, alpha, z, group):
     u, j = n // 8, n % 8
     s = (cc - 2 * j) % 16
     lane = 8 * g + j
-    p = s * q + i
-    off = (w * U + u) * T + (p // 16) * 512 + lane * 16 + p % 16
+    off = (w * U + u) * T + i * 512 + lane * 16 + s
     out[off.ravel()] = planes.ravel()
     G = alpha.shape[2]
     i, n, g = np.meshgrid(np.arange(q), np.arange(N), np.arange(G), indexing="ij")

@@ -270,6 +270,58 @@ def test_gemm_smallbatch(layout, N, K, q, group, B):
         assert np.array_equal(Y2.cpu().numpy().view(np.uint16), Yh[perm].view(np.uint16))
 
 
+@pytest.mark.parametrize("N,K,q,group,rb,ks,B", [
+    (264, 1024, 3, 128, 1, 1, 2),      # 33 units: an odd number, the last pair is a single tile
+    (264, 1024, 3, 128, 1, 2, 8),      # split-K, both windows apart
+    (264, 2048, 3, 128, 3, 2, 16),     # 11 units per block, two windows per split, wide
+    (1408, 1536, 3, 128, 1, 1, 5),     # 176 units: every warp four pairs, three windows
+    (1408, 1536, 3, 128, 1, 3, 9),
+    (776, 2560, 2, 128, 2, 1, 4),      # 97 units -> 48 + 49
+    (776, 2560, 2, 0, 2, 5, 16),       # one scale per row
+    (512, 1024, 1, 128, 4, 1, 3),
+    (512, 1024, 4, 128, 4, 2, 12),
+    (512, 1024, 4, 0, 1, 1, 7),
+    (8, 512, 3, 128, 1, 1, 2),         # one unit, one window
+    (16, 16384, 3, 128, 1, 1, 16),     # 32 windows in one block
+])
+def test_small_batch_kernel_explicit_plans(N, K, q, group, rb, ks, B):
+    """The tensor-core small-batch kernel under decompositions chosen by the caller."""
+    p, codes, alpha, z, X = make_layer(f"mma/{N}x{K}q{q}g{group}", N, K, q, group, B)
+    ref = oracle.forward_planes(p, alpha, z, X, group)
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    plan = bq.Plan(2, rb, ks, 0)
+    ws = bq.new_workspace(L.d, B, plan)
+    Y = torch.full((B, N), float("nan"), dtype=torch.float16, device=DEV)
+    for _ in range(2):   # the second call finds the counters as the first one left them
+        bq.gemm_smallbatch_plan(L.d, plan, L.packed, L.alpha, L.z, dev(X), Y, B, ws)
+    torch.cuda.synchronize()
+    bq.poll_status()
+    assert rel_err(Y.cpu().numpy(), ref) <= TOL
+    # column by column through the batch-1 kernel: the same numbers up to rounding
+    p1 = bq.plan_default(L.d, 1)
+    Y1 = torch.zeros_like(Y)
+    bq.gemm_smallbatch_plan(L.d, p1, L.packed, L.alpha, L.z, dev(X), Y1, B, bq.new_workspace(L.d, 1, p1))
+    torch.cuda.synchronize()
+    assert rel_err(Y1.cpu().numpy(), ref) <= TOL
+
+
+def test_small_batch_kernel_structured_inputs():
+    """Unit activations pick out single weights: exact values, every (row, k) position distinguishable."""
+    N, K, q, group, B = 64, 1024, 3, 128, 16
+    p, codes, alpha, z, _ = make_layer("mma/struct", N, K, q, group, B)
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    rng = np.random.default_rng(5)
+    ks = rng.choice(K, size=B, replace=False)
+    X = np.zeros((B, K), np.float16)
+    X[np.arange(B), ks] = 1.0
+    ref = oracle.forward_planes(p, alpha, z, X, group)     # = column ks[b] of the dequantised matrix
+    Y = torch.zeros((B, N), dtype=torch.float16, device=DEV)
+    bq.gemm_smallbatch(L.d, L.packed, L.alpha, L.z, dev(X), Y, B, bq.new_workspace(L.d, B))
+    torch.cuda.synchronize()
+    got = Y.cpu().numpy().astype(np.float64)
+    assert np.abs(got - ref).max() <= 2.0 ** -10 * np.abs(ref).max()
+
+
 def test_gemv_host_buffers():
     N, K, q, group = 520, 3584, 3, 128
     p, codes, alpha, z, x = make_layer("host", N, K, q, group)

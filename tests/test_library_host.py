@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(L, n), n
     assert set(names) == set(bq.SIGNATURES), "binding and header disagree"
-    assert bq.lib().bcq_version() == 103
+    assert bq.lib().bcq_version() == 104
 
 
 def test_status_strings():
@@ -137,5 +137,12 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * N * 4)
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
-    assert bq.plan_default(d, 4, 148).kernel == 1         # batches run the same kernel per column
+    for B in (2, 4, 16):                                   # batches: one pass of the tensor-core kernel
+        pb = bq.plan_default(d, B, 148)
+        assert pb.kernel == 2
+        assert 1 <= pb.row_blocks <= U and 1 <= pb.k_splits <= W
+        assert -(-U // pb.row_blocks) <= 176 and -(-W // pb.k_splits) <= 32
+        assert bq.workspace_bytes(d, B, pb) == (0 if pb.k_splits == 1 else 4096 * 4 + pb.k_splits * B * N * 4)
+        assert bq.workspace_bytes(d, B, p) == bq.workspace_bytes(d, 1, p)   # a batch-1 plan runs column by column
+    assert bq.workspace_bytes(d, 1, bq.plan_default(d, 4, 148)) == 0        # the small-batch kernel needs B >= 2
     assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
