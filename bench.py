@@ -149,7 +149,7 @@ class Stack:
             dt = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
             scales[(N, K)] = (torch.from_numpy(a).to(device), torch.from_numpy(z).to(device))
             xs[(N, K)] = torch.from_numpy(synth.activations(f"{wname}/{N}x{K}", B, K).reshape(-1)).to(device)
-            wss[(N, K)] = bq.new_workspace(dt, 1, device=device)
+            wss[(N, K)] = bq.new_workspace(dt, B, device=device)
         self.x_host = {k: v.cpu() for k, v in xs.items()}
         for layer in range(w["layers"]):
             for (pname, N, K) in layer_shapes(w):

@@ -277,6 +277,19 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
                     __syncwarp();
                     if (lane == 0) issue_next(d);
 
+                    // Independent accumulation chains (an MMA waits for the previous one into the same
+                    // registers): one per plane; folded into the pair's accumulators at the end.
+                    constexpr int NCH = WIDE ? (Q > 1 ? 2 : 1) : Q;
+                    float c[NCH][4], ch[WIDE ? NCH : 1][4];
+#pragma unroll
+                    for (int j = 0; j < NCH; ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) c[j][e] = 0.f;
+#pragma unroll
+                    for (int j = 0; j < (WIDE ? NCH : 1); ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) ch[j][e] = 0.f;
+
                     // offset term: rows m, m + 8 times (z, z) at k = 2t, 2t + 1; x sums (high, low) there
                     mma_16816(acc[pp], zz[0], zz[1], 0u, 0u, xs_lo, 0u);
                     if constexpr (WIDE) mma_16816(acc_hi[pp], zz[0], zz[1], 0u, 0u, xs_hi, 0u);
@@ -295,11 +308,18 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
                                 const uint32_t a1 = ((Wd[1][i][k] << sh0) & 0x80008000u) ^ nb[1][i];
                                 const uint32_t a2 = ((Wd[0][i][k] << sh1) & 0x80008000u) ^ nb[0][i];
                                 const uint32_t a3 = ((Wd[1][i][k] << sh1) & 0x80008000u) ^ nb[1][i];
-                                mma_16816(acc[pp], a0, a1, a2, a3, xf.x, xf.y);
-                                if constexpr (WIDE) mma_16816(acc_hi[pp], a0, a1, a2, a3, xg.x, xg.y);
+                                mma_16816(c[i % NCH], a0, a1, a2, a3, xf.x, xf.y);
+                                if constexpr (WIDE) mma_16816(ch[i % NCH], a0, a1, a2, a3, xg.x, xg.y);
                             }
                         });
                     });
+#pragma unroll
+                    for (int j = 0; j < NCH; ++j)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            acc[pp][e] += c[j][e];
+                            if constexpr (WIDE) acc_hi[pp][e] += ch[j][e];
+                        }
                 }
                 if (++d == D) {
                     d = 0;
