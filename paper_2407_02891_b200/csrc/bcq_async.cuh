@@ -61,13 +61,19 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)   
 }
 // Bounded wait.  Returns false if the block is aborting (this wait or another one ran out); the wait
 // that runs out raises the block's abort flag and records its code in the kernel's device status word.
+// Polls without blocking and naps in between (a warp suspended inside a blocking try_wait was seen to
+// resume only about a microsecond after the phase had completed).  LONG waits -- those that normally
+// last microseconds -- lengthen their naps up to 256 ns, so that waiting warps leave the issue slots
+// to the working ones; the time limit is about the same either way.
+template <bool LONG = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code, int *status_word)
 {
-    // Poll without blocking and nap briefly in between: a warp suspended inside a blocking
-    // try_wait was seen to resume only about a microsecond after the phase had completed.
-    for (int it = 0; it < kSpinLimit; ++it) {
+    for (int it = 0; it < (LONG ? kSpinLimit / 4 : kSpinLimit); ++it) {
         if (mbar_test_wait(bar, parity)) return true;
-        __nanosleep(32);
+        if (LONG && it >= 8)
+            __nanosleep(256);
+        else
+            __nanosleep(32);
         if ((it & 255) == 255 && *abort_flag) return false;
     }
     *abort_flag = 1;

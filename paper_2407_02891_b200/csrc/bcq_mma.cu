@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
         for (int s = 0; s < kMmaMaxSlots; ++s) mbar_init(bar_full + 8 * s, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_x_ready + 8 * b, BR / 8);   // lane 0 of every loader warp that stages columns
-            mbar_init(bar_x_free + 8 * b, kMmaWarps);
+            mbar_init(bar_x_free + 8 * b, P < kMmaWarps ? P : kMmaWarps);   // the consumer warps that have jobs
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
 #pragma unroll
                 for (int j = 0; j < 64; ++j) x2[j] = 0u;
             }
-            if (use > 0 && !mbar_wait(bar_x_free + 8 * buf, (use - 1) & 1, abort_flag, kMmaWaitXFree, &g_mma_status)) break;
+            if (use > 0 && !mbar_wait<true>(bar_x_free + 8 * buf, (use - 1) & 1, abort_flag, kMmaWaitXFree, &g_mma_status)) break;
             float sum = 0.f;
 #pragma unroll
             for (int j = 0; j < 64; ++j) {
@@ -222,9 +222,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
     bool alive = true;
     int d = 0, fill = 0;   // this warp's ring position: slot cw + kMmaWarps * d, fill number
 
-    for (int wi = 0; wi < nwin && alive; ++wi) {
+    for (int wi = 0; wi < nwin && alive && mine > 0; ++wi) {   // warps without jobs go straight to the end
         const int buf = wi & 1;
-        if (!mbar_wait(bar_x_ready + 8 * buf, (wi >> 1) & 1, abort_flag, kMmaWaitXReady, &g_mma_status)) {
+        if (!mbar_wait<true>(bar_x_ready + 8 * buf, (wi >> 1) & 1, abort_flag, kMmaWaitXReady, &g_mma_status)) {
             alive = false;
             break;
         }
