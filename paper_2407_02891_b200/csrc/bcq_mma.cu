@@ -232,8 +232,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
         const uint32_t xs_lo = xsum[(buf * BR + m) * 4 + t];
         const uint32_t xs_hi = WIDE ? xsum[(buf * BR + m + 8) * 4 + t] : 0u;
 
-        static_for<0, PMAX>([&](auto PP) {
-            constexpr int pp = decltype(PP)::value;
+        // One copy of the job's code (it is a few thousand instructions long): the loop over this
+        // warp's pairs is not unrolled, the pair at hand uses accumulator set 0 and the sets rotate
+        // after every pair, PMAX times per window, so that they are back in place for the next window.
+#pragma unroll 1
+        for (int pp = 0; pp < PMAX; ++pp) {
             if (alive && cw + kMmaWarps * pp < P) {
                 const int s = cw + kMmaWarps * d;
                 if (!mbar_wait(bar_full + 8 * s, fill & 1, abort_flag, kMmaWaitFull, &g_mma_status)) {
@@ -291,8 +294,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
                         for (int e = 0; e < 4; ++e) ch[j][e] = 0.f;
 
                     // offset term: rows m, m + 8 times (z, z) at k = 2t, 2t + 1; x sums (high, low) there
-                    mma_16816(acc[pp], zz[0], zz[1], 0u, 0u, xs_lo, 0u);
-                    if constexpr (WIDE) mma_16816(acc_hi[pp], zz[0], zz[1], 0u, 0u, xs_hi, 0u);
+                    mma_16816(acc[0], zz[0], zz[1], 0u, 0u, xs_lo, 0u);
+                    if constexpr (WIDE) mma_16816(acc_hi[0], zz[0], zz[1], 0u, 0u, xs_hi, 0u);
 
                     static_for<0, 4>([&](auto KK) {
                         constexpr int k = decltype(KK)::value;
@@ -317,8 +320,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
                     for (int j = 0; j < NCH; ++j)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            acc[pp][e] += c[j][e];
-                            if constexpr (WIDE) acc_hi[pp][e] += ch[j][e];
+                            acc[0][e] += c[j][e];
+                            if constexpr (WIDE) acc_hi[0][e] += ch[j][e];
                         }
                 }
                 if (++d == D) {
@@ -326,7 +329,20 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
                     ++fill;
                 }
             }
-        });
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float first = acc[0][e];
+#pragma unroll
+                for (int j = 0; j + 1 < PMAX; ++j) acc[j][e] = acc[j + 1][e];
+                acc[PMAX - 1][e] = first;
+                if constexpr (WIDE) {
+                    const float first_hi = acc_hi[0][e];
+#pragma unroll
+                    for (int j = 0; j + 1 < PMAX; ++j) acc_hi[j][e] = acc_hi[j + 1][e];
+                    acc_hi[PMAX - 1][e] = first_hi;
+                }
+            }
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_x_free + 8 * buf);
     }
