@@ -243,20 +243,20 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 8 * kMaxSlots + 32);
     int *s_last = const_cast<int *>(abort_flag) + 1;
 
-    if (tid == 0) {
-        TRACE(0);
+    if (tid == 0) TRACE(0);
 #ifdef BCQ_TRACE
-        g_trace[blockIdx.x % 1024][13] = 0; g_trace[blockIdx.x % 1024][14] = 0; g_trace[blockIdx.x % 1024][15] = 0;
+    if (tid == 0) { g_trace[blockIdx.x % 1024][13] = 0; g_trace[blockIdx.x % 1024][14] = 0; g_trace[blockIdx.x % 1024][15] = 0; }
 #endif
-        for (int s = 0; s < kMaxSlots; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
+    if (warp == 0) {   // one warp initialises the barriers, a few each
+        for (int s = lane; s < kMaxSlots; s += 32) mbar_init(bar_full + 8 * s, 1);
+        if (lane < 2) {
+            mbar_init(bar_tab_ready + 8 * lane, kBuilderThreads);
+            mbar_init(bar_tab_free + 8 * lane, kLutWarps);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_tab_ready + 8 * b, kBuilderThreads);
-            mbar_init(bar_tab_free + 8 * b, kLutWarps);
+        if (lane == 0) {
+            *abort_flag = (NS < kMinSlots) ? 1 : 0;
+            if (NS < kMinSlots) atomicExch(&g_lut_status, int(kTooFewSlots));
         }
-        *abort_flag = (NS < kMinSlots) ? 1 : 0;
-        if (NS < kMinSlots) atomicExch(&g_lut_status, int(kTooFewSlots));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }

@@ -123,13 +123,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
     volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 8 * kMmaMaxSlots + 32);
     int *s_last = const_cast<int *>(abort_flag) + 1;
 
-    if (tid == 0) {
-        for (int s = 0; s < kMmaMaxSlots; ++s) mbar_init(bar_full + 8 * s, 1);
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_x_ready + 8 * b, BR / 8);   // lane 0 of every loader warp that stages columns
-            mbar_init(bar_x_free + 8 * b, P < kMmaWarps ? P : kMmaWarps);   // the consumer warps that have jobs
+    if (warp == 0) {   // one warp initialises the barriers, a few each
+        for (int s = lane; s < kMmaMaxSlots; s += 32) mbar_init(bar_full + 8 * s, 1);
+        if (lane < 2) {
+            mbar_init(bar_x_ready + 8 * lane, BR / 8);   // lane 0 of every loader warp that stages columns
+            mbar_init(bar_x_free + 8 * lane, P < kMmaWarps ? P : kMmaWarps);   // the consumer warps that have jobs
         }
-        *abort_flag = 0;
+        if (lane == 0) *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
