@@ -115,6 +115,24 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, world: int, device) -> float:
+    """The slowest rank's time: replicas run independently, the job is as slow as its slowest rank.
+    A barrier, then an all-reduce(MAX) of one scalar -- the only collective of the multi-GPU path."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    dist.barrier()
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_metric(ms_per_step: float, world: int) -> float:
+    """us/token of the whole job: `world` replicas each finish one token per step (weak scaling)."""
+    return ms_per_step * 1e3 / world
+
+
 def physical_gpu_index(local: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -175,6 +193,15 @@ class Stack:
     def launch_all(self):
         for it in self.items:
             self.launch_one(it)
+
+    def launches_per_step(self):
+        """Kernel launches of one step: one per layer, or one per layer and column where the default
+        plan of the batch is the batch-1 kernel run column by column."""
+        n = 0
+        for it in self.items:
+            plan = self.bq.plan_default(it[0], self.B)
+            n += self.B if (self.B > 1 and plan.kernel == 1) else 1
+        return n
 
     def capture(self):
         torch = self.torch
@@ -374,23 +401,16 @@ def main():
     with ClockSampler(physical_gpu_index(local)) as clocks:
         ms = stack.time_steps(args.steps)
         torch.cuda.synchronize(device)
-    if world > 1:
-        dist.barrier()
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, device)
     ms_per_step = ms / args.steps
-    launches_per_step = len(stack.items)
+    launches_per_step = stack.launches_per_step()
 
     per_shape = stack.per_shape_us()
     e2e = None
     if not args.no_e2e and args.batch == 1:
         e_ms, h2d, d2h = stack.e2e_steps(max(3, min(args.steps, 20)))
-        if world > 1:
-            t = torch.tensor([e_ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e2e = {"value": e_ms * 1e3 / world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        e_ms = max_over_ranks(e_ms, world, device)
+        e2e = {"value": replica_metric(e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "api": "bcq_gemv_host per layer, pinned host x and y, one stream sync per token"}
 
     if rank != 0:
@@ -401,7 +421,7 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     achieved = stack.bytes / (ms_per_step * 1e-3) / 1e9
     out = {
-        "metric": METRIC, "value": ms_per_step * 1e3 / world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": replica_metric(ms_per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
         "tokens_per_s": world * 1e3 / ms_per_step,
@@ -414,7 +434,7 @@ def main():
                                  if bq.lib().bcq_version() == NCU_TRAFFIC["lib_version"]
                                  and args.workload == NCU_TRAFFIC["workload"] and args.layers == 0
                                  and args.batch == 1 else None),
-                     "kernel": f"lut_gemv_kernel<{w['q']}>" if args.batch == 1 else "bcq_gemm_smallbatch kernels",
+                     "kernel": f"lut_gemv_kernel<{w['q']}>" if args.batch <= 2 else f"mma_gemm_kernel<{w['q']}>",
                      "algorithmic_bytes_per_launch": stack.bytes // launches_per_step,
                      "launches_per_step": launches_per_step},
         "per_shape": per_shape,
