@@ -44,10 +44,17 @@ UNIT = "us/token"
 
 
 def layer_shapes(w):
-    """(name, N, K) of the six linear layers of one decoder layer (OPT, or Llama-2 with GQA)."""
+    """(name, N, K) of the six linear layers of one decoder layer (OPT, or Llama-2 with GQA).
+
+    With w["fuse"] the projections that read the same activation are stacked into one product
+    (q/k/v; gate/up): the same weights and the same arithmetic in fewer, longer launches."""
     h, f = w["hidden"], w["ffn"]
     if w.get("family") == "llama":
+        if w.get("fuse"):
+            return [("qkv", h + w["kv"], h), ("o", h, h), ("gate_up", 2 * f, h), ("down", h, f)]
         return [("q", h, h), ("kv", w["kv"], h), ("o", h, h), ("gate", f, h), ("up", f, h), ("down", h, f)]
+    if w.get("fuse"):
+        return [("qkv", 3 * h, h), ("out", h, h), ("fc1", f, h), ("fc2", h, f)]
     return [("q", h, h), ("k", h, h), ("v", h, h), ("out", h, h), ("fc1", f, h), ("fc2", h, f)]
 
 
@@ -333,6 +340,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--batch", type=int, default=1, help="activation vectors per product (1..16)")
+    ap.add_argument("--fuse", action="store_true",
+                    help="stack the projections that share an activation (q/k/v, gate/up) into one product each; "
+                         "not the default workload: a second number beside it")
     ap.add_argument("--layers", type=int, default=0, help="override the number of decoder layers (profiling)")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: plain launches instead of a CUDA graph, warm-up as given, "
@@ -345,10 +355,12 @@ def main():
     w = dict(WORKLOADS[args.workload])
     if args.layers > 0:
         w["layers"] = args.layers
+    if args.fuse:
+        w["fuse"] = True
     config = {"workload": args.workload,
               "shapes": ", ".join(f"{n}:{N}x{K}" for (n, N, K) in layer_shapes(w)) + " per layer",
               "hidden": w["hidden"], "ffn": w["ffn"], "layers": w["layers"], "q": w["q"], "group": w["group"],
-              "batch": args.batch,
+              "batch": args.batch, "fused_projections": bool(args.fuse),
               "cache": "inputs larger than L2 (every launch reads its own weights)", "parallelism": "replicas only"}
 
     if args.impl == "reference":
@@ -442,7 +454,7 @@ def main():
                      "traffic": (NCU_TRAFFIC["bytes_per_launch"]
                                  if bq.lib().bcq_version() == NCU_TRAFFIC["lib_version"]
                                  and args.workload == NCU_TRAFFIC["workload"] and args.layers == 0
-                                 and args.batch == 1 else None),
+                                 and args.batch == 1 and not args.fuse else None),
                      "kernel": f"lut_gemv_kernel<{w['q']}>" if args.batch <= 2 else f"mma_gemm_kernel<{w['q']}>",
                      "algorithmic_bytes_per_launch": stack.bytes // launches_per_step,
                      "launches_per_step": launches_per_step},
