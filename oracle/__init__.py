@@ -96,6 +96,21 @@ def round_to_bcchoice(w_int, n_bits: int, bit_to_plane) -> tuple[np.ndarray, np.
     return wq, codes
 
 
+def quantize_rtn(W, group: int, n_bits: int, s_factor: float = 1.0):
+    """Eq. gptqt step 1 with S = s_factor (Wmax - Wmin)/(2^n - 1), qbias = Wmin per (row, group).
+    W fp16 [N, K].  Returns (w_int [N,K] u8, S [N,G] f16, qbias [N,G] f16)."""
+    W = _c(W, np.float16)
+    N, K = W.shape
+    G = 1 if group == 0 else K // group
+    w_int = np.empty((N, K), np.uint8)
+    S = np.empty((N, G), np.float16)
+    qbias = np.empty((N, G), np.float16)
+    rc = _load().orc_quantize_rtn(_p(W), ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group), ctypes.c_int(n_bits),
+                                  ctypes.c_double(s_factor), _p(w_int), _p(S), _p(qbias))
+    _check(rc, "quantize_rtn")
+    return w_int, S, qbias
+
+
 def merge_linear(w_int, S, qbias, group: int, n_bits: int, bit_to_plane):
     """Eq. fuse_step3.  Returns (codes [N,K] u8, alpha [q,N,G] f16, z [N,G] f16)."""
     w = _c(w_int, np.uint8)

@@ -17,6 +17,9 @@
  *   Eq. round       every W_int is replaced by the nearest value the merged code reaches
  *                   (section "Quantize Weight Twice")
  *   Eq. fuse_step3  S and qbias fold in:  alpha_j = S m_j,  z = S (2^n - 1)/2 + qbias
+ *   Eq. gptqt step 1 (section "Quantize Weight Twice") with the scale of section
+ *                   "Re-explore Scaling Factor":  S = (Wmax - Wmin)/(2^n - 1), qbias = Wmin,
+ *                   W_int = round-to-nearest of the weight on that grid (orc_quantize_rtn)
  *   Eq. bcw         dequantised weight  w = sum_j alpha_j b_j  (+ z after the fusion)
  *
  * Readings taken where the paper is silent:
@@ -26,6 +29,12 @@
  *     parity unpinned for the tie rule alone (tests assert minimal distance and
  *     determinism, not which of two equidistant values is taken).
  *   - A plane set P is a partition of the n step-1 bits into q non-empty sets.
+ *   - Step 1 as printed, round(W/S - qbias), contradicts the dequantisation S W_int + qbias;
+ *     the quantiser is the inverse of the dequantisation:  W_int = round((W - qbias)/S),
+ *     clamped to 0 .. 2^n - 1, round = nearest, ties to even.  S is the fp16 value that
+ *     is stored (the range formula evaluated in fp64, rounded once), so that quantiser and
+ *     dequantiser use the same number.  A group whose weights are all equal gets S = 0,
+ *     W_int = 0.
  *   - Batch: every column of x is an independent matrix-vector product.
  *
  * Layouts (all row-major, the last index fastest):
@@ -144,10 +153,51 @@ int orc_round_to_bcchoice(const uint8_t *w_int, size_t count, int n_bits, int q,
     return ORC_OK;
 }
 
-/* ---- Eq. fuse_step3: fold S and qbias into the code ---------------------------- */
-
 static int n_groups(int K, int group) { return group == 0 ? 1 : K / group; }
 static int group_len(int K, int group) { return group == 0 ? K : group; }
+
+/* ---- Eq. gptqt, step 1: linear quantisation of fp16 weights to n bits ---------- */
+
+/* W fp16 [N][K].  Per (row, group): qbias = Wmin, S = fp16(s_factor (Wmax - Wmin)/(2^n - 1));
+ * s_factor = 1 is the step-1 scale, other values are the re-explored scales of Eq. reexplore.
+ * w_int = clamp(round((W - qbias)/S), 0, 2^n - 1). */
+int orc_quantize_rtn(const uint16_t *W, int N, int K, int group, int n_bits, double s_factor,
+                     uint8_t *w_int, uint16_t *S, uint16_t *qbias)
+{
+    if (N < 1 || K < 1 || group < 0 || (group && K % group) || n_bits < 1 || n_bits > 8) return ORC_BAD;
+    if (!(s_factor > 0.0) || !isfinite(s_factor)) return ORC_BAD;
+    int G = n_groups(K, group), L = group_len(K, group);
+    double top = ldexp(1.0, n_bits) - 1.0;
+    for (int n = 0; n < N; ++n)
+        for (int g = 0; g < G; ++g) {
+            const uint16_t *w = W + (size_t)n * K + (size_t)g * L;
+            double lo = orc_half_to_double(w[0]), hi = lo;
+            for (int k = 0; k < L; ++k) {
+                double v = orc_half_to_double(w[k]);
+                if (!isfinite(v)) return ORC_BAD;
+                if (v < lo) lo = v;
+                if (v > hi) hi = v;
+            }
+            uint16_t s_h = orc_double_to_half((s_factor * (hi - lo)) / top);
+            uint16_t b_h = orc_double_to_half(lo);   /* exact: lo is an fp16 value */
+            double s = orc_half_to_double(s_h);
+            if (!isfinite(s)) return ORC_BAD;
+            S[(size_t)n * G + g] = s_h;
+            qbias[(size_t)n * G + g] = b_h;
+            for (int k = 0; k < L; ++k) {
+                double r = 0.0;
+                if (s > 0.0) {
+                    r = rint((orc_half_to_double(w[k]) - lo) / s);   /* default rounding mode: ties to even */
+                    if (r > top) r = top;
+                    if (r < 0.0) r = 0.0;
+                }
+                w_int[(size_t)n * K + (size_t)g * L + k] = (uint8_t)r;
+            }
+        }
+    return ORC_OK;
+}
+
+/* ---- Eq. fuse_step3: fold S and qbias into the code ---------------------------- */
 
 int orc_merge_linear(const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias,
                      int N, int K, int group, int n_bits, int q, const uint8_t *bit_to_plane,

@@ -316,3 +316,109 @@ def test_group_boundaries_matter():
     x = np.ones((1, K), np.float16)
     y = oracle.forward_planes(p, alpha, z, x, group)
     assert np.array_equal(y[0], np.full(N, 128 * (1.0 + 0.5) + 128 * (-2.0 - 0.25)))
+
+
+# ---------------------------------------------------------------------------------------
+# Eq. gptqt step 1: linear quantisation of fp16 weights (oracle.quantize_rtn)
+# ---------------------------------------------------------------------------------------
+
+def _weights(name, N, K, scale=0.05):
+    return (scale * synth.normal(name + "/W", 0, N * K)).reshape(N, K).astype(np.float16)
+
+
+def test_rtn_exact_grid_is_recovered():
+    """Weights that lie on a grid qbias + S k (S a power of two) quantise to k, S and qbias exactly
+    (section "Re-explore Scaling Factor": S = (Wmax - Wmin)/(2^n - 1), qbias = Wmin)."""
+    for n in (2, 3, 4, 5):
+        top = 2 ** n - 1
+        rng = np.random.default_rng(n)
+        k = rng.integers(0, top + 1, size=(6, 64)).astype(np.float64)
+        k[:, 0], k[:, 1] = 0, top                                   # both ends occur in every group of 32
+        k[:, 32], k[:, 33] = 0, top
+        for S, b in ((2.0 ** -6, -0.75), (2.0 ** -9, 0.125)):
+            W = (b + S * k).astype(np.float16)
+            assert np.array_equal(W.astype(np.float64), b + S * k)  # representable: the case is exact
+            for group in (0, 32):
+                w_int, S_h, q_h = oracle.quantize_rtn(W, group, n)
+                assert np.array_equal(w_int, k.astype(np.uint8))
+                assert np.all(S_h.astype(np.float64) == S) and np.all(q_h.astype(np.float64) == b)
+
+
+@pytest.mark.parametrize("n,group", [(3, 0), (4, 128), (5, 64), (8, 32)])
+def test_rtn_is_the_nearest_grid_point_by_brute_force(n, group):
+    """Against enumeration of every level: the chosen integer minimises |W - (S k + qbias)|, the ends
+    of the range map to 0 and 2^n - 1, the error is at most S/2, and S is the range formula."""
+    N, K = 5, 256
+    W = _weights(f"rtn/{n}/{group}", N, K)
+    w_int, S_h, q_h = oracle.quantize_rtn(W, group, n)
+    L = K if group == 0 else group
+    Wd = W.astype(np.float64).reshape(N, K // L, L)
+    S = S_h.astype(np.float64)[:, :, None]
+    b = q_h.astype(np.float64)[:, :, None]
+    assert np.array_equal(b[:, :, 0], Wd.min(axis=2))
+    exact_S = (Wd.max(axis=2) - Wd.min(axis=2)) / (2 ** n - 1)
+    assert np.all(np.abs(S[:, :, 0] - exact_S) <= exact_S * 2.0 ** -11)       # one fp16 rounding
+    levels = np.arange(2 ** n, dtype=np.float64)
+    dist = np.abs(Wd[..., None] - (S[..., None] * levels + b[..., None]))     # [N, G, L, 2^n]
+    chosen = np.take_along_axis(dist, w_int.reshape(N, K // L, L, 1).astype(np.int64), axis=3)[..., 0]
+    assert np.all(chosen <= dist.min(axis=3) * (1 + 1e-12))
+    # the top of the range may sit half an fp16 rounding of S outside the grid, never more
+    assert np.all(chosen <= S / 2 + (2 ** n - 1) * exact_S[:, :, None] * 2.0 ** -11)
+    wi = w_int.reshape(N, K // L, L)
+    assert np.all(wi[Wd == Wd.min(axis=2, keepdims=True)] == 0)
+    assert np.all(wi[Wd == Wd.max(axis=2, keepdims=True)] == 2 ** n - 1)
+    # monotone: a larger weight never gets a smaller integer
+    order = np.argsort(Wd, axis=2, kind="stable")
+    assert np.all(np.diff(np.take_along_axis(wi.astype(np.int64), order, axis=2), axis=2) >= 0)
+
+
+def test_rtn_ties_go_to_even_and_clamp():
+    """Half-way points (exactly representable) round to the even integer; a re-explored, smaller S
+    (Eq. reexplore) pushes large weights past the grid and they clamp to 2^n - 1."""
+    n = 3
+    W = np.array([[0.0, 7.0, 0.5, 1.5, 2.5, 3.5, 4.5, 6.5]], np.float16)
+    w_int, S, b = oracle.quantize_rtn(W, 0, n)
+    assert float(S[0, 0]) == 1.0 and float(b[0, 0]) == 0.0
+    assert w_int.tolist() == [[0, 7, 0, 2, 2, 4, 4, 6]]
+    w2, S2, _ = oracle.quantize_rtn(W, 0, n, s_factor=0.5)         # S = 0.5: 3.5 -> 7, everything above clamps
+    assert float(S2[0, 0]) == 0.5
+    assert w2.tolist() == [[0, 7, 1, 3, 5, 7, 7, 7]]
+    w3, S3, _ = oracle.quantize_rtn(W, 0, n, s_factor=2.0)         # S = 2: half-way points 1, 3, 5, 7 do not occur
+    assert float(S3[0, 0]) == 2.0 and w3.tolist() == [[0, 4, 0, 1, 1, 2, 2, 3]]
+
+
+def test_rtn_constant_group_and_errors():
+    W = np.full((2, 64), 0.375, np.float16)
+    W[1, 32:] = [0.25] * 16 + [0.5] * 16
+    w_int, S, b = oracle.quantize_rtn(W, 32, 4)
+    assert np.all(w_int[0] == 0) and np.all(S[0] == 0) and np.all(b[0] == np.float16(0.375))
+    assert np.all(w_int[1, :32] == 0) and w_int[1, 32:].tolist() == [0] * 16 + [15] * 16
+    # S = 0 dequantises the constant group exactly through the merge as well
+    codes, alpha, z = oracle.merge_linear(w_int, S, b, 32, 4, [0, 1, 2, 2])
+    Wq = oracle.dequant(codes, alpha, z, 32)
+    assert np.array_equal(Wq[0], np.full(64, 0.375))
+    bad = W.copy()
+    bad[0, 3] = np.inf
+    with pytest.raises(Exception):
+        oracle.quantize_rtn(bad, 32, 4)
+    with pytest.raises(Exception):
+        oracle.quantize_rtn(W, 32, 4, s_factor=0.0)
+
+
+@pytest.mark.parametrize("n,q,b2p", [(4, 3, [0, 1, 2, 2]), (3, 3, [0, 1, 2]), (5, 2, [0, 0, 1, 1, 1])])
+def test_rtn_then_merge_reconstruction_error_bound(n, q, b2p):
+    """End to end (step 1, Eq. round, Eq. fuse_step3): the dequantised weight differs from the fp16
+    weight by at most S/2 (step 1) + S * the largest gap/2 of the reachable set (Eq. round)."""
+    N, K, group = 4, 256, 128
+    W = _weights(f"rtnmerge/{n}/{q}", N, K)
+    w_int, S, qb = oracle.quantize_rtn(W, group, n)
+    codes, alpha, z = oracle.merge_linear(w_int, S, qb, group, n, b2p)
+    Wq = oracle.dequant(codes, alpha, z, group)
+    _, values = oracle.bcchoice(n, b2p)
+    reach = np.sort(np.asarray(values, np.float64))
+    half_gap = max(np.diff(reach).max() / 2, reach[0], (2 ** n - 1) - reach[-1])
+    Sd = np.repeat(S.astype(np.float64), group, axis=1)
+    slack = (np.abs(W.astype(np.float64)).max() + 1) * 2.0 ** -9     # fp16 rounding of alpha and z
+    assert np.all(np.abs(Wq - W.astype(np.float64)) <= Sd * (0.5 + half_gap) + slack)
+    if q == n:
+        assert np.all(np.abs(Wq - W.astype(np.float64)) <= Sd * 0.5 + slack)
