@@ -140,6 +140,27 @@ int bcq_merge_linear(const bcq_desc *desc, const uint8_t *w_int_dev, const uint1
                      uint8_t *codes_dev, uint16_t *alpha_dev, uint16_t *z_dev, void *stream);
 
 /*
+ * fp16 weights -> packed binary-coded operand in desc->layout, in one call: step-1 linear
+ * quantisation (Eq. gptqt step 1 with the scale of section "Re-explore Scaling Factor"),
+ * nearest reachable integer (Eq. round), fusion (Eq. fuse_step3) and packing.
+ * Per (row, group) of W [N][K] (fp16, device, 16-byte aligned, finite values):
+ *   qbias = Wmin,   S = fp16( s_factor * (Wmax - Wmin) / (2^n_bits - 1) )
+ *   w_int = clamp( round((W - qbias) / S), 0, 2^n_bits - 1 )   nearest, ties to even, decided
+ *           in fp64 from the stored fp16 S; a group of equal weights gets S = 0, w_int = 0
+ * s_factor = 1 is the step-1 scale; Eq. reexplore searches s_factor between
+ * (2^n - 1)/(2^(n+1) - 1) and (2^n - 1)/(2^(n-1) - 1).  bit_to_plane_host as in bcq_merge_linear.
+ * Outputs (device, caller-owned): S, qbias [N][G] canonical (always written; they are also
+ * the kernels' scratch); w_int [N][K] or NULL; packed / alpha / z exactly as bcq_merge_linear
+ * followed by bcq_pack would produce them for desc->layout (alpha and z ignored when the tiles
+ * carry the scales).  Asynchronous on `stream`, no allocation.  The paper times no quantiser;
+ * this one reads W twice (range, then encode): about 4 bytes per weight of traffic.
+ */
+int bcq_quantize_rtn(const bcq_desc *desc, const uint16_t *W_dev, int n_bits,
+                     const uint8_t *bit_to_plane_host, double s_factor, uint16_t *S_dev,
+                     uint16_t *qbias_dev, uint8_t *w_int_dev, void *packed_dev, uint16_t *alpha_dev,
+                     uint16_t *z_dev, void *stream);
+
+/*
  * Codes + canonical scales -> packed bit-planes and scales in desc->layout.
  * Bit-exact: only bit extraction and permutation.  Canonical, or tiled with group 0:
  * alpha_in/z_in may be NULL together with alpha_out/z_out to pack the planes only.  Tiled with

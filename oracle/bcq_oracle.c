@@ -178,6 +178,7 @@ int orc_quantize_rtn(const uint16_t *W, int N, int K, int group, int n_bits, dou
                 if (v < lo) lo = v;
                 if (v > hi) hi = v;
             }
+            if (lo == 0.0) lo = 0.0;   /* a zero minimum is stored as +0 whichever zero was met first */
             uint16_t s_h = orc_double_to_half((s_factor * (hi - lo)) / top);
             uint16_t b_h = orc_double_to_half(lo);   /* exact: lo is an fp16 value */
             double s = orc_half_to_double(s_h);

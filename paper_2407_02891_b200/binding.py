@@ -73,6 +73,7 @@ SIGNATURES = {
     "bcq_workspace_bytes": (_sz, [_dp, _i, _pp]),
     "bcq_workspace_init": (_i, [_vp, _sz, _vp]),
     "bcq_merge_linear": (_i, [_dp, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp]),
+    "bcq_quantize_rtn": (_i, [_dp, _vp, _i, _vp, ctypes.c_double, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bcq_pack": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bcq_repack": (_i, [_dp, _vp, _vp, _vp, _dp, _vp, _vp, _vp, _vp]),
     "bcq_gemv": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -183,6 +184,17 @@ def merge_linear(d: Desc, w_int, S, qbias, n_bits: int, bit_to_plane, codes, alp
     _check(lib().bcq_merge_linear(ctypes.byref(d), _ptr(w_int), _ptr(S), _ptr(qbias), n_bits,
                                   ctypes.cast(b2p, ctypes.c_void_p), _ptr(codes), _ptr(alpha), _ptr(z),
                                   _stream()), "bcq_merge_linear")
+
+
+def quantize_rtn(d: Desc, W, n_bits: int, bit_to_plane, S, qbias, w_int, packed, alpha, z, s_factor: float = 1.0):
+    """bcq_quantize_rtn: fp16 weights W [N, K] -> S, qbias, (w_int), packed, alpha, z in d's layout."""
+    _dev(W, S, qbias, w_int, packed, alpha, z)
+    if len(bit_to_plane) != n_bits:
+        raise ValueError("bit_to_plane needs n_bits entries")
+    b2p = (ctypes.c_uint8 * len(bit_to_plane))(*[int(v) for v in bit_to_plane])
+    _check(lib().bcq_quantize_rtn(ctypes.byref(d), _ptr(W), n_bits, ctypes.cast(b2p, ctypes.c_void_p), float(s_factor),
+                                  _ptr(S), _ptr(qbias), _ptr(w_int), _ptr(packed), _ptr(alpha), _ptr(z), _stream()),
+           "bcq_quantize_rtn")
 
 
 def pack(d: Desc, codes, alpha_in, z_in, packed_out, alpha_out, z_out):

@@ -176,6 +176,36 @@ int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, con
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
 
+// The host-side table of the linear-int -> binary-code conversion (Eq. fuse_step2, Eq. round):
+// plane weights m_j and, for every step-1 integer, the code of the nearest reachable integer.
+int merge_table(int q, int n_bits, const uint8_t *bit_to_plane, double (&weight)[4], uint8_t (&code_of_int)[256])
+{
+    // A sign pattern (code) drives all step-1 bits of a plane together, so the integers it can
+    // reach are those whose binary digit (i-1) equals the code's bit for the plane of step-1 bit i.
+    for (int j = 0; j < 4; ++j) weight[j] = 0.0;
+    for (int i = 0; i < n_bits; ++i) {
+        if (bit_to_plane[i] >= q) return BCQ_ERR_INVALID_ARG;
+        weight[bit_to_plane[i]] += double(1u << i) * 0.5;  // step-1 bit i+1 weighs 2^(i-1)
+    }
+    for (int j = 0; j < q; ++j)
+        if (weight[j] == 0.0) return BCQ_ERR_INVALID_ARG;
+    int reach[16];
+    for (int c = 0; c < (1 << q); ++c) {
+        int v = 0;
+        for (int i = 0; i < n_bits; ++i) v |= ((c >> bit_to_plane[i]) & 1) << i;
+        reach[c] = v;
+    }
+    for (int t = 0; t < 256; ++t) {
+        int best = 0;
+        for (int c = 1; c < (1 << q); ++c) {
+            const int dc = abs(t - reach[c]), db = abs(t - reach[best]);
+            if (dc < db || (dc == db && reach[c] < reach[best])) best = c;
+        }
+        code_of_int[t] = uint8_t(best);
+    }
+    return BCQ_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -280,32 +310,36 @@ int bcq_merge_linear(const bcq_desc *desc, const uint8_t *w_int, const uint16_t 
         !aligned(z, 2))
         return BCQ_ERR_MISALIGNED;
 
-    // A sign pattern (code) drives all step-1 bits of a plane together, so the integers it can
-    // reach are those whose binary digit (i-1) equals the code's bit for the plane of step-1 bit i.
-    double weight[4] = {0, 0, 0, 0};
-    for (int i = 0; i < n_bits; ++i) {
-        if (bit_to_plane[i] >= d.q) return BCQ_ERR_INVALID_ARG;
-        weight[bit_to_plane[i]] += double(1u << i) * 0.5;  // step-1 bit i+1 weighs 2^(i-1)
-    }
-    for (int j = 0; j < d.q; ++j)
-        if (weight[j] == 0.0) return BCQ_ERR_INVALID_ARG;
-    int reach[16];
-    for (int c = 0; c < (1 << d.q); ++c) {
-        int v = 0;
-        for (int i = 0; i < n_bits; ++i) v |= ((c >> bit_to_plane[i]) & 1) << i;
-        reach[c] = v;
-    }
+    double weight[4];
     uint8_t code_of_int[256];
-    for (int t = 0; t < 256; ++t) {
-        int best = 0;
-        for (int c = 1; c < (1 << d.q); ++c) {
-            const int dc = abs(t - reach[c]), db = abs(t - reach[best]);
-            if (dc < db || (dc == db && reach[c] < reach[best])) best = c;
-        }
-        code_of_int[t] = uint8_t(best);
-    }
+    rc = merge_table(d.q, n_bits, bit_to_plane, weight, code_of_int);
+    if (rc != BCQ_OK) return rc;
     cudaError_t e = launch_merge(d, w_int, S, qbias, n_bits, code_of_int, weight, codes, alpha, z,
                                  static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_quantize_rtn(const bcq_desc *desc, const uint16_t *W, int n_bits, const uint8_t *bit_to_plane, double s_factor,
+                     uint16_t *S, uint16_t *qbias, uint8_t *w_int, void *packed, uint16_t *alpha, uint16_t *z, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!W || !bit_to_plane || !S || !qbias || !packed) return BCQ_ERR_INVALID_ARG;
+    if (n_bits < 1 || n_bits > 8 || desc->q > n_bits) return BCQ_ERR_INVALID_ARG;
+    if (!(s_factor > 0.0) || !(s_factor < 1e30)) return BCQ_ERR_INVALID_ARG;
+    if (interleaved(desc))
+        alpha = z = nullptr;
+    else if (!alpha || !z)
+        return BCQ_ERR_INVALID_ARG;
+    if (!aligned(W, 16) || !aligned(packed, 16) || !aligned(w_int, 8) || !aligned(S, 2) || !aligned(qbias, 2) ||
+        !aligned(alpha, 2) || !aligned(z, 2))
+        return BCQ_ERR_MISALIGNED;
+    double weight[4];
+    uint8_t code_of_int[256];
+    rc = merge_table(desc->q, n_bits, bit_to_plane, weight, code_of_int);
+    if (rc != BCQ_OK) return rc;
+    cudaError_t e = launch_quantize_rtn(W, n_bits, s_factor, code_of_int, weight, S, qbias, w_int,
+                                        make_view(*desc, packed, alpha, z), static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
 

@@ -91,6 +91,9 @@ inline View make_view(const bcq_desc &d, const void *packed, const uint16_t *alp
 cudaError_t launch_merge(const bcq_desc &d, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias,
                          int n_bits, const uint8_t *code_of_int /*[256]*/, const double *plane_weight /*[q]*/,
                          uint8_t *codes, uint16_t *alpha, uint16_t *z, cudaStream_t st);
+cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, const uint8_t *code_of_int /*[256]*/,
+                                const double *plane_weight /*[q]*/, uint16_t *S, uint16_t *qbias, uint8_t *w_int,
+                                const View &dst, cudaStream_t st);
 cudaError_t launch_pack(const uint8_t *codes, const View &dst, cudaStream_t st);
 cudaError_t launch_permute_planes(const View &src, const View &dst, cudaStream_t st);
 cudaError_t launch_permute_scales(const View &src, const View &dst, cudaStream_t st);

@@ -1,0 +1,137 @@
+// On-device quantiser front end: fp16 weights -> packed binary-coded operand in one call.
+//
+//   step 1 (Eq. gptqt, with the scale of section "Re-explore Scaling Factor"), per (row, group):
+//       qbias = Wmin,  S = fp16( s_factor (Wmax - Wmin) / (2^n - 1) ),
+//       W_int = clamp( round((W - qbias) / S), 0, 2^n - 1 )        (nearest, ties to even)
+//   step 2 (Eq. round): W_int -> code of the nearest integer the merged planes reach
+//   fusion (Eq. fuse_step3): alpha_j = S m_j,  z = S (2^n - 1)/2 + qbias
+//   packing: code bit i -> plane i, written straight into the layout of the descriptor.
+//
+// The quantiser is the inverse of the dequantisation S W_int + qbias and uses the fp16 S that is
+// stored.  The integer is decided in fp64: W - qbias is exact there, the quotient is rounded once,
+// so the decision does not depend on evaluation order.  Three small kernels, all bound by the
+// 2 bytes per weight they read (twice: once for the range, once to encode).
+#include "bcq_internal.cuh"
+
+namespace bcq {
+
+struct QuantTable {
+    uint8_t code_of_int[256];
+    double plane_weight[4];
+    double centre;      // (2^n - 1) / 2
+    double top;         // 2^n - 1
+    double s_factor;
+};
+
+// One warp per (row, group): the range of the group's weights, then S and qbias.
+__global__ void __launch_bounds__(256) rtn_range_kernel(const __half *__restrict__ W, int N, int K, int L, QuantTable tab,
+                                                        __half *__restrict__ S, __half *__restrict__ qbias)
+{
+    const int G = K / L;
+    const size_t unit = (size_t(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (unit >= size_t(N) * G) return;
+    const __half *w = W + (unit / G) * size_t(K) + (unit % G) * size_t(L);
+    float lo = __half2float(w[0]), hi = lo;
+    for (int k = 4 * lane; k < L; k += 128) {   // L is a multiple of 32: whole 8-byte pieces
+        const uint2 raw = *reinterpret_cast<const uint2 *>(w + k);
+        const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const float2 f = __half22float2(h[j]);
+            lo = fminf(lo, fminf(f.x, f.y));
+            hi = fmaxf(hi, fmaxf(f.x, f.y));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (lane == 0) {
+        if (lo == 0.f) lo = 0.f;   // a zero minimum is stored as +0
+        const double range = double(hi) - double(lo);   // exact
+        S[unit] = __double2half(__ddiv_rn(__dmul_rn(tab.s_factor, range), tab.top));
+        qbias[unit] = __float2half_rn(lo);              // exact: lo is an fp16 value
+    }
+}
+
+// One thread per (row, chunk of 8 weights): integers, codes, one byte per plane.
+__global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restrict__ W, const __half *__restrict__ S,
+                                                         const __half *__restrict__ qbias, int L, QuantTable tab,
+                                                         uint8_t *__restrict__ w_int, const View dst)
+{
+    __shared__ uint8_t lut[256];
+    for (int t = threadIdx.x; t < 256; t += blockDim.x) lut[t] = tab.code_of_int[t];
+    __syncthreads();
+    const int kbytes = dst.K / 8;
+    const size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t >= size_t(dst.N) * kbytes) return;
+    const int n = int(t / kbytes), kb = int(t % kbytes);
+    const int G = dst.K / L, g = (kb * 8) / L;
+    const double s = double(__half2float(S[size_t(n) * G + g]));
+    const double b = double(__half2float(qbias[size_t(n) * G + g]));
+    const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
+    const __half *h = reinterpret_cast<const __half *>(&raw);
+    uint32_t ints[8], planes[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        double r = 0.0;
+        if (s > 0.0) {
+            r = rint(__ddiv_rn(double(__half2float(h[j])) - b, s));   // the subtraction is exact in fp64
+            r = fmin(fmax(r, 0.0), tab.top);
+        }
+        ints[j] = uint32_t(int(r));
+        const uint32_t code = lut[ints[j]];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) planes[i] |= ((code >> i) & 1u) << j;
+    }
+    for (int i = 0; i < dst.q; ++i) *dst.plane_byte(i, n, kb) = uint8_t(planes[i]);
+    if (w_int) {
+        uint2 out;
+        out.x = ints[0] | (ints[1] << 8) | (ints[2] << 16) | (ints[3] << 24);
+        out.y = ints[4] | (ints[5] << 8) | (ints[6] << 16) | (ints[7] << 24);
+        *reinterpret_cast<uint2 *>(w_int + size_t(n) * dst.K + size_t(kb) * 8) = out;
+    }
+}
+
+// One thread per (row, group): alpha_j = S m_j and z = S centre + qbias, evaluated exactly in fp64
+// and rounded once, written where the destination layout keeps them.
+__global__ void __launch_bounds__(256) rtn_scales_kernel(const __half *__restrict__ S, const __half *__restrict__ qbias,
+                                                         QuantTable tab, const View dst)
+{
+    const int G = dst.G();
+    const size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t >= size_t(dst.N) * G) return;
+    const int n = int(t / G), g = int(t % G);
+    const double s = double(__half2float(S[t])), b = double(__half2float(qbias[t]));
+    for (int j = 0; j < dst.q; ++j) *dst.alpha_elem(j, n, g) = __half_as_ushort(__double2half(s * tab.plane_weight[j]));
+    *dst.z_elem(n, g) = __half_as_ushort(__double2half(s * tab.centre + b));
+}
+
+cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, const uint8_t *code_of_int /*[256]*/,
+                                const double *plane_weight /*[q]*/, uint16_t *S, uint16_t *qbias, uint8_t *w_int,
+                                const View &dst, cudaStream_t st)
+{
+    QuantTable tab;
+    for (int t = 0; t < 256; ++t) tab.code_of_int[t] = code_of_int[t];
+    for (int j = 0; j < 4; ++j) tab.plane_weight[j] = j < dst.q ? plane_weight[j] : 0.0;
+    tab.top = double((1u << n_bits) - 1u);
+    tab.centre = tab.top / 2.0;
+    tab.s_factor = s_factor;
+    const int L = dst.group == 0 ? dst.K : dst.group;
+    const size_t units = size_t(dst.N) * dst.G();
+    const __half *w = reinterpret_cast<const __half *>(W);
+    __half *s = reinterpret_cast<__half *>(S), *b = reinterpret_cast<__half *>(qbias);
+    rtn_range_kernel<<<unsigned((units + 7) / 8), 256, 0, st>>>(w, dst.N, dst.K, L, tab, s, b);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t chunks = size_t(dst.N) * (dst.K / 8);
+    rtn_encode_kernel<<<unsigned((chunks + 255) / 256), 256, 0, st>>>(w, s, b, L, tab, w_int, dst);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    rtn_scales_kernel<<<unsigned((units + 255) / 256), 256, 0, st>>>(s, b, tab, dst);
+    return cudaGetLastError();
+}
+
+}  // namespace bcq
