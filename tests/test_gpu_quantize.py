@@ -92,7 +92,7 @@ def test_quantize_rtn_structured_weights():
 
 def test_quantize_rtn_without_integer_output_and_product():
     """w_int is optional; the operand that comes out multiplies like the oracle's dequantised matrix."""
-    N, K, q, group, n_bits, b2p = 520, 2048, 3, 128, 4, [0, 1, 2, 2]
+    N, K, q, group, n_bits, b2p = 520, 2048, 3, 128, 4, [0, 0, 1, 2]
     W = weights("q/prod", N, K)
     d = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
     S, qb, wi, packed, a, z = run(W, q, group, bq.LAYOUT_TILED, n_bits, b2p, want_int=False)
@@ -106,9 +106,9 @@ def test_quantize_rtn_without_integer_output_and_product():
     torch.cuda.synchronize()
     ref = oracle.forward_dequant(codes, alpha, zz, x, group)[0]
     assert rel_err(y.cpu().numpy(), ref) <= TOL
-    # and stays close to the unquantised product: 4-bit step 1 merged into 3 planes
+    # and stays near the unquantised product (4-bit step 1 merged into 3 planes with gaps of at most 3 S)
     exact = W.astype(np.float64) @ x[0].astype(np.float64)
-    assert rel_err(ref, exact) < 0.2
+    assert rel_err(ref, exact) < 0.5
 
 
 def test_quantize_rtn_full_size_sampled_rows():
