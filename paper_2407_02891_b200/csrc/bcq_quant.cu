@@ -8,7 +8,7 @@
 //   packing: code bit i -> plane i, written straight into the layout of the descriptor.
 //
 // The quantiser is the inverse of the dequantisation S W_int + qbias and uses the fp16 S that is
-// stored.  The integer is decided in fp64: W - qbias is exact there, the quotient is rounded once,
+// stored.  The integer is defined in fp64: W - qbias is exact there, the quotient is rounded once,
 // so the decision does not depend on evaluation order.  Three small kernels, all bound by the
 // 2 bytes per weight they read (twice: once for the range, once to encode).
 #include "bcq_internal.cuh"
@@ -73,13 +73,29 @@ __global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restric
     const double b = double(__half2float(qbias[size_t(n) * G + g]));
     const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
     const __half *h = reinterpret_cast<const __half *>(&raw);
+    // The integer is DEFINED by the fp64 quotient.  An fp32 estimate of it (three roundings, relative
+    // error below 1.8e-7) decides whenever it is further from a rounding boundary than its own error
+    // bound; the few weights that are not (and exact ties) take the fp64 division.  Same integers,
+    // a fraction of the fp64 work.
+    const float sf = __half2float(S[size_t(n) * G + g]), bf = __half2float(qbias[size_t(n) * G + g]);
+    const float inv_s = sf > 0.f ? __frcp_rn(sf) : 0.f;
+    const float topf = float(tab.top);
     uint32_t ints[8], planes[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         double r = 0.0;
         if (s > 0.0) {
-            r = rint(__ddiv_rn(double(__half2float(h[j])) - b, s));   // the subtraction is exact in fp64
-            r = fmin(fmax(r, 0.0), tab.top);
+            const float t = __fmul_rn(__fsub_rn(__half2float(h[j]), bf), inv_s);   // >= 0: qbias is the minimum
+            const float err = fmaf(t, 4e-7f, 1e-6f);
+            const float fl = floorf(t);
+            if (t - err > topf + 0.5f) {
+                r = tab.top;
+            } else if (fabsf(t - fl - 0.5f) > err) {
+                r = fmin(double(rintf(t)), tab.top);
+            } else {
+                r = rint(__ddiv_rn(double(__half2float(h[j])) - b, s));   // the subtraction is exact in fp64
+                r = fmin(fmax(r, 0.0), tab.top);
+            }
         }
         ints[j] = uint32_t(int(r));
         const uint32_t code = lut[ints[j]];
