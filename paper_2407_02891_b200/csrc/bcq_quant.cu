@@ -9,8 +9,8 @@
 //
 // The quantiser is the inverse of the dequantisation S W_int + qbias and uses the fp16 S that is
 // stored.  The integer is defined in fp64: W - qbias is exact there, the quotient is rounded once,
-// so the decision does not depend on evaluation order.  Three small kernels, all bound by the
-// 2 bytes per weight they read (twice: once for the range, once to encode).
+// so the decision does not depend on evaluation order.  Groups of 128 take one pass over W (a
+// group's 16 chunks sit in 16 lanes); other group lengths take a range pass and an encode pass.
 #include "bcq_internal.cuh"
 
 namespace bcq {
@@ -33,11 +33,12 @@ __global__ void __launch_bounds__(256) rtn_range_kernel(const __half *__restrict
     if (unit >= size_t(N) * G) return;
     const __half *w = W + (unit / G) * size_t(K) + (unit % G) * size_t(L);
     float lo = __half2float(w[0]), hi = lo;
-    for (int k = 4 * lane; k < L; k += 128) {   // L is a multiple of 32: whole 8-byte pieces
-        const uint2 raw = *reinterpret_cast<const uint2 *>(w + k);
+#pragma unroll 4
+    for (int k = 8 * lane; k < L; k += 256) {   // L is a multiple of 32: whole 16-byte pieces
+        const uint4 raw = *reinterpret_cast<const uint4 *>(w + k);
         const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < 4; ++j) {
             const float2 f = __half22float2(h[j]);
             lo = fminf(lo, fminf(f.x, f.y));
             hi = fmaxf(hi, fmaxf(f.x, f.y));
@@ -56,45 +57,33 @@ __global__ void __launch_bounds__(256) rtn_range_kernel(const __half *__restrict
     }
 }
 
-// One thread per (row, chunk of 8 weights): integers, codes, one byte per plane.
-__global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restrict__ W, const __half *__restrict__ S,
-                                                         const __half *__restrict__ qbias, int L, QuantTable tab,
-                                                         uint8_t *__restrict__ w_int, const View dst)
+// Integers, codes and plane bytes of one chunk of 8 weights (row n, bytes kb of the planes).
+// The integer is DEFINED by the fp64 quotient (W - qbias)/S.  An fp32 estimate of it (three
+// roundings, relative error below 1.8e-7) decides whenever it is further from a rounding boundary
+// than its own error bound; the few weights that are not (and exact ties) take the fp64 division.
+// Same integers, a fraction of the fp64 work.
+__device__ __forceinline__ void encode_chunk(const uint4 raw, __half s_h, __half b_h, const QuantTable &tab,
+                                             const uint8_t *lut, uint8_t *__restrict__ w_int, const View &dst, int n, int kb)
 {
-    __shared__ uint8_t lut[256];
-    for (int t = threadIdx.x; t < 256; t += blockDim.x) lut[t] = tab.code_of_int[t];
-    __syncthreads();
-    const int kbytes = dst.K / 8;
-    const size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (t >= size_t(dst.N) * kbytes) return;
-    const int n = int(t / kbytes), kb = int(t % kbytes);
-    const int G = dst.K / L, g = (kb * 8) / L;
-    const double s = double(__half2float(S[size_t(n) * G + g]));
-    const double b = double(__half2float(qbias[size_t(n) * G + g]));
-    const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
-    const __half *h = reinterpret_cast<const __half *>(&raw);
-    // The integer is DEFINED by the fp64 quotient.  An fp32 estimate of it (three roundings, relative
-    // error below 1.8e-7) decides whenever it is further from a rounding boundary than its own error
-    // bound; the few weights that are not (and exact ties) take the fp64 division.  Same integers,
-    // a fraction of the fp64 work.
-    const float sf = __half2float(S[size_t(n) * G + g]), bf = __half2float(qbias[size_t(n) * G + g]);
+    const float sf = __half2float(s_h), bf = __half2float(b_h);
+    const double s = double(sf), b = double(bf);
     const float inv_s = sf > 0.f ? __frcp_rn(sf) : 0.f;
     const float topf = float(tab.top);
+    const __half *h = reinterpret_cast<const __half *>(&raw);
     uint32_t ints[8], planes[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        double r = 0.0;
-        if (s > 0.0) {
+        float r = 0.f;
+        if (sf > 0.f) {
             const float t = __fmul_rn(__fsub_rn(__half2float(h[j]), bf), inv_s);   // >= 0: qbias is the minimum
             const float err = fmaf(t, 4e-7f, 1e-6f);
-            const float fl = floorf(t);
             if (t - err > topf + 0.5f) {
-                r = tab.top;
-            } else if (fabsf(t - fl - 0.5f) > err) {
-                r = fmin(double(rintf(t)), tab.top);
+                r = topf;
+            } else if (fabsf(t - floorf(t) - 0.5f) > err) {
+                r = fminf(rintf(t), topf);
             } else {
-                r = rint(__ddiv_rn(double(__half2float(h[j])) - b, s));   // the subtraction is exact in fp64
-                r = fmin(fmax(r, 0.0), tab.top);
+                const double r64 = rint(__ddiv_rn(double(__half2float(h[j])) - b, s));   // the subtraction is exact in fp64
+                r = float(fmin(fmax(r64, 0.0), tab.top));
             }
         }
         ints[j] = uint32_t(int(r));
@@ -111,18 +100,91 @@ __global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restric
     }
 }
 
-// One thread per (row, group): alpha_j = S m_j and z = S centre + qbias, evaluated exactly in fp64
-// and rounded once, written where the destination layout keeps them.
+// alpha_j = S m_j and z = S centre + qbias of one (row, group): exact in fp64, rounded once.
+__device__ __forceinline__ void write_scales(__half s_h, __half b_h, const QuantTable &tab, const View &dst, int n, int g)
+{
+    const double s = double(__half2float(s_h)), b = double(__half2float(b_h));
+    for (int j = 0; j < dst.q; ++j) *dst.alpha_elem(j, n, g) = __half_as_ushort(__double2half(s * tab.plane_weight[j]));
+    *dst.z_elem(n, g) = __half_as_ushort(__double2half(s * tab.centre + b));
+}
+
+__device__ __forceinline__ void range_to_scale(float lo, float hi, const QuantTable &tab, __half &s_h, __half &b_h)
+{
+    if (lo == 0.f) lo = 0.f;   // a zero minimum is stored as +0
+    const double range = double(hi) - double(lo);   // exact
+    s_h = __double2half(__ddiv_rn(__dmul_rn(tab.s_factor, range), tab.top));
+    b_h = __float2half_rn(lo);                      // exact: lo is an fp16 value
+}
+
+// Any group length: one thread per (row, chunk), S and qbias from the range kernel.  Block x of row
+// blockIdx.x covers chunks 256 blockIdx.y .. + 255.
+__global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restrict__ W, const __half *__restrict__ S,
+                                                         const __half *__restrict__ qbias, int L, QuantTable tab,
+                                                         uint8_t *__restrict__ w_int, const View dst)
+{
+    __shared__ uint8_t lut[256];
+    for (int t = threadIdx.x; t < 256; t += blockDim.x) lut[t] = tab.code_of_int[t];
+    __syncthreads();
+    const int n = blockIdx.x, kb = blockIdx.y * 256 + threadIdx.x;
+    if (kb >= dst.K / 8) return;
+    const int G = dst.K / L, g = (kb * 8) / L;
+    const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
+    encode_chunk(raw, S[size_t(n) * G + g], qbias[size_t(n) * G + g], tab, lut, w_int, dst, n, kb);
+}
+
+// Groups of 128: everything in one pass.  A group is 16 chunks = 16 consecutive lanes, each holding
+// its chunk in registers: range by shuffles, S and qbias by the group's first lane, then the encoding.
+__global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restrict__ W, QuantTable tab,
+                                                           __half *__restrict__ S, __half *__restrict__ qbias,
+                                                           uint8_t *__restrict__ w_int, const View dst)
+{
+    __shared__ uint8_t lut[256];
+    for (int t = threadIdx.x; t < 256; t += blockDim.x) lut[t] = tab.code_of_int[t];
+    __syncthreads();
+    const int kbytes = dst.K / 8;   // a multiple of 16: a half-warp is inside the row or outside
+    const int n = blockIdx.x, kb = blockIdx.y * 256 + threadIdx.x;
+    const bool in = kb < kbytes;
+    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+    if (in) raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
+    const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+    float lo, hi;
+    {
+        const float2 f = __half22float2(h2[0]);
+        lo = fminf(f.x, f.y), hi = fmaxf(f.x, f.y);
+#pragma unroll
+        for (int j = 1; j < 4; ++j) {
+            const float2 e = __half22float2(h2[j]);
+            lo = fminf(lo, fminf(e.x, e.y));
+            hi = fmaxf(hi, fmaxf(e.x, e.y));
+        }
+    }
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    __half s_h = __float2half_rn(0.f), b_h = s_h;
+    const bool first = (threadIdx.x & 15) == 0;
+    const int g = kb >> 4, G = dst.K / 128;
+    if (first && in) {
+        range_to_scale(lo, hi, tab, s_h, b_h);
+        S[size_t(n) * G + g] = s_h;
+        qbias[size_t(n) * G + g] = b_h;
+        write_scales(s_h, b_h, tab, dst, n, g);
+    }
+    const unsigned pair = uint32_t(__half_as_ushort(s_h)) | (uint32_t(__half_as_ushort(b_h)) << 16);
+    const unsigned got = __shfl_sync(0xffffffffu, pair, (threadIdx.x & 31) & 16);
+    if (in) encode_chunk(raw, __ushort_as_half(uint16_t(got & 0xffffu)), __ushort_as_half(uint16_t(got >> 16)), tab, lut, w_int, dst, n, kb);
+}
+
+// One thread per (row, group): the fused scales, written where the destination layout keeps them.
 __global__ void __launch_bounds__(256) rtn_scales_kernel(const __half *__restrict__ S, const __half *__restrict__ qbias,
                                                          QuantTable tab, const View dst)
 {
     const int G = dst.G();
     const size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (t >= size_t(dst.N) * G) return;
-    const int n = int(t / G), g = int(t % G);
-    const double s = double(__half2float(S[t])), b = double(__half2float(qbias[t]));
-    for (int j = 0; j < dst.q; ++j) *dst.alpha_elem(j, n, g) = __half_as_ushort(__double2half(s * tab.plane_weight[j]));
-    *dst.z_elem(n, g) = __half_as_ushort(__double2half(s * tab.centre + b));
+    write_scales(S[t], qbias[t], tab, dst, int(t / G), int(t % G));
 }
 
 cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, const uint8_t *code_of_int /*[256]*/,
@@ -139,11 +201,15 @@ cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, 
     const size_t units = size_t(dst.N) * dst.G();
     const __half *w = reinterpret_cast<const __half *>(W);
     __half *s = reinterpret_cast<__half *>(S), *b = reinterpret_cast<__half *>(qbias);
+    const dim3 grid(unsigned(dst.N), unsigned((dst.K / 8 + 255) / 256));   // one row per blockIdx.x
+    if (L == 128) {
+        rtn_fused128_kernel<<<grid, 256, 0, st>>>(w, tab, s, b, w_int, dst);
+        return cudaGetLastError();
+    }
     rtn_range_kernel<<<unsigned((units + 7) / 8), 256, 0, st>>>(w, dst.N, dst.K, L, tab, s, b);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const size_t chunks = size_t(dst.N) * (dst.K / 8);
-    rtn_encode_kernel<<<unsigned((chunks + 255) / 256), 256, 0, st>>>(w, s, b, L, tab, w_int, dst);
+    rtn_encode_kernel<<<grid, 256, 0, st>>>(w, s, b, L, tab, w_int, dst);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     rtn_scales_kernel<<<unsigned((units + 255) / 256), 256, 0, st>>>(s, b, tab, dst);
