@@ -57,47 +57,60 @@ __global__ void __launch_bounds__(256) rtn_range_kernel(const __half *__restrict
     }
 }
 
+// Shared-memory table of a block: entry t = the code of step-1 integer t with code bit i moved to
+// bit 8 i, so that OR-ing (entry << j) over the 8 weights j of a chunk leaves plane i's byte in byte i.
+__device__ __forceinline__ void load_spread_table(const QuantTable &tab, uint32_t *lut)
+{
+    for (int t = threadIdx.x; t < 256; t += blockDim.x) {
+        const uint32_t c = tab.code_of_int[t];
+        lut[t] = (c & 1u) | ((c & 2u) << 7) | ((c & 4u) << 14) | ((c & 8u) << 21);
+    }
+    __syncthreads();
+}
+
 // Integers, codes and plane bytes of one chunk of 8 weights (row n, bytes kb of the planes).
-// The integer is DEFINED by the fp64 quotient (W - qbias)/S.  An fp32 estimate of it (three
-// roundings, relative error below 1.8e-7) decides whenever it is further from a rounding boundary
-// than its own error bound; the few weights that are not (and exact ties) take the fp64 division.
-// Same integers, a fraction of the fp64 work.
+// The integer is DEFINED by the fp64 quotient (W - qbias)/S, rounded to nearest, ties to even.  An
+// fp32 estimate t of the quotient (three roundings, relative error below 1.8e-7) decides whenever it
+// is further from a rounding boundary than its own error bound; the few weights that are not (and
+// exact ties) take the fp64 division.  Same integers, a fraction of the fp64 work.  Rounding t: adding
+// 1.5 * 2^23 leaves the nearest integer in the low mantissa bits (valid below 2^22; larger t clamp).
 __device__ __forceinline__ void encode_chunk(const uint4 raw, __half s_h, __half b_h, const QuantTable &tab,
-                                             const uint8_t *lut, uint8_t *__restrict__ w_int, const View &dst, int n, int kb)
+                                             const uint32_t *lut, uint8_t *__restrict__ w_int, const View &dst, int n, int kb)
 {
     const float sf = __half2float(s_h), bf = __half2float(b_h);
-    const double s = double(sf), b = double(bf);
-    const float inv_s = sf > 0.f ? __frcp_rn(sf) : 0.f;
+    const float inv_s = sf > 0.f ? __frcp_rn(sf) : 0.f;   // S = 0: every t is 0, every integer 0
     const float topf = float(tab.top);
-    const __half *h = reinterpret_cast<const __half *>(&raw);
-    uint32_t ints[8], planes[4] = {0u, 0u, 0u, 0u};
+    const int topi = int(tab.top);
+    const float magic = 12582912.f;
+    const uint32_t word[4] = {raw.x, raw.y, raw.z, raw.w};
+    uint32_t spread = 0u, ints_lo = 0u, ints_hi = 0u;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        float r = 0.f;
-        if (sf > 0.f) {
-            const float t = __fmul_rn(__fsub_rn(__half2float(h[j]), bf), inv_s);   // >= 0: qbias is the minimum
-            const float err = fmaf(t, 4e-7f, 1e-6f);
-            if (t - err > topf + 0.5f) {
-                r = topf;
-            } else if (fabsf(t - floorf(t) - 0.5f) > err) {
-                r = fminf(rintf(t), topf);
+        const __half hw = __ushort_as_half(uint16_t(word[j >> 1] >> (16 * (j & 1))));
+        const float w = __half2float(hw);
+        const float t = __fmul_rn(__fsub_rn(w, bf), inv_s);   // >= 0: qbias is the minimum
+        const float err = fmaf(t, 4e-7f, 1e-6f);
+        int r;
+        if (t - err > topf + 0.5f) {
+            r = topi;
+        } else {
+            const float shifted = __fadd_rn(t, magic);
+            const float nearest = __fsub_rn(shifted, magic);
+            if (fabsf(t - nearest) < 0.5f - err) {
+                r = min(__float_as_int(shifted) - __float_as_int(magic), topi);
             } else {
-                const double r64 = rint(__ddiv_rn(double(__half2float(h[j])) - b, s));   // the subtraction is exact in fp64
-                r = float(fmin(fmax(r64, 0.0), tab.top));
+                const double r64 = rint(__ddiv_rn(double(w) - double(bf), double(sf)));   // the subtraction is exact in fp64
+                r = int(fmin(fmax(r64, 0.0), tab.top));
             }
         }
-        ints[j] = uint32_t(int(r));
-        const uint32_t code = lut[ints[j]];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) planes[i] |= ((code >> i) & 1u) << j;
+        spread |= lut[r] << j;
+        if (j < 4)
+            ints_lo |= uint32_t(r) << (8 * j);
+        else
+            ints_hi |= uint32_t(r) << (8 * (j - 4));
     }
-    for (int i = 0; i < dst.q; ++i) *dst.plane_byte(i, n, kb) = uint8_t(planes[i]);
-    if (w_int) {
-        uint2 out;
-        out.x = ints[0] | (ints[1] << 8) | (ints[2] << 16) | (ints[3] << 24);
-        out.y = ints[4] | (ints[5] << 8) | (ints[6] << 16) | (ints[7] << 24);
-        *reinterpret_cast<uint2 *>(w_int + size_t(n) * dst.K + size_t(kb) * 8) = out;
-    }
+    for (int i = 0; i < dst.q; ++i) *dst.plane_byte(i, n, kb) = uint8_t(spread >> (8 * i));
+    if (w_int) *reinterpret_cast<uint2 *>(w_int + size_t(n) * dst.K + size_t(kb) * 8) = make_uint2(ints_lo, ints_hi);
 }
 
 // alpha_j = S m_j and z = S centre + qbias of one (row, group): exact in fp64, rounded once.
@@ -122,9 +135,8 @@ __global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restric
                                                          const __half *__restrict__ qbias, int L, QuantTable tab,
                                                          uint8_t *__restrict__ w_int, const View dst)
 {
-    __shared__ uint8_t lut[256];
-    for (int t = threadIdx.x; t < 256; t += blockDim.x) lut[t] = tab.code_of_int[t];
-    __syncthreads();
+    __shared__ uint32_t lut[256];
+    load_spread_table(tab, lut);
     const int n = blockIdx.x, kb = blockIdx.y * 256 + threadIdx.x;
     if (kb >= dst.K / 8) return;
     const int G = dst.K / L, g = (kb * 8) / L;
@@ -138,9 +150,8 @@ __global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restr
                                                            __half *__restrict__ S, __half *__restrict__ qbias,
                                                            uint8_t *__restrict__ w_int, const View dst)
 {
-    __shared__ uint8_t lut[256];
-    for (int t = threadIdx.x; t < 256; t += blockDim.x) lut[t] = tab.code_of_int[t];
-    __syncthreads();
+    __shared__ uint32_t lut[256];
+    load_spread_table(tab, lut);
     const int kbytes = dst.K / 8;   // a multiple of 16: a half-warp is inside the row or outside
     const int n = blockIdx.x, kb = blockIdx.y * 256 + threadIdx.x;
     const bool in = kb < kbytes;
