@@ -174,18 +174,30 @@ __global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restr
         lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
         hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
     }
+    // S and qbias by the group's first lane, handed to the other 15; then lanes 0 .. q of the group
+    // each produce one fused scale (alpha_0 .. alpha_{q-1}, z = S centre + qbias) in the same pass.
     __half s_h = __float2half_rn(0.f), b_h = s_h;
-    const bool first = (threadIdx.x & 15) == 0;
+    const int sub = threadIdx.x & 15;
     const int g = kb >> 4, G = dst.K / 128;
-    if (first && in) {
+    if (sub == 0 && in) {
         range_to_scale(lo, hi, tab, s_h, b_h);
         S[size_t(n) * G + g] = s_h;
         qbias[size_t(n) * G + g] = b_h;
-        write_scales(s_h, b_h, tab, dst, n, g);
     }
     const unsigned pair = uint32_t(__half_as_ushort(s_h)) | (uint32_t(__half_as_ushort(b_h)) << 16);
     const unsigned got = __shfl_sync(0xffffffffu, pair, (threadIdx.x & 31) & 16);
-    if (in) encode_chunk(raw, __ushort_as_half(uint16_t(got & 0xffffu)), __ushort_as_half(uint16_t(got >> 16)), tab, lut, w_int, dst, n, kb);
+    s_h = __ushort_as_half(uint16_t(got & 0xffffu));
+    b_h = __ushort_as_half(uint16_t(got >> 16));
+    if (in && sub <= dst.q) {
+        const double mult = sub < dst.q ? tab.plane_weight[sub & 3] : tab.centre;
+        const double add = sub < dst.q ? 0.0 : double(__half2float(b_h));
+        const uint16_t v = __half_as_ushort(__double2half(double(__half2float(s_h)) * mult + add));   // exact, rounded once
+        if (sub < dst.q)
+            *dst.alpha_elem(sub, n, g) = v;
+        else
+            *dst.z_elem(n, g) = v;
+    }
+    if (in) encode_chunk(raw, s_h, b_h, tab, lut, w_int, dst, n, kb);
 }
 
 // One thread per (row, group): the fused scales, written where the destination layout keeps them.
