@@ -58,6 +58,11 @@ struct View {
         const int lane = 8 * g + j;
         return packed + tile_base(w, u) + size_t(i) * 512 + size_t(lane) * 16 + s;
     }
+    // distance in bytes from plane_byte(i, n, kb) to plane_byte(i + 1, n, kb)
+    __host__ __device__ size_t plane_stride() const
+    {
+        return layout == BCQ_LAYOUT_CANONICAL ? size_t(N) * size_t(K / 8) : size_t(512);
+    }
     __host__ __device__ uint16_t *alpha_elem(int i, int n, int g) const
     {
         if (layout == BCQ_LAYOUT_CANONICAL) return alpha + (size_t(i) * N + n) * G() + g;

@@ -109,7 +109,9 @@ __device__ __forceinline__ void encode_chunk(const uint4 raw, __half s_h, __half
         else
             ints_hi |= uint32_t(r) << (8 * (j - 4));
     }
-    for (int i = 0; i < dst.q; ++i) *dst.plane_byte(i, n, kb) = uint8_t(spread >> (8 * i));
+    unsigned char *out = dst.plane_byte(0, n, kb);
+    const size_t stride = dst.plane_stride();
+    for (int i = 0; i < dst.q; ++i) out[i * stride] = uint8_t(spread >> (8 * i));
     if (w_int) *reinterpret_cast<uint2 *>(w_int + size_t(n) * dst.K + size_t(kb) * 8) = make_uint2(ints_lo, ints_hi);
 }
 
