@@ -12,7 +12,7 @@
  * offset).  g(k) = k / group is the scaling unit along K; group == 0 means one scale per
  * row, which is the granularity the paper states.  This library computes y at batch 1
  * (bcq_gemv) and for 2..16 activation vectors (bcq_gemm_smallbatch), and prepares the
- * operands (bcq_merge_linear, bcq_pack, bcq_repack).
+ * operands (bcq_quantize_rtn from fp16 weights; bcq_merge_linear, bcq_pack, bcq_repack).
  *
  * Conventions
  *   - Every pointer named *_dev is DEVICE memory owned by the caller; *_host is host memory.
@@ -202,10 +202,12 @@ int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed
 /*
  * Y[b] = W X[b] for b < B, 1 <= B <= 16; X [B][K], Y [B][N] row-major fp16.  Every column is
  * an independent product (the paper defines batch 1 only; Eq. bcw + Eq. fuse_step3 per column).
- * B == 1 is bcq_gemv.  Tiled layout, B >= 2: ONE pass over the packed weights for all columns
- * (tensor-core kernel: a weight bit becomes the fp16 value +-alpha of its row and group, the
- * products with x are exact, all sums fp32; the offset term uses the fp32 group sums of x,
- * kept to 22 bits).  The workspace depends on B: bcq_workspace_bytes(desc, B, plan).
+ * B == 1 is bcq_gemv.  Tiled layout: by default B >= 3 takes ONE pass over the packed weights
+ * for all columns (plan kernel 2, the tensor-core kernel: a weight bit becomes the fp16 value
+ * +-alpha of its row and group, the products with x are exact, all sums fp32; the offset term
+ * uses the fp32 group sums of x, kept to 22 bits) and B == 2 runs the lookup-table kernel once
+ * per column, which is faster for two columns (bcq_plan_default tells which).  The workspace
+ * depends on B: bcq_workspace_bytes(desc, B, plan).
  * Canonical layout: one pass of the generic kernel for all columns.
  * bcq_gemm_smallbatch_plan takes the decomposition from the caller; a plan with kernel 1 runs
  * the lookup-table kernel once per column (B passes, workspace as for bcq_gemv).
