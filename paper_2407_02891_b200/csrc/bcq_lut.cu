@@ -235,7 +235,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     const int n_b = (fixed_in_back ? back - kFixedBytes : back) / SL::kBytes;
     const int NS = min(n_a + n_b, kMaxSlots);
     const int D = min(NS / kLutWarps, kMaxSlotsPerWarp);   // ring slots per consumer warp
-    auto slot_ptr = [&](int s) -> unsigned char * { return s < n_a ? ring_a + s * SL::kBytes : ring_b + (s - n_a) * SL::kBytes; };
+    unsigned char *const ring_b0 = ring_b - n_a * SL::kBytes;   // so that slot s of either piece is at piece + s * kBytes
+    auto slot_ptr = [&](int s) -> unsigned char * { return (s < n_a ? ring_a : ring_b0) + s * SL::kBytes; };
 
     const uint32_t bars = smem_u32(fixed);
     const uint32_t bar_full = bars;
@@ -275,18 +276,22 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     const int cw = warp - kFirstConsumerWarp;   // 0 .. kLutWarps-1 for consumers, negative for builders
     const int mine = (cw >= 0 && V > cw) ? (V - cw + kLutWarps - 1) / kLutWarps : 0;   // units of this warp per window
     const int total_jobs = mine * nwin;
-    int issued = 0, consumed = 0, iw = 0, it = 0;
+    int issued = 0, consumed = 0, it = 0;
+    // the next tile to fetch: this warp's units of a window are kLutWarps tiles apart, then on to the next window
+    const uint8_t *src = p.tiles + (size_t(w0) * p.U + u0 + (cw < 0 ? 0 : cw)) * SL::kBytes;
+    const long long unit_step = (long long)kLutWarps * SL::kBytes;
+    const long long window_step = ((long long)p.U - (long long)kLutWarps * mine) * SL::kBytes;
     auto issue_next = [&](int slot_d) {   // lane 0 of a consumer warp only
         if (issued < total_jobs) {
-            const size_t tile = size_t(w0 + iw) * p.U + u0 + cw + kLutWarps * it;
             const int s = cw + kLutWarps * slot_d;
             const uint32_t full = bar_full + 8 * s;
             mbar_expect_tx(full, SL::kBytes);
-            bulk_g2s(smem_u32(slot_ptr(s)), p.tiles + tile * SL::kBytes, SL::kBytes, full);   // planes + alphas + offsets
+            bulk_g2s(smem_u32(slot_ptr(s)), src, SL::kBytes, full);   // planes + alphas + offsets
             ++issued;
+            src += unit_step;
             if (++it == mine) {
                 it = 0;
-                ++iw;
+                src += window_step;
             }
         }
     };
