@@ -319,7 +319,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             const int b = wi & 1, use = wi >> 1;
             f32x2 x01[8], x23[8];
             load_quad(xblk + wi * kWindow, tid & 15, x01, x23);   // in flight while waiting for the buffer
-            if (use > 0 && !mbar_wait(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, &g_lut_status)) break;
+            if (use > 0 && !mbar_wait<true>(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, &g_lut_status)) break;   // a long wait: nap longer
             build_quad(tables + b * 128, x01, x23, tid & 15, tid >> 4, kBuilderThreads / 16);
             mbar_arrive(bar_tab_ready + 8 * b);
         }
