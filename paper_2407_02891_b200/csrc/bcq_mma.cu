@@ -23,7 +23,7 @@
 // batch-1 kernel's bank mapping); the lane undoes that while loading -- word rotation through the
 // load address, the odd half-word through one byte-permute -- so that all rows of an MMA see the
 // same weights k.  X is staged per 512-wide window by two loader warps, already in operand order
-// (one 8-byte shared-memory load per MMA and lane), three windows in flight.
+// (one 8-byte shared-memory load per MMA and lane), double buffered.
 //
 // The block structure is that of the batch-1 kernel: one block per SM owns a range of row units and
 // a range of windows; every consumer warp owns a few ring slots (one slot = one tile pair = one
@@ -43,9 +43,8 @@ constexpr int kMmaMaxSlotsPerWarp = 4;
 constexpr int kMmaMaxSlots = kMmaWarps * kMmaMaxSlotsPerWarp;
 constexpr int kXGroupBytes = 264;        // 256 B of operand-ordered x of one (column, group) + 8 B: no bank conflicts
 constexpr int kXRowBytes = 4 * kXGroupBytes;
-constexpr int kXBuffers = 3;             // windows of staged x in flight: the loaders run up to two windows ahead
 
-static_assert(8 * kMmaMaxSlots + 16 * kXBuffers + 16 <= kMmaFixedBytes, "barrier area");
+static_assert(8 * kMmaMaxSlots + 64 <= kMmaFixedBytes, "barrier area");
 
 __device__ int g_mma_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
 
@@ -108,26 +107,25 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
     const int V = u1 - u0, P = (V + 1) >> 1;   // row units and unit pairs of this block
     const int nwin = w1 - w0;
 
-    // ---- shared memory: [barriers | x operands (3 buffers) | group sums of x (3 buffers) | ring] ----
+    // ---- shared memory: [barriers | x operands (2 buffers) | group sums of x (2 buffers) | ring] ----
     unsigned char *fixed = smem;
     unsigned char *xs = smem + kMmaFixedBytes;
-    uint32_t *xsum = reinterpret_cast<uint32_t *>(xs + kXBuffers * kXBufBytes);   // [buffer][BR][4] fp16 (high, low)
-    constexpr int kXAllBytes = (kXBuffers * (kXBufBytes + BR * 16) + 127) / 128 * 128;
-    unsigned char *ring = xs + kXAllBytes;
-    constexpr int kRingBytes = kMmaSmemBytes - kMmaFixedBytes - kXAllBytes;
+    uint32_t *xsum = reinterpret_cast<uint32_t *>(xs + 2 * kXBufBytes);   // [2][BR][4] fp16 (high, low)
+    unsigned char *ring = xs + 2 * kXBufBytes + 2 * BR * 16;
+    constexpr int kRingBytes = kMmaSmemBytes - kMmaFixedBytes - 2 * kXBufBytes - 2 * BR * 16;
     constexpr int NS = kRingBytes / kSlotBytes < kMmaMaxSlots ? kRingBytes / kSlotBytes : kMmaMaxSlots;
     constexpr int D = NS / kMmaWarps;   // ring slots per consumer warp
     static_assert(D >= 1, "ring too small");
 
     const uint32_t bars = smem_u32(fixed);
     const uint32_t bar_full = bars;
-    const uint32_t bar_x_ready = bars + 8 * kMmaMaxSlots, bar_x_free = bar_x_ready + 8 * kXBuffers;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 8 * kMmaMaxSlots + 16 * kXBuffers);
+    const uint32_t bar_x_ready = bars + 8 * kMmaMaxSlots, bar_x_free = bar_x_ready + 16;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 8 * kMmaMaxSlots + 32);
     int *s_last = const_cast<int *>(abort_flag) + 1;
 
     if (warp == 0) {   // one warp initialises the barriers, a few each
         for (int s = lane; s < kMmaMaxSlots; s += 32) mbar_init(bar_full + 8 * s, 1);
-        if (lane < kXBuffers) {
+        if (lane < 2) {
             mbar_init(bar_x_ready + 8 * lane, BR / 8);   // lane 0 of every loader warp that stages columns
             mbar_init(bar_x_free + 8 * lane, P < kMmaWarps ? P : kMmaWarps);   // the consumer warps that have jobs
         }
@@ -175,7 +173,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
         const int b = tid >> 2, t = tid & 3;
         if (b >= BR) return;
         for (int wi = 0; wi < nwin; ++wi) {
-            const int buf = wi % kXBuffers, use = wi / kXBuffers;
+            const int buf = wi & 1, use = wi >> 1;
             uint32_t x2[64];   // x2[j] = (x[2j], x[2j+1]) of the group
             if (b < p.B) {
                 const uint4 *src = reinterpret_cast<const uint4 *>(p.X + size_t(b) * p.K + size_t(w0 + wi) * kWindow + 128 * t);
@@ -246,9 +244,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
     int d = 0, fill = 0;   // this warp's ring position: slot cw + kMmaWarps * d, fill number
 
     for (int wi = 0; wi < nwin && alive && mine > 0; ++wi) {   // warps without jobs go straight to the end
-        const int buf = wi % kXBuffers;
+        const int buf = wi & 1;
         MTRACE_T(t_x0);
-        if (!mbar_wait<true>(bar_x_ready + 8 * buf, (wi / kXBuffers) & 1, abort_flag, kMmaWaitXReady, &g_mma_status)) {
+        if (!mbar_wait<true>(bar_x_ready + 8 * buf, (wi >> 1) & 1, abort_flag, kMmaWaitXReady, &g_mma_status)) {
             alive = false;
             break;
         }
