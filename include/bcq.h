@@ -93,7 +93,7 @@ typedef struct bcq_desc {
  * shape, either layout), 1 = lookup-table kernel (tiled layout, one column per launch),
  * 2 = tensor-core small-batch kernel (tiled layout, 2..16 columns per launch); kernels 1 and 2
  * are launched as row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace.
- * Limits: at most 192 (kernel 1) or 200 (kernel 2) row units of 8 rows per block, at most 32
+ * Limits: at most 192 (kernel 1) or 176 (kernel 2) row units of 8 rows per block, at most 32
  * windows of 512 weights per K split. */
 typedef struct bcq_plan {
     int32_t kernel;

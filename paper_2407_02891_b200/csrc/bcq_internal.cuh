@@ -17,7 +17,7 @@ constexpr int kLutWarps = 24;       // warps per block of the lookup-table kerne
 constexpr int kLutUnitsPerWarp = 8; // row units a warp keeps accumulators for
 constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
 constexpr int kMaxWindowsPerBlock = 32; // windows one block may walk (bounds the planner's search)
-constexpr int kMmaWarps = 25;        // consumer warps per block of the small-batch kernel
+constexpr int kMmaWarps = 22;        // consumer warps per block of the small-batch kernel
 constexpr int kMmaPairsPerWarp = 4;  // pairs of row units a warp keeps accumulators for
 constexpr int kMmaMaxUnitsPerBlock = 2 * kMmaWarps * kMmaPairsPerWarp;
 constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace

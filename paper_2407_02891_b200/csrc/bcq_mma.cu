@@ -35,7 +35,7 @@
 namespace bcq {
 
 constexpr int kMmaLoaderWarps = 2;
-constexpr int kMmaThreads = (kMmaLoaderWarps + kMmaWarps) * 32;   // 864
+constexpr int kMmaThreads = (kMmaLoaderWarps + kMmaWarps) * 32;   // 768
 constexpr int kMmaConsumerThreads = kMmaWarps * 32;
 constexpr int kMmaSmemBytes = 232448;    // 227 KB: the per-block opt-in maximum
 constexpr int kMmaFixedBytes = 2048;     // barriers and flags

@@ -143,7 +143,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
         pb = bq.plan_default(d, B, 148)
         assert pb.kernel == 2
         assert 1 <= pb.row_blocks <= U and 1 <= pb.k_splits <= W
-        assert -(-U // pb.row_blocks) <= 200 and -(-W // pb.k_splits) <= 32
+        assert -(-U // pb.row_blocks) <= 176 and -(-W // pb.k_splits) <= 32
         assert bq.workspace_bytes(d, B, pb) == (0 if pb.k_splits == 1 else 4096 * 4 + pb.k_splits * B * N * 4)
         assert bq.workspace_bytes(d, B, p) == bq.workspace_bytes(d, 1, p)   # a batch-1 plan runs column by column
     assert bq.workspace_bytes(d, 1, bq.plan_default(d, 4, 148)) == 0        # the small-batch kernel needs B >= 2
