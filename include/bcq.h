@@ -90,7 +90,7 @@ typedef struct bcq_desc {
 } bcq_desc;
 
 /* How a product is decomposed over the GPU.  kernel: 0 = generic (one warp per row; any valid
- * shape, either layout), 1 = lookup-table kernel (tiled layout, one column per launch),
+ * shape, either layout), 1 = lookup-table kernel (tiled layout, one or two columns per launch),
  * 2 = tensor-core small-batch kernel (tiled layout, 2..16 columns per launch); kernels 1 and 2
  * are launched as row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace.
  * Limits: at most 192 (kernel 1) or 176 (kernel 2) row units of 8 rows per block, at most 32
@@ -205,12 +205,15 @@ int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed
  * B == 1 is bcq_gemv.  Tiled layout: by default B >= 3 takes ONE pass over the packed weights
  * for all columns (plan kernel 2, the tensor-core kernel: a weight bit becomes the fp16 value
  * +-alpha of its row and group, the products with x are exact, all sums fp32; the offset term
- * uses the fp32 group sums of x, kept to 22 bits) and B == 2 runs the lookup-table kernel once
- * per column, which is faster for two columns (bcq_plan_default tells which).  The workspace
- * depends on B: bcq_workspace_bytes(desc, B, plan).
+ * uses the fp32 group sums of x, kept to 22 bits) and B == 2 runs the lookup-table kernel on the
+ * column pair (plan kernel 1 with tables that hold both columns' sums side by side: one pass
+ * over the weights, one 4-byte lookup per weight byte for both columns), which is faster for
+ * two columns (bcq_plan_default tells which).  The workspace depends on B:
+ * bcq_workspace_bytes(desc, B, plan).
  * Canonical layout: one pass of the generic kernel for all columns.
  * bcq_gemm_smallbatch_plan takes the decomposition from the caller; a plan with kernel 1 runs
- * the lookup-table kernel once per column (B passes, workspace as for bcq_gemv).
+ * the lookup-table kernel on two columns at a time when the scales live in the tiles (group
+ * 128: ceil(B/2) passes) and column by column otherwise (one scale per row: B passes).
  */
 int bcq_gemm_smallbatch(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
                         const uint16_t *z_dev, const uint16_t *X_dev, uint16_t *Y_dev, int B,

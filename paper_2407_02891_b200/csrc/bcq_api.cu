@@ -145,13 +145,15 @@ int check_plan(const bcq_desc *d, const bcq_plan *p, int B)
 size_t plan_workspace(const bcq_desc *d, const bcq_plan *p, int B)
 {
     if (p->k_splits <= 1) return 0;
-    if (p->kernel == 1) return kCounterBytes + size_t(p->k_splits) * d->N * sizeof(float);
+    // kernel 1 runs one column per launch, or two when the scales live in the tiles
+    if (p->kernel == 1) return kCounterBytes + size_t(p->k_splits) * ((B >= 2 && interleaved(d)) ? 2 : 1) * d->N * sizeof(float);
     if (p->kernel == 2) return kCounterBytes + size_t(p->k_splits) * B * d->N * sizeof(float);
     return 0;
 }
 
+// cols: 1, or 2 (lookup-table kernel with the scales in the tiles): x and y hold two columns
 int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, const uint16_t *alpha, const uint16_t *z,
-             const uint16_t *x, uint16_t *y, void *ws, size_t ws_bytes, void *stream)
+             const uint16_t *x, uint16_t *y, void *ws, size_t ws_bytes, void *stream, int cols = 1)
 {
     if (!packed || !x || !y) return BCQ_ERR_INVALID_ARG;
     if (interleaved(desc))
@@ -165,13 +167,13 @@ int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, con
     if (plan->kernel == 0) {
         e = launch_generic(*desc, packed, alpha, z, x, y, 1, st);
     } else {
-        const size_t need = plan_workspace(desc, plan, 1);
+        const size_t need = plan_workspace(desc, plan, cols);
         if (need > 0) {
             if (!ws) return BCQ_ERR_INVALID_ARG;
             if (!aligned(ws, 16)) return BCQ_ERR_MISALIGNED;
             if (ws_bytes < need) return BCQ_ERR_WORKSPACE_TOO_SMALL;
         }
-        e = launch_lut_gemv(*desc, *plan, packed, alpha, z, x, y, need ? ws : nullptr, st);
+        e = launch_lut_gemv(*desc, *plan, packed, alpha, z, x, y, need ? ws : nullptr, st, cols);
     }
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
@@ -436,9 +438,13 @@ int bcq_gemm_smallbatch_plan(const bcq_desc *desc, const bcq_plan *plan, const v
         return BCQ_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (plan->kernel == 1) {
-        // The lookup-table kernel once per column: B passes over the weights, each at the batch-1 rate.
-        for (int b = 0; b < B; ++b) {
-            rc = run_gemv(desc, plan, packed, alpha, z, X + size_t(b) * desc->K, Y + size_t(b) * desc->N, ws, ws_bytes, stream);
+        // The lookup-table kernel column by column -- or, with the scales in the tiles, two columns at a
+        // time (tables that hold both columns' sums side by side: one pass over the weights per pair).
+        const int step = interleaved(desc) ? 2 : 1;
+        for (int b = 0; b < B; b += step) {
+            const int cols = (b + step <= B) ? step : 1;
+            rc = run_gemv(desc, plan, packed, alpha, z, X + size_t(b) * desc->K, Y + size_t(b) * desc->N, ws, ws_bytes, stream,
+                          cols);
             if (rc != BCQ_OK) return rc;
         }
         return BCQ_OK;

@@ -106,7 +106,8 @@ cudaError_t launch_permute_scales(const View &src, const View &dst, cudaStream_t
 cudaError_t launch_generic(const bcq_desc &d, const void *packed, const uint16_t *alpha, const uint16_t *z,
                            const uint16_t *X, uint16_t *Y, int B, cudaStream_t st);
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
-                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st);
+                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st,
+                            int cols = 1);
 
 cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *X, uint16_t *Y, int B, void *workspace, cudaStream_t st);

@@ -41,7 +41,6 @@ constexpr int kBuilderThreads = kBuilderWarps * 32;
 constexpr int kFirstConsumerWarp = kBuilderWarps;
 constexpr int kConsumerThreads = kLutWarps * 32;
 constexpr int kLutThreads = (kBuilderWarps + kLutWarps) * 32;      // 896
-constexpr int kTablesBytes = 256 * 256;                            // both fp16 tables, entry stride 256 B
 constexpr int kLutSmemBytes = 232448;                              // 227 KB: the per-block opt-in maximum
 constexpr int kMaxSlotsPerWarp = 5;
 constexpr int kMaxSlots = kLutWarps * kMaxSlotsPerWarp;
@@ -49,7 +48,7 @@ constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
 constexpr int kFixedBytes = 2048;      // barriers and flags
 
 static_assert(8 * kMaxSlots + 64 <= kFixedBytes, "barrier area");
-static_assert(2 * kFixedBytes <= kLutSmemBytes - kTablesBytes, "barriers must fit before or after the tables");
+static_assert(2 * kFixedBytes <= kLutSmemBytes - 2 * 65536, "barriers must fit before or after the tables");
 
 __device__ int g_lut_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
 
@@ -99,6 +98,19 @@ __device__ __forceinline__ void lut_add(float &acc, uint32_t addr)
         "ld.shared.b16 h, [%1+%2];\n\t"
         "add.rn.f32.f16 %0, h, %0;\n\t}"
         : "+f"(acc)
+        : "r"(addr), "n"(OFF));
+}
+// the same for two columns at once: the 4-byte entry holds (column 0, column 1) as fp16
+template <int OFF>
+__device__ __forceinline__ void lut_add2(float &acc0, float &acc1, uint32_t addr)
+{
+    asm volatile(
+        "{\n\t.reg .b16 l, h;\n\t.reg .b32 v;\n\t"
+        "ld.shared.b32 v, [%2+%3];\n\t"
+        "mov.b32 {l, h}, v;\n\t"
+        "add.rn.f32.f16 %0, l, %0;\n\t"
+        "add.rn.f32.f16 %1, h, %1;\n\t}"
+        : "+f"(acc0), "+f"(acc1)
         : "r"(addr), "n"(OFF));
 }
 template <int OFF>
@@ -204,12 +216,77 @@ __device__ __forceinline__ void build_quad(unsigned char *table, const f32x2 (&x
     }
 }
 
+// Two columns.  Table entry e (256 B) = [even chunks: 32 words][odd chunks: 32 words], a word = the fp16
+// sums of (column 0, column 1) for that chunk and entry.  A thread owns the chunk pair cp (chunks 2cp,
+// 2cp + 1) of both columns: xa / xb hold activation j of the two chunks for column 0 / column 1.
+__device__ __forceinline__ void load_pair(const __half *xw, size_t col_stride, int cp, f32x2 (&xa)[8], f32x2 (&xb)[8])
+{
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        const __half *src = xw + c * col_stride + 16 * cp;
+        const uint4 r0 = *reinterpret_cast<const uint4 *>(src), r1 = *reinterpret_cast<const uint4 *>(src + 8);
+        const __half2 *h0 = reinterpret_cast<const __half2 *>(&r0), *h1 = reinterpret_cast<const __half2 *>(&r1);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 f0 = __half22float2(h0[j]), f1 = __half22float2(h1[j]);
+            if (c == 0) {
+                xa[2 * j] = pack2(f0.x, f1.x);
+                xa[2 * j + 1] = pack2(f0.y, f1.y);
+            } else {
+                xb[2 * j] = pack2(f0.x, f1.x);
+                xb[2 * j + 1] = pack2(f0.y, f1.y);
+            }
+        }
+    }
+}
+__device__ __forceinline__ void build_pair(unsigned char *table, const f32x2 (&xa)[8], const f32x2 (&xb)[8], int cp, int hi0,
+                                           int hi_step)
+{
+    const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
+    f32x2 lowa = pack2(0.f, 0.f), lowb = lowa;
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        lowa = fma2(m1, xa[j], lowa);
+        lowb = fma2(m1, xb[j], lowb);
+    }
+    for (int hi = hi0; hi < 32; hi += hi_step) {
+        f32x2 ca = lowa, cb = lowb;
+#pragma unroll
+        for (int j = 3; j < 8; ++j) {
+            const float sg = ((hi >> (j - 3)) & 1) ? 1.f : -1.f;
+            const f32x2 s2 = pack2(sg, sg);
+            ca = fma2(s2, xa[j], ca);
+            cb = fma2(s2, xb[j], cb);
+        }
+        unsigned char *dst = table + cp * 4 + hi * (8 * 256);
+        static_for<0, 8>([&](auto step_c) {
+            constexpr int step = decltype(step_c)::value;
+            constexpr int gray = step ^ (step >> 1);
+            if constexpr (step > 0) {
+                constexpr int bit = (step & 1) ? 0 : ((step & 2) ? 1 : 2);
+                constexpr bool on = (gray >> bit) & 1;
+                ca = fma2(on ? p2 : m2, xa[bit], ca);
+                cb = fma2(on ? p2 : m2, xb[bit], cb);
+            }
+            const float2 a = unpack2(ca), b = unpack2(cb);   // a: column 0 of chunks 2cp, 2cp+1; b: column 1
+            const __half2 even = __floats2half2_rn(a.x, b.x), odd = __floats2half2_rn(a.y, b.y);
+            *reinterpret_cast<uint32_t *>(dst + gray * 256) = *reinterpret_cast<const uint32_t *>(&even);
+            *reinterpret_cast<uint32_t *>(dst + gray * 256 + 128) = *reinterpret_cast<const uint32_t *>(&odd);
+        });
+    }
+}
+
 enum { kWaitEmpty = 1, kWaitFull = 2, kWaitTableReady = 3, kWaitTableFree = 4, kWaitDrain = 5, kTooFewSlots = 6 };
 
-template <int Q, bool GROUPED>
+// NB columns per launch: 1, or 2 (grouped scales only) with tables that hold both columns' sums side by
+// side, so that one 4-byte lookup serves two products; each of the two table buffers then fills a
+// 64 KB region of its own.
+template <int Q, bool GROUPED, int NB>
 __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParams p)
 {
+    static_assert(NB == 1 || (NB == 2 && GROUPED), "two columns need the scales inside the tiles");
     extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int kTablesBytes = NB * 65536;
     using SL = Slot<Q, GROUPED>;
     constexpr int NACC = GROUPED ? 1 : Q;   // accumulators per unit and lane: the row's sum, or one per plane
     constexpr int UMAX = kLutUnitsPerWarp;
@@ -304,9 +381,15 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     // ---- start-up: everybody builds the first window's table -------------------------------------
     if (tid < 512) {
-        f32x2 x01[8], x23[8];
-        load_quad(xblk, tid & 15, x01, x23);
-        build_quad(tables, x01, x23, tid & 15, tid >> 4, 32);
+        if constexpr (NB == 1) {
+            f32x2 x01[8], x23[8];
+            load_quad(xblk, tid & 15, x01, x23);
+            build_quad(tables, x01, x23, tid & 15, tid >> 4, 32);
+        } else {
+            f32x2 xa[8], xb[8];
+            load_pair(xblk, size_t(p.K), tid & 31, xa, xb);
+            build_pair(tables, xa, xb, tid & 31, tid >> 5, 16);
+        }
     }
     __syncthreads();
     if (tid == 0) TRACE(3);
@@ -317,10 +400,16 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         // buffer 0 are windows 2, 4, ... and of buffer 1 windows 1, 3, ...
         for (int wi = 1; wi < nwin; ++wi) {
             const int b = wi & 1, use = wi >> 1;
-            f32x2 x01[8], x23[8];
-            load_quad(xblk + wi * kWindow, tid & 15, x01, x23);   // in flight while waiting for the buffer
+            f32x2 x01[8], x23[8];   // one column: a chunk quad; two columns: a chunk pair of each
+            if constexpr (NB == 1)
+                load_quad(xblk + wi * kWindow, tid & 15, x01, x23);   // in flight while waiting for the buffer
+            else
+                load_pair(xblk + wi * kWindow, size_t(p.K), tid & 31, x01, x23);
             if (use > 0 && !mbar_wait<true>(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, &g_lut_status)) break;   // a long wait: nap longer
-            build_quad(tables + b * 128, x01, x23, tid & 15, tid >> 4, kBuilderThreads / 16);
+            if constexpr (NB == 1)
+                build_quad(tables + b * 128, x01, x23, tid & 15, tid >> 4, kBuilderThreads / 16);
+            else
+                build_pair(tables + b * 65536, x01, x23, tid & 31, tid >> 5, kBuilderThreads / 32);
             mbar_arrive(bar_tab_ready + 8 * b);
         }
         return;
@@ -333,12 +422,14 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
     const int ctid = tid - kFirstConsumerWarp * 32;
     const int g4 = lane >> 3, jr = lane & 7;
-    float acc[UMAX][NACC];
+    float acc[UMAX][NACC], acc1[NB == 2 ? UMAX : 1];   // acc1: the second column
     float xacc = 0.f;   // per-row scales: sum of x over this lane's groups of all windows
 #pragma unroll
     for (int t = 0; t < UMAX; ++t)
 #pragma unroll
         for (int i = 0; i < NACC; ++i) acc[t][i] = 0.f;
+#pragma unroll
+    for (int t = 0; t < (NB == 2 ? UMAX : 1); ++t) acc1[t] = 0.f;
     bool alive = !*abort_flag;
     int d = 0, k = 0;   // this warp's ring position: slot cw + kLutWarps * d, fill number k
 
@@ -361,11 +452,23 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         // next one share the 4-byte column 8 g + ((h + j) mod 8); the odd chunk is its upper half.
         uint32_t off[8];
 #pragma unroll
-        for (int h = 0; h < 8; ++h) off[h] = tab0 + uint32_t(b * 128 + 4 * (8 * g4 + ((h + jr) & 7)));
+        for (int h = 0; h < 8; ++h) off[h] = tab0 + uint32_t(b * (NB == 1 ? 128 : 65536) + 4 * (8 * g4 + ((h + jr) & 7)));
         // sum of x over this lane's group: the all-ones entries of the group's 16 chunks (two per lane)
-        const uint32_t ones = lds_b32<255 * 256>(off[0]);
-        const float2 ones_f = __half22float2(*reinterpret_cast<const __half2 *>(&ones));
-        float xsum = ones_f.x + ones_f.y;
+        float xsum, xsum1 = 0.f;
+        if constexpr (NB == 1) {
+            const uint32_t ones = lds_b32<255 * 256>(off[0]);
+            const float2 ones_f = __half22float2(*reinterpret_cast<const __half2 *>(&ones));
+            xsum = ones_f.x + ones_f.y;
+        } else {
+            const uint32_t even = lds_b32<255 * 256>(off[0]), odd = lds_b32<255 * 256 + 128>(off[0]);
+            const float2 e = __half22float2(*reinterpret_cast<const __half2 *>(&even));
+            const float2 o = __half22float2(*reinterpret_cast<const __half2 *>(&odd));
+            xsum = e.x + o.x;
+            xsum1 = e.y + o.y;
+            xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 1);
+            xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 2);
+            xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 4);
+        }
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
@@ -415,16 +518,21 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                     __syncwarp();
                     if (lane == 0) issue_next(d);
 
-                    float sum[Q][2];
+                    float sum[Q][2], sum1[NB == 2 ? Q : 1][2];
 #pragma unroll
                     for (int i = 0; i < Q; ++i) sum[i][0] = sum[i][1] = 0.f;
+#pragma unroll
+                    for (int i = 0; i < (NB == 2 ? Q : 1); ++i) sum1[i][0] = sum1[i][1] = 0.f;
                     static_for<0, 16>([&](auto S) {
                         constexpr int st = decltype(S)::value;
                         static_for<0, Q>([&](auto I) {
                             constexpr int i = decltype(I)::value;
                             constexpr int pb = i * 16 + st;
                             const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
-                            lut_add<(st & 1) * 2>(sum[i][st & 1], addr);
+                            if constexpr (NB == 1)
+                                lut_add<(st & 1) * 2>(sum[i][st & 1], addr);
+                            else
+                                lut_add2<(st & 1) * 128>(sum[i][st & 1], sum1[i][st & 1], addr);
                         });
                     });
                     if constexpr (GROUPED) {
@@ -432,6 +540,12 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 #pragma unroll
                         for (int i = 0; i < Q; ++i) a = fmaf(__half2float(sc[i]), sum[i][0] + sum[i][1], a);
                         acc[t][0] = a;
+                        if constexpr (NB == 2) {
+                            float a1 = fmaf(__half2float(sc[Q]), xsum1, acc1[t]);
+#pragma unroll
+                            for (int i = 0; i < Q; ++i) a1 = fmaf(__half2float(sc[i]), sum1[i][0] + sum1[i][1], a1);
+                            acc1[t] = a1;
+                        }
                     } else {
 #pragma unroll
                         for (int i = 0; i < Q; ++i) acc[t][i % NACC] += sum[i][0] + sum[i][1];
@@ -460,7 +574,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     }
 
     // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up, lanes 0..7 store ---------
-    float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * p.N : nullptr;
+    // (two columns: y and the partials of column 1 follow those of column 0, N elements further on)
+    float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * NB * p.N : nullptr;
 #pragma unroll
     for (int t = 0; t < UMAX; ++t) {
         float v = acc[t][0];
@@ -476,12 +591,24 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         }
         v += __shfl_xor_sync(0xffffffffu, v, 8);
         v += __shfl_xor_sync(0xffffffffu, v, 16);
+        float v1 = 0.f;
+        if constexpr (NB == 2) {
+            v1 = acc1[t];
+            v1 += __shfl_xor_sync(0xffffffffu, v1, 8);
+            v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
+        }
         if (lane < 8 && cw + kLutWarps * t < V) {
             const int n = (u0 + cw + kLutWarps * t) * kUnitRows + lane;
             if (partial)
                 partial[n] = v;
             else
                 p.y[n] = __float2half_rn(v);
+            if constexpr (NB == 2) {
+                if (partial)
+                    partial[size_t(p.N) + n] = v1;
+                else
+                    p.y[size_t(p.N) + n] = __float2half_rn(v1);
+            }
         }
     }
 
@@ -498,17 +625,20 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         if (*s_last) {
             __threadfence();
             // fixed summation order (deterministic); the loads of 8 splits are issued together
-            for (int n = u0 * kUnitRows + ctid; n < u1 * kUnitRows; n += kConsumerThreads) {
+            const int R = V * kUnitRows;
+            for (int idx = ctid; idx < NB * R; idx += kConsumerThreads) {
+                const int col = idx >= R ? 1 : 0;
+                const size_t at = size_t(col) * p.N + size_t(u0) * kUnitRows + (idx - col * R);
                 float v = 0.f;
                 for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
                     float part[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        part[k] = (k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * p.N + n) : 0.f;
+                        part[k] = (k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at) : 0.f;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) v += part[k];
                 }
-                p.y[n] = __float2half_rn(v);
+                p.y[at] = __float2half_rn(v);
             }
             if (ctid == 0) p.counters[rbi] = 0;
         }
@@ -516,7 +646,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     if (ctid == 0) TRACE(11);
 }
 
-template <int Q, bool GROUPED>
+template <int Q, bool GROUPED, int NB>
 static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
 {
     // The opt-in to more than 48 KB of dynamic shared memory is per function and per device:
@@ -526,7 +656,7 @@ static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(lut_gemv_kernel<Q, GROUPED>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
+        e = cudaFuncSetAttribute(lut_gemv_kernel<Q, GROUPED, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
@@ -540,11 +670,12 @@ static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, GROUPED>, prm);
+    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, GROUPED, NB>, prm);
 }
 
+// cols = 1: y = W x.  cols = 2 (grouped scales only): x and y hold two columns, K and N elements apart.
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
-                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st)
+                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st, int cols)
 {
     LutParams prm;
     prm.tiles = static_cast<const uint8_t *>(packed);
@@ -561,11 +692,21 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
     prm.row_blocks = plan.row_blocks;
     prm.k_splits = plan.k_splits;
     const bool grouped = d.group != 0;
+    if (cols == 2) {
+        if (!grouped) return cudaErrorInvalidValue;
+        switch (d.q) {
+            case 1: return launch_lut_q<1, true, 2>(prm, st);
+            case 2: return launch_lut_q<2, true, 2>(prm, st);
+            case 3: return launch_lut_q<3, true, 2>(prm, st);
+            case 4: return launch_lut_q<4, true, 2>(prm, st);
+        }
+        return cudaErrorInvalidValue;
+    }
     switch (d.q) {
-        case 1: return grouped ? launch_lut_q<1, true>(prm, st) : launch_lut_q<1, false>(prm, st);
-        case 2: return grouped ? launch_lut_q<2, true>(prm, st) : launch_lut_q<2, false>(prm, st);
-        case 3: return grouped ? launch_lut_q<3, true>(prm, st) : launch_lut_q<3, false>(prm, st);
-        case 4: return grouped ? launch_lut_q<4, true>(prm, st) : launch_lut_q<4, false>(prm, st);
+        case 1: return grouped ? launch_lut_q<1, true, 1>(prm, st) : launch_lut_q<1, false, 1>(prm, st);
+        case 2: return grouped ? launch_lut_q<2, true, 1>(prm, st) : launch_lut_q<2, false, 1>(prm, st);
+        case 3: return grouped ? launch_lut_q<3, true, 1>(prm, st) : launch_lut_q<3, false, 1>(prm, st);
+        case 4: return grouped ? launch_lut_q<4, true, 1>(prm, st) : launch_lut_q<4, false, 1>(prm, st);
     }
     return cudaErrorInvalidValue;
 }

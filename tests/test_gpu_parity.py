@@ -297,12 +297,48 @@ def test_small_batch_kernel_explicit_plans(N, K, q, group, rb, ks, B):
     torch.cuda.synchronize()
     bq.poll_status()
     assert rel_err(Y.cpu().numpy(), ref) <= TOL
-    # column by column through the batch-1 kernel: the same numbers up to rounding
+    # through the lookup-table kernel (two columns per pass with group 128, one with per-row scales):
+    # the same numbers up to rounding
     p1 = bq.plan_default(L.d, 1)
     Y1 = torch.zeros_like(Y)
-    bq.gemm_smallbatch_plan(L.d, p1, L.packed, L.alpha, L.z, dev(X), Y1, B, bq.new_workspace(L.d, 1, p1))
+    bq.gemm_smallbatch_plan(L.d, p1, L.packed, L.alpha, L.z, dev(X), Y1, B, bq.new_workspace(L.d, B, p1))
     torch.cuda.synchronize()
+    bq.poll_status()
     assert rel_err(Y1.cpu().numpy(), ref) <= TOL
+
+
+@pytest.mark.parametrize("N,K,q,rb,ks,B", [
+    (264, 1024, 3, 1, 1, 2),       # 33 units, both windows in one block
+    (264, 1024, 3, 1, 2, 2),       # split-K
+    (1536, 1536, 3, 1, 3, 2),      # 192 units: every warp eight units
+    (776, 2560, 2, 2, 5, 3),       # a pair and a single column
+    (512, 1024, 1, 4, 1, 4),
+    (512, 1024, 4, 4, 2, 5),
+    (8, 512, 3, 1, 1, 2),          # one unit, one window
+    (16, 16384, 3, 1, 1, 2),       # 32 windows in one block
+])
+def test_lookup_kernel_on_column_pairs(N, K, q, rb, ks, B):
+    """Plan kernel 1 with group 128 runs two columns per launch (both columns' sums in one table entry)."""
+    group = 128
+    p, codes, alpha, z, X = make_layer(f"pair/{N}x{K}q{q}", N, K, q, group, B)
+    ref = oracle.forward_planes(p, alpha, z, X, group)
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    plan = bq.Plan(1, rb, ks, 0)
+    ws = bq.new_workspace(L.d, B, plan)
+    Y = torch.full((B, N), float("nan"), dtype=torch.float16, device=DEV)
+    for _ in range(2):   # the second call finds the counters as the first one left them
+        bq.gemm_smallbatch_plan(L.d, plan, L.packed, L.alpha, L.z, dev(X), Y, B, ws)
+    torch.cuda.synchronize()
+    bq.poll_status()
+    Yh = Y.cpu().numpy()
+    assert rel_err(Yh, ref) <= TOL
+    # each column equals the batch-1 product of that column bit for bit (same table values, same order of sums)
+    y1 = torch.zeros(N, dtype=torch.float16, device=DEV)
+    ws1 = bq.new_workspace(L.d, 1, plan)
+    for b in range(B):
+        bq.gemv_plan(L.d, plan, L.packed, L.alpha, L.z, dev(X[b]), y1, ws1)
+        torch.cuda.synchronize()
+        assert np.array_equal(y1.cpu().numpy().view(np.uint16), Yh[b].view(np.uint16))
 
 
 def test_small_batch_kernel_structured_inputs():

@@ -137,7 +137,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * N * 4)
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
-    p2 = bq.plan_default(d, 2, 148)                        # two columns: the batch-1 kernel, column by column
+    p2 = bq.plan_default(d, 2, 148)                        # two columns: the lookup-table kernel on a column pair
     assert (p2.kernel, p2.row_blocks, p2.k_splits) == (p.kernel, p.row_blocks, p.k_splits)
     for B in (3, 4, 16):                                   # more: one pass of the tensor-core kernel
         pb = bq.plan_default(d, B, 148)
@@ -145,6 +145,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
         assert 1 <= pb.row_blocks <= U and 1 <= pb.k_splits <= W
         assert -(-U // pb.row_blocks) <= 176 and -(-W // pb.k_splits) <= 32
         assert bq.workspace_bytes(d, B, pb) == (0 if pb.k_splits == 1 else 4096 * 4 + pb.k_splits * B * N * 4)
-        assert bq.workspace_bytes(d, B, p) == bq.workspace_bytes(d, 1, p)   # a batch-1 plan runs column by column
+        # a lookup-table plan runs the columns two at a time: partial sums of two columns
+        assert bq.workspace_bytes(d, B, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * 2 * N * 4)
     assert bq.workspace_bytes(d, 1, bq.plan_default(d, 4, 148)) == 0        # the small-batch kernel needs B >= 2
     assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
