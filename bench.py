@@ -202,12 +202,13 @@ class Stack:
             self.launch_one(it)
 
     def launches_per_step(self):
-        """Kernel launches of one step: one per layer, or one per layer and column where the default
-        plan of the batch is the batch-1 kernel run column by column."""
+        """Kernel launches of one step: one per layer, except where the default plan of the batch is the
+        lookup-table kernel, which takes two columns per launch (one with per-row scales)."""
         n = 0
         for it in self.items:
             plan = self.bq.plan_default(it[0], self.B)
-            n += self.B if (self.B > 1 and plan.kernel == 1) else 1
+            per_launch = 2 if self.bq.scales_in_tiles(it[0]) else 1
+            n += -(-self.B // per_launch) if (self.B > 1 and plan.kernel == 1) else 1
         return n
 
     def capture(self):
@@ -455,7 +456,7 @@ def main():
                                  if bq.lib().bcq_version() == NCU_TRAFFIC["lib_version"]
                                  and args.workload == NCU_TRAFFIC["workload"] and args.layers == 0
                                  and args.batch == 1 and not args.fuse else None),
-                     "kernel": f"lut_gemv_kernel<{w['q']}>" if args.batch <= 2 else f"mma_gemm_kernel<{w['q']}>",
+                     "kernel": f"lut_gemv_kernel<{w['q']}>" if args.batch <= 3 else f"mma_gemm_kernel<{w['q']}>",
                      "algorithmic_bytes_per_launch": stack.bytes // launches_per_step,
                      "launches_per_step": launches_per_step},
         "per_shape": per_shape,

@@ -202,14 +202,14 @@ int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed
 /*
  * Y[b] = W X[b] for b < B, 1 <= B <= 16; X [B][K], Y [B][N] row-major fp16.  Every column is
  * an independent product (the paper defines batch 1 only; Eq. bcw + Eq. fuse_step3 per column).
- * B == 1 is bcq_gemv.  Tiled layout: by default B >= 3 takes ONE pass over the packed weights
+ * B == 1 is bcq_gemv.  Tiled layout: by default B >= 4 takes ONE pass over the packed weights
  * for all columns (plan kernel 2, the tensor-core kernel: a weight bit becomes the fp16 value
  * +-alpha of its row and group, the products with x are exact, all sums fp32; the offset term
- * uses the fp32 group sums of x, kept to 22 bits) and B == 2 runs the lookup-table kernel on the
- * column pair (plan kernel 1 with tables that hold both columns' sums side by side: one pass
- * over the weights, one 4-byte lookup per weight byte for both columns), which is faster for
- * two columns (bcq_plan_default tells which).  The workspace depends on B:
- * bcq_workspace_bytes(desc, B, plan).
+ * uses the fp32 group sums of x, kept to 22 bits) and B == 2, 3 run the lookup-table kernel on
+ * column pairs (plan kernel 1 with tables that hold two columns' sums side by side: one pass
+ * over the weights and one 4-byte lookup per weight byte for both columns of a pair; every
+ * column is bit-identical to bcq_gemv on it), which is faster there (bcq_plan_default tells
+ * which).  The workspace depends on B: bcq_workspace_bytes(desc, B, plan).
  * Canonical layout: one pass of the generic kernel for all columns.
  * bcq_gemm_smallbatch_plan takes the decomposition from the caller; a plan with kernel 1 runs
  * the lookup-table kernel on two columns at a time when the scales live in the tiles (group

@@ -48,7 +48,7 @@ int device_sm_count(int *out)
     return BCQ_OK;
 }
 
-constexpr int kSmallBatchMin = 3;   // from this many columns on the default plan is the tensor-core kernel
+constexpr int kSmallBatchMin = 4;   // from this many columns on the default plan is the tensor-core kernel
 
 bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED; }   // group 128 or one scale per row
 
