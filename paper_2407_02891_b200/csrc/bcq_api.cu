@@ -61,7 +61,7 @@ bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d-
 // It ranks decompositions; it does not predict time exactly.
 long long lut_cost(int U, int W, int rb, int ks, int sm)
 {
-    const long long fixed = 4500, per_window = 700, round = 1200, per_split = 150;
+    const long long fixed = 3600, per_window = 510, round = 920, per_split = 200;
     const long long waves = (static_cast<long long>(rb) * ks + sm - 1) / sm;
     const long long wc = (W + ks - 1) / ks;
     const long long units = (U + rb - 1) / rb;
