@@ -133,7 +133,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert -(-U // p.row_blocks) <= 192 and -(-W // p.k_splits) <= 32
     blocks = p.row_blocks * p.k_splits
     if U * W >= 148 * 8:
-        assert blocks >= 0.75 * 148
+        assert blocks >= 0.7 * 148
     assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * N * 4)
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
