@@ -61,9 +61,10 @@ bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d-
 // row units of a block per window (each consumer warp does one tile), a throughput term per tile and
 // a split-K combine that grows with the number of splits; per launch, the time to get the blocks going.
 // It ranks decompositions; it does not predict time exactly.
-long long lut_cost(int U, int W, int rb, int ks, int sm)
+long long lut_cost(int U, int W, int rb, int ks, int sm, bool grouped)
 {
-    const long long per_window = 620, round = 420, per_tile = 25, per_split = 105, per_block = 37;
+    // (a split costs more with one scale per row: every split applies the row's scales to its sums)
+    const long long per_window = 620, round = 420, per_tile = 25, per_split = grouped ? 105 : 250, per_block = 37;
     const long long blocks = static_cast<long long>(rb) * ks;
     const long long waves = (blocks + sm - 1) / sm;
     const long long wc = (W + ks - 1) / ks;
@@ -86,7 +87,7 @@ int plan_lut(const bcq_desc *d, int sm, bcq_plan *out)
                 const int rb = k == 0 ? rb_min : (k * sm) / ks - j;
                 if (rb < rb_min || rb < 1 || rb > U || rb > kMaxRowBlocks) continue;
                 if (j > 0 && 10LL * rb * ks < 7LL * sm) continue;   // the fit covers plans down to 0.7 of the GPU
-                const long long c = lut_cost(U, W, rb, ks, sm);
+                const long long c = lut_cost(U, W, rb, ks, sm, d->group != 0);
                 if (best < 0 || c < best) {
                     best = c;
                     out->kernel = 1;
