@@ -63,7 +63,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 106
+#define BCQ_VERSION 107
 
 typedef enum bcq_status {
     BCQ_OK = 0,
