@@ -38,7 +38,7 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "opt30b_q3_g128"
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
 # profiles/lut_gemv_kernel_opt30b_q3_g128.md; valid only for the library revision it was taken on.
-NCU_TRAFFIC = {"lib_version": 107, "workload": "opt30b_q3_g128", "bytes_per_launch": 46.1e6}
+NCU_TRAFFIC = {"lib_version": 107, "workload": "opt30b_q3_g128", "bytes_per_launch": 46.4e6}
 METRIC = "BCQ GEMV us/token (sum of all linear layers of the decoder stack, bs=1)"
 UNIT = "us/token"
 
