@@ -3,6 +3,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "bcq_internal.cuh"
 
 using namespace bcq;
@@ -144,6 +146,39 @@ int plan_mma(const bcq_desc *d, int sm, int B, bcq_plan *out)
         }
     }
     return best < 0 ? BCQ_ERR_UNSUPPORTED_SHAPE : BCQ_OK;
+}
+
+// The search above costs a few microseconds; products are launched far more often than shapes change,
+// so the last plans are remembered (a small table, replaced round-robin).
+int cached_plan(const bcq_desc *d, int B, int sm, bcq_plan *out)
+{
+    struct Entry {
+        bcq_desc d;
+        int B, sm;
+        bcq_plan plan;
+    };
+    static Entry table[32];
+    static int used = 0, next = 0;
+    static std::mutex lock;
+    {
+        std::lock_guard<std::mutex> g(lock);
+        for (int i = 0; i < used; ++i) {
+            const Entry &e = table[i];
+            if (e.B == B && e.sm == sm && e.d.N == d->N && e.d.K == d->K && e.d.q == d->q && e.d.group == d->group &&
+                e.d.layout == d->layout) {
+                *out = e.plan;
+                return BCQ_OK;
+            }
+        }
+    }
+    const int rc = B < kSmallBatchMin ? plan_lut(d, sm, out) : plan_mma(d, sm, B, out);
+    if (rc != BCQ_OK) return rc;
+    std::lock_guard<std::mutex> g(lock);
+    Entry &e = table[next];
+    e.d = *d, e.B = B, e.sm = sm, e.plan = *out;
+    next = (next + 1) % 32;
+    if (used < 32) ++used;
+    return BCQ_OK;
 }
 
 // B: the number of columns the plan is for (kernel 1 handles one column per launch, kernel 2 needs 2..16)
@@ -291,7 +326,7 @@ int bcq_plan_default(const bcq_desc *desc, int B, int sm_count, bcq_plan *out)
             rc = device_sm_count(&sm_count);
             if (rc != BCQ_OK) return rc;
         }
-        return B < kSmallBatchMin ? plan_lut(desc, sm_count, out) : plan_mma(desc, sm_count, B, out);
+        return cached_plan(desc, B, sm_count, out);
     }
     return BCQ_OK;
 }

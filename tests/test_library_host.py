@@ -150,3 +150,23 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
         assert bq.workspace_bytes(d, B, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * 2 * N * 4)
     assert bq.workspace_bytes(d, 1, bq.plan_default(d, 4, 148)) == 0        # the small-batch kernel needs B >= 2
     assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
+
+
+def test_default_plans_are_remembered_consistently():
+    """bcq_plan_default keeps its last plans in a small table: more shapes than the table holds, asked
+    twice in different orders and for different batches, always give the same plan."""
+    shapes = [(512 * k, 4096) for k in range(1, 50)]
+    first = {}
+    for B in (1, 8):
+        for (N, K) in shapes:
+            p = bq.plan_default(bq.desc(N, K, 3, 128, bq.LAYOUT_TILED), B, 148)
+            first[(N, K, B)] = (p.kernel, p.row_blocks, p.k_splits)
+    for (N, K) in reversed(shapes):
+        for B in (8, 1):
+            p = bq.plan_default(bq.desc(N, K, 3, 128, bq.LAYOUT_TILED), B, 148)
+            assert first[(N, K, B)] == (p.kernel, p.row_blocks, p.k_splits)
+    # a different GPU size is a different entry
+    a = bq.plan_default(bq.desc(7168, 7168, 3, 128, bq.LAYOUT_TILED), 1, 148)
+    b = bq.plan_default(bq.desc(7168, 7168, 3, 128, bq.LAYOUT_TILED), 1, 64)
+    assert a.row_blocks * a.k_splits <= 148 and b.row_blocks * b.k_splits <= 2 * 64
+    assert (a.row_blocks, a.k_splits) != (b.row_blocks, b.k_splits)
