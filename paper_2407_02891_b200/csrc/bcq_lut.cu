@@ -500,7 +500,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                         wbuf[4 * j + 2] = v.z;
                         wbuf[4 * j + 3] = v.w;
                     }
-                    __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
+                    [[maybe_unused]] __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
                     if constexpr (GROUPED) {
                         const unsigned char *sp = slot + SL::kPlaneBytes + lane * (2 * (Q + 1));
                         if constexpr (Q == 3) {
