@@ -378,6 +378,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     // The weights above are constants; everything from here on (x, partial sums, counters, y) may
     // depend on the previous kernel in the stream: wait for it to be complete and visible.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) TRACE(12);
 
     // ---- start-up: everybody builds the first window's table -------------------------------------
     if (tid < 512) {
@@ -444,8 +445,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             break;
         }
 #ifdef BCQ_TRACE
+        if (ctid == 0 && wi == 0) TRACE(2);   // before the accumulating trace slots: those read global memory
         if (ctid == 0) TRACE_ADD(15, gtime() - tt0);
-        if (ctid == 0 && wi == 0) TRACE(2);
 #endif
         if (ctid == 0 && wi == 0) TRACE(4);
         // Table address part of the lookups of step pair h: chunk 16 g + ((2h + 2j) mod 16) and the
