@@ -626,31 +626,20 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         if (*s_last) {
             __threadfence();
             // fixed summation order (deterministic); the loads of 8 splits are issued together
-            // two rows per thread at a time, all their loads in flight together (a block has at most 2 NB rows per thread)
             const int R = V * kUnitRows;
-            for (int idx = ctid; idx < NB * R; idx += 2 * kConsumerThreads) {
-                const int idx2 = idx + kConsumerThreads;
-                const bool two = idx2 < NB * R;
-                const int col = idx >= R ? 1 : 0, col2 = idx2 >= R ? 1 : 0;
+            for (int idx = ctid; idx < NB * R; idx += kConsumerThreads) {
+                const int col = idx >= R ? 1 : 0;
                 const size_t at = size_t(col) * p.N + size_t(u0) * kUnitRows + (idx - col * R);
-                const size_t at2 = two ? size_t(col2) * p.N + size_t(u0) * kUnitRows + (idx2 - col2 * R) : at;
-                float v = 0.f, v2 = 0.f;
+                float v = 0.f;
                 for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
-                    float part[8], part2[8];
+                    float part[8];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const bool in = k0 + k < p.k_splits;
-                        part[k] = in ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at) : 0.f;
-                        part2[k] = (in && two) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at2) : 0.f;
-                    }
+                    for (int k = 0; k < 8; ++k)
+                        part[k] = (k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at) : 0.f;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        v += part[k];
-                        v2 += part2[k];
-                    }
+                    for (int k = 0; k < 8; ++k) v += part[k];
                 }
                 p.y[at] = __float2half_rn(v);
-                if (two) p.y[at2] = __float2half_rn(v2);
             }
             if (ctid == 0) p.counters[rbi] = 0;
         }
