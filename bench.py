@@ -433,7 +433,7 @@ def main():
         e_ms, h2d, d2h = stack.e2e_steps(max(3, min(args.steps, 20)))
         e_ms = max_over_ranks(e_ms, world, device)
         e2e = {"value": replica_metric(e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "api": "bcq_gemv_host per layer (pinned host x and y), the token captured once in a CUDA graph, one replay + stream sync per token"}
+               "api": "bcq_gemv_host per layer (pinned host x copied in, y stored by the kernel straight into pinned host memory), the token captured once in a CUDA graph, one replay + stream sync per token"}
 
     if rank != 0:
         if world > 1:

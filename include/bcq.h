@@ -227,7 +227,8 @@ int bcq_gemm_smallbatch_plan(const bcq_desc *desc, const bcq_plan *plan, const v
  * bcq_gemv with the activation and the result in HOST memory: enqueues x_host -> x_stage_dev,
  * the product, y_stage_dev -> y_host on `stream` and returns without synchronising (the
  * caller synchronises the stream before reading y_host).  Use page-locked host memory for
- * the copies to be asynchronous.  x_stage_dev [K] and y_stage_dev [N] are caller-owned
+ * the copies to be asynchronous; when y_host is page-locked the kernel stores y into it
+ * directly and y_stage_dev is not used.  x_stage_dev [K] and y_stage_dev [N] are caller-owned
  * device buffers.
  */
 int bcq_gemv_host(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,

@@ -537,8 +537,16 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed, const uint16_t *alph
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(x_stage, x_host, size_t(desc->K) * 2, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e);
-    rc = bcq_gemv(desc, packed, alpha, z, x_stage, y_stage, ws, ws_bytes, stream);
-    if (rc != BCQ_OK) return rc;
+    // Page-locked host memory is addressable from the device: the kernel then stores y there itself
+    // (N fp16 values over the bus, once) and the copy back, a stream operation of its own, is saved.
+    cudaPointerAttributes attr;
+    uint16_t *y_direct = nullptr;
+    if (cudaPointerGetAttributes(&attr, y_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+        y_direct = static_cast<uint16_t *>(attr.devicePointer);
+    else
+        (void)cudaGetLastError();   // pageable memory is not an error here
+    rc = bcq_gemv(desc, packed, alpha, z, x_stage, y_direct ? y_direct : y_stage, ws, ws_bytes, stream);
+    if (rc != BCQ_OK || y_direct) return rc;
     e = cudaMemcpyAsync(y_host, y_stage, size_t(desc->N) * 2, cudaMemcpyDeviceToHost, st);
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }

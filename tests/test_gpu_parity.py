@@ -371,6 +371,13 @@ def test_gemv_host_buffers():
     torch.cuda.synchronize()
     ref = oracle.forward_planes(p, alpha, z, x, group)[0]
     assert rel_err(yh.numpy(), ref) <= TOL
+    # pageable host buffers take the staged path
+    yp = torch.zeros(N, dtype=torch.float16)
+    ys.zero_()
+    bq.gemv_host(L.d, L.packed, L.alpha, L.z, torch.from_numpy(x.reshape(-1).copy()), yp, xs, ys, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(yp.numpy().view(np.uint16), yh.numpy().view(np.uint16))
+    assert np.array_equal(ys.cpu().numpy().view(np.uint16), yh.numpy().view(np.uint16))   # staged through y_stage
 
 
 def test_device_errors_are_reported_not_raised_as_faults():
