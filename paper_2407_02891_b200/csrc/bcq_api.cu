@@ -535,25 +535,17 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed, const uint16_t *alph
     if (rc != BCQ_OK) return rc;
     if (!x_host || !y_host || !x_stage || !y_stage) return BCQ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // Page-locked host memory is addressable from the device: the kernel then reads x from it and stores
-    // y into it itself, and the two copies -- stream operations of their own, each a few microseconds
-    // of latency around a product that takes ten -- are saved.  (Every row block reads its slice of x
-    // over the bus, so x crosses it several times; it is a few kilobytes.)
-    auto mapped = [](const void *host) -> void * {
-        cudaPointerAttributes attr;
-        if (cudaPointerGetAttributes(&attr, host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
-            return attr.devicePointer;
+    cudaError_t e = cudaMemcpyAsync(x_stage, x_host, size_t(desc->K) * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    // Page-locked host memory is addressable from the device: the kernel then stores y there itself
+    // (N fp16 values over the bus, once) and the copy back, a stream operation of its own, is saved.
+    cudaPointerAttributes attr;
+    uint16_t *y_direct = nullptr;
+    if (cudaPointerGetAttributes(&attr, y_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+        y_direct = static_cast<uint16_t *>(attr.devicePointer);
+    else
         (void)cudaGetLastError();   // pageable memory is not an error here
-        return nullptr;
-    };
-    const uint16_t *x_direct = static_cast<const uint16_t *>(mapped(x_host));
-    uint16_t *y_direct = static_cast<uint16_t *>(mapped(y_host));
-    cudaError_t e = cudaSuccess;
-    if (!x_direct) {
-        e = cudaMemcpyAsync(x_stage, x_host, size_t(desc->K) * 2, cudaMemcpyHostToDevice, st);
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
-    rc = bcq_gemv(desc, packed, alpha, z, x_direct ? x_direct : x_stage, y_direct ? y_direct : y_stage, ws, ws_bytes, stream);
+    rc = bcq_gemv(desc, packed, alpha, z, x_stage, y_direct ? y_direct : y_stage, ws, ws_bytes, stream);
     if (rc != BCQ_OK || y_direct) return rc;
     e = cudaMemcpyAsync(y_host, y_stage, size_t(desc->N) * 2, cudaMemcpyDeviceToHost, st);
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
