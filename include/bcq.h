@@ -23,6 +23,10 @@
  *   - fp16 values are IEEE binary16 bit patterns in uint16_t.  Accumulation is fp32;
  *     y is rounded to fp16 (nearest even) once, at the end.  (The lookup-table kernel keeps
  *     its table of 8-activation partial sums in fp16: each is computed in fp32 and rounded once.)
+ *   - Packed operands are constants to the products: bcq_gemv and bcq_gemm_smallbatch may start
+ *     fetching them before the previous kernel in the stream has finished (programmatic dependent
+ *     launch), so write them with this library's calls or plain kernels and copies, which finish
+ *     before the product is launched; x, y and the workspace are ordered as usual.
  *   - Device pointers must be 16-byte aligned (y: 2-byte) or BCQ_ERR_MISALIGNED is returned.
  *   - Return value: BCQ_OK (0) or a negative bcq_status.  No exceptions, no exit().
  *

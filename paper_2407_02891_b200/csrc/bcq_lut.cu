@@ -1,4 +1,5 @@
-// Lookup-table BCQ GEMV (batch 1, tiled layout, group 128) for sm_100a.
+// Lookup-table BCQ GEMV for sm_100a: batch 1 (tiled layout, scales per group of 128 or per row), and a
+// two-column variant for group 128.
 //
 //   y = sum_g ( sum_i alpha_i (B_i x)_g + z (sum x)_g )          (Eq. bcw + Eq. fuse_step3)
 //
@@ -28,6 +29,16 @@
 // own (row, group) scales.  With the 256-byte entry stride and the 64 KB alignment ONE byte-permute
 // builds the complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + column): a
 // lookup is PRMT + LDS.U16 + one mixed-precision add (fp32 += fp16).
+//
+// Two columns (NB = 2).  A lookup moves 2 bytes per lane, half of what the shared-memory pipe delivers
+// per access; with two activation vectors the entry becomes 4 bytes -- the sums of (column 0, column 1)
+// for the same chunk and index -- and one lookup feeds two adds.  Entry e (256 B) is then [even chunks:
+// 32 words][odd chunks: 32 words]; all lanes of a warp are at chunks of one parity at any step, so they
+// still read 32 different words.  Each table buffer fills a 64 KB region of its own.
+//
+// The kernel is launched with programmatic stream serialisation: it lets its dependents start as soon as
+// it runs and waits for its own predecessor only before it touches x, the workspace or y; the packed
+// weights are treated as constants that are complete before the launch.
 //
 // Every wait on an mbarrier is bounded; if one runs out the block sets an abort flag and a
 // device status word, stops waiting, drains its own copies and returns (see lut_status_take).
