@@ -388,3 +388,31 @@ def test_device_errors_are_reported_not_raised_as_faults():
         bq.gemv(d, t, t, t, t, t)
     assert e.value.status == bq.ERR_UNSUPPORTED_SHAPE
     bq.poll_status()        # no bounded wait ran out in any kernel launched so far
+
+
+def test_random_shapes_batches_and_plans():
+    """Seeded random cases over every kernel of the tiled layout: shapes (1..260 row units, 1..11 windows),
+    q, scale granularity, batch, and decompositions (given and default), each against the oracle."""
+    rng = np.random.default_rng(240702891)
+    for case in range(48):
+        q = int(rng.integers(1, 5))
+        group = int(rng.choice([0, 128]))
+        U, W = int(rng.integers(1, 260)), int(rng.integers(1, 12))
+        N, K = 8 * U, 512 * W
+        B = int(rng.choice([1, 1, 2, 3, 4, 5, 8, 9, 16]))
+        kernel = int(rng.choice([1, 2])) if B >= 2 else 1
+        ks = int(rng.integers(1, W + 1))
+        rb_min = -(-U // (192 if kernel == 1 else 176))
+        rb = int(rng.integers(rb_min, min(U, rb_min + 6) + 1))
+        p, codes, alpha, z, X = make_layer(f"random/{case}", N, K, q, group, B)
+        ref = oracle.forward_planes(p, alpha, z, X, group)
+        L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+        Y = torch.empty((B, N), dtype=torch.float16, device=DEV)
+        for plan in (bq.Plan(kernel, rb, ks, 0), bq.plan_default(L.d, B)):
+            ws = bq.new_workspace(L.d, B, plan)
+            Y.fill_(float("nan"))
+            for _ in range(2):
+                bq.gemm_smallbatch_plan(L.d, plan, L.packed, L.alpha, L.z, dev(X), Y, B, ws)
+            torch.cuda.synchronize()
+            bq.poll_status()
+            assert rel_err(Y.cpu().numpy(), ref) <= TOL, (case, N, K, q, group, B, plan.kernel, plan.row_blocks, plan.k_splits)
