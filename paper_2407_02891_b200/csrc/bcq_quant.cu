@@ -126,17 +126,9 @@ __device__ __forceinline__ void write_scales(__half s_h, __half b_h, const Quant
 __device__ __forceinline__ void range_to_scale(float lo, float hi, const QuantTable &tab, __half &s_h, __half &b_h)
 {
     if (lo == 0.f) lo = 0.f;   // a zero minimum is stored as +0
-    // S is DEFINED as the fp64 value s_factor * range / top rounded once to fp16.  An fp32 estimate (four
-    // roundings, relative error below 2.4e-7) rounds to the same fp16 value unless it lies within its error
-    // of a rounding boundary; only then is the fp64 quotient computed.
-    const float range = hi - lo;
-    const float est = __fdiv_rn(__fmul_rn(float(tab.s_factor), range), float(tab.top));
-    const __half below = __float2half_rn(est * (1.f - 4e-7f)), above = __float2half_rn(est * (1.f + 4e-7f));
-    if (__half_as_ushort(below) == __half_as_ushort(above) && est < 60000.f)
-        s_h = below;
-    else
-        s_h = __double2half(__ddiv_rn(__dmul_rn(tab.s_factor, double(hi) - double(lo)), tab.top));
-    b_h = __float2half_rn(lo);   // exact: lo is an fp16 value
+    const double range = double(hi) - double(lo);   // exact
+    s_h = __double2half(__ddiv_rn(__dmul_rn(tab.s_factor, range), tab.top));
+    b_h = __float2half_rn(lo);                      // exact: lo is an fp16 value
 }
 
 // Any group length: one thread per (row, chunk), S and qbias from the range kernel.  Block x of row
