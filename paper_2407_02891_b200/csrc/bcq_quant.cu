@@ -15,6 +15,8 @@
 
 namespace bcq {
 
+constexpr int kQuantRows = 16;   // rows a block walks: the block's table set-up is shared by them
+
 struct QuantTable {
     uint8_t code_of_int[256];
     double plane_weight[4];
@@ -131,19 +133,21 @@ __device__ __forceinline__ void range_to_scale(float lo, float hi, const QuantTa
     b_h = __float2half_rn(lo);                      // exact: lo is an fp16 value
 }
 
-// Any group length: one thread per (row, chunk), S and qbias from the range kernel.  Block x of row
-// blockIdx.x covers chunks 256 blockIdx.y .. + 255.
+// Any group length: one thread per (row, chunk), S and qbias from the range kernel.  Block (x, y) covers
+// rows kQuantRows x .. + kQuantRows - 1 and chunks 256 y .. + 255.
 __global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restrict__ W, const __half *__restrict__ S,
                                                          const __half *__restrict__ qbias, int L, QuantTable tab,
                                                          uint8_t *__restrict__ w_int, const View dst)
 {
     __shared__ uint32_t lut[256];
     load_spread_table(tab, lut);
-    const int n = blockIdx.x, kb = blockIdx.y * 256 + threadIdx.x;
+    const int kb = blockIdx.y * 256 + threadIdx.x;
     if (kb >= dst.K / 8) return;
     const int G = dst.K / L, g = (kb * 8) / L;
-    const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
-    encode_chunk(raw, S[size_t(n) * G + g], qbias[size_t(n) * G + g], tab, lut, w_int, dst, n, kb);
+    for (int n = blockIdx.x * kQuantRows; n < min(dst.N, (blockIdx.x + 1) * kQuantRows); ++n) {
+        const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
+        encode_chunk(raw, S[size_t(n) * G + g], qbias[size_t(n) * G + g], tab, lut, w_int, dst, n, kb);
+    }
 }
 
 // Groups of 128: everything in one pass.  A group is 16 chunks = 16 consecutive lanes, each holding
@@ -155,51 +159,53 @@ __global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restr
     __shared__ uint32_t lut[256];
     load_spread_table(tab, lut);
     const int kbytes = dst.K / 8;   // a multiple of 16: a half-warp is inside the row or outside
-    const int n = blockIdx.x, kb = blockIdx.y * 256 + threadIdx.x;
+    const int kb = blockIdx.y * 256 + threadIdx.x;
     const bool in = kb < kbytes;
-    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-    if (in) raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
-    const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
-    float lo, hi;
-    {
-        const float2 f = __half22float2(h2[0]);
-        lo = fminf(f.x, f.y), hi = fmaxf(f.x, f.y);
+    for (int n = blockIdx.x * kQuantRows; n < min(dst.N, (blockIdx.x + 1) * kQuantRows); ++n) {
+        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+        if (in) raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
+        const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+        float lo, hi;
+        {
+            const float2 f = __half22float2(h2[0]);
+            lo = fminf(f.x, f.y), hi = fmaxf(f.x, f.y);
 #pragma unroll
-        for (int j = 1; j < 4; ++j) {
-            const float2 e = __half22float2(h2[j]);
-            lo = fminf(lo, fminf(e.x, e.y));
-            hi = fmaxf(hi, fmaxf(e.x, e.y));
+            for (int j = 1; j < 4; ++j) {
+                const float2 e = __half22float2(h2[j]);
+                lo = fminf(lo, fminf(e.x, e.y));
+                hi = fmaxf(hi, fmaxf(e.x, e.y));
+            }
         }
-    }
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) {
-        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        for (int o = 8; o > 0; o >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        }
+        // S and qbias by the group's first lane, handed to the other 15; then lanes 0 .. q of the group
+        // each produce one fused scale (alpha_0 .. alpha_{q-1}, z = S centre + qbias) in the same pass.
+        __half s_h = __float2half_rn(0.f), b_h = s_h;
+        const int sub = threadIdx.x & 15;
+        const int g = kb >> 4, G = dst.K / 128;
+        if (sub == 0 && in) {
+            range_to_scale(lo, hi, tab, s_h, b_h);
+            S[size_t(n) * G + g] = s_h;
+            qbias[size_t(n) * G + g] = b_h;
+        }
+        const unsigned pair = uint32_t(__half_as_ushort(s_h)) | (uint32_t(__half_as_ushort(b_h)) << 16);
+        const unsigned got = __shfl_sync(0xffffffffu, pair, (threadIdx.x & 31) & 16);
+        s_h = __ushort_as_half(uint16_t(got & 0xffffu));
+        b_h = __ushort_as_half(uint16_t(got >> 16));
+        if (in && sub <= dst.q) {
+            const double mult = sub < dst.q ? tab.plane_weight[sub & 3] : tab.centre;
+            const double add = sub < dst.q ? 0.0 : double(__half2float(b_h));
+            const uint16_t v = __half_as_ushort(__double2half(double(__half2float(s_h)) * mult + add));   // exact, rounded once
+            if (sub < dst.q)
+                *dst.alpha_elem(sub, n, g) = v;
+            else
+                *dst.z_elem(n, g) = v;
+        }
+        if (in) encode_chunk(raw, s_h, b_h, tab, lut, w_int, dst, n, kb);
     }
-    // S and qbias by the group's first lane, handed to the other 15; then lanes 0 .. q of the group
-    // each produce one fused scale (alpha_0 .. alpha_{q-1}, z = S centre + qbias) in the same pass.
-    __half s_h = __float2half_rn(0.f), b_h = s_h;
-    const int sub = threadIdx.x & 15;
-    const int g = kb >> 4, G = dst.K / 128;
-    if (sub == 0 && in) {
-        range_to_scale(lo, hi, tab, s_h, b_h);
-        S[size_t(n) * G + g] = s_h;
-        qbias[size_t(n) * G + g] = b_h;
-    }
-    const unsigned pair = uint32_t(__half_as_ushort(s_h)) | (uint32_t(__half_as_ushort(b_h)) << 16);
-    const unsigned got = __shfl_sync(0xffffffffu, pair, (threadIdx.x & 31) & 16);
-    s_h = __ushort_as_half(uint16_t(got & 0xffffu));
-    b_h = __ushort_as_half(uint16_t(got >> 16));
-    if (in && sub <= dst.q) {
-        const double mult = sub < dst.q ? tab.plane_weight[sub & 3] : tab.centre;
-        const double add = sub < dst.q ? 0.0 : double(__half2float(b_h));
-        const uint16_t v = __half_as_ushort(__double2half(double(__half2float(s_h)) * mult + add));   // exact, rounded once
-        if (sub < dst.q)
-            *dst.alpha_elem(sub, n, g) = v;
-        else
-            *dst.z_elem(n, g) = v;
-    }
-    if (in) encode_chunk(raw, s_h, b_h, tab, lut, w_int, dst, n, kb);
 }
 
 // One thread per (row, group): the fused scales, written where the destination layout keeps them.
@@ -226,7 +232,7 @@ cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, 
     const size_t units = size_t(dst.N) * dst.G();
     const __half *w = reinterpret_cast<const __half *>(W);
     __half *s = reinterpret_cast<__half *>(S), *b = reinterpret_cast<__half *>(qbias);
-    const dim3 grid(unsigned(dst.N), unsigned((dst.K / 8 + 255) / 256));   // one row per blockIdx.x
+    const dim3 grid(unsigned((dst.N + kQuantRows - 1) / kQuantRows), unsigned((dst.K / 8 + 255) / 256));   // kQuantRows rows per block
     if (L == 128) {
         rtn_fused128_kernel<<<grid, 256, 0, st>>>(w, tab, s, b, w_int, dst);
         return cudaGetLastError();
