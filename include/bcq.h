@@ -21,8 +21,13 @@
  *     enqueue work; they never synchronise.  Errors found on the host return before any
  *     launch.  The current CUDA device must be the one that owns the pointers.
  *   - fp16 values are IEEE binary16 bit patterns in uint16_t.  Accumulation is fp32;
- *     y is rounded to fp16 (nearest even) once, at the end.  (The lookup-table kernel keeps
- *     its table of 8-activation partial sums in fp16: each is computed in fp32 and rounded once.)
+ *     y is rounded to fp16 (nearest even) once, at the end.  The lookup-table kernel keeps
+ *     its table of 8-activation partial sums in fp16: each signed sum of 8 consecutive
+ *     activations x[8c .. 8c+7] is computed in fp32 and rounded once (relative 2^-11 per table
+ *     entry; everything added afterwards is fp32).  Input range: such a sum must stay finite in
+ *     fp16, i.e. |x[8c]| + ... + |x[8c+7]| < 65520 for every chunk c; beyond that the entry becomes
+ *     infinite and so does every y that uses it (the generic kernel, plan kernel 0, has no table
+ *     and no such limit).
  *   - Packed operands are constants to the products: bcq_gemv and bcq_gemm_smallbatch may start
  *     fetching them before the previous kernel in the stream has finished (programmatic dependent
  *     launch), so write them with this library's calls or plain kernels and copies, which finish
@@ -67,7 +72,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 107
+#define BCQ_VERSION 200
 
 typedef enum bcq_status {
     BCQ_OK = 0,
@@ -97,14 +102,20 @@ typedef struct bcq_desc {
  * shape, either layout), 1 = lookup-table kernel (tiled layout, one or two columns per launch),
  * 2 = tensor-core small-batch kernel (tiled layout, 2..16 columns per launch); kernels 1 and 2
  * are launched as row_blocks x k_splits thread blocks; k_splits > 1 needs the workspace.
- * Limits: at most 192 (kernel 1) or 176 (kernel 2) row units of 8 rows per block, at most 32
- * windows of 512 weights per K split. */
+ * Limits: at most 184 (kernel 1; 160 for q = 4 with two columns per launch) or 176 (kernel 2)
+ * row units of 8 rows per block, at most 32 windows of 512 weights per K split.
+ * reserved: 0.  The library's own tests set BCQ_PLAN_TEST_* bits there (kernel 1 only) to see a
+ * bounded wait inside the kernel run out without anything faulting: SHORT_WAITS shortens the
+ * limit of every wait to about a millisecond, WITHHOLD_TABLE makes the table builders keep a
+ * completed table to themselves, so that the warps waiting for it give up.  y is then undefined
+ * and bcq_poll_status reports BCQ_ERR_TIMEOUT. */
 typedef struct bcq_plan {
     int32_t kernel;
     int32_t row_blocks;
     int32_t k_splits;
     int32_t reserved;
 } bcq_plan;
+enum { BCQ_PLAN_TEST_SHORT_WAITS = 1, BCQ_PLAN_TEST_WITHHOLD_TABLE = 2 };
 
 /* ---- sizes (pure host functions; 0 when the descriptor is invalid) -------------------- */
 size_t bcq_packed_bytes(const bcq_desc *desc);   /* q*N*K/8, plus 2*(q+1)*N*G when tiled with group 128 */
@@ -123,7 +134,8 @@ int bcq_plan_default(const bcq_desc *desc, int B, int sm_count, bcq_plan *plan_o
  * workspace holds split-K partial sums and arrival counters.  It must be zero-filled once
  * (bcq_workspace_init) before its first use; every call leaves the counters zero again, so
  * it can be reused by later calls ON THE SAME STREAM.  Two products in flight at once
- * need two workspaces. */
+ * need two workspaces.  After a call that bcq_poll_status reported as timed out the counters
+ * may be left non-zero: zero-fill the workspace again before the next use. */
 size_t bcq_workspace_bytes(const bcq_desc *desc, int B, const bcq_plan *plan /* NULL = default */);
 int bcq_workspace_init(void *workspace_dev, size_t bytes, void *stream);
 
@@ -157,7 +169,8 @@ int bcq_merge_linear(const bcq_desc *desc, const uint8_t *w_int_dev, const uint1
  * the kernels' scratch); w_int [N][K] or NULL; packed / alpha / z exactly as bcq_merge_linear
  * followed by bcq_pack would produce them for desc->layout (alpha and z ignored when the tiles
  * carry the scales).  Asynchronous on `stream`, no allocation.  The paper times no quantiser;
- * this one reads W twice (range, then encode): about 4 bytes per weight of traffic.
+ * this one reads W once for groups of 128 (2 bytes per weight plus the operand written) and
+ * twice (range, then encode) for every other group length.
  */
 int bcq_quantize_rtn(const bcq_desc *desc, const uint16_t *W_dev, int n_bits,
                      const uint8_t *bit_to_plane_host, double s_factor, uint16_t *S_dev,
@@ -193,7 +206,7 @@ int bcq_repack(const bcq_desc *src, const void *packed_src_dev, const uint16_t *
  * y = W x at batch 1 (the definition at the top of this file; Eq. bcw + Eq. fuse_step3).
  * x [K], y [N] fp16.  y is overwritten.  workspace may be NULL when bcq_workspace_bytes is 0.
  * bcq_gemv_plan is the same product with an explicit decomposition (for tuning and tests):
- * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 192 row units (1536 rows)
+ * the plan must have 1 <= row_blocks, 1 <= k_splits <= K/512, at most 184 row units (1472 rows)
  * per row block and at most 32 windows (16384 weights along K) per K split.
  */
 int bcq_gemv(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
@@ -255,10 +268,12 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed_dev, const uint16_t *
  *   - every GPU on which this library is loaded gives up that much memory until the process
  *     exits, whether or not this function is ever called;
  *   - a product whose default decomposition needs more scratch (k_splits * N * 4 bytes plus
- *     16 KiB of counters) is refused with BCQ_ERR_SCRATCH_LIMIT and nothing is launched;
+ *     128 bytes of counters per row block) is refused with BCQ_ERR_SCRATCH_LIMIT and nothing is
+ *     launched;
  *   - the first call on each device looks up the array's device address (a host-side runtime
- *     query, done with that device current).  Make that first call during start-up, before
- *     any stream capture is begun;
+ *     query, done with that device current) and keeps it for as long as the device's primary
+ *     context lives (a cudaDeviceReset invalidates it).  Make that first call during start-up,
+ *     before any stream capture is begun;
  *   - all calls on a device share the one array.  Calls on the same stream are ordered and
  *     safe; calls whose kernels can overlap on the GPU (different streams, no dependency)
  *     race on it and give wrong results.  The array keeps the previous call's contents; the
@@ -274,8 +289,9 @@ int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, const uint16_
  * Every wait inside the kernels (on an mbarrier fed by an asynchronous copy or by other warps)
  * is bounded.  If one ever runs out, the block stops waiting, lets its outstanding copies land,
  * returns without a fault, and records the event in a device status word; y is then undefined.
- * bcq_poll_status synchronises with the device, returns BCQ_ERR_TIMEOUT if that happened since
- * the last poll (detail via bcq_last_cuda_error) and clears the word; BCQ_OK otherwise.
+ * bcq_poll_status waits for all work submitted to the current device (cudaDeviceSynchronize:
+ * non-blocking streams included), returns BCQ_ERR_TIMEOUT if a wait ran out since the last poll
+ * (detail via bcq_last_cuda_error) and clears the word; BCQ_OK otherwise.
  */
 int bcq_poll_status(void);
 

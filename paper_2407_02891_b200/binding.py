@@ -27,6 +27,8 @@ ERR_CUDA = -5
 ERR_SCRATCH_LIMIT = -6
 ERR_TIMEOUT = -7
 NOALLOC_SCRATCH_BYTES = 2 << 20
+PLAN_TEST_SHORT_WAITS = 1      # bcq_plan.reserved bits used by the library's own tests (see include/bcq.h)
+PLAN_TEST_WITHHOLD_TABLE = 2
 
 
 class Desc(ctypes.Structure):

@@ -10,14 +10,19 @@
 using namespace bcq;
 
 namespace {
-
 thread_local char g_cuda_error[256] = "";
+}
 
-int cuda_fail(cudaError_t e)
+// Remember the text of a failed CUDA runtime call for bcq_last_cuda_error(); returns BCQ_ERR_CUDA.
+int bcq::record_cuda_error(cudaError_t e)
 {
     snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
     return BCQ_ERR_CUDA;
 }
+
+namespace {
+
+int cuda_fail(cudaError_t e) { return bcq::record_cuda_error(e); }
 
 bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -57,30 +62,44 @@ bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED
 // tiled layout with grouped scales: alpha and z live inside `packed`
 bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group != 0; }
 
-// Time model of the lookup-table kernel in nanoseconds, fitted to a sweep of decompositions over the
-// layer shapes of the OPT and Llama-2 workloads on B200 (it picks a plan within 1 % of the fastest
-// measured one on average, 4 % at worst): per block, a per-window overhead, one "round" per kLutWarps
-// row units of a block per window (each consumer warp does one tile), a throughput term per tile and
-// a split-K combine that grows with the number of splits; per launch, the time to get the blocks going.
-// It ranks decompositions; it does not predict time exactly.
+// Row units one block of the lookup-table kernel can take for `cols` columns per launch (B >= 2 with the
+// scales in the tiles runs column pairs, and a last single column with the same plan).
+int lut_max_units(const bcq_desc *d, int B)
+{
+    const bool grouped = d->group != 0;
+    int cons = lut_consumer_warps(d->q, grouped, 1);
+    if (B >= 2 && interleaved(d)) {
+        const int c2 = lut_consumer_warps(d->q, grouped, 2);
+        if (c2 < cons) cons = c2;
+    }
+    return cons * kLutUnitsPerWarp;
+}
+
+// Time model of the lookup-table kernel in nanoseconds, from sweeps of decompositions over the layer shapes
+// of the OPT workloads on B200.  The lookups are bound by the shared-memory pipe, so a block's time is
+// its tiles times a constant, plus a cost per window (a table switch), plus the split-K publication and
+// combine; a window cannot take less than the three builder warps need for its table.  It ranks
+// decompositions; it does not predict time exactly.
 long long lut_cost(int U, int W, int rb, int ks, int sm, bool grouped)
 {
     // (a split costs more with one scale per row: every split applies the row's scales to its sums)
-    const long long per_window = 620, round = 420, per_tile = 25, per_split = grouped ? 105 : 250, per_block = 37;
+    const long long per_tile = 38, per_window = 250, table_build = 1200, split_fixed = 1500, per_split = grouped ? 40 : 100,
+                    per_block = 20;
     const long long blocks = static_cast<long long>(rb) * ks;
     const long long waves = (blocks + sm - 1) / sm;
     const long long wc = (W + ks - 1) / ks;
     const long long units = (U + rb - 1) / rb;
-    long long rounds = (units + kLutWarps - 1) / kLutWarps;
-    if (rounds < 1) rounds = 1;
-    const long long block_time = wc * (per_window + rounds * round + units * per_tile) + (ks > 1 ? per_split * ks : 0);
+    long long window_time = units * per_tile + per_window;
+    if (wc > 1 && window_time < table_build) window_time = table_build;
+    const long long block_time = wc * window_time + (ks > 1 ? split_fixed + per_split * ks : 0);
     return waves * block_time + per_block * (blocks < sm ? blocks : sm);
 }
 
-int plan_lut(const bcq_desc *d, int sm, bcq_plan *out)
+int plan_lut(const bcq_desc *d, int B, int sm, bcq_plan *out)
 {
     const int U = d->N / kUnitRows, W = d->K / kWindow;
-    const int rb_min = (U + kMaxUnitsPerBlock - 1) / kMaxUnitsPerBlock;
+    const int max_units = lut_max_units(d, B);
+    const int rb_min = (U + max_units - 1) / max_units;
     long long best = -1;
     for (int ks = (W + kMaxWindowsPerBlock - 1) / kMaxWindowsPerBlock; ks <= W && ks <= 64; ++ks) {
         // row blocks that fill whole waves of the GPU, or a little less than that, and the fewest possible
@@ -171,7 +190,7 @@ int cached_plan(const bcq_desc *d, int B, int sm, bcq_plan *out)
             }
         }
     }
-    const int rc = B < kSmallBatchMin ? plan_lut(d, sm, out) : plan_mma(d, sm, B, out);
+    const int rc = B < kSmallBatchMin ? plan_lut(d, B, sm, out) : plan_mma(d, sm, B, out);
     if (rc != BCQ_OK) return rc;
     std::lock_guard<std::mutex> g(lock);
     Entry &e = table[next];
@@ -186,9 +205,10 @@ int check_plan(const bcq_desc *d, const bcq_plan *p, int B)
 {
     if (p->kernel == 0) return BCQ_OK;
     if ((p->kernel != 1 && p->kernel != 2) || !lut_kernel_covers(d)) return BCQ_ERR_INVALID_ARG;
+    if (p->reserved & ~(BCQ_PLAN_TEST_SHORT_WAITS | BCQ_PLAN_TEST_WITHHOLD_TABLE)) return BCQ_ERR_INVALID_ARG;
     if (p->kernel == 2 && B < 2) return BCQ_ERR_INVALID_ARG;
     const int U = d->N / kUnitRows, W = d->K / kWindow;
-    const int max_units = p->kernel == 1 ? kMaxUnitsPerBlock : kMmaMaxUnitsPerBlock;
+    const int max_units = p->kernel == 1 ? lut_max_units(d, B) : kMmaMaxUnitsPerBlock;
     if (p->row_blocks < 1 || p->row_blocks > U || p->row_blocks > kMaxRowBlocks) return BCQ_ERR_INVALID_ARG;
     if (p->k_splits < 1 || p->k_splits > W) return BCQ_ERR_INVALID_ARG;
     if ((W + p->k_splits - 1) / p->k_splits > kMaxWindowsPerBlock) return BCQ_ERR_INVALID_ARG;
@@ -200,7 +220,7 @@ size_t plan_workspace(const bcq_desc *d, const bcq_plan *p, int B)
 {
     if (p->k_splits <= 1) return 0;
     // kernel 1 runs one column per launch, or two when the scales live in the tiles
-    if (p->kernel == 1) return kCounterBytes + size_t(p->k_splits) * ((B >= 2 && interleaved(d)) ? 2 : 1) * d->N * sizeof(float);
+    if (p->kernel == 1) return lut_counter_bytes(*p) + size_t(p->k_splits) * ((B >= 2 && interleaved(d)) ? 2 : 1) * d->N * sizeof(float);
     if (p->kernel == 2) return kCounterBytes + size_t(p->k_splits) * B * d->N * sizeof(float);
     return 0;
 }
@@ -289,7 +309,8 @@ int bcq_poll_status(void)
 {
     int v = 0;
     int w = 0;
-    cudaError_t e = lut_status_take(&v);
+    cudaError_t e = cudaDeviceSynchronize();   // kernels on non-blocking streams included
+    if (e == cudaSuccess) e = lut_status_take(&v);
     if (e == cudaSuccess) e = mma_status_take(&w);
     if (e != cudaSuccess) return cuda_fail(e);
     if (v != 0 || w != 0) {

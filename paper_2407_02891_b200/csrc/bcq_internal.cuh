@@ -13,15 +13,21 @@ namespace bcq {
 constexpr int kWindow = 512;        // weights along K covered by one lookup-table build
 constexpr int kUnitRows = 8;        // rows of one row unit
 constexpr int kGroupsPerWindow = 4; // 128-weight groups in a window
-constexpr int kLutWarps = 24;       // warps per block of the lookup-table kernel
-constexpr int kLutUnitsPerWarp = 8; // row units a warp keeps accumulators for
-constexpr int kMaxUnitsPerBlock = kLutWarps * kLutUnitsPerWarp;
+constexpr int kLutConsumersMax = 23; // consumer warps per block of the lookup-table kernel (some instantiations have fewer)
+constexpr int kLutUnitsPerWarp = 8;  // row units a consumer warp keeps accumulators for
 constexpr int kMaxWindowsPerBlock = 32; // windows one block may walk (bounds the planner's search)
 constexpr int kMmaWarps = 22;        // consumer warps per block of the small-batch kernel
 constexpr int kMmaPairsPerWarp = 4;  // pairs of row units a warp keeps accumulators for
 constexpr int kMmaMaxUnitsPerBlock = 2 * kMmaWarps * kMmaPairsPerWarp;
 constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace
-constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);
+constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);   // small-batch kernel: one counter per row block
+
+// The lookup-table kernel counts arrivals per (row block, consumer warp): 32 counters per row block at the
+// head of its workspace, the fp32 partial rows behind them.
+inline size_t lut_counter_bytes(const bcq_plan &plan) { return (size_t(plan.row_blocks) * 32 * sizeof(int) + 255) & ~size_t(255); }
+// consumer warps and tiles per copy of the instantiation for (q, scales per group?, columns per launch)
+int lut_consumer_warps(int q, bool grouped, int cols);
+int lut_tiles_per_job(int q, bool grouped, int cols);
 
 inline int n_groups(const bcq_desc &d) { return d.group == 0 ? 1 : d.K / d.group; }
 
@@ -111,6 +117,8 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
 
 cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *X, uint16_t *Y, int B, void *workspace, cudaStream_t st);
+
+int record_cuda_error(cudaError_t e);   // text for bcq_last_cuda_error(); returns BCQ_ERR_CUDA
 
 cudaError_t lut_status_take(int *status);
 cudaError_t mma_status_take(int *status);

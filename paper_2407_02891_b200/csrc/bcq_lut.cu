@@ -4,29 +4,34 @@
 //   y = sum_g ( sum_i alpha_i (B_i x)_g + z (sum x)_g )          (Eq. bcw + Eq. fuse_step3)
 //
 // Per 512-wide window of K the block builds, in shared memory, all 2^8 signed sums of every
-// 8-activation chunk; packed weight bytes index those tables directly.  One block per SM, two
+// 8-activation chunk; packed weight bytes index those tables directly.  One block per SM, three
 // kinds of warps:
 //
-//   builders  (warps 0-3)   build the window tables from x, one window ahead of the consumers
-//                           (two tables, double buffered);
-//   consumers (warps 4-27)  each owns a few shared-memory slots that it keeps filled with bulk
-//                           async copies (cp.async.bulk, completion on an mbarrier), one slot =
-//                           one tile = q*512 B of plane bytes + the unit's alphas and offsets of
-//                           one (window, row unit).  A consumer waits for its next tile, copies
-//                           it into registers, immediately re-uses the slot for the tile that
-//                           many jobs ahead, then looks every weight byte up in the window table
-//                           and accumulates in fp32.  (One warp can start only about 18 bulk
-//                           copies per microsecond: the copies have to be issued by many warps.)
+//   producers (1 or 2 warps) lane c keeps the private ring of consumer warp c filled with bulk async
+//                            copies (cp.async.bulk, completion on the slot's mbarrier).  A slot holds one
+//                            job = kJ consecutive tiles of one window (one contiguous piece of memory), a
+//                            ring kD slots.  The packed weights are constants, so the first slot of every
+//                            ring is requested before the kernel waits for its predecessor in the stream;
+//                            the rest follows once the first table stands (requests queued earlier
+//                            would delay the activations on their way to the block).
+//   builders  (3 warps)      build the window tables from x, one window ahead of the consumers
+//                            (two tables, double buffered);
+//   consumers (kCons warps)  wait for a slot, copy its tiles to registers (handing the slot back after the
+//                            last one), look every weight byte up in the window table and accumulate in
+//                            fp32.  One tile = q*512 B of plane bytes + the unit's alphas and offsets of one
+//                            (window, row unit).
+//
+// The lookup itself is bound by the shared-memory pipe: one 32-lane lookup is one wavefront, a tile of
+// q = 3 planes costs 48 of them plus 14 to bring the tile to registers and 14 for the copy engine to
+// write it; per-tile bookkeeping is kept off the consumers for that reason.
 //
 // Tables.  The sums are computed in fp32 and stored as fp16 (one rounding, relative 2^-11; the
-// accumulation of the looked-up values stays fp32).  Halving the tables to 32 KB each is what
-// leaves 140 KB of shared memory for tiles in flight -- the stream is otherwise bound by the DRAM
-// latency.  Both tables share one 64 KB region at a shared-window address that is a multiple of
-// 64 KB: entry e of table b, chunk c at byte  e*256 + b*128 + (c>>1)*4 + (c&1)*2.  Lane l = 8 g + j
-// of a consumer warp handles row j of a unit and the g-th group of 128 weights of the window; it
-// walks the group's 16 chunks skewed by 2 j, so at every step the 32 lanes address 32 different
-// 4-byte columns -- 32 distinct banks whatever the weight bytes are -- and a lane needs only its
-// own (row, group) scales.  With the 256-byte entry stride and the 64 KB alignment ONE byte-permute
+// accumulation of the looked-up values stays fp32).  Both tables share one 64 KB region at a shared-window
+// address that is a multiple of 64 KB: entry e of table b, chunk c at byte  e*256 + b*128 + (c>>1)*4 +
+// (c&1)*2.  Lane l = 8 g + j of a consumer warp handles row j of a unit and the g-th group of 128 weights
+// of the window; it walks the group's 16 chunks skewed by 2 j, so at every step the 32 lanes address 32
+// different 4-byte columns -- 32 distinct banks whatever the weight bytes are -- and a lane needs only
+// its own (row, group) scales.  With the 256-byte entry stride and the 64 KB alignment ONE byte-permute
 // builds the complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + column): a
 // lookup is PRMT + LDS.U16 + one mixed-precision add (fp32 += fp16).
 //
@@ -36,56 +41,93 @@
 // 32 words][odd chunks: 32 words]; all lanes of a warp are at chunks of one parity at any step, so they
 // still read 32 different words.  Each table buffer fills a 64 KB region of its own.
 //
+// Split K.  The rows of consumer warp c are the same in every K split of a row block.  Each warp stores its
+// partial rows, publishes them (fence + one atomic on the counter of (row block, c)) and is done unless it
+// was the last of the k_splits warps to arrive: that one adds the partial rows in split order
+// (deterministic), rounds and stores y.  No block-wide barrier and no waiting on other blocks.
+//
 // The kernel is launched with programmatic stream serialisation: it lets its dependents start as soon as
 // it runs and waits for its own predecessor only before it touches x, the workspace or y; the packed
 // weights are treated as constants that are complete before the launch.
 //
-// Every wait on an mbarrier is bounded; if one runs out the block sets an abort flag and a
-// device status word, stops waiting, drains its own copies and returns (see lut_status_take).
+// Every wait is bounded; if one runs out the block sets an abort flag and a device status word, stops
+// waiting, sees its own copies land and returns (see lut_status_take).
 #include "bcq_async.cuh"
 #include "bcq_internal.cuh"
 
 namespace bcq {
 
-constexpr int kBuilderWarps = 4;
+constexpr int kLutThreads = 896;                  // 28 warps at 72 registers fill the register file
+constexpr int kLutSmemBytes = 232448;             // 227 KB: the per-block opt-in maximum
+constexpr int kFixedBytes = 2048;                 // barriers and flags
+constexpr int kBuilderWarps = 3;
 constexpr int kBuilderThreads = kBuilderWarps * 32;
-constexpr int kFirstConsumerWarp = kBuilderWarps;
-constexpr int kConsumerThreads = kLutWarps * 32;
-constexpr int kLutThreads = (kBuilderWarps + kLutWarps) * 32;      // 896
-constexpr int kLutSmemBytes = 232448;                              // 227 KB: the per-block opt-in maximum
-constexpr int kMaxSlotsPerWarp = 5;
-constexpr int kMaxSlots = kLutWarps * kMaxSlotsPerWarp;
-constexpr int kMinSlots = kLutWarps;   // one slot per consumer warp at least
-constexpr int kFixedBytes = 2048;      // barriers and flags
-
-static_assert(8 * kMaxSlots + 64 <= kFixedBytes, "barrier area");
-static_assert(2 * kFixedBytes <= kLutSmemBytes - 2 * 65536, "barriers must fit before or after the tables");
+constexpr int kUnitsPerWarp = kLutUnitsPerWarp;   // row units a consumer warp keeps accumulators for
+constexpr int kEarlyJobs = 1;                     // jobs per ring requested before the first table stands
+constexpr int kTestSpinLimit = 1 << 12;           // polls per wait when a test shortens the limit
 
 __device__ int g_lut_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
 
-#ifdef BCQ_TRACE
-// Development aid (not compiled into the product): per-block event times in ns.
-__device__ unsigned long long g_trace[1024][16];
-__device__ __forceinline__ unsigned long long gtime()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define TRACE(slot) do { if (blockIdx.x < 1024) g_trace[blockIdx.x][slot] = gtime(); } while (0)
-#define TRACE_ADD(slot, v) do { if (blockIdx.x < 1024) g_trace[blockIdx.x][slot] += (v); } while (0)
-#else
-#define TRACE(slot) do { } while (0)
-#define TRACE_ADD(slot, v) do { } while (0)
-#endif
-
-// One tile = one ring slot.  GROUPED (group 128): planes + the tile's alphas and offsets;
-// otherwise (one scale per row) the planes only, alphas and offsets live in their own arrays.
-template <int Q, bool GROUPED>
-struct Slot {
-    static constexpr int kPlaneBytes = Q * 512;
-    static constexpr int kBytes = kPlaneBytes + (GROUPED ? Q * 64 + 64 : 0);
+// Geometry of one instantiation: tile bytes, tiles per job (kJ), slots per ring (kD), consumer warps.
+// The rings are cut from the two pieces of shared memory before and after the 64 KB-aligned tables; the
+// sizes below assume the usual 1 KB offset of a block's shared window (the kernel checks what it finds).
+template <int Q, bool GROUPED, int NB>
+struct LutCfg {
+    static constexpr int kTile = Q * 512 + (GROUPED ? Q * 64 + 64 : 0);
+    static constexpr int kTables = NB * 65536;
+    static constexpr int kFront = 65536 - 1024;
+    static constexpr int kBack = kLutSmemBytes - kFront - kTables - kFixedBytes;
+    static constexpr int rings(int j, int d) { return kFront / (j * d * kTile) + kBack / (j * d * kTile); }
+    // preference: two tiles per copy and two slots; then one tile per copy with three or two slots
+    static constexpr int kChoice = rings(2, 2) >= kLutConsumersMax ? 0 : (rings(1, 3) >= kLutConsumersMax ? 1 : 2);
+    static constexpr int kJ = kChoice == 0 ? 2 : 1;
+    static constexpr int kD = kChoice == 0 ? 2 : (kChoice == 1 ? 3 : 2);
+    static constexpr int kCons = rings(kJ, kD) < kLutConsumersMax ? rings(kJ, kD) : kLutConsumersMax;
+    static constexpr int kProducers = kJ == 1 ? 2 : 1;   // one warp starts about 18 copies per microsecond
+    static constexpr int kFirstCons = kProducers + kBuilderWarps;
+    static constexpr int kWorking = kBuilderWarps + kCons;   // warps that take part after the producers split off
+    static constexpr int kJobsPerWarp = kUnitsPerWarp / kJ;
+    static constexpr int kRingBytes = kJ * kD * kTile;
+    static_assert(kCons >= 16 && kFirstCons + kCons <= kLutThreads / 32, "warp budget");
+    static_assert(16 * kCons * kD + 64 <= kFixedBytes, "barrier area");
 };
+
+int lut_consumer_warps(int q, bool grouped, int cols)
+{
+    switch (q * 4 + (grouped ? 2 : 0) + (cols == 2 ? 1 : 0)) {
+        case 4: return LutCfg<1, false, 1>::kCons;
+        case 6: return LutCfg<1, true, 1>::kCons;
+        case 7: return LutCfg<1, true, 2>::kCons;
+        case 8: return LutCfg<2, false, 1>::kCons;
+        case 10: return LutCfg<2, true, 1>::kCons;
+        case 11: return LutCfg<2, true, 2>::kCons;
+        case 12: return LutCfg<3, false, 1>::kCons;
+        case 14: return LutCfg<3, true, 1>::kCons;
+        case 15: return LutCfg<3, true, 2>::kCons;
+        case 16: return LutCfg<4, false, 1>::kCons;
+        case 18: return LutCfg<4, true, 1>::kCons;
+        case 19: return LutCfg<4, true, 2>::kCons;
+    }
+    return 0;
+}
+int lut_tiles_per_job(int q, bool grouped, int cols)
+{
+    switch (q * 4 + (grouped ? 2 : 0) + (cols == 2 ? 1 : 0)) {
+        case 4: return LutCfg<1, false, 1>::kJ;
+        case 6: return LutCfg<1, true, 1>::kJ;
+        case 7: return LutCfg<1, true, 2>::kJ;
+        case 8: return LutCfg<2, false, 1>::kJ;
+        case 10: return LutCfg<2, true, 1>::kJ;
+        case 11: return LutCfg<2, true, 2>::kJ;
+        case 12: return LutCfg<3, false, 1>::kJ;
+        case 14: return LutCfg<3, true, 1>::kJ;
+        case 15: return LutCfg<3, true, 2>::kJ;
+        case 16: return LutCfg<4, false, 1>::kJ;
+        case 18: return LutCfg<4, true, 1>::kJ;
+        case 19: return LutCfg<4, true, 2>::kJ;
+    }
+    return 1;
+}
 
 struct LutParams {
     const uint8_t *tiles;  // tiled operand: per (window, unit) planes (+ alphas, offsets when grouped)
@@ -93,10 +135,11 @@ struct LutParams {
     const __half *z;       // per-row scales only: [u][r]
     const __half *x;
     __half *y;
-    float *partial;  // [k_splits][N] when k_splits > 1
-    int *counters;   // [row_blocks]
+    float *partial;  // [k_splits][cols][N] when k_splits > 1
+    int *counters;   // [row_blocks][32] when k_splits > 1
     int N, K, U, W;
     int row_blocks, k_splits;
+    int test_flags;  // BCQ_PLAN_TEST_* (0 in production)
 };
 
 // table lookup + accumulate: the address register already holds the complete shared-window
@@ -111,6 +154,19 @@ __device__ __forceinline__ void lut_add(float &acc, uint32_t addr)
         : "+f"(acc)
         : "r"(addr), "n"(OFF));
 }
+// the first lookup of a sum: acc = entry
+template <int OFF>
+__device__ __forceinline__ float lut_first(uint32_t addr)
+{
+    float f;
+    asm volatile(
+        "{\n\t.reg .b16 h;\n\t"
+        "ld.shared.b16 h, [%1+%2];\n\t"
+        "cvt.f32.f16 %0, h;\n\t}"
+        : "=f"(f)
+        : "r"(addr), "n"(OFF));
+    return f;
+}
 // the same for two columns at once: the 4-byte entry holds (column 0, column 1) as fp16
 template <int OFF>
 __device__ __forceinline__ void lut_add2(float &acc0, float &acc1, uint32_t addr)
@@ -122,6 +178,18 @@ __device__ __forceinline__ void lut_add2(float &acc0, float &acc1, uint32_t addr
         "add.rn.f32.f16 %0, l, %0;\n\t"
         "add.rn.f32.f16 %1, h, %1;\n\t}"
         : "+f"(acc0), "+f"(acc1)
+        : "r"(addr), "n"(OFF));
+}
+template <int OFF>
+__device__ __forceinline__ void lut_first2(float &acc0, float &acc1, uint32_t addr)
+{
+    asm volatile(
+        "{\n\t.reg .b16 l, h;\n\t.reg .b32 v;\n\t"
+        "ld.shared.b32 v, [%2+%3];\n\t"
+        "mov.b32 {l, h}, v;\n\t"
+        "cvt.f32.f16 %0, l;\n\t"
+        "cvt.f32.f16 %1, h;\n\t}"
+        : "=f"(acc0), "=f"(acc1)
         : "r"(addr), "n"(OFF));
 }
 template <int OFF>
@@ -146,12 +214,6 @@ __device__ __forceinline__ float2 unpack2(f32x2 v)
     asm("mov.b64 {%0,%1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));
     return r;
 }
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
-{
-    f32x2 d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
 {
     f32x2 d;
@@ -168,24 +230,22 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
 // so that a builder can have the next window's activations on their way while it waits for the buffer.
 __device__ __forceinline__ void load_quad(const __half *xw, int cq, f32x2 (&x01)[8], f32x2 (&x23)[8])
 {
-    {
-        float xf[4][8];
+    float xf[4][8];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint4 raw = *reinterpret_cast<const uint4 *>(xw + 32 * cq + 8 * k);
-            const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+    for (int k = 0; k < 4; ++k) {
+        const uint4 raw = *reinterpret_cast<const uint4 *>(xw + 32 * cq + 8 * k);
+        const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float2 f = __half22float2(h2[j]);
-                xf[k][2 * j] = f.x;
-                xf[k][2 * j + 1] = f.y;
-            }
+        for (int j = 0; j < 4; ++j) {
+            const float2 f = __half22float2(h2[j]);
+            xf[k][2 * j] = f.x;
+            xf[k][2 * j + 1] = f.y;
         }
+    }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            x01[j] = pack2(xf[0][j], xf[1][j]);
-            x23[j] = pack2(xf[2][j], xf[3][j]);
-        }
+    for (int j = 0; j < 8; ++j) {
+        x01[j] = pack2(xf[0][j], xf[1][j]);
+        x23[j] = pack2(xf[2][j], xf[3][j]);
     }
 }
 __device__ __forceinline__ void build_quad(unsigned char *table, const f32x2 (&x01)[8], const f32x2 (&x23)[8], int cq, int hi0,
@@ -287,7 +347,24 @@ __device__ __forceinline__ void build_pair(unsigned char *table, const f32x2 (&x
     }
 }
 
-enum { kWaitEmpty = 1, kWaitFull = 2, kWaitTableReady = 3, kWaitTableFree = 4, kWaitDrain = 5, kTooFewSlots = 6 };
+enum { kWaitEmpty = 1, kWaitFull = 2, kWaitTableReady = 3, kWaitTableFree = 4, kWaitDrain = 5, kTooFewRings = 6, kWaitStart = 7 };
+
+// A bounded wait whose limit a test can shorten (see BCQ_PLAN_TEST_SHORT_WAITS).
+template <bool LONG = false>
+__device__ __forceinline__ bool lut_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code, int limit)
+{
+    for (int it = 0; it < limit; ++it) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if (LONG && it >= 8)
+            __nanosleep(256);
+        else
+            __nanosleep(32);
+        if ((it & 255) == 255 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicExch(&g_lut_status, code);
+    return false;
+}
 
 // NB columns per launch: 1, or 2 (grouped scales only) with tables that hold both columns' sums side by
 // side, so that one 4-byte lookup serves two products; each of the two table buffers then fills a
@@ -296,133 +373,171 @@ template <int Q, bool GROUPED, int NB>
 __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParams p)
 {
     static_assert(NB == 1 || (NB == 2 && GROUPED), "two columns need the scales inside the tiles");
+    using C = LutCfg<Q, GROUPED, NB>;
     extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int kTablesBytes = NB * 65536;
-    using SL = Slot<Q, GROUPED>;
+    constexpr int kTile = C::kTile, kJ = C::kJ, kD = C::kD, kCons = C::kCons;
+    constexpr int kSlotBytes = kJ * kTile;
     constexpr int NACC = GROUPED ? 1 : Q;   // accumulators per unit and lane: the row's sum, or one per plane
-    constexpr int UMAX = kLutUnitsPerWarp;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     const int rbi = blockIdx.x % p.row_blocks, ks = blockIdx.x / p.row_blocks;
     const int u0 = int((long long)rbi * p.U / p.row_blocks), u1 = int((long long)(rbi + 1) * p.U / p.row_blocks);
     const int w0 = int((long long)ks * p.W / p.k_splits), w1 = int((long long)(ks + 1) * p.W / p.k_splits);
-    const int V = u1 - u0;       // row units of this block
-    const int nwin = w1 - w0;    // windows of this block
+    const int V = u1 - u0;                       // row units of this block
+    const int nwin = w1 - w0;                    // windows of this block
+    const int njobs = (V + kJ - 1) / kJ;         // jobs per window
+    const int spin_limit = (p.test_flags & BCQ_PLAN_TEST_SHORT_WAITS) ? kTestSpinLimit : kSpinLimit;
 
-    // ---- carve shared memory: [front | tables (64 KB, 64 KB aligned) | back] ----------------------
+    // ---- carve shared memory: [front | tables (64 KB each, 64 KB aligned) | barriers | back] --------------
     const uint32_t base = smem_u32(smem);
     const uint32_t tab0 = (base + 0xFFFFu) & ~0xFFFFu;  // shared-window address of the tables
-    const int front = int(tab0 - base), back = kLutSmemBytes - front - kTablesBytes;
+    const int front = int(tab0 - base), back = kLutSmemBytes - front - C::kTables;
     unsigned char *tables = smem + front;
-    unsigned char *after = tables + kTablesBytes;
+    unsigned char *after = tables + C::kTables;
     const bool fixed_in_back = back >= kFixedBytes;
     unsigned char *fixed = fixed_in_back ? after : smem;
     unsigned char *ring_a = fixed_in_back ? smem : smem + kFixedBytes;
     unsigned char *ring_b = fixed_in_back ? after + kFixedBytes : after;
-    const int n_a = (fixed_in_back ? front : front - kFixedBytes) / SL::kBytes;
-    const int n_b = (fixed_in_back ? back - kFixedBytes : back) / SL::kBytes;
-    const int NS = min(n_a + n_b, kMaxSlots);
-    const int D = min(NS / kLutWarps, kMaxSlotsPerWarp);   // ring slots per consumer warp
-    unsigned char *const ring_b0 = ring_b - n_a * SL::kBytes;   // so that slot s of either piece is at piece + s * kBytes
-    auto slot_ptr = [&](int s) -> unsigned char * { return (s < n_a ? ring_a : ring_b0) + s * SL::kBytes; };
+    const int rings_a = (fixed_in_back ? front : front - kFixedBytes) / C::kRingBytes;
+    const int rings_b = (fixed_in_back ? back - kFixedBytes : back) / C::kRingBytes;
+    auto ring_ptr = [&](int c) -> unsigned char * {
+        return c < rings_a ? ring_a + c * C::kRingBytes : ring_b + (c - rings_a) * C::kRingBytes;
+    };
 
     const uint32_t bars = smem_u32(fixed);
-    const uint32_t bar_full = bars;
-    const uint32_t bar_tab_ready = bars + 8 * kMaxSlots, bar_tab_free = bar_tab_ready + 16;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 8 * kMaxSlots + 32);
-    int *s_last = const_cast<int *>(abort_flag) + 1;
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kCons * kD;     // [consumer][slot]
+    const uint32_t bar_tab_ready = bars + 16 * kCons * kD, bar_tab_free = bar_tab_ready + 16;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 16 * kCons * kD + 32);
+    volatile int *started = abort_flag + 1;
 
-    if (tid == 0) TRACE(0);
-#ifdef BCQ_TRACE
-    if (tid == 0) { g_trace[blockIdx.x % 1024][13] = 0; g_trace[blockIdx.x % 1024][14] = 0; g_trace[blockIdx.x % 1024][15] = 0; }
-#endif
     if (warp == 0) {   // one warp initialises the barriers, a few each
-        for (int s = lane; s < kMaxSlots; s += 32) mbar_init(bar_full + 8 * s, 1);
+        for (int s = lane; s < kCons * kD; s += 32) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
         if (lane < 2) {
             mbar_init(bar_tab_ready + 8 * lane, kBuilderThreads);
-            mbar_init(bar_tab_free + 8 * lane, kLutWarps);
+            mbar_init(bar_tab_free + 8 * lane, kCons);
         }
         if (lane == 0) {
-            *abort_flag = (NS < kMinSlots) ? 1 : 0;
-            if (NS < kMinSlots) atomicExch(&g_lut_status, int(kTooFewSlots));
+            // every consumer warp needs its ring, and the block's row units must fit the consumers
+            const bool bad = rings_a + rings_b < kCons || njobs > kCons * C::kJobsPerWarp;
+            *abort_flag = bad ? 1 : 0;
+            *started = 0;
+            if (bad) atomicExch(&g_lut_status, int(kTooFewRings));
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    if (tid == 0) TRACE(1);
     // Programmatic dependent launch: the next kernel in the stream may start taking SMs as soon as
     // this kernel's blocks leave them (it still waits, below, for its predecessor to finish before
     // it reads x or writes anything).  Without the launch attribute both instructions do nothing.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+    // Work of consumer c: jobs jb = c, c + kCons, ... of every window, in that order; its m-th job uses slot
+    // m % kD of its ring in fill number m / kD.
     // =============================================================================================
-    const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
-    // ---- consumer warps: job bookkeeping, and the first D tiles of each warp on their way -----------
-    // A warp's jobs, in the order it consumes them: windows outermost, its units innermost.  Lane 0
-    // keeps D of them in flight; the issue cursor (iw, it) runs D jobs ahead of the consumption.
-    const int cw = warp - kFirstConsumerWarp;   // 0 .. kLutWarps-1 for consumers, negative for builders
-    const int mine = (cw >= 0 && V > cw) ? (V - cw + kLutWarps - 1) / kLutWarps : 0;   // units of this warp per window
-    const int total_jobs = mine * nwin;
-    int issued = 0, consumed = 0, it = 0;
-    // the next tile to fetch: this warp's units of a window are kLutWarps tiles apart, then on to the next window
-    const uint8_t *src = p.tiles + (size_t(w0) * p.U + u0 + (cw < 0 ? 0 : cw)) * SL::kBytes;
-    const long long unit_step = (long long)kLutWarps * SL::kBytes;
-    const long long window_step = ((long long)p.U - (long long)kLutWarps * mine) * SL::kBytes;
-    auto issue_next = [&](int slot_d) {   // lane 0 of a consumer warp only
-        if (issued < total_jobs) {
-            const int s = cw + kLutWarps * slot_d;
-            const uint32_t full = bar_full + 8 * s;
-            mbar_expect_tx(full, SL::kBytes);
-            bulk_g2s(smem_u32(slot_ptr(s)), src, SL::kBytes, full);   // planes + alphas + offsets
-            ++issued;
-            src += unit_step;
-            if (++it == mine) {
-                it = 0;
-                src += window_step;
+    // ---- producers: lane -> consumer c; keeps that consumer's ring filled ---------------------------
+    if (warp < C::kProducers) {
+        const int c = lane * C::kProducers + warp;
+        const int mine = (c < kCons && njobs > c) ? (njobs - c + kCons - 1) / kCons : 0;   // jobs per window
+        if (mine > 0 && !*abort_flag) {
+            const uint32_t ring = smem_u32(ring_ptr(c));
+            const uint32_t full0 = bar_full + 8 * kD * c, empty0 = bar_empty + 8 * kD * c;
+            int slot = 0, fill = 0, issued = 0;
+            const uint8_t *src_w = p.tiles + (size_t(w0) * p.U + u0) * kTile;
+            bool ok = true;
+            for (int wi = 0; wi < nwin && ok; ++wi) {
+                for (int jb = c; jb < njobs; jb += kCons) {
+                    if (issued == kEarlyJobs) {
+                        // The rest of the ring waits until the first table stands.  First wait, like the other
+                        // warps, for the previous kernel (however long it runs); the flag follows shortly.
+                        asm volatile("griddepcontrol.wait;" ::: "memory");
+                        int itr = 0;
+                        while (!*started && !*abort_flag && itr < spin_limit) {
+                            __nanosleep(64);
+                            ++itr;
+                        }
+                        if (!*started) {
+                            if (!*abort_flag) {
+                                *abort_flag = 1;
+                                atomicExch(&g_lut_status, int(kWaitStart));
+                            }
+                            ok = false;
+                            break;
+                        }
+                    }
+                    if (fill > 0 && !lut_wait(empty0 + 8 * slot, (fill - 1) & 1, abort_flag, kWaitEmpty, spin_limit)) {
+                        ok = false;
+                        break;
+                    }
+                    const int nt = min(kJ, V - kJ * jb);
+                    mbar_expect_tx(full0 + 8 * slot, nt * kTile);
+                    bulk_g2s(ring + slot * kSlotBytes, src_w + size_t(kJ * jb) * kTile, nt * kTile, full0 + 8 * slot);
+                    ++issued;
+                    if (++slot == kD) {
+                        slot = 0;
+                        ++fill;
+                    }
+                }
+                src_w += size_t(p.U) * kTile;
+            }
+            // See the lane's last copies land before the block's shared memory can be handed to another
+            // block (they have landed long ago unless the block is giving up).
+            for (int m = max(0, issued - kD); m < issued; ++m) {
+                bool landed = false;
+                for (int itr = 0; itr < kSpinLimit && !landed; ++itr) {
+                    landed = mbar_test_wait(full0 + 8 * (m % kD), uint32_t((m / kD) & 1));
+                    if (!landed) __nanosleep(256);
+                }
+                if (!landed) atomicExch(&g_lut_status, int(kWaitDrain));
             }
         }
-    };
-    if (cw >= 0 && lane == 0 && !*abort_flag)
-        for (int q5 = 0; q5 < D; ++q5) issue_next(q5);
+        return;
+    }
+    if (warp >= C::kFirstCons + kCons) return;   // warps this instantiation has no use for
 
+    // =============================================================================================
     // The weights above are constants; everything from here on (x, partial sums, counters, y) may
     // depend on the previous kernel in the stream: wait for it to be complete and visible.
+    const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (tid == 0) TRACE(12);
 
-    // ---- start-up: everybody builds the first window's table -------------------------------------
-    if (tid < 512) {
+    // ---- start-up: builders and consumers build the first window's table together -----------------
+    const int bt = tid - C::kProducers * 32;   // 0 .. kWorking*32-1
+    if (bt < 512) {
         if constexpr (NB == 1) {
             f32x2 x01[8], x23[8];
-            load_quad(xblk, tid & 15, x01, x23);
-            build_quad(tables, x01, x23, tid & 15, tid >> 4, 32);
+            load_quad(xblk, bt & 15, x01, x23);
+            build_quad(tables, x01, x23, bt & 15, bt >> 4, 32);
         } else {
             f32x2 xa[8], xb[8];
-            load_pair(xblk, size_t(p.K), tid & 31, xa, xb);
-            build_pair(tables, xa, xb, tid & 31, tid >> 5, 16);
+            load_pair(xblk, size_t(p.K), bt & 31, xa, xb);
+            build_pair(tables, xa, xb, bt & 31, bt >> 5, 16);
         }
     }
-    __syncthreads();
-    if (tid == 0) TRACE(3);
+    named_barrier(1, C::kWorking * 32);
+    if (bt == 0) *started = 1;
 
-    if (warp < kBuilderWarps) {
+    if (warp < C::kFirstCons) {
         // ---- builders: one table per window, one window ahead of the consumers ----------------------
-        // Window 0 was built by everybody above (published by __syncthreads); the builders' fills of
-        // buffer 0 are windows 2, 4, ... and of buffer 1 windows 1, 3, ...
+        // Window 0 was built above; the builders' fills of buffer 0 are windows 2, 4, ... and of
+        // buffer 1 windows 1, 3, ...
+        const bool withhold = (p.test_flags & BCQ_PLAN_TEST_WITHHOLD_TABLE) != 0;
         for (int wi = 1; wi < nwin; ++wi) {
             const int b = wi & 1, use = wi >> 1;
             f32x2 x01[8], x23[8];   // one column: a chunk quad; two columns: a chunk pair of each
             if constexpr (NB == 1)
-                load_quad(xblk + wi * kWindow, tid & 15, x01, x23);   // in flight while waiting for the buffer
+                load_quad(xblk + wi * kWindow, bt & 15, x01, x23);   // in flight while waiting for the buffer
             else
-                load_pair(xblk + wi * kWindow, size_t(p.K), tid & 31, x01, x23);
-            if (use > 0 && !mbar_wait<true>(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, &g_lut_status)) break;   // a long wait: nap longer
+                load_pair(xblk + wi * kWindow, size_t(p.K), bt & 31, x01, x23);
+            if (use > 0 && !lut_wait<true>(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, spin_limit)) break;
             if constexpr (NB == 1)
-                build_quad(tables + b * 128, x01, x23, tid & 15, tid >> 4, kBuilderThreads / 16);
+                build_quad(tables + b * 128, x01, x23, bt & 15, bt >> 4, kBuilderThreads / 16);
             else
-                build_pair(tables + b * 65536, x01, x23, tid & 31, tid >> 5, kBuilderThreads / 32);
-            mbar_arrive(bar_tab_ready + 8 * b);
+                build_pair(tables + b * 65536, x01, x23, bt & 31, bt >> 5, kBuilderThreads / 32);
+            if (!withhold) mbar_arrive(bar_tab_ready + 8 * b);   // (a test withholds it to see the consumers give up)
         }
         return;
     }
@@ -432,34 +547,27 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     // Lane l = 8 g + j owns row 8u + j of every unit and the g-th group of 128 weights of every
     // window: its 16q bytes of a tile are the group's 16 chunks (skewed by 2 j, see the layout), so
     // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
-    const int ctid = tid - kFirstConsumerWarp * 32;
+    const int cw = warp - C::kFirstCons;
     const int g4 = lane >> 3, jr = lane & 7;
-    float acc[UMAX][NACC], acc1[NB == 2 ? UMAX : 1];   // acc1: the second column
+    float acc[kUnitsPerWarp][NACC], acc1[NB == 2 ? kUnitsPerWarp : 1];   // acc1: the second column
     float xacc = 0.f;   // per-row scales: sum of x over this lane's groups of all windows
 #pragma unroll
-    for (int t = 0; t < UMAX; ++t)
+    for (int t = 0; t < kUnitsPerWarp; ++t)
 #pragma unroll
         for (int i = 0; i < NACC; ++i) acc[t][i] = 0.f;
 #pragma unroll
-    for (int t = 0; t < (NB == 2 ? UMAX : 1); ++t) acc1[t] = 0.f;
+    for (int t = 0; t < (NB == 2 ? kUnitsPerWarp : 1); ++t) acc1[t] = 0.f;
     bool alive = !*abort_flag;
-    int d = 0, k = 0;   // this warp's ring position: slot cw + kLutWarps * d, fill number k
-
+    const unsigned char *ring = ring_ptr(cw);
+    const uint32_t full0 = bar_full + 8 * kD * cw, empty0 = bar_empty + 8 * kD * cw;
+    int slot = 0, fill = 0;
 
     for (int wi = 0; wi < nwin && alive; ++wi) {
         const int b = wi & 1;
-#ifdef BCQ_TRACE
-        const unsigned long long tt0 = gtime();
-#endif
-        if (wi > 0 && !mbar_wait(bar_tab_ready + 8 * b, ((wi >> 1) - (b == 0 ? 1 : 0)) & 1, abort_flag, kWaitTableReady, &g_lut_status)) {
+        if (wi > 0 && !lut_wait(bar_tab_ready + 8 * b, ((wi >> 1) - (b == 0 ? 1 : 0)) & 1, abort_flag, kWaitTableReady, spin_limit)) {
             alive = false;
             break;
         }
-#ifdef BCQ_TRACE
-        if (ctid == 0 && wi == 0) TRACE(2);   // before the accumulating trace slots: those read global memory
-        if (ctid == 0) TRACE_ADD(15, gtime() - tt0);
-#endif
-        if (ctid == 0 && wi == 0) TRACE(4);
         // Table address part of the lookups of step pair h: chunk 16 g + ((2h + 2j) mod 16) and the
         // next one share the 4-byte column 8 g + ((h + j) mod 8); the odd chunk is its upper half.
         uint32_t off[8];
@@ -486,118 +594,108 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
         xacc += xsum;
 
-        static_for<0, UMAX>([&](auto T) {
+        static_for<0, C::kJobsPerWarp>([&](auto T) {
             constexpr int t = decltype(T)::value;
-            if (alive && cw + kLutWarps * t < V) {
-                const int s = cw + kLutWarps * d;
-#ifdef BCQ_TRACE
-                const unsigned long long tw0 = gtime();
-#endif
-                const bool got = mbar_wait(bar_full + 8 * s, k & 1, abort_flag, kWaitFull, &g_lut_status);
-#ifdef BCQ_TRACE
-                if (ctid == 0) { TRACE_ADD(13, gtime() - tw0); TRACE_ADD(14, 1); if (wi == 0 && t == 0) TRACE(5); }
-#endif
-                if (!got) {
+            const int jb = cw + kCons * t;
+            if (alive && jb < njobs) {
+                if (!lut_wait(full0 + 8 * slot, fill & 1, abort_flag, kWaitFull, spin_limit)) {
                     alive = false;
                 } else {
-                    ++consumed;
-                    // slot -> registers, then hand the slot back to the producer
-                    const unsigned char *slot = slot_ptr(s);
-                    uint32_t wbuf[4 * Q];
+                    const unsigned char *sl = ring + slot * kSlotBytes;
+                    const int nt = min(kJ, V - kJ * jb);   // the last job of a window may be short
+                    static_for<0, kJ>([&](auto TT) {
+                        constexpr int tt = decltype(TT)::value;
+                        constexpr int a = t * kJ + tt;     // accumulator slot of this unit
+                        if (tt < nt) {
+                            const unsigned char *tile = sl + tt * kTile;
+                            uint32_t wbuf[4 * Q];
 #pragma unroll
-                    for (int j = 0; j < Q; ++j) {
-                        const uint4 v = *reinterpret_cast<const uint4 *>(slot + j * 512 + lane * 16);
-                        wbuf[4 * j + 0] = v.x;
-                        wbuf[4 * j + 1] = v.y;
-                        wbuf[4 * j + 2] = v.z;
-                        wbuf[4 * j + 3] = v.w;
-                    }
-                    [[maybe_unused]] __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
-                    if constexpr (GROUPED) {
-                        const unsigned char *sp = slot + SL::kPlaneBytes + lane * (2 * (Q + 1));
-                        if constexpr (Q == 3) {
-                            *reinterpret_cast<uint2 *>(sc) = *reinterpret_cast<const uint2 *>(sp);
-                        } else if constexpr (Q == 1) {
-                            *reinterpret_cast<uint32_t *>(sc) = *reinterpret_cast<const uint32_t *>(sp);
-                        } else {
+                            for (int j = 0; j < Q; ++j) {
+                                const uint4 v = *reinterpret_cast<const uint4 *>(tile + j * 512 + lane * 16);
+                                wbuf[4 * j + 0] = v.x;
+                                wbuf[4 * j + 1] = v.y;
+                                wbuf[4 * j + 2] = v.z;
+                                wbuf[4 * j + 3] = v.w;
+                            }
+                            [[maybe_unused]] __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
+                            if constexpr (GROUPED) {
+                                const unsigned char *sp = tile + Q * 512 + lane * (2 * (Q + 1));
+                                if constexpr (Q == 3) {
+                                    *reinterpret_cast<uint2 *>(sc) = *reinterpret_cast<const uint2 *>(sp);
+                                } else if constexpr (Q == 1) {
+                                    *reinterpret_cast<uint32_t *>(sc) = *reinterpret_cast<const uint32_t *>(sp);
+                                } else {
 #pragma unroll
-                            for (int i = 0; i <= Q; ++i) sc[i] = reinterpret_cast<const __half *>(sp)[i];
+                                    for (int i = 0; i <= Q; ++i) sc[i] = reinterpret_cast<const __half *>(sp)[i];
+                                }
+                            }
+                            if (tt == nt - 1) {   // the slot's last tile is in registers: hand the slot back
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(empty0 + 8 * slot);
+                            }
+                            float sum[Q], sum1[NB == 2 ? Q : 1];
+                            static_for<0, 16>([&](auto S) {
+                                constexpr int st = decltype(S)::value;
+                                static_for<0, Q>([&](auto I) {
+                                    constexpr int i = decltype(I)::value;
+                                    constexpr int pb = i * 16 + st;
+                                    const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
+                                    if constexpr (NB == 1) {
+                                        if constexpr (st == 0)
+                                            sum[i] = lut_first<0>(addr);
+                                        else
+                                            lut_add<(st & 1) * 2>(sum[i], addr);
+                                    } else {
+                                        if constexpr (st == 0)
+                                            lut_first2<0>(sum[i], sum1[i], addr);
+                                        else
+                                            lut_add2<(st & 1) * 128>(sum[i], sum1[i], addr);
+                                    }
+                                });
+                            });
+                            if constexpr (GROUPED) {
+                                float v = fmaf(__half2float(sc[Q]), xsum, acc[a][0]);
+#pragma unroll
+                                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(sc[i]), sum[i], v);
+                                acc[a][0] = v;
+                                if constexpr (NB == 2) {
+                                    float v1 = fmaf(__half2float(sc[Q]), xsum1, acc1[a]);
+#pragma unroll
+                                    for (int i = 0; i < Q; ++i) v1 = fmaf(__half2float(sc[i]), sum1[i], v1);
+                                    acc1[a] = v1;
+                                }
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < Q; ++i) acc[a][i] += sum[i];
+                            }
                         }
-                    }
-                    // The tile is in registers: order those reads before the next copy into the slot
-                    // (generic-proxy reads, then an async-proxy write), then refill the slot.
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) issue_next(d);
-
-                    float sum[Q][2], sum1[NB == 2 ? Q : 1][2];
-#pragma unroll
-                    for (int i = 0; i < Q; ++i) sum[i][0] = sum[i][1] = 0.f;
-#pragma unroll
-                    for (int i = 0; i < (NB == 2 ? Q : 1); ++i) sum1[i][0] = sum1[i][1] = 0.f;
-                    static_for<0, 16>([&](auto S) {
-                        constexpr int st = decltype(S)::value;
-                        static_for<0, Q>([&](auto I) {
-                            constexpr int i = decltype(I)::value;
-                            constexpr int pb = i * 16 + st;
-                            const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
-                            if constexpr (NB == 1)
-                                lut_add<(st & 1) * 2>(sum[i][st & 1], addr);
-                            else
-                                lut_add2<(st & 1) * 128>(sum[i][st & 1], sum1[i][st & 1], addr);
-                        });
                     });
-                    if constexpr (GROUPED) {
-                        float a = fmaf(__half2float(sc[Q]), xsum, acc[t][0]);
-#pragma unroll
-                        for (int i = 0; i < Q; ++i) a = fmaf(__half2float(sc[i]), sum[i][0] + sum[i][1], a);
-                        acc[t][0] = a;
-                        if constexpr (NB == 2) {
-                            float a1 = fmaf(__half2float(sc[Q]), xsum1, acc1[t]);
-#pragma unroll
-                            for (int i = 0; i < Q; ++i) a1 = fmaf(__half2float(sc[i]), sum1[i][0] + sum1[i][1], a1);
-                            acc1[t] = a1;
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < Q; ++i) acc[t][i % NACC] += sum[i][0] + sum[i][1];
+                    if (++slot == kD) {
+                        slot = 0;
+                        ++fill;
                     }
-                }
-                if (++d == D) {
-                    d = 0;
-                    ++k;
                 }
             }
         });
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tab_free + 8 * b);
-        if (ctid == 0 && wi < 4) TRACE(6 + wi);
     }
+    if (!alive) return;   // the block is giving up: y is undefined (bcq_poll_status reports it)
 
-    // Gave up on a wait: copies this warp started may still be in flight.  See them land (bounded)
-    // before the block's shared memory can be handed to another block.
-    if (!alive && lane == 0) {
-        for (int m = consumed; m < issued; ++m) {
-            bool landed = false;
-            for (int itr = 0; itr < kSpinLimit && !landed; ++itr)
-                landed = mbar_try_wait(bar_full + 8 * (cw + kLutWarps * (m % D)), uint32_t((m / D) & 1));
-            if (!landed) atomicExch(&g_lut_status, int(kWaitDrain));
-        }
-    }
-
-    // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up, lanes 0..7 store ---------
-    // (two columns: y and the partials of column 1 follow those of column 0, N elements further on)
+    // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up; lanes 0..7 store y, or this K
+    // split's partial rows (two columns: those of column 1 follow column 0, N elements further on) ------
     float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * NB * p.N : nullptr;
 #pragma unroll
-    for (int t = 0; t < UMAX; ++t) {
-        float v = acc[t][0];
+    for (int a = 0; a < kUnitsPerWarp; ++a) {
+        const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;   // the unit, counted inside the block
+        float v = acc[a][0];
         if constexpr (!GROUPED) {
             // one scale per row: apply the row's alphas and offset to the sums over this block's K range
-            const int u = u0 + cw + kLutWarps * t;
             v = 0.f;
-            if (u < u1) {
+            if (ul < V) {
+                const int u = u0 + ul;
 #pragma unroll
-                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(p.alpha[(size_t(u) * Q + i) * kUnitRows + jr]), acc[t][i % NACC], v);
+                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(p.alpha[(size_t(u) * Q + i) * kUnitRows + jr]), acc[a][i % NACC], v);
                 v = fmaf(__half2float(p.z[size_t(u) * kUnitRows + jr]), xacc, v);
             }
         }
@@ -605,12 +703,12 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         v += __shfl_xor_sync(0xffffffffu, v, 16);
         float v1 = 0.f;
         if constexpr (NB == 2) {
-            v1 = acc1[t];
+            v1 = acc1[a];
             v1 += __shfl_xor_sync(0xffffffffu, v1, 8);
             v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
         }
-        if (lane < 8 && cw + kLutWarps * t < V) {
-            const int n = (u0 + cw + kLutWarps * t) * kUnitRows + lane;
+        if (lane < 8 && ul < V) {
+            const size_t n = size_t(u0 + ul) * kUnitRows + lane;
             if (partial)
                 partial[n] = v;
             else
@@ -624,38 +722,51 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
         }
     }
 
-    if (ctid == 0) TRACE(10);
-    // ---- split-K: the last block to arrive for this row block adds the partials in fixed order --
-    if (p.k_splits > 1) {
-        __threadfence();
-        named_barrier(2, kConsumerThreads);
-        if (ctid == 0) {
-            const int old = atomicAdd(p.counters + rbi, 1);
-            *s_last = (old == p.k_splits - 1);
+    // ---- split K: the last warp to arrive for (row block, consumer warp) adds the partial rows ------
+    if (p.k_splits > 1 && kJ * cw < V) {
+        __syncwarp();                     // the lanes' partial rows are ordered before lane 0's fence
+        int last = 0;
+        int *counter = p.counters + rbi * 32 + cw;
+        if (lane == 0) {
+            __threadfence();              // cumulative: publishes the whole warp's rows
+            last = (atomicAdd(counter, 1) == p.k_splits - 1);
+            if (last) __threadfence();    // the other splits' rows are visible to what follows
         }
-        named_barrier(2, kConsumerThreads);
-        if (*s_last) {
-            __threadfence();
-            // fixed summation order (deterministic); the loads of 8 splits are issued together
-            const int R = V * kUnitRows;
-            for (int idx = ctid; idx < NB * R; idx += kConsumerThreads) {
-                const int col = idx >= R ? 1 : 0;
-                const size_t at = size_t(col) * p.N + size_t(u0) * kUnitRows + (idx - col * R);
-                float v = 0.f;
-                for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
-                    float part[8];
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+            __syncwarp();
+            // lane -> two rows per column: (accumulator slot lane >> 3, row lane & 7) and slot + 4; fixed
+            // summation order; the loads of 8 splits of all the lane's rows are issued together
+            constexpr int R = 2 * NB;
+            size_t n[R];
+            bool on[R];
+            float v[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int a = (lane >> 3) + 4 * (r & 1);
+                const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;
+                on[r] = ul < V;
+                n[r] = size_t(r >> 1) * p.N + size_t(u0 + (on[r] ? ul : 0)) * kUnitRows + (lane & 7);
+                v[r] = 0.f;
+            }
+            for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
+                float part[R][8];
+#pragma unroll
+                for (int r = 0; r < R; ++r)
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        part[k] = (k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at) : 0.f;
+                        part[r][k] = (on[r] && k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + n[r]) : 0.f;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) v += part[k];
-                }
-                p.y[at] = __float2half_rn(v);
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) v[r] += part[r][k];
             }
-            if (ctid == 0) p.counters[rbi] = 0;
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if (on[r]) p.y[n[r]] = __float2half_rn(v[r]);
+            if (lane == 0) *counter = 0;
         }
     }
-    if (ctid == 0) TRACE(11);
 }
 
 template <int Q, bool GROUPED, int NB>
@@ -696,13 +807,14 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
     prm.x = reinterpret_cast<const __half *>(x);
     prm.y = reinterpret_cast<__half *>(y);
     prm.counters = static_cast<int *>(workspace);
-    prm.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + kCounterBytes) : nullptr;
+    prm.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + lut_counter_bytes(plan)) : nullptr;
     prm.N = d.N;
     prm.K = d.K;
     prm.U = d.N / kUnitRows;
     prm.W = d.K / kWindow;
     prm.row_blocks = plan.row_blocks;
     prm.k_splits = plan.k_splits;
+    prm.test_flags = plan.reserved;
     const bool grouped = d.group != 0;
     if (cols == 2) {
         if (!grouped) return cudaErrorInvalidValue;
@@ -723,14 +835,7 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
     return cudaErrorInvalidValue;
 }
 
-#ifdef BCQ_TRACE
-extern "C" int bcq_debug_read_trace(unsigned long long *host, int blocks)
-{
-    return int(cudaMemcpyFromSymbol(host, g_trace, size_t(blocks) * 16 * sizeof(unsigned long long)));
-}
-#endif
-
-// Read and clear the device status word (synchronises with the device).
+// Read and clear the device status word.
 cudaError_t lut_status_take(int *status)
 {
     int v = 0;

@@ -5,8 +5,7 @@
 // the call neither takes a workspace nor allocates one.
 #include <mutex>
 
-#include "bcq.h"
-#include <cuda_runtime.h>
+#include "bcq_internal.cuh"
 
 // Lives in the device memory of every GPU that loads this library, from load until exit.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[BCQ_NOALLOC_SCRATCH_BYTES];
@@ -14,7 +13,6 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[BCQ_NOALLOC_SCR
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr size_t kCounterRegion = 4096 * sizeof(int);   // head of the scratch: arrival counters
 std::mutex g_mutex;
 void *g_scratch_addr[kMaxDevices] = {};
 
@@ -23,11 +21,15 @@ void *g_scratch_addr[kMaxDevices] = {};
 int scratch_address(void **out)
 {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BCQ_ERR_CUDA;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return bcq::record_cuda_error(e);
+    if (dev < 0 || dev >= kMaxDevices) return bcq::record_cuda_error(cudaErrorInvalidDevice);
     std::lock_guard<std::mutex> lock(g_mutex);
     if (!g_scratch_addr[dev]) {
         void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return BCQ_ERR_CUDA;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return bcq::record_cuda_error(e);
+        if (!p) return bcq::record_cuda_error(cudaErrorInvalidSymbol);
         g_scratch_addr[dev] = p;
     }
     *out = g_scratch_addr[dev];
@@ -49,10 +51,10 @@ extern "C" int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, co
     void *scratch = nullptr;
     rc = scratch_address(&scratch);
     if (rc != BCQ_OK) return rc;
-    // The array keeps whatever the previous call left.  The kernel needs its arrival counters to
-    // start at zero; the partial sums are fully overwritten before they are read.
-    if (cudaMemsetAsync(scratch, 0, kCounterRegion, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-        return BCQ_ERR_CUDA;
+    // The array keeps whatever the previous call left.  The kernel needs its arrival counters (the head
+    // of the scratch) to start at zero; the partial sums are fully overwritten before they are read.
+    const cudaError_t e = cudaMemsetAsync(scratch, 0, bcq::lut_counter_bytes(plan), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return bcq::record_cuda_error(e);
     return bcq_gemv_plan(desc, &plan, packed_dev, alpha_dev, z_dev, x_dev, y_dev, scratch,
                          size_t(BCQ_NOALLOC_SCRATCH_BYTES), stream);
 }

@@ -55,3 +55,9 @@ def tiled_operands(planes, alpha, z, group):
 def rel_err(y_gpu, y_ref):
     y_ref = np.asarray(y_ref, np.float64)
     return float(np.abs(np.asarray(y_gpu, np.float64) - y_ref).max() / np.abs(y_ref).max())
+
+
+def lut_max_units(q, group, B=1):
+    """Row units (8 rows) one block of the lookup-table kernel takes, as include/bcq.h states the limit:
+    184, or 160 for q = 4 when two columns share a launch (group 128 with B >= 2)."""
+    return 160 if (q == 4 and group != 0 and B >= 2) else 184

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import TOL, make_layer, rel_err, tiled_operands
+from helpers import lut_max_units, TOL, make_layer, rel_err, tiled_operands
 from paper_2407_02891_b200 import binding as bq
 from paper_2407_02891_b200 import synth
 
@@ -185,7 +185,7 @@ def test_gemv_lut_kernel_default_plan(N, K, q, group):
 @pytest.mark.parametrize("N,K,q,rb,ks", [(520, 3584, 3, 2, 1), (520, 3584, 3, 2, 7), (520, 3584, 3, 3, 2),
                                          (520, 3584, 3, 65, 3), (520, 3584, 3, 5, 4), (512, 1024, 2, 1, 1),
                                          (512, 1024, 2, 1, 2), (1000, 1536, 2, 125, 3), (1000, 1536, 2, 2, 1),
-                                         (1536, 1024, 3, 1, 2), (4000, 512, 2, 3, 1)])
+                                         (1472, 1024, 3, 1, 2), (4000, 512, 2, 3, 1)])
 def test_gemv_lut_kernel_explicit_plans(N, K, q, rb, ks, group):
     """Ragged row blocks, one and several windows per block, with and without split-K."""
     p, codes, alpha, z, x = make_layer(f"lutp/{N}x{K}", N, K, q, group)
@@ -310,7 +310,7 @@ def test_small_batch_kernel_explicit_plans(N, K, q, group, rb, ks, B):
 @pytest.mark.parametrize("N,K,q,rb,ks,B", [
     (264, 1024, 3, 1, 1, 2),       # 33 units, both windows in one block
     (264, 1024, 3, 1, 2, 2),       # split-K
-    (1536, 1536, 3, 1, 3, 2),      # 192 units: every warp eight units
+    (1472, 1536, 3, 1, 3, 2),      # 184 units: every consumer warp eight units
     (776, 2560, 2, 2, 5, 3),       # a pair and a single column
     (512, 1024, 1, 4, 1, 4),
     (512, 1024, 4, 4, 2, 5),
@@ -402,7 +402,7 @@ def test_random_shapes_batches_and_plans():
         B = int(rng.choice([1, 1, 2, 3, 4, 5, 8, 9, 16]))
         kernel = int(rng.choice([1, 2])) if B >= 2 else 1
         ks = int(rng.integers(1, W + 1))
-        rb_min = -(-U // (192 if kernel == 1 else 176))
+        rb_min = -(-U // (lut_max_units(q, group, B) if kernel == 1 else 176))
         rb = int(rng.integers(rb_min, min(U, rb_min + 6) + 1))
         p, codes, alpha, z, X = make_layer(f"random/{case}", N, K, q, group, B)
         ref = oracle.forward_planes(p, alpha, z, X, group)

@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(L, n), n
     assert set(names) == set(bq.SIGNATURES), "binding and header disagree"
-    assert bq.lib().bcq_version() == 107
+    assert bq.lib().bcq_version() == 200
 
 
 def test_status_strings():
@@ -78,7 +78,7 @@ def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
     dt = bq.desc(64, 1024, 3, 128, bq.LAYOUT_TILED)
     split = bq.Plan(1, 1, 2, 0)
     need = bq.workspace_bytes(dt, 1, split)
-    assert need == 4096 * 4 + 2 * 64 * 4
+    assert need == 256 + 2 * 64 * 4          # 32 counters per row block (rounded up to 256 bytes) + [2][64] fp32
     args = (ctypes.byref(dt), ctypes.byref(split), ok, ok, ok, ok, ok)
     assert L.bcq_gemv_plan(*args, None, 0, None) == bq.ERR_INVALID_ARG
     assert L.bcq_gemv_plan(*args, ok, need - 1, None) == bq.ERR_WORKSPACE_TOO_SMALL
@@ -86,7 +86,7 @@ def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
     # plans that break the limits
     for p in (bq.Plan(1, 0, 1, 0), bq.Plan(1, 9, 1, 0), bq.Plan(1, 1, 3, 0), bq.Plan(2, 1, 1, 0)):
         assert L.bcq_gemv_plan(ctypes.byref(dt), ctypes.byref(p), ok, ok, ok, ok, ok, ok, 1 << 20, None) == bq.ERR_INVALID_ARG
-    big = bq.desc(2048, 512, 3, 128, bq.LAYOUT_TILED)     # 256 units in one row block > 128
+    big = bq.desc(2048, 512, 3, 128, bq.LAYOUT_TILED)     # 256 units in one row block > 184
     p = bq.Plan(1, 1, 1, 0)
     assert L.bcq_gemv_plan(ctypes.byref(big), ctypes.byref(p), ok, ok, ok, ok, ok, None, 0, None) == bq.ERR_INVALID_ARG
     # batch limits
@@ -130,11 +130,12 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert p.kernel == 1
     U, W = N // 8, K // 512
     assert 1 <= p.row_blocks <= U and 1 <= p.k_splits <= W
-    assert -(-U // p.row_blocks) <= 192 and -(-W // p.k_splits) <= 32
+    assert -(-U // p.row_blocks) <= 184 and -(-W // p.k_splits) <= 32
     blocks = p.row_blocks * p.k_splits
     if U * W >= 148 * 8:
         assert blocks >= 0.7 * 148
-    assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * N * 4)
+    counters = -(-p.row_blocks * 128 // 256) * 256          # lookup-table kernel: 32 counters per row block
+    assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else counters + p.k_splits * N * 4)
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
     for B in (2, 3):                                       # two or three columns: the lookup-table kernel on column pairs
@@ -147,7 +148,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
         assert -(-U // pb.row_blocks) <= 176 and -(-W // pb.k_splits) <= 32
         assert bq.workspace_bytes(d, B, pb) == (0 if pb.k_splits == 1 else 4096 * 4 + pb.k_splits * B * N * 4)
         # a lookup-table plan runs the columns two at a time: partial sums of two columns
-        assert bq.workspace_bytes(d, B, p) == (0 if p.k_splits == 1 else 4096 * 4 + p.k_splits * 2 * N * 4)
+        assert bq.workspace_bytes(d, B, p) == (0 if p.k_splits == 1 else counters + p.k_splits * 2 * N * 4)
     assert bq.workspace_bytes(d, 1, bq.plan_default(d, 4, 148)) == 0        # the small-batch kernel needs B >= 2
     assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
 
