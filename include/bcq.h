@@ -28,10 +28,13 @@
  *     fp16, i.e. |x[8c]| + ... + |x[8c+7]| < 65520 for every chunk c; beyond that the entry becomes
  *     infinite and so does every y that uses it (the generic kernel, plan kernel 0, has no table
  *     and no such limit).
- *   - Packed operands are constants to the products: bcq_gemv and bcq_gemm_smallbatch may start
- *     fetching them before the previous kernel in the stream has finished (programmatic dependent
- *     launch), so write them with this library's calls or plain kernels and copies, which finish
- *     before the product is launched; x, y and the workspace are ordered as usual.
+ *   - Packed operands are constants to the products: bcq_gemv and bcq_gemm_smallbatch start
+ *     fetching them before they wait for the previous kernel in the stream (programmatic dependent
+ *     launch).  Operands written by this library's calls (bcq_pack, bcq_repack, bcq_quantize_rtn)
+ *     or by copies may be multiplied right away on the same stream.  A kernel of your own that
+ *     writes packed operands immediately in front of a product must make its writes visible
+ *     before its blocks end (__threadfence() after the last store), or be separated from the
+ *     product by any other stream operation; x, y and the workspace are ordered as usual.
  *   - Device pointers must be 16-byte aligned (y: 2-byte) or BCQ_ERR_MISALIGNED is returned.
  *   - Return value: BCQ_OK (0) or a negative bcq_status.  No exceptions, no exit().
  *

@@ -48,24 +48,6 @@ static_assert(8 * kMmaMaxSlots + 64 <= kMmaFixedBytes, "barrier area");
 
 __device__ int g_mma_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
 
-#ifdef BCQ_TRACE
-// Development aid (not compiled into the product): per consumer warp, ns spent per phase.
-__device__ unsigned long long g_mma_trace[148 * 32][8];
-__device__ __forceinline__ unsigned long long mma_now()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define MTRACE_T(var) const unsigned long long var = mma_now()
-#define MTRACE_ADD(slot, v) do { if (lane == 0 && blockIdx.x < 148) g_mma_trace[blockIdx.x * 32 + warp][slot] += (v); } while (0)
-#define MTRACE_SET(slot, v) do { if (lane == 0 && blockIdx.x < 148) g_mma_trace[blockIdx.x * 32 + warp][slot] = (v); } while (0)
-#else
-#define MTRACE_T(var) do { } while (0)
-#define MTRACE_ADD(slot, v) do { } while (0)
-#define MTRACE_SET(slot, v) do { } while (0)
-#endif
-
 struct MmaParams {
     const uint8_t *tiles;
     const uint16_t *alpha;   // per-row scales only: [u][i][r]
@@ -139,9 +121,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- consumer warps: their jobs (window-major, then their pairs), D of them in flight ---------
-    MTRACE_T(t_begin);
-    MTRACE_SET(0, t_begin);
-    MTRACE_SET(1, 0); MTRACE_SET(2, 0); MTRACE_SET(3, 0); MTRACE_SET(4, 0); MTRACE_SET(5, 0);
     const int cw = warp - kMmaLoaderWarps;
     const int mine = (cw >= 0 && P > cw) ? (P - cw + kMmaWarps - 1) / kMmaWarps : 0;   // pairs of this warp per window
     const int total_jobs = mine * nwin;
@@ -245,12 +224,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
 
     for (int wi = 0; wi < nwin && alive && mine > 0; ++wi) {   // warps without jobs go straight to the end
         const int buf = wi & 1;
-        MTRACE_T(t_x0);
         if (!mbar_wait<true>(bar_x_ready + 8 * buf, (wi >> 1) & 1, abort_flag, kMmaWaitXReady, &g_mma_status)) {
             alive = false;
             break;
         }
-        MTRACE_ADD(1, mma_now() - t_x0);
         const unsigned char *xb = xs + buf * kXBufBytes + m * kXRowBytes + t * kXGroupBytes;   // column m (and m + 8)
         const uint32_t xs_lo = xsum[(buf * BR + m) * 4 + t];
         const uint32_t xs_hi = WIDE ? xsum[(buf * BR + m + 8) * 4 + t] : 0u;
@@ -259,13 +236,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
             constexpr int pp = decltype(PP)::value;
             if (alive && cw + kMmaWarps * pp < P) {
                 const int s = cw + kMmaWarps * d;
-                MTRACE_T(t_f0);
                 if (!mbar_wait(bar_full + 8 * s, fill & 1, abort_flag, kMmaWaitFull, &g_mma_status)) {
                     alive = false;
                 } else {
-                    MTRACE_T(t_f1);
-                    MTRACE_ADD(2, t_f1 - t_f0);
-                    MTRACE_ADD(5, 1);
                     ++consumed;
                     const unsigned char *slot = ring + s * kSlotBytes;
                     [[maybe_unused]] const int ua = u0 + 2 * (cw + kMmaWarps * pp);
@@ -303,8 +276,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) issue_next(d);
-                    MTRACE_T(t_f2);
-                    MTRACE_ADD(3, t_f2 - t_f1);
 
                     // Independent accumulation chains (an MMA waits for the previous one into the same
                     // registers): one per plane; folded into the pair's accumulators at the end.
@@ -349,7 +320,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
                             acc[pp][e] += c[j][e];
                             if constexpr (WIDE) acc_hi[pp][e] += ch[j][e];
                         }
-                    MTRACE_ADD(4, mma_now() - t_f2 + (acc[pp][0] == 12345.678f ? 1 : 0));
                 }
                 if (++d == D) {
                     d = 0;
@@ -372,7 +342,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) mma_gemm_kernel(const MmaParam
         }
     }
 
-    MTRACE_SET(6, mma_now());
     // ---- store: lane (m, t) holds rows m of both units for columns 2t, 2t+1 (and 8 + those) -------
     float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * p.B * p.N : nullptr;
     auto put = [&](int b, int n, float v) {
@@ -492,13 +461,6 @@ cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void 
     }
     return cudaErrorInvalidValue;
 }
-
-#ifdef BCQ_TRACE
-extern "C" int bcq_debug_read_mma_trace(unsigned long long *host)
-{
-    return int(cudaMemcpyFromSymbol(host, g_mma_trace, sizeof(g_mma_trace)));
-}
-#endif
 
 // Read and clear the device status word (synchronises with the device).
 cudaError_t mma_status_take(int *status)

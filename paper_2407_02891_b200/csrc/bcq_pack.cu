@@ -75,6 +75,9 @@ __global__ void pack_kernel(const uint8_t *__restrict__ codes, const View dst)
         }
         *dst.plane_byte(i, n, kb) = uint8_t(byte);
     }
+    // The products start fetching packed operands before they wait for the kernel in front of them: every
+    // kernel that writes operands makes its writes visible device-wide before its blocks count as finished.
+    __threadfence();
 }
 
 cudaError_t launch_pack(const uint8_t *codes, const View &dst, cudaStream_t st)
@@ -95,6 +98,7 @@ __global__ void permute_planes_kernel(const View src, const View dst)
     const int n = int((t / kbytes) % src.N);
     const int i = int(t / (size_t(kbytes) * src.N));
     *dst.plane_byte(i, n, kb) = *src.plane_byte(i, n, kb);
+    __threadfence();   // see pack_kernel
 }
 
 __global__ void permute_scales_kernel(const View src, const View dst)
@@ -105,6 +109,7 @@ __global__ void permute_scales_kernel(const View src, const View dst)
     const int n = int(t / G), g = int(t % G);
     for (int i = 0; i < src.q; ++i) *dst.alpha_elem(i, n, g) = *src.alpha_elem(i, n, g);
     *dst.z_elem(n, g) = *src.z_elem(n, g);
+    __threadfence();   // see pack_kernel
 }
 
 cudaError_t launch_permute_planes(const View &src, const View &dst, cudaStream_t st)

@@ -148,6 +148,7 @@ __global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restric
         const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
         encode_chunk(raw, S[size_t(n) * G + g], qbias[size_t(n) * G + g], tab, lut, w_int, dst, n, kb);
     }
+    __threadfence();   // operands visible device-wide before the block counts as finished (products fetch them early)
 }
 
 // Groups of 128: everything in one pass.  A group is 16 chunks = 16 consecutive lanes, each holding
@@ -206,6 +207,7 @@ __global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restr
         }
         if (in) encode_chunk(raw, s_h, b_h, tab, lut, w_int, dst, n, kb);
     }
+    __threadfence();   // operands visible device-wide before the block counts as finished (products fetch them early)
 }
 
 // One thread per (row, group): the fused scales, written where the destination layout keeps them.
@@ -216,6 +218,7 @@ __global__ void __launch_bounds__(256) rtn_scales_kernel(const __half *__restric
     const size_t t = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (t >= size_t(dst.N) * G) return;
     write_scales(S[t], qbias[t], tab, dst, int(t / G), int(t % G));
+    __threadfence();   // as in the encoding kernels
 }
 
 cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, const uint8_t *code_of_int /*[256]*/,

@@ -25,6 +25,12 @@ CASES = [
     ("opt66b/attn_q2_row", 9216, 9216, 2, 0),
     ("llama70b/kv", 2048, 8192, 3, 128),
     ("llama70b/down", 8192, 28672, 3, 128),
+    ("llama70b/gate", 28672, 8192, 3, 128),
+    ("llama70b/q", 8192, 8192, 3, 128),
+    ("opt6.7b/fc2", 4096, 16384, 3, 128),
+    ("opt66b/fc1_q2_row", 36864, 9216, 2, 0),        # the paper's own granularity at the largest shapes
+    ("opt66b/fc2_q2_row", 9216, 36864, 2, 0),
+    ("opt66b/fc1_q2", 36864, 9216, 2, 128),
 ]
 
 
@@ -84,15 +90,25 @@ def test_fullsize_repack_round_trip_sampled():
     assert np.array_equal(z2.view(N, -1).cpu().numpy().view(np.uint16), z.view(np.uint16))
 
 
-@pytest.mark.parametrize("B", [2, 16])
-def test_fullsize_smallbatch_sampled_rows(B):
-    name, N, K, q, group = "llama70b/kv", 2048, 8192, 3, 128
+@pytest.mark.parametrize("name,N,K,B", [
+    ("llama70b/kv", 2048, 8192, 2), ("llama70b/kv", 2048, 8192, 16),
+    ("llama70b/gate", 28672, 8192, 2), ("llama70b/gate", 28672, 8192, 3), ("llama70b/gate", 28672, 8192, 4),
+    ("llama70b/gate", 28672, 8192, 8), ("llama70b/gate", 28672, 8192, 16),
+    ("llama70b/down", 8192, 28672, 4), ("llama70b/down", 8192, 28672, 9),
+    ("llama70b/q", 8192, 8192, 8),
+])
+def test_fullsize_smallbatch_sampled_rows(name, N, K, B):
+    """Every small-batch path at the sizes of the Llama-2-70B-shaped layer: column pairs through the
+    lookup-table kernel (B = 2, 3), the tensor-core kernel with one and with two MMAs per step (B <= 8, B > 8)."""
+    q, group = 3, 128
     dt, packed, at, zt, alpha, z = _build(name, N, K, q, group)
     X = synth.activations(name, B, K)
     Y = torch.full((B, N), float("nan"), dtype=torch.float16, device=DEV)
     bq.gemm_smallbatch(dt, packed, at, zt, torch.from_numpy(X).to(DEV), Y, B, bq.new_workspace(dt, B))
     torch.cuda.synchronize()
+    bq.poll_status()
     Yh = Y.cpu().numpy().astype(np.float64)
+    assert np.isfinite(Yh).all()
     rows = _sample_rows(name, N)
     ref = oracle.forward_planes(synth.plane_rows(name, N, K, q, rows), alpha[:, rows], z[rows], X, group)
     assert np.abs(Yh[:, rows] - ref).max() <= TOL * np.abs(ref).max()

@@ -416,3 +416,76 @@ def test_random_shapes_batches_and_plans():
             torch.cuda.synchronize()
             bq.poll_status()
             assert rel_err(Y.cpu().numpy(), ref) <= TOL, (case, N, K, q, group, B, plan.kernel, plan.row_blocks, plan.k_splits)
+
+
+def _heavy_tailed(kind, K, name):
+    """Activations with the outliers LLM hidden states have: fp16, the bulk N(0,1)."""
+    x = synth.normal(name + "/x", 0, K)
+    u = synth.uniform(name + "/pick", 0, K)
+    if kind == "outliers_x50":               # one value in a hundred is fifty times larger
+        x = np.where(u < 0.01, 50.0 * x, x)
+    elif kind == "spikes_1e2_1e4":           # a few spikes of 1e2 .. 1e4 in every window of 512
+        for w in range(K // 512):
+            for j, mag in enumerate((1e2, -1e3, 1e4)):
+                x[512 * w + int(u[512 * w + j] * 512)] = mag
+    elif kind == "near_table_limit":         # one chunk of eight same-sign values whose sum is just below the
+        x[8 * 37:8 * 37 + 8] = 8000.0        # largest finite fp16 (64000 < 65504), another with the opposite sign
+        x[8 * 101:8 * 101 + 8] = -8000.0
+    elif kind == "cancelling":               # large values that cancel inside a chunk: the table entry is small,
+        x[8 * 5:8 * 5 + 8] = [3000.0, -3000.0, 2000.0, -2000.0, 1000.0, -1000.0, 0.5, -0.25]   # its terms are not
+    return x.astype(np.float16).reshape(1, K)
+
+
+@pytest.mark.parametrize("group", [128, 0])
+@pytest.mark.parametrize("kind", ["outliers_x50", "spikes_1e2_1e4", "near_table_limit", "cancelling"])
+def test_gemv_heavy_tailed_activations(kind, group):
+    """The lookup tables hold fp16 sums of 8 activations (one rounding each, relative 2^-11): the product
+    must stay inside the stated tolerance when the activations have outliers, up to the documented limit
+    (every 8-activation sum finite in fp16)."""
+    N, K, q = 1024, 4096, 3
+    p, codes, alpha, z, _ = make_layer(f"tails/{group}", N, K, q, group)
+    x = _heavy_tailed(kind, K, f"tails/{kind}")
+    ref = oracle.forward_planes(p, alpha, z, x, group)[0]
+    L = gpu_layer(N, K, q, group, bq.LAYOUT_TILED, codes, alpha, z)
+    assert bq.plan_default(L.d).kernel == 1
+    y = run_gemv(L, x)
+    assert np.isfinite(y).all()
+    assert rel_err(y, ref) <= TOL
+    # two columns per launch build their tables the same way
+    if group:
+        X = np.concatenate([x, synth.activations("tails/col1", 1, K)])
+        Y = torch.zeros((2, N), dtype=torch.float16, device=DEV)
+        bq.gemm_smallbatch(L.d, L.packed, L.alpha, L.z, dev(X), Y, 2, bq.new_workspace(L.d, 2))
+        torch.cuda.synchronize()
+        assert rel_err(Y.cpu().numpy(), oracle.forward_planes(p, alpha, z, X, group)) <= TOL
+
+
+def test_operands_rewritten_in_place_between_two_products():
+    """The products fetch packed operands before they wait for the kernel in front of them; operands
+    written by the library's own calls must still be complete.  Pack layer A, multiply, pack layer B into
+    the SAME buffers, multiply again at once: the second result is B's, for each way of writing operands."""
+    N, K, q, group = 2048, 4096, 3, 128
+    pa, ca, aa, za, x = make_layer("inplace/A", N, K, q, group)
+    pb, cb, ab, zb, _ = make_layer("inplace/B", N, K, q, group)
+    ref_b = oracle.forward_planes(pb, ab, zb, x, group)[0]
+    d = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
+    dc = d.with_layout(bq.LAYOUT_CANONICAL)
+    packed, _, _ = bq.empty_operands(d, DEV)
+    xd = dev(x.reshape(-1))
+    ws = bq.new_workspace(d, 1)
+    ya = torch.zeros(N, dtype=torch.float16, device=DEV)
+    yb = torch.zeros(N, dtype=torch.float16, device=DEV)
+    codes_a, codes_b = dev(ca), dev(cb)
+    canon_b = dev(pb.reshape(-1))
+    for how in ("pack", "repack"):
+        for _ in range(3):
+            bq.pack(d, codes_a, dev(aa), dev(za), packed, None, None)
+            bq.gemv(d, packed, None, None, xd, ya, ws)
+            if how == "pack":
+                bq.pack(d, codes_b, dev(ab), dev(zb), packed, None, None)
+            else:
+                bq.repack(dc, canon_b, dev(ab), dev(zb), d, packed, None, None)
+            bq.gemv(d, packed, None, None, xd, yb, ws)          # no synchronisation in between
+        torch.cuda.synchronize()
+        bq.poll_status()
+        assert rel_err(yb.cpu().numpy(), ref_b) <= TOL, how

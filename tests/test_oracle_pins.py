@@ -422,3 +422,26 @@ def test_rtn_then_merge_reconstruction_error_bound(n, q, b2p):
     assert np.all(np.abs(Wq - W.astype(np.float64)) <= Sd * (0.5 + half_gap) + slack)
     if q == n:
         assert np.all(np.abs(Wq - W.astype(np.float64)) <= Sd * 0.5 + slack)
+
+
+def test_rtn_zero_minimum_is_stored_as_plus_zero_whichever_zero_comes_first():
+    """A group whose minimum is zero: -0.0 and +0.0 compare equal, so which of the two the minimum search
+    ends on depends on the order of the weights; the stored qbias must not.  Both orders give the bit
+    pattern 0x0000, the same S and the same integers; a strictly negative minimum keeps its sign."""
+    neg0, pos0 = np.uint16(0x8000).view(np.float16), np.float16(0.0)
+    top = np.float16(0.75)
+    first = np.array([[neg0, np.float16(0.25), pos0, top]], np.float16)      # -0 met first
+    last = np.array([[pos0, np.float16(0.25), top, neg0]], np.float16)       # -0 met last
+    only = np.array([[neg0, np.float16(0.25), np.float16(0.5), top]], np.float16)   # no +0 in the group at all
+    for W in (first, last, only):
+        w_int, S, qb = oracle.quantize_rtn(W, 0, 2)
+        assert qb.view(np.uint16).tolist() == [[0x0000]]
+        assert S.view(np.uint16).tolist() == np.array([[0.25]], np.float16).view(np.uint16).tolist()   # 0.75 / 3
+        zero_at = [i for i in range(4) if W[0, i] == 0]
+        assert all(w_int[0, i] == 0 for i in zero_at) and w_int[0].max() == 3
+    # the offset that merge derives from it is then S * centre exactly (no -0 leaking into z)
+    _, alpha, z = oracle.merge_linear(oracle.quantize_rtn(first, 0, 2)[0], *oracle.quantize_rtn(first, 0, 2)[1:], 0, 2, [0, 1])
+    assert z.view(np.uint16).tolist() == np.array([[0.375]], np.float16).view(np.uint16).tolist()
+    # a negative minimum is kept as it is
+    W = np.array([[np.float16(-0.5), neg0, np.float16(0.25), np.float16(1.0)]], np.float16)
+    assert oracle.quantize_rtn(W, 0, 2)[2].view(np.uint16).tolist() == np.array([[-0.5]], np.float16).view(np.uint16).tolist()
