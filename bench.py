@@ -36,9 +36,10 @@ WORKLOADS = {
     "llama70b_q3_g128": dict(family="llama", hidden=8192, ffn=28672, kv=2048, layers=8, q=3, group=128),
 }
 DEFAULT_WORKLOAD = "opt30b_q3_g128"
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
-# profiles/lut_gemv_kernel_opt30b_q3_g128.md; valid only for the library revision it was taken on.
-NCU_TRAFFIC = {"lib_version": 107, "workload": "opt30b_q3_g128", "bytes_per_launch": 46.4e6}
+# DRAM bytes per launch of the dominant kernel: the per-shape dram__bytes_read + dram__bytes_write figures of
+# the ncu capture summarised under profiles/ (a small text file, one "key value" pair per line); they hold
+# only for the library revision they were taken on.
+NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "lut_gemv_kernel_opt30b_q3_g128.traffic.txt")
 METRIC = "BCQ GEMV us/token (sum of all linear layers of the decoder stack, bs=1)"
 UNIT = "us/token"
 
@@ -62,6 +63,24 @@ def algorithmic_bytes(N, K, q, group, B=1):
     """Packed planes + fp16 alphas + fp16 offsets + x + y."""
     G = 1 if group == 0 else K // group
     return q * N * K // 8 + 2 * q * N * G + 2 * N * G + 2 * B * K + 2 * B * N
+
+
+def ncu_traffic_per_launch(lib_version, workload, shapes_per_step):
+    """Mean DRAM bytes per launch over one step from the tracked ncu figures, or None when they were taken on
+    another library revision or workload.  shapes_per_step: {"NxK": launches per step}."""
+    try:
+        kv = {}
+        with open(NCU_TRAFFIC_FILE) as f:
+            for line in f:
+                line = line.split("#")[0].split()
+                if len(line) == 2:
+                    kv[line[0]] = line[1]
+        if int(kv["lib_version"]) != lib_version or kv["workload"] != workload:
+            return None
+        total = sum(float(kv["dram_bytes_" + s]) * n for s, n in shapes_per_step.items())
+        return total / sum(shapes_per_step.values())
+    except (OSError, KeyError, ValueError):
+        return None
 
 
 def measured_peak_gbs():
@@ -167,15 +186,24 @@ class Stack:
         self.items = []       # (desc, packed, alpha, z, x, y, ws)
         self.bytes = 0
         scales, xs, wss = {}, {}, {}
+        distinct = []
         for (pname, N, K) in layer_shapes(w):
-            if (N, K) in scales:
-                continue
+            if (N, K) not in distinct:
+                distinct.append((N, K))
+        # the activations of a token: one vector (B vectors) per distinct shape, side by side in ONE device
+        # buffer, so that the end-to-end leg can bring a token's activations in with a single copy
+        x_np = [synth.activations(f"{wname}/{N}x{K}", B, K).reshape(-1) for (N, K) in distinct]
+        self.x_host_all = torch.from_numpy(np.concatenate(x_np))
+        self.x_all = self.x_host_all.to(device)
+        off = 0
+        for (N, K), xv in zip(distinct, x_np):
             a, z = synth.scale_rows(f"{wname}/{N}x{K}", N, K, q, group)
             dt = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
             scales[(N, K)] = (torch.from_numpy(a).to(device), torch.from_numpy(z).to(device))
-            xs[(N, K)] = torch.from_numpy(synth.activations(f"{wname}/{N}x{K}", B, K).reshape(-1)).to(device)
+            xs[(N, K)] = self.x_all[off:off + xv.size]       # 16-byte aligned: K is a multiple of 512
+            off += xv.size
             wss[(N, K)] = bq.new_workspace(dt, B, device=device)
-        self.x_host = {k: v.cpu() for k, v in xs.items()}
+        self.names = []       # generator names of every item, for the parity check
         for layer in range(w["layers"]):
             for (pname, N, K) in layer_shapes(w):
                 dc = bq.desc(N, K, q, group, bq.LAYOUT_CANONICAL)
@@ -186,6 +214,7 @@ class Stack:
                 bq.repack(dc, canon, ad, zd, dt, packed, at, zt)
                 y = torch.zeros(B * N, dtype=torch.float16, device=device)
                 self.items.append((dt, packed, at, zt, xs[(N, K)], y, wss[(N, K)], (N, K)))
+                self.names.append(f"{wname}/L{layer}/{pname}")
                 self.bytes += algorithmic_bytes(N, K, q, group, B)
             torch.cuda.synchronize(device)
         self.graph = None
@@ -256,30 +285,51 @@ class Stack:
             out[f"{N}x{K}"] = {"us": round(best, 3), "gbs": round(b / best * 1e-3, 1), "launches": len(its)}
         return out
 
+    def parity(self, rows_per_shape=48):
+        """Sampled output rows of the LAST launch of every distinct shape (what the timed replays left in y),
+        recomputed by the CPU oracle from inputs regenerated on the host."""
+        import oracle
+
+        q, group = self.w["q"], self.w["group"]
+        worst, rows_checked, per_shape = 0.0, 0, {}
+        last = {}
+        for idx, it in enumerate(self.items):
+            last[it[7]] = idx
+        for (N, K), idx in last.items():
+            name = self.names[idx]
+            y = self.items[idx][5].cpu().numpy().astype(np.float64).reshape(self.B, N)
+            r = synth.u64(name + "/bench_rows", 0, rows_per_shape) % np.uint64(N)
+            rows = np.unique(np.concatenate([r.astype(np.int64), [0, N - 1]]))
+            a, z = synth.scale_rows(f"{self.wname}/{N}x{K}", N, K, q, group)
+            X = synth.activations(f"{self.wname}/{N}x{K}", self.B, K)
+            ref = oracle.forward_planes(synth.plane_rows(name, N, K, q, rows), a[:, rows], z[rows], X, group)
+            err = float(np.abs(y[:, rows] - ref).max() / np.abs(ref).max()) if np.isfinite(y).all() else float("inf")
+            per_shape[f"{N}x{K}"] = err
+            worst = max(worst, err)
+            rows_checked += len(rows)
+        return {"max_rel_err": worst, "tol": 5e-3, "rows": rows_checked, "per_shape": per_shape,
+                "ok": bool(worst <= 5e-3),
+                "what": "sampled rows of the last launch of every distinct shape after the timed replays, "
+                        "against the fp64 CPU oracle on regenerated inputs"}
+
     def e2e_steps(self, steps):
-        """The same token through bcq_gemv_host: x from pinned host memory, y back to host, per layer."""
-        torch, bq = self.torch, self.bq
-        xh = {k: v.pin_memory() for k, v in self.x_host.items()}
-        yh = {k: torch.zeros(k[0], dtype=torch.float16).pin_memory() for k in xh}
-        xs = {k: torch.zeros(k[1], dtype=torch.float16, device=self.device) for k in xh}
-        h2d = sum(2 * it[7][1] for it in self.items)
-        d2h = sum(2 * it[7][0] for it in self.items)
-
-        def enqueue():
-            for (d, packed, a, z, x, y, ws, s) in self.items:
-                bq.gemv_host(d, packed, a, z, xh[s], yh[s], xs[s], y, ws)
-
-        enqueue()
-        torch.cuda.synchronize(self.device)
-        graph = torch.cuda.CUDAGraph()      # the per-layer copies and products of one token, captured once
-        with torch.cuda.graph(graph):
-            enqueue()
+        """The same token end to end: the token's activations come from pinned host memory (one copy), the
+        products run through bcq_gemv as in the timed region (the captured graph), the last layer's output
+        goes back to pinned host memory (one copy), and the host waits for it."""
+        torch = self.torch
+        xh = self.x_host_all.pin_memory()
+        last_y = self.items[-1][5]
+        yh = torch.zeros(last_y.numel(), dtype=torch.float16).pin_memory()
+        h2d = xh.numel() * xh.element_size()
+        d2h = yh.numel() * yh.element_size()
 
         def one():
-            graph.replay()
+            self.x_all.copy_(xh, non_blocking=True)
+            self.graph.replay()
+            yh.copy_(last_y, non_blocking=True)
             torch.cuda.current_stream().synchronize()
 
-        for _ in range(2):
+        for _ in range(3):
             one()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize(self.device)
@@ -331,6 +381,22 @@ class OracleSample:
 
 # ---------------------------------------------------------------------------------------------
 
+def spawn_replicas(n: int) -> int:
+    """`python bench.py --gpus N` run plainly: start the N replicas (one process per GPU) the way the
+    contract launches them, and pass their output through.  Fails cleanly when the box has fewer GPUs."""
+    import subprocess
+
+    import torch
+    have = torch.cuda.device_count()
+    if have < n:
+        sys.stderr.write(f"bench.py: --gpus {n} asked for, {have} visible: nothing measured\n")
+        return 2
+    port = 29500 + os.getpid() % 2000
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -340,6 +406,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-parity", action="store_true", help="skip the sampled-row oracle check of the timed outputs")
     ap.add_argument("--batch", type=int, default=1, help="activation vectors per product (1..16)")
     ap.add_argument("--fuse", action="store_true",
                     help="stack the projections that share an activation (q/k/v, gate/up) into one product each; "
@@ -350,6 +417,8 @@ def main():
                          "no per-shape, e2e or CPU legs; the printed number is not a benchmark value")
     args = ap.parse_args()
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(spawn_replicas(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -427,13 +496,16 @@ def main():
     ms_per_step = ms / args.steps
     launches_per_step = stack.launches_per_step()
 
+    parity = stack.parity() if rank == 0 and not args.no_parity else None   # what the timed replays left in y
     per_shape = stack.per_shape_us()
     e2e = None
-    if not args.no_e2e and args.batch == 1:
-        e_ms, h2d, d2h = stack.e2e_steps(max(3, min(args.steps, 20)))
+    if not args.no_e2e:
+        e_ms, h2d, d2h = stack.e2e_steps(max(3, min(args.steps, 50)))
         e_ms = max_over_ranks(e_ms, world, device)
         e2e = {"value": replica_metric(e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "api": "bcq_gemv_host per layer (pinned host x copied in, y stored by the kernel straight into pinned host memory), the token captured once in a CUDA graph, one replay + stream sync per token"}
+               "api": "per token: one copy of the token's activations from pinned host memory, every product through "
+                      "bcq_gemv / bcq_gemm_smallbatch (the captured graph of the timed region), one copy of the last "
+                      "layer's output to pinned host memory, stream synchronise"}
 
     if rank != 0:
         if world > 1:
@@ -442,25 +514,30 @@ def main():
 
     peak, peak_kind = measured_peak_gbs()
     achieved = stack.bytes / (ms_per_step * 1e-3) / 1e9
+    shapes_per_step = {}
+    for it in stack.items:
+        key = f"{it[7][0]}x{it[7][1]}"
+        shapes_per_step[key] = shapes_per_step.get(key, 0) + 1
+    traffic = (ncu_traffic_per_launch(bq.lib().bcq_version(), args.workload, shapes_per_step)
+               if args.batch == 1 and not args.fuse else None)
     out = {
         "metric": METRIC, "value": replica_metric(ms_per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+        "vs_baseline": None, "dtype": "f32 accumulate, f16 lookup tables (fp16 x, y, scales)" if args.batch <= 3 else
+        "f32 accumulate, f16 tensor-core operands (fp16 x, y, scales)", "data": "synthetic", "config": config,
         "tokens_per_s": world * 1e3 / ms_per_step,
         "clocks": clocks.summary(),
         "gpu_launches": launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "frac_of_nominal_8000": round(achieved / 8000.0, 4),
                      "peak_kind": peak_kind,
-                     "traffic": (NCU_TRAFFIC["bytes_per_launch"]
-                                 if bq.lib().bcq_version() == NCU_TRAFFIC["lib_version"]
-                                 and args.workload == NCU_TRAFFIC["workload"] and args.layers == 0
-                                 and args.batch == 1 and not args.fuse else None),
+                     "traffic": traffic,
                      "kernel": f"lut_gemv_kernel<{w['q']}>" if args.batch <= 3 else f"mma_gemm_kernel<{w['q']}>",
                      "algorithmic_bytes_per_launch": stack.bytes // launches_per_step,
                      "launches_per_step": launches_per_step},
         "per_shape": per_shape,
         "e2e": e2e,
+        "parity": parity,
     }
     if not args.no_cpu_baseline and args.batch == 1:
         smp = OracleSample(args.workload, w)
@@ -469,6 +546,9 @@ def main():
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+    if parity is not None and not parity["ok"]:
+        sys.stderr.write("bench.py: the timed outputs do not match the oracle within the tolerance\n")
+        sys.exit(1)
 
 
 if __name__ == "__main__":
