@@ -220,6 +220,41 @@ int bcq_gemv_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed
                   uint16_t *y_dev, void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /*
+ * Several layers that read the SAME activation, in one launch: y_o = W_o x for o < count (batch 1).
+ * At decode the query, key and value projections of a layer (and the gate and up projections of a
+ * gated feed-forward block) multiply one and the same vector -- the per-token measurement of the
+ * paper's section "Setup" runs every linear module of every decoder layer once per token -- and
+ * launching them together builds each window's lookup table once per thread block instead of once
+ * per projection and pays the fixed cost of a launch once.  Every operand keeps its own packed
+ * tensor and its own y; nothing is concatenated.
+ *   desc   K, q, group and layout (BCQ_LAYOUT_TILED) of all operands; desc->N = sum of ops[o].N
+ *   ops    host array of 1..4 operands: packed_dev (and alpha_dev / z_dev when the scales are not in
+ *          the tiles), y_dev [N] and N (a multiple of 8) of each; read during the call only
+ *   plan   kernel 1; its row_blocks are shared out among the operands in proportion to their rows
+ *          (largest remainders; bcq_multi_row_blocks tells how), its k_splits apply to all.  An operand
+ *          that would get no row block, or more than 184 row units per block, makes the plan invalid.
+ *          bcq_gemv_multi uses bcq_plan_default of `desc` (enlarged, if need be, until it is valid).
+ * Workspace: bcq_workspace_bytes(desc, 1, plan), as for a single product of desc->N rows.
+ * With the same k_splits and the same row blocks per operand as a bcq_gemv_plan call on that operand
+ * alone, y_o is bit-identical to that call's result.  Errors as bcq_gemv.
+ */
+typedef struct bcq_operand {
+    const void *packed_dev;
+    const uint16_t *alpha_dev;
+    const uint16_t *z_dev;
+    uint16_t *y_dev;
+    int32_t N;
+    int32_t reserved;   /* 0 */
+} bcq_operand;
+int bcq_gemv_multi(const bcq_desc *desc, const bcq_operand *ops_host, int count, const uint16_t *x_dev,
+                   void *workspace_dev, size_t workspace_bytes, void *stream);
+int bcq_gemv_multi_plan(const bcq_desc *desc, const bcq_plan *plan, const bcq_operand *ops_host, int count,
+                        const uint16_t *x_dev, void *workspace_dev, size_t workspace_bytes, void *stream);
+/* The row blocks each operand gets under `plan` (pure host logic): row_blocks_out[o], o < count. */
+int bcq_multi_row_blocks(const bcq_desc *desc, const bcq_plan *plan, const int32_t *N_host, int count,
+                         int32_t *row_blocks_out);
+
+/*
  * Y[b] = W X[b] for b < B, 1 <= B <= 16; X [B][K], Y [B][N] row-major fp16.  Every column is
  * an independent product (the paper defines batch 1 only; Eq. bcw + Eq. fuse_step3 per column).
  * B == 1 is bcq_gemv.  Tiled layout: by default B >= 4 takes ONE pass over the packed weights

@@ -50,6 +50,12 @@ class Plan(ctypes.Structure):
                 ("k_splits", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
+class Operand(ctypes.Structure):
+    """bcq_operand"""
+    _fields_ = [("packed_dev", ctypes.c_void_p), ("alpha_dev", ctypes.c_void_p), ("z_dev", ctypes.c_void_p),
+                ("y_dev", ctypes.c_void_p), ("N", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
 class BcqError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
@@ -80,6 +86,9 @@ SIGNATURES = {
     "bcq_repack": (_i, [_dp, _vp, _vp, _vp, _dp, _vp, _vp, _vp, _vp]),
     "bcq_gemv": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_gemv_multi": (_i, [_dp, _vp, _i, _vp, _vp, _sz, _vp]),
+    "bcq_gemv_multi_plan": (_i, [_dp, _pp, _vp, _i, _vp, _vp, _sz, _vp]),
+    "bcq_multi_row_blocks": (_i, [_dp, _pp, _vp, _i, _vp]),
     "bcq_gemm_smallbatch": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "bcq_gemm_smallbatch_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp]),
     "bcq_gemv_host": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -224,6 +233,35 @@ def gemv_plan(d: Desc, plan: Plan, packed, alpha, z, x, y, workspace=None):
     wp, wn = _ws_args(workspace)
     _check(lib().bcq_gemv_plan(ctypes.byref(d), ctypes.byref(plan), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x),
                                _ptr(y), wp, wn, _stream()), "bcq_gemv_plan")
+
+
+def _operands(layers, ys):
+    arr = (Operand * len(layers))()
+    for o, (L, y) in enumerate(zip(layers, ys)):
+        _dev(L.packed, L.alpha, L.z, y)
+        arr[o] = Operand(_ptr(L.packed), _ptr(L.alpha), _ptr(L.z), _ptr(y), L.d.N, 0)
+    return arr
+
+
+def gemv_multi(d: Desc, layers, x, ys, workspace=None, plan: Plan | None = None):
+    """bcq_gemv_multi(_plan): the layers (Layer objects that share K, q, group) times one x; d.N = sum of rows."""
+    _dev(x)
+    arr = _operands(layers, ys)
+    wp, wn = _ws_args(workspace)
+    if plan is None:
+        _check(lib().bcq_gemv_multi(ctypes.byref(d), ctypes.cast(arr, ctypes.c_void_p), len(layers), _ptr(x), wp, wn,
+                                    _stream()), "bcq_gemv_multi")
+    else:
+        _check(lib().bcq_gemv_multi_plan(ctypes.byref(d), ctypes.byref(plan), ctypes.cast(arr, ctypes.c_void_p),
+                                         len(layers), _ptr(x), wp, wn, _stream()), "bcq_gemv_multi_plan")
+
+
+def multi_row_blocks(d: Desc, plan: Plan, Ns) -> list[int]:
+    n = (ctypes.c_int32 * len(Ns))(*[int(v) for v in Ns])
+    out = (ctypes.c_int32 * len(Ns))()
+    _check(lib().bcq_multi_row_blocks(ctypes.byref(d), ctypes.byref(plan), ctypes.cast(n, ctypes.c_void_p), len(Ns),
+                                      ctypes.cast(out, ctypes.c_void_p)), "bcq_multi_row_blocks")
+    return list(out)
 
 
 def gemm_smallbatch(d: Desc, packed, alpha, z, X, Y, B: int, workspace=None):

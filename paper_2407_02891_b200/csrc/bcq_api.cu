@@ -252,6 +252,77 @@ int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, con
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
 
+// Share the plan's row blocks out among operands of N[o] rows in proportion to their rows (largest remainders,
+// at least one each); BCQ_ERR_INVALID_ARG when that is impossible or a block would get too many row units.
+int share_row_blocks(const bcq_desc *d, const bcq_plan *plan, const int32_t *N, int count, int32_t *out)
+{
+    const int max_units = lut_max_units(d, 1);
+    long long total = 0;
+    for (int o = 0; o < count; ++o) {
+        if (N[o] <= 0 || N[o] % kUnitRows != 0) return BCQ_ERR_INVALID_ARG;
+        total += N[o];
+    }
+    if (total != d->N || plan->row_blocks < count) return BCQ_ERR_INVALID_ARG;
+    long long rem[kLutMaxOperands];
+    int given = 0;
+    for (int o = 0; o < count; ++o) {
+        const long long share = static_cast<long long>(plan->row_blocks) * N[o];
+        out[o] = static_cast<int32_t>(share / total);
+        rem[o] = share % total;
+        if (out[o] < 1) out[o] = 1, rem[o] = -1;
+        given += out[o];
+    }
+    while (given < plan->row_blocks) {   // hand the rest to the largest remainders (ties: the earlier operand)
+        int best = 0;
+        for (int o = 1; o < count; ++o)
+            if (rem[o] > rem[best]) best = o;
+        ++out[best], rem[best] = -1, ++given;
+        bool all_used = true;
+        for (int o = 0; o < count; ++o) all_used = all_used && rem[o] < 0;
+        if (all_used)
+            for (int o = 0; o < count; ++o) rem[o] = N[o];   // more left than operands: go round again by size
+    }
+    if (given != plan->row_blocks) return BCQ_ERR_INVALID_ARG;   // the one-block minimum exceeded the plan
+    for (int o = 0; o < count; ++o) {
+        const int U = N[o] / kUnitRows;
+        if (out[o] > U || (U + out[o] - 1) / out[o] > max_units) return BCQ_ERR_INVALID_ARG;
+    }
+    return BCQ_OK;
+}
+
+int run_multi(const bcq_desc *desc, const bcq_plan *plan, const bcq_operand *ops, int count, const uint16_t *x, void *ws,
+              size_t ws_bytes, void *stream)
+{
+    if (!ops || !x || count < 1 || count > kLutMaxOperands) return BCQ_ERR_INVALID_ARG;
+    if (!lut_kernel_covers(desc) || plan->kernel != 1) return BCQ_ERR_INVALID_ARG;
+    int32_t N[kLutMaxOperands], rb[kLutMaxOperands];
+    for (int o = 0; o < count; ++o) N[o] = ops[o].N;
+    int rc = share_row_blocks(desc, plan, N, count, rb);
+    if (rc != BCQ_OK) return rc;
+    LutOperand lo[kLutMaxOperands];
+    for (int o = 0; o < count; ++o) {
+        const bcq_operand &op = ops[o];
+        if (!op.packed_dev || !op.y_dev) return BCQ_ERR_INVALID_ARG;
+        lo[o].alpha = lo[o].z = nullptr;
+        if (!interleaved(desc)) {
+            if (!op.alpha_dev || !op.z_dev) return BCQ_ERR_INVALID_ARG;
+            lo[o].alpha = op.alpha_dev, lo[o].z = op.z_dev;
+        }
+        if (!aligned(op.packed_dev, 16) || !aligned(lo[o].alpha, 16) || !aligned(lo[o].z, 16) || !aligned(op.y_dev, 2))
+            return BCQ_ERR_MISALIGNED;
+        lo[o].packed = op.packed_dev, lo[o].y = op.y_dev, lo[o].N = op.N, lo[o].row_blocks = rb[o];
+    }
+    if (!aligned(x, 16)) return BCQ_ERR_MISALIGNED;
+    const size_t need = plan_workspace(desc, plan, 1);
+    if (need > 0) {
+        if (!ws) return BCQ_ERR_INVALID_ARG;
+        if (!aligned(ws, 16)) return BCQ_ERR_MISALIGNED;
+        if (ws_bytes < need) return BCQ_ERR_WORKSPACE_TOO_SMALL;
+    }
+    const cudaError_t e = launch_lut_multi(*desc, *plan, lo, count, x, need ? ws : nullptr, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
 // The host-side table of the linear-int -> binary-code conversion (Eq. fuse_step2, Eq. round):
 // plane weights m_j and, for every step-1 integer, the code of the nearest reachable integer.
 int merge_table(int q, int n_bits, const uint8_t *bit_to_plane, double (&weight)[4], uint8_t (&code_of_int)[256])
@@ -493,6 +564,50 @@ int bcq_gemv(const bcq_desc *desc, const void *packed, const uint16_t *alpha, co
     int rc = bcq_plan_default(desc, 1, 0, &plan);
     if (rc != BCQ_OK) return rc;
     return run_gemv(desc, &plan, packed, alpha, z, x, y, ws, ws_bytes, stream);
+}
+
+int bcq_multi_row_blocks(const bcq_desc *desc, const bcq_plan *plan, const int32_t *N, int count, int32_t *out)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!plan || !N || !out || count < 1 || count > kLutMaxOperands) return BCQ_ERR_INVALID_ARG;
+    rc = check_plan(desc, plan, 1);
+    if (rc != BCQ_OK) return rc;
+    if (plan->kernel != 1) return BCQ_ERR_INVALID_ARG;
+    return share_row_blocks(desc, plan, N, count, out);
+}
+
+int bcq_gemv_multi_plan(const bcq_desc *desc, const bcq_plan *plan, const bcq_operand *ops, int count, const uint16_t *x,
+                        void *ws, size_t ws_bytes, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!plan) return BCQ_ERR_INVALID_ARG;
+    if (plan->kernel != 1 || !lut_kernel_covers(desc)) return BCQ_ERR_INVALID_ARG;
+    // the limits on row units per block apply per operand (share_row_blocks); the rest as for one product
+    if (plan->reserved & ~(BCQ_PLAN_TEST_SHORT_WAITS | BCQ_PLAN_TEST_WITHHOLD_TABLE)) return BCQ_ERR_INVALID_ARG;
+    const int W = desc->K / kWindow;
+    if (plan->row_blocks < 1 || plan->row_blocks > kMaxRowBlocks || plan->k_splits < 1 || plan->k_splits > W ||
+        (W + plan->k_splits - 1) / plan->k_splits > kMaxWindowsPerBlock)
+        return BCQ_ERR_INVALID_ARG;
+    return run_multi(desc, plan, ops, count, x, ws, ws_bytes, stream);
+}
+
+int bcq_gemv_multi(const bcq_desc *desc, const bcq_operand *ops, int count, const uint16_t *x, void *ws, size_t ws_bytes,
+                   void *stream)
+{
+    bcq_plan plan;
+    int rc = bcq_plan_default(desc, 1, 0, &plan);
+    if (rc != BCQ_OK) return rc;
+    if (plan.kernel != 1 || !ops || count < 1 || count > kLutMaxOperands) return BCQ_ERR_INVALID_ARG;
+    // the default plan of the rows taken together, with more row blocks if an operand would not fit its share
+    int32_t N[kLutMaxOperands], rb[kLutMaxOperands];
+    for (int o = 0; o < count; ++o) N[o] = ops[o].N;
+    while ((rc = share_row_blocks(desc, &plan, N, count, rb)) != BCQ_OK && plan.row_blocks < desc->N / kUnitRows &&
+           plan.row_blocks < kMaxRowBlocks)
+        ++plan.row_blocks;
+    if (rc != BCQ_OK) return rc;
+    return run_multi(desc, &plan, ops, count, x, ws, ws_bytes, stream);
 }
 
 int bcq_gemm_smallbatch_plan(const bcq_desc *desc, const bcq_plan *plan, const void *packed, const uint16_t *alpha,

@@ -114,6 +114,17 @@ cudaError_t launch_generic(const bcq_desc &d, const void *packed, const uint16_t
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st,
                             int cols = 1);
+// Several operands that share x, K, q and the scaling unit, one launch: d.N = all their rows, the operands' row
+// blocks add up to plan.row_blocks.
+constexpr int kLutMaxOperands = 4;
+struct LutOperand {
+    const void *packed;
+    const uint16_t *alpha, *z;
+    uint16_t *y;
+    int N, row_blocks;
+};
+cudaError_t launch_lut_multi(const bcq_desc &d, const bcq_plan &plan, const LutOperand *ops, int count, const uint16_t *x,
+                             void *workspace, cudaStream_t st, int cols = 1);
 
 cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *X, uint16_t *Y, int B, void *workspace, cudaStream_t st);

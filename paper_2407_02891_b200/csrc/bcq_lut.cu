@@ -129,15 +129,22 @@ int lut_tiles_per_job(int q, bool grouped, int cols)
     return 1;
 }
 
+// Up to kLutMaxOperands matrices that share x, K, q and the scaling unit are multiplied in one launch: every
+// row block belongs to exactly one operand (row blocks rb_first[o] .. rb_first[o + 1] - 1 split operand o's
+// row units evenly), so a block works on one operand exactly as it would in a launch of its own.
 struct LutParams {
-    const uint8_t *tiles;  // tiled operand: per (window, unit) planes (+ alphas, offsets when grouped)
-    const __half *alpha;   // per-row scales only: [u][i][r]
-    const __half *z;       // per-row scales only: [u][r]
+    const uint8_t *tiles[kLutMaxOperands];  // tiled operand: per (window, unit) planes (+ alphas, offsets when grouped)
+    const __half *alpha[kLutMaxOperands];   // per-row scales only: [u][i][r]
+    const __half *z[kLutMaxOperands];       // per-row scales only: [u][r]
+    __half *y[kLutMaxOperands];
+    int U[kLutMaxOperands];                 // row units of each operand
+    int row0[kLutMaxOperands];              // first row of each operand among all rows of the launch
+    int rb_first[kLutMaxOperands + 1];
+    int count;
     const __half *x;
-    __half *y;
     float *partial;  // [k_splits][cols][N] when k_splits > 1
     int *counters;   // [row_blocks][32] when k_splits > 1
-    int N, K, U, W;
+    int N, K, W;     // N: rows of all operands together
     int row_blocks, k_splits;
     int test_flags;  // BCQ_PLAN_TEST_* (0 in production)
 };
@@ -381,7 +388,11 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     const int rbi = blockIdx.x % p.row_blocks, ks = blockIdx.x / p.row_blocks;
-    const int u0 = int((long long)rbi * p.U / p.row_blocks), u1 = int((long long)(rbi + 1) * p.U / p.row_blocks);
+    int op = 0;                                  // the operand this row block belongs to
+    while (op + 1 < p.count && rbi >= p.rb_first[op + 1]) ++op;
+    const int rbl = rbi - p.rb_first[op], rbn = p.rb_first[op + 1] - p.rb_first[op];
+    const int U = p.U[op];
+    const int u0 = int((long long)rbl * U / rbn), u1 = int((long long)(rbl + 1) * U / rbn);
     const int w0 = int((long long)ks * p.W / p.k_splits), w1 = int((long long)(ks + 1) * p.W / p.k_splits);
     const int V = u1 - u0;                       // row units of this block
     const int nwin = w1 - w0;                    // windows of this block
@@ -446,7 +457,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             const uint32_t ring = smem_u32(ring_ptr(c));
             const uint32_t full0 = bar_full + 8 * kD * c, empty0 = bar_empty + 8 * kD * c;
             int slot = 0, fill = 0, issued = 0;
-            const uint8_t *src_w = p.tiles + (size_t(w0) * p.U + u0) * kTile;
+            const uint8_t *src_w = p.tiles[op] + (size_t(w0) * U + u0) * kTile;
             bool ok = true;
             for (int wi = 0; wi < nwin && ok; ++wi) {
                 for (int jb = c; jb < njobs; jb += kCons) {
@@ -481,7 +492,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                         ++fill;
                     }
                 }
-                src_w += size_t(p.U) * kTile;
+                src_w += size_t(U) * kTile;
             }
             // See the lane's last copies land before the block's shared memory can be handed to another
             // block (they have landed long ago unless the block is giving up).
@@ -684,7 +695,9 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
 
     // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up; lanes 0..7 store y, or this K
     // split's partial rows (two columns: those of column 1 follow column 0, N elements further on) ------
-    float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * NB * p.N : nullptr;
+    float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * NB * p.N + p.row0[op] : nullptr;
+    __half *y = p.y[op];
+    const size_t Nop = size_t(U) * kUnitRows;   // rows of this operand: its second column of y starts there
 #pragma unroll
     for (int a = 0; a < kUnitsPerWarp; ++a) {
         const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;   // the unit, counted inside the block
@@ -695,8 +708,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             if (ul < V) {
                 const int u = u0 + ul;
 #pragma unroll
-                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(p.alpha[(size_t(u) * Q + i) * kUnitRows + jr]), acc[a][i % NACC], v);
-                v = fmaf(__half2float(p.z[size_t(u) * kUnitRows + jr]), xacc, v);
+                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(p.alpha[op][(size_t(u) * Q + i) * kUnitRows + jr]), acc[a][i % NACC], v);
+                v = fmaf(__half2float(p.z[op][size_t(u) * kUnitRows + jr]), xacc, v);
             }
         }
         v += __shfl_xor_sync(0xffffffffu, v, 8);
@@ -708,16 +721,16 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
         }
         if (lane < 8 && ul < V) {
-            const size_t n = size_t(u0 + ul) * kUnitRows + lane;
+            const size_t n = size_t(u0 + ul) * kUnitRows + lane;   // row inside the operand
             if (partial)
                 partial[n] = v;
             else
-                p.y[n] = __float2half_rn(v);
+                y[n] = __float2half_rn(v);
             if constexpr (NB == 2) {
                 if (partial)
                     partial[size_t(p.N) + n] = v1;
                 else
-                    p.y[size_t(p.N) + n] = __float2half_rn(v1);
+                    y[Nop + n] = __float2half_rn(v1);
             }
         }
     }
@@ -738,7 +751,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             // lane -> two rows per column: (accumulator slot lane >> 3, row lane & 7) and slot + 4; fixed
             // summation order; the loads of 8 splits of all the lane's rows are issued together
             constexpr int R = 2 * NB;
-            size_t n[R];
+            size_t n[R];   // row inside the operand (+ the operand's rows for the second column)
+            size_t at[R];  // the same row among all rows of the launch, per column: index into a split's partials
             bool on[R];
             float v[R];
 #pragma unroll
@@ -746,7 +760,9 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                 const int a = (lane >> 3) + 4 * (r & 1);
                 const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;
                 on[r] = ul < V;
-                n[r] = size_t(r >> 1) * p.N + size_t(u0 + (on[r] ? ul : 0)) * kUnitRows + (lane & 7);
+                const size_t row = size_t(u0 + (on[r] ? ul : 0)) * kUnitRows + (lane & 7);
+                n[r] = size_t(r >> 1) * Nop + row;
+                at[r] = size_t(r >> 1) * p.N + p.row0[op] + row;
                 v[r] = 0.f;
             }
             for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
@@ -755,7 +771,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
                 for (int r = 0; r < R; ++r)
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        part[r][k] = (on[r] && k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + n[r]) : 0.f;
+                        part[r][k] = (on[r] && k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at[r]) : 0.f;
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -763,7 +779,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParam
             }
 #pragma unroll
             for (int r = 0; r < R; ++r)
-                if (on[r]) p.y[n[r]] = __float2half_rn(v[r]);
+                if (on[r]) y[n[r]] = __float2half_rn(v[r]);
             if (lane == 0) *counter = 0;
         }
     }
@@ -796,29 +812,11 @@ static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
     return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, GROUPED, NB>, prm);
 }
 
-// cols = 1: y = W x.  cols = 2 (grouped scales only): x and y hold two columns, K and N elements apart.
-cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
-                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st, int cols)
+static cudaError_t launch_lut_params(int q, bool grouped, int cols, const LutParams &prm, cudaStream_t st)
 {
-    LutParams prm;
-    prm.tiles = static_cast<const uint8_t *>(packed);
-    prm.alpha = reinterpret_cast<const __half *>(alpha);   // used with per-row scales only
-    prm.z = reinterpret_cast<const __half *>(z);
-    prm.x = reinterpret_cast<const __half *>(x);
-    prm.y = reinterpret_cast<__half *>(y);
-    prm.counters = static_cast<int *>(workspace);
-    prm.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + lut_counter_bytes(plan)) : nullptr;
-    prm.N = d.N;
-    prm.K = d.K;
-    prm.U = d.N / kUnitRows;
-    prm.W = d.K / kWindow;
-    prm.row_blocks = plan.row_blocks;
-    prm.k_splits = plan.k_splits;
-    prm.test_flags = plan.reserved;
-    const bool grouped = d.group != 0;
     if (cols == 2) {
         if (!grouped) return cudaErrorInvalidValue;
-        switch (d.q) {
+        switch (q) {
             case 1: return launch_lut_q<1, true, 2>(prm, st);
             case 2: return launch_lut_q<2, true, 2>(prm, st);
             case 3: return launch_lut_q<3, true, 2>(prm, st);
@@ -826,13 +824,56 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
         }
         return cudaErrorInvalidValue;
     }
-    switch (d.q) {
+    switch (q) {
         case 1: return grouped ? launch_lut_q<1, true, 1>(prm, st) : launch_lut_q<1, false, 1>(prm, st);
         case 2: return grouped ? launch_lut_q<2, true, 1>(prm, st) : launch_lut_q<2, false, 1>(prm, st);
         case 3: return grouped ? launch_lut_q<3, true, 1>(prm, st) : launch_lut_q<3, false, 1>(prm, st);
         case 4: return grouped ? launch_lut_q<4, true, 1>(prm, st) : launch_lut_q<4, false, 1>(prm, st);
     }
     return cudaErrorInvalidValue;
+}
+
+// cols = 1: y = W x.  cols = 2 (grouped scales only): x and y hold two columns, K and N elements apart.
+cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
+                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st, int cols)
+{
+    LutOperand one;
+    one.packed = packed, one.alpha = alpha, one.z = z, one.y = y, one.N = d.N, one.row_blocks = plan.row_blocks;
+    return launch_lut_multi(d, plan, &one, 1, x, workspace, st, cols);
+}
+
+// Several operands that share x in one launch (batch 1 unless count == 1); d.N is the sum of their rows and
+// ops[o].row_blocks the row blocks given to operand o (they add up to plan.row_blocks).
+cudaError_t launch_lut_multi(const bcq_desc &d, const bcq_plan &plan, const LutOperand *ops, int count, const uint16_t *x,
+                             void *workspace, cudaStream_t st, int cols)
+{
+    if (count < 1 || count > kLutMaxOperands || (count > 1 && cols != 1)) return cudaErrorInvalidValue;
+    LutParams prm = {};
+    int rows = 0, rb = 0;
+    for (int o = 0; o < count; ++o) {
+        prm.tiles[o] = static_cast<const uint8_t *>(ops[o].packed);
+        prm.alpha[o] = reinterpret_cast<const __half *>(ops[o].alpha);   // used with per-row scales only
+        prm.z[o] = reinterpret_cast<const __half *>(ops[o].z);
+        prm.y[o] = reinterpret_cast<__half *>(ops[o].y);
+        prm.U[o] = ops[o].N / kUnitRows;
+        prm.row0[o] = rows;
+        prm.rb_first[o] = rb;
+        rows += ops[o].N;
+        rb += ops[o].row_blocks;
+    }
+    for (int o = count; o <= kLutMaxOperands; ++o) prm.rb_first[o] = rb;
+    if (rows != d.N || rb != plan.row_blocks) return cudaErrorInvalidValue;
+    prm.count = count;
+    prm.x = reinterpret_cast<const __half *>(x);
+    prm.counters = static_cast<int *>(workspace);
+    prm.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + lut_counter_bytes(plan)) : nullptr;
+    prm.N = d.N;
+    prm.K = d.K;
+    prm.W = d.K / kWindow;
+    prm.row_blocks = plan.row_blocks;
+    prm.k_splits = plan.k_splits;
+    prm.test_flags = plan.reserved;
+    return launch_lut_params(d.q, d.group != 0, cols, prm, st);
 }
 
 // Read and clear the device status word.

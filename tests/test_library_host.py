@@ -171,3 +171,18 @@ def test_default_plans_are_remembered_consistently():
     b = bq.plan_default(bq.desc(7168, 7168, 3, 128, bq.LAYOUT_TILED), 1, 64)
     assert a.row_blocks * a.k_splits <= 148 and b.row_blocks * b.k_splits <= 2 * 64
     assert (a.row_blocks, a.k_splits) != (b.row_blocks, b.k_splits)
+
+
+def test_multi_row_blocks_are_shared_in_proportion():
+    d = bq.desc(7168 * 3, 7168, 3, 128, bq.LAYOUT_TILED)
+    assert bq.multi_row_blocks(d, bq.Plan(1, 60, 7, 0), [7168, 7168, 7168]) == [20, 20, 20]
+    assert bq.multi_row_blocks(d, bq.Plan(1, 61, 7, 0), [7168, 7168, 7168]) == [21, 20, 20]
+    d = bq.desc(8192 + 2048, 8192, 3, 128, bq.LAYOUT_TILED)          # a query projection and a fused k/v (GQA)
+    assert bq.multi_row_blocks(d, bq.Plan(1, 20, 7, 0), [8192, 2048]) == [16, 4]
+    assert bq.multi_row_blocks(d, bq.Plan(1, 18, 7, 0), [8192, 2048]) == [14, 4]      # 14.4 and 3.6: the remainder goes to 3.6
+    with pytest.raises(bq.BcqError):                                  # rows do not add up to desc.N
+        bq.multi_row_blocks(d, bq.Plan(1, 20, 7, 0), [8192, 1024])
+    with pytest.raises(bq.BcqError):                                  # 1024 row units in 5 row blocks: more than 184 each
+        bq.multi_row_blocks(d, bq.Plan(1, 6, 7, 0), [8192, 2048])
+    with pytest.raises(bq.BcqError):                                  # fewer row blocks than operands
+        bq.multi_row_blocks(d, bq.Plan(1, 1, 7, 0), [8192, 2048])
