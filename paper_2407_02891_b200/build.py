@@ -10,7 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbcq.so")
-SOURCES = ["bcq_api.cu", "bcq_pack.cu", "bcq_gemv.cu", "bcq_lut.cu", "bcq_mma.cu", "bcq_quant.cu", "bcq_noalloc.cu"]
+SOURCES = ["bcq_api.cu", "bcq_pack.cu", "bcq_gemv.cu", "bcq_lut.cu", "bcq_lut_q1.cu", "bcq_lut_q2.cu", "bcq_lut_q3.cu",
+           "bcq_lut_q4.cu", "bcq_mma.cu", "bcq_quant.cu", "bcq_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
@@ -44,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if r.returncode:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
 
-    with ThreadPoolExecutor(max_workers=4) as ex:
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 4)) as ex:
         list(ex.map(run, jobs))
     if jobs or force or _stale(LIB, objs):
         run([nvcc, "-shared", "-o", LIB, *objs, "-lcudart"])

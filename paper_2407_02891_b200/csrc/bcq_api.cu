@@ -585,6 +585,7 @@ int bcq_gemv_multi_plan(const bcq_desc *desc, const bcq_plan *plan, const bcq_op
     if (!plan) return BCQ_ERR_INVALID_ARG;
     if (plan->kernel != 1 || !lut_kernel_covers(desc)) return BCQ_ERR_INVALID_ARG;
     // the limits on row units per block apply per operand (share_row_blocks); the rest as for one product
+    if (plan->reserved != 0 && count > 1) return BCQ_ERR_INVALID_ARG;   // the test bits apply to single products
     if (plan->reserved & ~(BCQ_PLAN_TEST_SHORT_WAITS | BCQ_PLAN_TEST_WITHHOLD_TABLE)) return BCQ_ERR_INVALID_ARG;
     const int W = desc->K / kWindow;
     if (plan->row_blocks < 1 || plan->row_blocks > kMaxRowBlocks || plan->k_splits < 1 || plan->k_splits > W ||

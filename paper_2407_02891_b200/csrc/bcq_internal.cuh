@@ -124,7 +124,7 @@ struct LutOperand {
     int N, row_blocks;
 };
 cudaError_t launch_lut_multi(const bcq_desc &d, const bcq_plan &plan, const LutOperand *ops, int count, const uint16_t *x,
-                             void *workspace, cudaStream_t st, int cols = 1);
+                             void *workspace, cudaStream_t st);
 
 cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *X, uint16_t *Y, int B, void *workspace, cudaStream_t st);

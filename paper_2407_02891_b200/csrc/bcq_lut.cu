@@ -1,96 +1,17 @@
-// Lookup-table BCQ GEMV for sm_100a: batch 1 (tiled layout, scales per group of 128 or per row), and a
-// two-column variant for group 128.
-//
-//   y = sum_g ( sum_i alpha_i (B_i x)_g + z (sum x)_g )          (Eq. bcw + Eq. fuse_step3)
-//
-// Per 512-wide window of K the block builds, in shared memory, all 2^8 signed sums of every
-// 8-activation chunk; packed weight bytes index those tables directly.  One block per SM, three
-// kinds of warps:
-//
-//   producers (1 or 2 warps) lane c keeps the private ring of consumer warp c filled with bulk async
-//                            copies (cp.async.bulk, completion on the slot's mbarrier).  A slot holds one
-//                            job = kJ consecutive tiles of one window (one contiguous piece of memory), a
-//                            ring kD slots.  The packed weights are constants, so the first slot of every
-//                            ring is requested before the kernel waits for its predecessor in the stream;
-//                            the rest follows once the first table stands (requests queued earlier
-//                            would delay the activations on their way to the block).
-//   builders  (3 warps)      build the window tables from x, one window ahead of the consumers
-//                            (two tables, double buffered);
-//   consumers (kCons warps)  wait for a slot, copy its tiles to registers (handing the slot back after the
-//                            last one), look every weight byte up in the window table and accumulate in
-//                            fp32.  One tile = q*512 B of plane bytes + the unit's alphas and offsets of one
-//                            (window, row unit).
-//
-// The lookup itself is bound by the shared-memory pipe: one 32-lane lookup is one wavefront, a tile of
-// q = 3 planes costs 48 of them plus 14 to bring the tile to registers and 14 for the copy engine to
-// write it; per-tile bookkeeping is kept off the consumers for that reason.
-//
-// Tables.  The sums are computed in fp32 and stored as fp16 (one rounding, relative 2^-11; the
-// accumulation of the looked-up values stays fp32).  Both tables share one 64 KB region at a shared-window
-// address that is a multiple of 64 KB: entry e of table b, chunk c at byte  e*256 + b*128 + (c>>1)*4 +
-// (c&1)*2.  Lane l = 8 g + j of a consumer warp handles row j of a unit and the g-th group of 128 weights
-// of the window; it walks the group's 16 chunks skewed by 2 j, so at every step the 32 lanes address 32
-// different 4-byte columns -- 32 distinct banks whatever the weight bytes are -- and a lane needs only
-// its own (row, group) scales.  With the 256-byte entry stride and the 64 KB alignment ONE byte-permute
-// builds the complete address (byte 1 <- weight byte, bytes 0,2,3 <- table address + column): a
-// lookup is PRMT + LDS.U16 + one mixed-precision add (fp32 += fp16).
-//
-// Two columns (NB = 2).  A lookup moves 2 bytes per lane, half of what the shared-memory pipe delivers
-// per access; with two activation vectors the entry becomes 4 bytes -- the sums of (column 0, column 1)
-// for the same chunk and index -- and one lookup feeds two adds.  Entry e (256 B) is then [even chunks:
-// 32 words][odd chunks: 32 words]; all lanes of a warp are at chunks of one parity at any step, so they
-// still read 32 different words.  Each table buffer fills a 64 KB region of its own.
-//
-// Split K.  The rows of consumer warp c are the same in every K split of a row block.  Each warp stores its
-// partial rows, publishes them (fence + one atomic on the counter of (row block, c)) and is done unless it
-// was the last of the k_splits warps to arrive: that one adds the partial rows in split order
-// (deterministic), rounds and stores y.  No block-wide barrier and no waiting on other blocks.
-//
-// The kernel is launched with programmatic stream serialisation: it lets its dependents start as soon as
-// it runs and waits for its own predecessor only before it touches x, the workspace or y; the packed
-// weights are treated as constants that are complete before the launch.
-//
-// Every wait is bounded; if one runs out the block sets an abort flag and a device status word, stops
-// waiting, sees its own copies land and returns (see lut_status_take).
-#include "bcq_async.cuh"
-#include "bcq_internal.cuh"
+// Host side of the lookup-table BCQ GEMV: geometry queries, parameter marshalling and dispatch to the
+// instantiations (bcq_lut_kernel.cuh holds the kernel; bcq_lut_q1.cu .. q4.cu instantiate it per plane count).
+#include "bcq_lut_kernel.cuh"
 
 namespace bcq {
 
-constexpr int kLutThreads = 896;                  // 28 warps at 72 registers fill the register file
-constexpr int kLutSmemBytes = 232448;             // 227 KB: the per-block opt-in maximum
-constexpr int kFixedBytes = 2048;                 // barriers and flags
-constexpr int kBuilderWarps = 3;
-constexpr int kBuilderThreads = kBuilderWarps * 32;
-constexpr int kUnitsPerWarp = kLutUnitsPerWarp;   // row units a consumer warp keeps accumulators for
-constexpr int kEarlyJobs = 1;                     // jobs per ring requested before the first table stands
-constexpr int kTestSpinLimit = 1 << 12;           // polls per wait when a test shortens the limit
-
-__device__ int g_lut_status = 0;  // 0, or the code of the wait that ran out (sticky until taken)
-
-// Geometry of one instantiation: tile bytes, tiles per job (kJ), slots per ring (kD), consumer warps.
-// The rings are cut from the two pieces of shared memory before and after the 64 KB-aligned tables; the
-// sizes below assume the usual 1 KB offset of a block's shared window (the kernel checks what it finds).
-template <int Q, bool GROUPED, int NB>
-struct LutCfg {
-    static constexpr int kTile = Q * 512 + (GROUPED ? Q * 64 + 64 : 0);
-    static constexpr int kTables = NB * 65536;
-    static constexpr int kFront = 65536 - 1024;
-    static constexpr int kBack = kLutSmemBytes - kFront - kTables - kFixedBytes;
-    static constexpr int rings(int j, int d) { return kFront / (j * d * kTile) + kBack / (j * d * kTile); }
-    // preference: two tiles per copy and two slots; then one tile per copy with three or two slots
-    static constexpr int kChoice = rings(2, 2) >= kLutConsumersMax ? 0 : (rings(1, 3) >= kLutConsumersMax ? 1 : 2);
-    static constexpr int kJ = kChoice == 0 ? 2 : 1;
-    static constexpr int kD = kChoice == 0 ? 2 : (kChoice == 1 ? 3 : 2);
-    static constexpr int kCons = rings(kJ, kD) < kLutConsumersMax ? rings(kJ, kD) : kLutConsumersMax;
-    static constexpr int kProducers = kJ == 1 ? 2 : 1;   // one warp starts about 18 copies per microsecond
-    static constexpr int kFirstCons = kProducers + kBuilderWarps;
-    static constexpr int kWorking = kBuilderWarps + kCons;   // warps that take part after the producers split off
-    static constexpr int kJobsPerWarp = kUnitsPerWarp / kJ;
-    static constexpr int kRingBytes = kJ * kD * kTile;
-    static_assert(kCons >= 16 && kFirstCons + kCons <= kLutThreads / 32, "warp budget");
-    static_assert(16 * kCons * kD + 64 <= kFixedBytes, "barrier area");
-};
+cudaError_t launch_lut_q1(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t launch_lut_q2(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t launch_lut_q3(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t launch_lut_q4(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t lut_status_take_q1(int *status);
+cudaError_t lut_status_take_q2(int *status);
+cudaError_t lut_status_take_q3(int *status);
+cudaError_t lut_status_take_q4(int *status);
 
 int lut_consumer_warps(int q, bool grouped, int cols)
 {
@@ -129,764 +50,82 @@ int lut_tiles_per_job(int q, bool grouped, int cols)
     return 1;
 }
 
-// Up to kLutMaxOperands matrices that share x, K, q and the scaling unit are multiplied in one launch: every
-// row block belongs to exactly one operand (row blocks rb_first[o] .. rb_first[o + 1] - 1 split operand o's
-// row units evenly), so a block works on one operand exactly as it would in a launch of its own.
-struct LutParams {
-    const uint8_t *tiles[kLutMaxOperands];  // tiled operand: per (window, unit) planes (+ alphas, offsets when grouped)
-    const __half *alpha[kLutMaxOperands];   // per-row scales only: [u][i][r]
-    const __half *z[kLutMaxOperands];       // per-row scales only: [u][r]
-    __half *y[kLutMaxOperands];
-    int U[kLutMaxOperands];                 // row units of each operand
-    int row0[kLutMaxOperands];              // first row of each operand among all rows of the launch
-    int rb_first[kLutMaxOperands + 1];
-    int count;
-    const __half *x;
-    float *partial;  // [k_splits][cols][N] when k_splits > 1
-    int *counters;   // [row_blocks][32] when k_splits > 1
-    int N, K, W;     // N: rows of all operands together
-    int row_blocks, k_splits;
-    int test_flags;  // BCQ_PLAN_TEST_* (0 in production)
-};
-
-// table lookup + accumulate: the address register already holds the complete shared-window
-// address of an fp16 entry; acc (fp32) += entry, in one mixed-precision add
-template <int OFF>
-__device__ __forceinline__ void lut_add(float &acc, uint32_t addr)
+static cudaError_t launch_lut_any(int q, bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
 {
-    asm volatile(
-        "{\n\t.reg .b16 h;\n\t"
-        "ld.shared.b16 h, [%1+%2];\n\t"
-        "add.rn.f32.f16 %0, h, %0;\n\t}"
-        : "+f"(acc)
-        : "r"(addr), "n"(OFF));
-}
-// the first lookup of a sum: acc = entry
-template <int OFF>
-__device__ __forceinline__ float lut_first(uint32_t addr)
-{
-    float f;
-    asm volatile(
-        "{\n\t.reg .b16 h;\n\t"
-        "ld.shared.b16 h, [%1+%2];\n\t"
-        "cvt.f32.f16 %0, h;\n\t}"
-        : "=f"(f)
-        : "r"(addr), "n"(OFF));
-    return f;
-}
-// the same for two columns at once: the 4-byte entry holds (column 0, column 1) as fp16
-template <int OFF>
-__device__ __forceinline__ void lut_add2(float &acc0, float &acc1, uint32_t addr)
-{
-    asm volatile(
-        "{\n\t.reg .b16 l, h;\n\t.reg .b32 v;\n\t"
-        "ld.shared.b32 v, [%2+%3];\n\t"
-        "mov.b32 {l, h}, v;\n\t"
-        "add.rn.f32.f16 %0, l, %0;\n\t"
-        "add.rn.f32.f16 %1, h, %1;\n\t}"
-        : "+f"(acc0), "+f"(acc1)
-        : "r"(addr), "n"(OFF));
-}
-template <int OFF>
-__device__ __forceinline__ void lut_first2(float &acc0, float &acc1, uint32_t addr)
-{
-    asm volatile(
-        "{\n\t.reg .b16 l, h;\n\t.reg .b32 v;\n\t"
-        "ld.shared.b32 v, [%2+%3];\n\t"
-        "mov.b32 {l, h}, v;\n\t"
-        "cvt.f32.f16 %0, l;\n\t"
-        "cvt.f32.f16 %1, h;\n\t}"
-        : "=f"(acc0), "=f"(acc1)
-        : "r"(addr), "n"(OFF));
-}
-template <int OFF>
-__device__ __forceinline__ uint32_t lds_b32(uint32_t addr)
-{
-    uint32_t v;
-    asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(OFF));
-    return v;
-}
-
-// two fp32 lanes in one 64-bit register
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi)
-{
-    f32x2 r;
-    asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ float2 unpack2(f32x2 v)
-{
-    float2 r;
-    asm("mov.b64 {%0,%1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));
-    return r;
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
-{
-    f32x2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-
-// Table build.  A thread owns four consecutive chunks (quad cq: chunks 4cq .. 4cq+3, i.e. 32
-// activations read straight from x): it converts them once, then for each of its values of the
-// entry bits 3..7 (hi = hi0, hi0 + hi_step, ... < 32) walks the 8 entries sharing those bits in
-// Gray-code order: one packed fp32 FMA per entry and chunk pair, the four sums rounded to fp16 and
-// stored with one 64-bit store (16 quads = 128 contiguous bytes per entry: no bank conflicts).
-// `table` points at entry 0 of the buffer being built.  Loading (load_quad) and building are separate
-// so that a builder can have the next window's activations on their way while it waits for the buffer.
-__device__ __forceinline__ void load_quad(const __half *xw, int cq, f32x2 (&x01)[8], f32x2 (&x23)[8])
-{
-    float xf[4][8];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const uint4 raw = *reinterpret_cast<const uint4 *>(xw + 32 * cq + 8 * k);
-        const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float2 f = __half22float2(h2[j]);
-            xf[k][2 * j] = f.x;
-            xf[k][2 * j + 1] = f.y;
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        x01[j] = pack2(xf[0][j], xf[1][j]);
-        x23[j] = pack2(xf[2][j], xf[3][j]);
-    }
-}
-__device__ __forceinline__ void build_quad(unsigned char *table, const f32x2 (&x01)[8], const f32x2 (&x23)[8], int cq, int hi0,
-                                           int hi_step)
-{
-    const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
-    f32x2 low01 = pack2(0.f, 0.f), low23 = low01;   // -(x0 + x1 + x2): entry bits 0..2 clear
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-        low01 = fma2(m1, x01[j], low01);
-        low23 = fma2(m1, x23[j], low23);
-    }
-    for (int hi = hi0; hi < 32; hi += hi_step) {
-        f32x2 c01 = low01, c23 = low23;
-#pragma unroll
-        for (int j = 3; j < 8; ++j) {
-            const float sg = ((hi >> (j - 3)) & 1) ? 1.f : -1.f;
-            const f32x2 s2 = pack2(sg, sg);
-            c01 = fma2(s2, x01[j], c01);
-            c23 = fma2(s2, x23[j], c23);
-        }
-        unsigned char *dst = table + cq * 8 + hi * (8 * 256);
-        static_for<0, 8>([&](auto step_c) {
-            constexpr int step = decltype(step_c)::value;
-            constexpr int gray = step ^ (step >> 1);
-            if constexpr (step > 0) {
-                constexpr int bit = (step & 1) ? 0 : ((step & 2) ? 1 : 2);  // lowest set bit of step
-                constexpr bool on = (gray >> bit) & 1;
-                c01 = fma2(on ? p2 : m2, x01[bit], c01);
-                c23 = fma2(on ? p2 : m2, x23[bit], c23);
-            }
-            const float2 a = unpack2(c01), b = unpack2(c23);
-            const __half2 h01 = __floats2half2_rn(a.x, a.y), h23 = __floats2half2_rn(b.x, b.y);
-            uint2 out;
-            out.x = *reinterpret_cast<const uint32_t *>(&h01);
-            out.y = *reinterpret_cast<const uint32_t *>(&h23);
-            *reinterpret_cast<uint2 *>(dst + gray * 256) = out;
-        });
-    }
-}
-
-// Two columns.  Table entry e (256 B) = [even chunks: 32 words][odd chunks: 32 words], a word = the fp16
-// sums of (column 0, column 1) for that chunk and entry.  A thread owns the chunk pair cp (chunks 2cp,
-// 2cp + 1) of both columns: xa / xb hold activation j of the two chunks for column 0 / column 1.
-__device__ __forceinline__ void load_pair(const __half *xw, size_t col_stride, int cp, f32x2 (&xa)[8], f32x2 (&xb)[8])
-{
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-        const __half *src = xw + c * col_stride + 16 * cp;
-        const uint4 r0 = *reinterpret_cast<const uint4 *>(src), r1 = *reinterpret_cast<const uint4 *>(src + 8);
-        const __half2 *h0 = reinterpret_cast<const __half2 *>(&r0), *h1 = reinterpret_cast<const __half2 *>(&r1);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float2 f0 = __half22float2(h0[j]), f1 = __half22float2(h1[j]);
-            if (c == 0) {
-                xa[2 * j] = pack2(f0.x, f1.x);
-                xa[2 * j + 1] = pack2(f0.y, f1.y);
-            } else {
-                xb[2 * j] = pack2(f0.x, f1.x);
-                xb[2 * j + 1] = pack2(f0.y, f1.y);
-            }
-        }
-    }
-}
-__device__ __forceinline__ void build_pair(unsigned char *table, const f32x2 (&xa)[8], const f32x2 (&xb)[8], int cp, int hi0,
-                                           int hi_step)
-{
-    const f32x2 m1 = pack2(-1.f, -1.f), p2 = pack2(2.f, 2.f), m2 = pack2(-2.f, -2.f);
-    f32x2 lowa = pack2(0.f, 0.f), lowb = lowa;
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-        lowa = fma2(m1, xa[j], lowa);
-        lowb = fma2(m1, xb[j], lowb);
-    }
-    for (int hi = hi0; hi < 32; hi += hi_step) {
-        f32x2 ca = lowa, cb = lowb;
-#pragma unroll
-        for (int j = 3; j < 8; ++j) {
-            const float sg = ((hi >> (j - 3)) & 1) ? 1.f : -1.f;
-            const f32x2 s2 = pack2(sg, sg);
-            ca = fma2(s2, xa[j], ca);
-            cb = fma2(s2, xb[j], cb);
-        }
-        unsigned char *dst = table + cp * 4 + hi * (8 * 256);
-        static_for<0, 8>([&](auto step_c) {
-            constexpr int step = decltype(step_c)::value;
-            constexpr int gray = step ^ (step >> 1);
-            if constexpr (step > 0) {
-                constexpr int bit = (step & 1) ? 0 : ((step & 2) ? 1 : 2);
-                constexpr bool on = (gray >> bit) & 1;
-                ca = fma2(on ? p2 : m2, xa[bit], ca);
-                cb = fma2(on ? p2 : m2, xb[bit], cb);
-            }
-            const float2 a = unpack2(ca), b = unpack2(cb);   // a: column 0 of chunks 2cp, 2cp+1; b: column 1
-            const __half2 even = __floats2half2_rn(a.x, b.x), odd = __floats2half2_rn(a.y, b.y);
-            *reinterpret_cast<uint32_t *>(dst + gray * 256) = *reinterpret_cast<const uint32_t *>(&even);
-            *reinterpret_cast<uint32_t *>(dst + gray * 256 + 128) = *reinterpret_cast<const uint32_t *>(&odd);
-        });
-    }
-}
-
-enum { kWaitEmpty = 1, kWaitFull = 2, kWaitTableReady = 3, kWaitTableFree = 4, kWaitDrain = 5, kTooFewRings = 6, kWaitStart = 7 };
-
-// A bounded wait whose limit a test can shorten (see BCQ_PLAN_TEST_SHORT_WAITS).
-template <bool LONG = false>
-__device__ __forceinline__ bool lut_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code, int limit)
-{
-    for (int it = 0; it < limit; ++it) {
-        if (mbar_test_wait(bar, parity)) return true;
-        if (LONG && it >= 8)
-            __nanosleep(256);
-        else
-            __nanosleep(32);
-        if ((it & 255) == 255 && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    atomicExch(&g_lut_status, code);
-    return false;
-}
-
-// NB columns per launch: 1, or 2 (grouped scales only) with tables that hold both columns' sums side by
-// side, so that one 4-byte lookup serves two products; each of the two table buffers then fills a
-// 64 KB region of its own.
-template <int Q, bool GROUPED, int NB>
-__global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const LutParams p)
-{
-    static_assert(NB == 1 || (NB == 2 && GROUPED), "two columns need the scales inside the tiles");
-    using C = LutCfg<Q, GROUPED, NB>;
-    extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int kTile = C::kTile, kJ = C::kJ, kD = C::kD, kCons = C::kCons;
-    constexpr int kSlotBytes = kJ * kTile;
-    constexpr int NACC = GROUPED ? 1 : Q;   // accumulators per unit and lane: the row's sum, or one per plane
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    const int rbi = blockIdx.x % p.row_blocks, ks = blockIdx.x / p.row_blocks;
-    int op = 0;                                  // the operand this row block belongs to
-    while (op + 1 < p.count && rbi >= p.rb_first[op + 1]) ++op;
-    const int rbl = rbi - p.rb_first[op], rbn = p.rb_first[op + 1] - p.rb_first[op];
-    const int U = p.U[op];
-    const int u0 = int((long long)rbl * U / rbn), u1 = int((long long)(rbl + 1) * U / rbn);
-    const int w0 = int((long long)ks * p.W / p.k_splits), w1 = int((long long)(ks + 1) * p.W / p.k_splits);
-    const int V = u1 - u0;                       // row units of this block
-    const int nwin = w1 - w0;                    // windows of this block
-    const int njobs = (V + kJ - 1) / kJ;         // jobs per window
-    const int spin_limit = (p.test_flags & BCQ_PLAN_TEST_SHORT_WAITS) ? kTestSpinLimit : kSpinLimit;
-
-    // ---- carve shared memory: [front | tables (64 KB each, 64 KB aligned) | barriers | back] --------------
-    const uint32_t base = smem_u32(smem);
-    const uint32_t tab0 = (base + 0xFFFFu) & ~0xFFFFu;  // shared-window address of the tables
-    const int front = int(tab0 - base), back = kLutSmemBytes - front - C::kTables;
-    unsigned char *tables = smem + front;
-    unsigned char *after = tables + C::kTables;
-    const bool fixed_in_back = back >= kFixedBytes;
-    unsigned char *fixed = fixed_in_back ? after : smem;
-    unsigned char *ring_a = fixed_in_back ? smem : smem + kFixedBytes;
-    unsigned char *ring_b = fixed_in_back ? after + kFixedBytes : after;
-    const int rings_a = (fixed_in_back ? front : front - kFixedBytes) / C::kRingBytes;
-    const int rings_b = (fixed_in_back ? back - kFixedBytes : back) / C::kRingBytes;
-    auto ring_ptr = [&](int c) -> unsigned char * {
-        return c < rings_a ? ring_a + c * C::kRingBytes : ring_b + (c - rings_a) * C::kRingBytes;
-    };
-
-    const uint32_t bars = smem_u32(fixed);
-    const uint32_t bar_full = bars, bar_empty = bars + 8 * kCons * kD;     // [consumer][slot]
-    const uint32_t bar_tab_ready = bars + 16 * kCons * kD, bar_tab_free = bar_tab_ready + 16;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(fixed + 16 * kCons * kD + 32);
-    volatile int *started = abort_flag + 1;
-
-    if (warp == 0) {   // one warp initialises the barriers, a few each
-        for (int s = lane; s < kCons * kD; s += 32) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
-        }
-        if (lane < 2) {
-            mbar_init(bar_tab_ready + 8 * lane, kBuilderThreads);
-            mbar_init(bar_tab_free + 8 * lane, kCons);
-        }
-        if (lane == 0) {
-            // every consumer warp needs its ring, and the block's row units must fit the consumers
-            const bool bad = rings_a + rings_b < kCons || njobs > kCons * C::kJobsPerWarp;
-            *abort_flag = bad ? 1 : 0;
-            *started = 0;
-            if (bad) atomicExch(&g_lut_status, int(kTooFewRings));
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-    // Programmatic dependent launch: the next kernel in the stream may start taking SMs as soon as
-    // this kernel's blocks leave them (it still waits, below, for its predecessor to finish before
-    // it reads x or writes anything).  Without the launch attribute both instructions do nothing.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-    // Work of consumer c: jobs jb = c, c + kCons, ... of every window, in that order; its m-th job uses slot
-    // m % kD of its ring in fill number m / kD.
-    // =============================================================================================
-    // ---- producers: lane -> consumer c; keeps that consumer's ring filled ---------------------------
-    if (warp < C::kProducers) {
-        const int c = lane * C::kProducers + warp;
-        const int mine = (c < kCons && njobs > c) ? (njobs - c + kCons - 1) / kCons : 0;   // jobs per window
-        if (mine > 0 && !*abort_flag) {
-            const uint32_t ring = smem_u32(ring_ptr(c));
-            const uint32_t full0 = bar_full + 8 * kD * c, empty0 = bar_empty + 8 * kD * c;
-            int slot = 0, fill = 0, issued = 0;
-            const uint8_t *src_w = p.tiles[op] + (size_t(w0) * U + u0) * kTile;
-            bool ok = true;
-            for (int wi = 0; wi < nwin && ok; ++wi) {
-                for (int jb = c; jb < njobs; jb += kCons) {
-                    if (issued == kEarlyJobs) {
-                        // The rest of the ring waits until the first table stands.  First wait, like the other
-                        // warps, for the previous kernel (however long it runs); the flag follows shortly.
-                        asm volatile("griddepcontrol.wait;" ::: "memory");
-                        int itr = 0;
-                        while (!*started && !*abort_flag && itr < spin_limit) {
-                            __nanosleep(64);
-                            ++itr;
-                        }
-                        if (!*started) {
-                            if (!*abort_flag) {
-                                *abort_flag = 1;
-                                atomicExch(&g_lut_status, int(kWaitStart));
-                            }
-                            ok = false;
-                            break;
-                        }
-                    }
-                    if (fill > 0 && !lut_wait(empty0 + 8 * slot, (fill - 1) & 1, abort_flag, kWaitEmpty, spin_limit)) {
-                        ok = false;
-                        break;
-                    }
-                    const int nt = min(kJ, V - kJ * jb);
-                    mbar_expect_tx(full0 + 8 * slot, nt * kTile);
-                    bulk_g2s(ring + slot * kSlotBytes, src_w + size_t(kJ * jb) * kTile, nt * kTile, full0 + 8 * slot);
-                    ++issued;
-                    if (++slot == kD) {
-                        slot = 0;
-                        ++fill;
-                    }
-                }
-                src_w += size_t(U) * kTile;
-            }
-            // See the lane's last copies land before the block's shared memory can be handed to another
-            // block (they have landed long ago unless the block is giving up).
-            for (int m = max(0, issued - kD); m < issued; ++m) {
-                bool landed = false;
-                for (int itr = 0; itr < kSpinLimit && !landed; ++itr) {
-                    landed = mbar_test_wait(full0 + 8 * (m % kD), uint32_t((m / kD) & 1));
-                    if (!landed) __nanosleep(256);
-                }
-                if (!landed) atomicExch(&g_lut_status, int(kWaitDrain));
-            }
-        }
-        return;
-    }
-    if (warp >= C::kFirstCons + kCons) return;   // warps this instantiation has no use for
-
-    // =============================================================================================
-    // The weights above are constants; everything from here on (x, partial sums, counters, y) may
-    // depend on the previous kernel in the stream: wait for it to be complete and visible.
-    const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-
-    // ---- start-up: builders and consumers build the first window's table together -----------------
-    const int bt = tid - C::kProducers * 32;   // 0 .. kWorking*32-1
-    if (bt < 512) {
-        if constexpr (NB == 1) {
-            f32x2 x01[8], x23[8];
-            load_quad(xblk, bt & 15, x01, x23);
-            build_quad(tables, x01, x23, bt & 15, bt >> 4, 32);
-        } else {
-            f32x2 xa[8], xb[8];
-            load_pair(xblk, size_t(p.K), bt & 31, xa, xb);
-            build_pair(tables, xa, xb, bt & 31, bt >> 5, 16);
-        }
-    }
-    named_barrier(1, C::kWorking * 32);
-    if (bt == 0) *started = 1;
-
-    if (warp < C::kFirstCons) {
-        // ---- builders: one table per window, one window ahead of the consumers ----------------------
-        // Window 0 was built above; the builders' fills of buffer 0 are windows 2, 4, ... and of
-        // buffer 1 windows 1, 3, ...
-        const bool withhold = (p.test_flags & BCQ_PLAN_TEST_WITHHOLD_TABLE) != 0;
-        for (int wi = 1; wi < nwin; ++wi) {
-            const int b = wi & 1, use = wi >> 1;
-            f32x2 x01[8], x23[8];   // one column: a chunk quad; two columns: a chunk pair of each
-            if constexpr (NB == 1)
-                load_quad(xblk + wi * kWindow, bt & 15, x01, x23);   // in flight while waiting for the buffer
-            else
-                load_pair(xblk + wi * kWindow, size_t(p.K), bt & 31, x01, x23);
-            if (use > 0 && !lut_wait<true>(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, spin_limit)) break;
-            if constexpr (NB == 1)
-                build_quad(tables + b * 128, x01, x23, bt & 15, bt >> 4, kBuilderThreads / 16);
-            else
-                build_pair(tables + b * 65536, x01, x23, bt & 31, bt >> 5, kBuilderThreads / 32);
-            if (!withhold) mbar_arrive(bar_tab_ready + 8 * b);   // (a test withholds it to see the consumers give up)
-        }
-        return;
-    }
-
-    // =============================================================================================
-    // ---- consumers ---------------------------------------------------------------------------------
-    // Lane l = 8 g + j owns row 8u + j of every unit and the g-th group of 128 weights of every
-    // window: its 16q bytes of a tile are the group's 16 chunks (skewed by 2 j, see the layout), so
-    // it needs only its own q alphas and one offset per tile and keeps ONE accumulator per unit.
-    const int cw = warp - C::kFirstCons;
-    const int g4 = lane >> 3, jr = lane & 7;
-    float acc[kUnitsPerWarp][NACC], acc1[NB == 2 ? kUnitsPerWarp : 1];   // acc1: the second column
-    float xacc = 0.f;   // per-row scales: sum of x over this lane's groups of all windows
-#pragma unroll
-    for (int t = 0; t < kUnitsPerWarp; ++t)
-#pragma unroll
-        for (int i = 0; i < NACC; ++i) acc[t][i] = 0.f;
-#pragma unroll
-    for (int t = 0; t < (NB == 2 ? kUnitsPerWarp : 1); ++t) acc1[t] = 0.f;
-    bool alive = !*abort_flag;
-    const unsigned char *ring = ring_ptr(cw);
-    const uint32_t full0 = bar_full + 8 * kD * cw, empty0 = bar_empty + 8 * kD * cw;
-    int slot = 0, fill = 0;
-
-    for (int wi = 0; wi < nwin && alive; ++wi) {
-        const int b = wi & 1;
-        if (wi > 0 && !lut_wait(bar_tab_ready + 8 * b, ((wi >> 1) - (b == 0 ? 1 : 0)) & 1, abort_flag, kWaitTableReady, spin_limit)) {
-            alive = false;
-            break;
-        }
-        // Table address part of the lookups of step pair h: chunk 16 g + ((2h + 2j) mod 16) and the
-        // next one share the 4-byte column 8 g + ((h + j) mod 8); the odd chunk is its upper half.
-        uint32_t off[8];
-#pragma unroll
-        for (int h = 0; h < 8; ++h) off[h] = tab0 + uint32_t(b * (NB == 1 ? 128 : 65536) + 4 * (8 * g4 + ((h + jr) & 7)));
-        // sum of x over this lane's group: the all-ones entries of the group's 16 chunks (two per lane)
-        float xsum, xsum1 = 0.f;
-        if constexpr (NB == 1) {
-            const uint32_t ones = lds_b32<255 * 256>(off[0]);
-            const float2 ones_f = __half22float2(*reinterpret_cast<const __half2 *>(&ones));
-            xsum = ones_f.x + ones_f.y;
-        } else {
-            const uint32_t even = lds_b32<255 * 256>(off[0]), odd = lds_b32<255 * 256 + 128>(off[0]);
-            const float2 e = __half22float2(*reinterpret_cast<const __half2 *>(&even));
-            const float2 o = __half22float2(*reinterpret_cast<const __half2 *>(&odd));
-            xsum = e.x + o.x;
-            xsum1 = e.y + o.y;
-            xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 1);
-            xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 2);
-            xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 4);
-        }
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
-        xacc += xsum;
-
-        static_for<0, C::kJobsPerWarp>([&](auto T) {
-            constexpr int t = decltype(T)::value;
-            const int jb = cw + kCons * t;
-            if (alive && jb < njobs) {
-                if (!lut_wait(full0 + 8 * slot, fill & 1, abort_flag, kWaitFull, spin_limit)) {
-                    alive = false;
-                } else {
-                    const unsigned char *sl = ring + slot * kSlotBytes;
-                    const int nt = min(kJ, V - kJ * jb);   // the last job of a window may be short
-                    static_for<0, kJ>([&](auto TT) {
-                        constexpr int tt = decltype(TT)::value;
-                        constexpr int a = t * kJ + tt;     // accumulator slot of this unit
-                        if (tt < nt) {
-                            const unsigned char *tile = sl + tt * kTile;
-                            uint32_t wbuf[4 * Q];
-#pragma unroll
-                            for (int j = 0; j < Q; ++j) {
-                                const uint4 v = *reinterpret_cast<const uint4 *>(tile + j * 512 + lane * 16);
-                                wbuf[4 * j + 0] = v.x;
-                                wbuf[4 * j + 1] = v.y;
-                                wbuf[4 * j + 2] = v.z;
-                                wbuf[4 * j + 3] = v.w;
-                            }
-                            [[maybe_unused]] __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
-                            if constexpr (GROUPED) {
-                                const unsigned char *sp = tile + Q * 512 + lane * (2 * (Q + 1));
-                                if constexpr (Q == 3) {
-                                    *reinterpret_cast<uint2 *>(sc) = *reinterpret_cast<const uint2 *>(sp);
-                                } else if constexpr (Q == 1) {
-                                    *reinterpret_cast<uint32_t *>(sc) = *reinterpret_cast<const uint32_t *>(sp);
-                                } else {
-#pragma unroll
-                                    for (int i = 0; i <= Q; ++i) sc[i] = reinterpret_cast<const __half *>(sp)[i];
-                                }
-                            }
-                            if (tt == nt - 1) {   // the slot's last tile is in registers: hand the slot back
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(empty0 + 8 * slot);
-                            }
-                            float sum[Q], sum1[NB == 2 ? Q : 1];
-                            static_for<0, 16>([&](auto S) {
-                                constexpr int st = decltype(S)::value;
-                                static_for<0, Q>([&](auto I) {
-                                    constexpr int i = decltype(I)::value;
-                                    constexpr int pb = i * 16 + st;
-                                    const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
-                                    if constexpr (NB == 1) {
-                                        if constexpr (st == 0)
-                                            sum[i] = lut_first<0>(addr);
-                                        else
-                                            lut_add<(st & 1) * 2>(sum[i], addr);
-                                    } else {
-                                        if constexpr (st == 0)
-                                            lut_first2<0>(sum[i], sum1[i], addr);
-                                        else
-                                            lut_add2<(st & 1) * 128>(sum[i], sum1[i], addr);
-                                    }
-                                });
-                            });
-                            if constexpr (GROUPED) {
-                                float v = fmaf(__half2float(sc[Q]), xsum, acc[a][0]);
-#pragma unroll
-                                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(sc[i]), sum[i], v);
-                                acc[a][0] = v;
-                                if constexpr (NB == 2) {
-                                    float v1 = fmaf(__half2float(sc[Q]), xsum1, acc1[a]);
-#pragma unroll
-                                    for (int i = 0; i < Q; ++i) v1 = fmaf(__half2float(sc[i]), sum1[i], v1);
-                                    acc1[a] = v1;
-                                }
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < Q; ++i) acc[a][i] += sum[i];
-                            }
-                        }
-                    });
-                    if (++slot == kD) {
-                        slot = 0;
-                        ++fill;
-                    }
-                }
-            }
-        });
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_tab_free + 8 * b);
-    }
-    if (!alive) return;   // the block is giving up: y is undefined (bcq_poll_status reports it)
-
-    // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up; lanes 0..7 store y, or this K
-    // split's partial rows (two columns: those of column 1 follow column 0, N elements further on) ------
-    float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * NB * p.N + p.row0[op] : nullptr;
-    __half *y = p.y[op];
-    const size_t Nop = size_t(U) * kUnitRows;   // rows of this operand: its second column of y starts there
-#pragma unroll
-    for (int a = 0; a < kUnitsPerWarp; ++a) {
-        const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;   // the unit, counted inside the block
-        float v = acc[a][0];
-        if constexpr (!GROUPED) {
-            // one scale per row: apply the row's alphas and offset to the sums over this block's K range
-            v = 0.f;
-            if (ul < V) {
-                const int u = u0 + ul;
-#pragma unroll
-                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(p.alpha[op][(size_t(u) * Q + i) * kUnitRows + jr]), acc[a][i % NACC], v);
-                v = fmaf(__half2float(p.z[op][size_t(u) * kUnitRows + jr]), xacc, v);
-            }
-        }
-        v += __shfl_xor_sync(0xffffffffu, v, 8);
-        v += __shfl_xor_sync(0xffffffffu, v, 16);
-        float v1 = 0.f;
-        if constexpr (NB == 2) {
-            v1 = acc1[a];
-            v1 += __shfl_xor_sync(0xffffffffu, v1, 8);
-            v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
-        }
-        if (lane < 8 && ul < V) {
-            const size_t n = size_t(u0 + ul) * kUnitRows + lane;   // row inside the operand
-            if (partial)
-                partial[n] = v;
-            else
-                y[n] = __float2half_rn(v);
-            if constexpr (NB == 2) {
-                if (partial)
-                    partial[size_t(p.N) + n] = v1;
-                else
-                    y[Nop + n] = __float2half_rn(v1);
-            }
-        }
-    }
-
-    // ---- split K: the last warp to arrive for (row block, consumer warp) adds the partial rows ------
-    if (p.k_splits > 1 && kJ * cw < V) {
-        __syncwarp();                     // the lanes' partial rows are ordered before lane 0's fence
-        int last = 0;
-        int *counter = p.counters + rbi * 32 + cw;
-        if (lane == 0) {
-            __threadfence();              // cumulative: publishes the whole warp's rows
-            last = (atomicAdd(counter, 1) == p.k_splits - 1);
-            if (last) __threadfence();    // the other splits' rows are visible to what follows
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-            __syncwarp();
-            // lane -> two rows per column: (accumulator slot lane >> 3, row lane & 7) and slot + 4; fixed
-            // summation order; the loads of 8 splits of all the lane's rows are issued together
-            constexpr int R = 2 * NB;
-            size_t n[R];   // row inside the operand (+ the operand's rows for the second column)
-            size_t at[R];  // the same row among all rows of the launch, per column: index into a split's partials
-            bool on[R];
-            float v[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const int a = (lane >> 3) + 4 * (r & 1);
-                const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;
-                on[r] = ul < V;
-                const size_t row = size_t(u0 + (on[r] ? ul : 0)) * kUnitRows + (lane & 7);
-                n[r] = size_t(r >> 1) * Nop + row;
-                at[r] = size_t(r >> 1) * p.N + p.row0[op] + row;
-                v[r] = 0.f;
-            }
-            for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
-                float part[R][8];
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        part[r][k] = (on[r] && k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at[r]) : 0.f;
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) v[r] += part[r][k];
-            }
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                if (on[r]) y[n[r]] = __float2half_rn(v[r]);
-            if (lane == 0) *counter = 0;
-        }
-    }
-}
-
-template <int Q, bool GROUPED, int NB>
-static cudaError_t launch_lut_q(const LutParams &prm, cudaStream_t st)
-{
-    // The opt-in to more than 48 KB of dynamic shared memory is per function and per device:
-    // done on the first launch on each device, remembered afterwards.
-    static bool configured[64] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(lut_gemv_kernel<Q, GROUPED, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(prm.row_blocks * prm.k_splits);
-    cfg.blockDim = dim3(kLutThreads);
-    cfg.dynamicSmemBytes = kLutSmemBytes;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol in the kernel
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, GROUPED, NB>, prm);
-}
-
-static cudaError_t launch_lut_params(int q, bool grouped, int cols, const LutParams &prm, cudaStream_t st)
-{
-    if (cols == 2) {
-        if (!grouped) return cudaErrorInvalidValue;
-        switch (q) {
-            case 1: return launch_lut_q<1, true, 2>(prm, st);
-            case 2: return launch_lut_q<2, true, 2>(prm, st);
-            case 3: return launch_lut_q<3, true, 2>(prm, st);
-            case 4: return launch_lut_q<4, true, 2>(prm, st);
-        }
-        return cudaErrorInvalidValue;
-    }
     switch (q) {
-        case 1: return grouped ? launch_lut_q<1, true, 1>(prm, st) : launch_lut_q<1, false, 1>(prm, st);
-        case 2: return grouped ? launch_lut_q<2, true, 1>(prm, st) : launch_lut_q<2, false, 1>(prm, st);
-        case 3: return grouped ? launch_lut_q<3, true, 1>(prm, st) : launch_lut_q<3, false, 1>(prm, st);
-        case 4: return grouped ? launch_lut_q<4, true, 1>(prm, st) : launch_lut_q<4, false, 1>(prm, st);
+        case 1: return launch_lut_q1(grouped, cols, test, one, many, st);
+        case 2: return launch_lut_q2(grouped, cols, test, one, many, st);
+        case 3: return launch_lut_q3(grouped, cols, test, one, many, st);
+        case 4: return launch_lut_q4(grouped, cols, test, one, many, st);
     }
     return cudaErrorInvalidValue;
 }
 
+static void fill_common(LutOne &one, const bcq_desc &d, const bcq_plan &plan, const uint16_t *x, void *workspace)
+{
+    one.x = reinterpret_cast<const __half *>(x);
+    one.counters = static_cast<int *>(workspace);
+    one.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + lut_counter_bytes(plan)) : nullptr;
+    one.N = d.N;
+    one.K = d.K;
+    one.row_blocks = plan.row_blocks;
+    one.k_splits = plan.k_splits;
+    one.test_flags = plan.reserved;
+}
+
 // cols = 1: y = W x.  cols = 2 (grouped scales only): x and y hold two columns, K and N elements apart.
+// A plan with test bits set runs the test instantiation (one column only).
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st, int cols)
 {
-    LutOperand one;
-    one.packed = packed, one.alpha = alpha, one.z = z, one.y = y, one.N = d.N, one.row_blocks = plan.row_blocks;
-    return launch_lut_multi(d, plan, &one, 1, x, workspace, st, cols);
+    LutOne one = {};
+    one.tiles = static_cast<const uint8_t *>(packed);
+    one.alpha = reinterpret_cast<const __half *>(alpha);   // used with per-row scales only
+    one.z = reinterpret_cast<const __half *>(z);
+    one.y = reinterpret_cast<__half *>(y);
+    fill_common(one, d, plan, x, workspace);
+    return launch_lut_any(d.q, d.group != 0, cols, plan.reserved != 0, &one, nullptr, st);
 }
 
-// Several operands that share x in one launch (batch 1 unless count == 1); d.N is the sum of their rows and
-// ops[o].row_blocks the row blocks given to operand o (they add up to plan.row_blocks).
+// Several operands that share x in one launch (batch 1); d.N is the sum of their rows and ops[o].row_blocks the
+// row blocks given to operand o (they add up to plan.row_blocks).  One operand is launch_lut_gemv.
 cudaError_t launch_lut_multi(const bcq_desc &d, const bcq_plan &plan, const LutOperand *ops, int count, const uint16_t *x,
-                             void *workspace, cudaStream_t st, int cols)
+                             void *workspace, cudaStream_t st)
 {
-    if (count < 1 || count > kLutMaxOperands || (count > 1 && cols != 1)) return cudaErrorInvalidValue;
-    LutParams prm = {};
+    if (count < 1 || count > kLutMaxOperands) return cudaErrorInvalidValue;
     int rows = 0, rb = 0;
+    for (int o = 0; o < count; ++o) rows += ops[o].N, rb += ops[o].row_blocks;
+    if (rows != d.N || rb != plan.row_blocks) return cudaErrorInvalidValue;
+    if (count == 1) return launch_lut_gemv(d, plan, ops[0].packed, ops[0].alpha, ops[0].z, x, ops[0].y, workspace, st, 1);
+    if (plan.reserved != 0) return cudaErrorInvalidValue;   // the test instantiation takes one operand
+    LutMany many = {};
+    rows = rb = 0;
     for (int o = 0; o < count; ++o) {
-        prm.tiles[o] = static_cast<const uint8_t *>(ops[o].packed);
-        prm.alpha[o] = reinterpret_cast<const __half *>(ops[o].alpha);   // used with per-row scales only
-        prm.z[o] = reinterpret_cast<const __half *>(ops[o].z);
-        prm.y[o] = reinterpret_cast<__half *>(ops[o].y);
-        prm.U[o] = ops[o].N / kUnitRows;
-        prm.row0[o] = rows;
-        prm.rb_first[o] = rb;
+        many.tiles[o] = static_cast<const uint8_t *>(ops[o].packed);
+        many.alpha[o] = reinterpret_cast<const __half *>(ops[o].alpha);   // used with per-row scales only
+        many.z[o] = reinterpret_cast<const __half *>(ops[o].z);
+        many.y[o] = reinterpret_cast<__half *>(ops[o].y);
+        many.U[o] = ops[o].N / kUnitRows;
+        many.row0[o] = rows;
+        many.rb_first[o] = rb;
         rows += ops[o].N;
         rb += ops[o].row_blocks;
     }
-    for (int o = count; o <= kLutMaxOperands; ++o) prm.rb_first[o] = rb;
-    if (rows != d.N || rb != plan.row_blocks) return cudaErrorInvalidValue;
-    prm.count = count;
-    prm.x = reinterpret_cast<const __half *>(x);
-    prm.counters = static_cast<int *>(workspace);
-    prm.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + lut_counter_bytes(plan)) : nullptr;
-    prm.N = d.N;
-    prm.K = d.K;
-    prm.W = d.K / kWindow;
-    prm.row_blocks = plan.row_blocks;
-    prm.k_splits = plan.k_splits;
-    prm.test_flags = plan.reserved;
-    return launch_lut_params(d.q, d.group != 0, cols, prm, st);
+    for (int o = count; o <= kLutMaxOperands; ++o) many.rb_first[o] = rb;
+    many.count = count;
+    fill_common(many.one, d, plan, x, workspace);
+    return launch_lut_any(d.q, d.group != 0, 1, false, nullptr, &many, st);
 }
 
-// Read and clear the device status word.
+// Read and clear the device status words of the kernels (one per translation unit that instantiates them).
 cudaError_t lut_status_take(int *status)
 {
-    int v = 0;
-    cudaError_t e = cudaMemcpyFromSymbol(&v, g_lut_status, sizeof(int));
-    if (e != cudaSuccess) return e;
-    if (v != 0) {
-        const int zero = 0;
-        e = cudaMemcpyToSymbol(g_lut_status, &zero, sizeof(int));
-    }
-    *status = v;
+    int v[4] = {0, 0, 0, 0};
+    cudaError_t e = lut_status_take_q1(&v[0]);
+    if (e == cudaSuccess) e = lut_status_take_q2(&v[1]);
+    if (e == cudaSuccess) e = lut_status_take_q3(&v[2]);
+    if (e == cudaSuccess) e = lut_status_take_q4(&v[3]);
+    *status = v[0] ? v[0] : (v[1] ? v[1] : (v[2] ? v[2] : v[3]));
     return e;
 }
 

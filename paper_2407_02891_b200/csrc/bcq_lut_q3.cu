@@ -1,0 +1,12 @@
+// The lookup-table kernel's instantiations for q = 3 bit-planes (a translation unit per q keeps the build parallel).
+#include "bcq_lut_kernel.cuh"
+
+namespace bcq {
+
+cudaError_t launch_lut_q3(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
+{
+    return launch_lut_for_q<3>(grouped, cols, test, one, many, st);
+}
+cudaError_t lut_status_take_q3(int *status) { return lut_status_take_here(status); }
+
+}  // namespace bcq
