@@ -134,8 +134,10 @@ int bcq_check_desc(const bcq_desc *desc);
 int bcq_plan_default(const bcq_desc *desc, int B, int sm_count, bcq_plan *plan_out);
 
 /* Bytes of workspace the plan needs (0 when k_splits == 1 and the generic kernel).  The
- * workspace holds split-K partial sums and arrival counters.  It must be zero-filled once
- * (bcq_workspace_init) before its first use; every call leaves the counters zero again, so
+ * workspace holds the split-K partial sums and arrival counts (kernel 1: one 64-bit word per
+ * row and column, in which the K splits' sums meet as fixed-point numbers in units of 2^-26;
+ * a split's partial sum beyond +-131071 saturates).  It must be zero-filled once
+ * (bcq_workspace_init) before its first use; every call leaves it zero where it has to be, so
  * it can be reused by later calls ON THE SAME STREAM.  Two products in flight at once
  * need two workspaces.  After a call that bcq_poll_status reported as timed out the counters
  * may be left non-zero: zero-fill the workspace again before the next use. */
@@ -305,8 +307,8 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed_dev, const uint16_t *
  * Consequences to know about:
  *   - every GPU on which this library is loaded gives up that much memory until the process
  *     exits, whether or not this function is ever called;
- *   - a product whose default decomposition needs more scratch (k_splits * N * 4 bytes plus
- *     128 bytes of counters per row block) is refused with BCQ_ERR_SCRATCH_LIMIT and nothing is
+ *   - a product whose default decomposition needs more scratch (8 bytes per row when K is
+ *     split, i.e. more than 262144 rows) is refused with BCQ_ERR_SCRATCH_LIMIT and nothing is
  *     launched;
  *   - the first call on each device looks up the array's device address (a host-side runtime
  *     query, done with that device current) and keeps it for as long as the device's primary

@@ -220,7 +220,7 @@ size_t plan_workspace(const bcq_desc *d, const bcq_plan *p, int B)
 {
     if (p->k_splits <= 1) return 0;
     // kernel 1 runs one column per launch, or two when the scales live in the tiles
-    if (p->kernel == 1) return lut_counter_bytes(*p) + size_t(p->k_splits) * ((B >= 2 && interleaved(d)) ? 2 : 1) * d->N * sizeof(float);
+    if (p->kernel == 1) return lut_workspace_bytes(d->N, (B >= 2 && interleaved(d)) ? 2 : 1);
     if (p->kernel == 2) return kCounterBytes + size_t(p->k_splits) * B * d->N * sizeof(float);
     return 0;
 }

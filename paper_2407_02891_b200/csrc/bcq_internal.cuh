@@ -19,12 +19,12 @@ constexpr int kMaxWindowsPerBlock = 32; // windows one block may walk (bounds th
 constexpr int kMmaWarps = 22;        // consumer warps per block of the small-batch kernel
 constexpr int kMmaPairsPerWarp = 4;  // pairs of row units a warp keeps accumulators for
 constexpr int kMmaMaxUnitsPerBlock = 2 * kMmaWarps * kMmaPairsPerWarp;
-constexpr int kMaxRowBlocks = 4096; // arrival counters at the head of the workspace
+constexpr int kMaxRowBlocks = 4096; // small-batch kernel: arrival counters at the head of its workspace
 constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);   // small-batch kernel: one counter per row block
 
-// The lookup-table kernel counts arrivals per (row block, consumer warp): 32 counters per row block at the
-// head of its workspace, the fp32 partial rows behind them.
-inline size_t lut_counter_bytes(const bcq_plan &plan) { return (size_t(plan.row_blocks) * 32 * sizeof(int) + 255) & ~size_t(255); }
+// The lookup-table kernel's split-K workspace: one 64-bit word per row and column (sum and arrival count in
+// one word, see bcq_lut_kernel.cuh); all zero between launches.
+inline size_t lut_workspace_bytes(int N, int cols) { return size_t(cols) * size_t(N) * sizeof(unsigned long long); }
 // consumer warps and tiles per copy of the instantiation for (q, scales per group?, columns per launch)
 int lut_consumer_warps(int q, bool grouped, int cols);
 int lut_tiles_per_job(int q, bool grouped, int cols);

@@ -64,8 +64,7 @@ static cudaError_t launch_lut_any(int q, bool grouped, int cols, bool test, cons
 static void fill_common(LutOne &one, const bcq_desc &d, const bcq_plan &plan, const uint16_t *x, void *workspace)
 {
     one.x = reinterpret_cast<const __half *>(x);
-    one.counters = static_cast<int *>(workspace);
-    one.partial = workspace ? reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + lut_counter_bytes(plan)) : nullptr;
+    one.accum = static_cast<unsigned long long *>(workspace);
     one.N = d.N;
     one.K = d.K;
     one.row_blocks = plan.row_blocks;

@@ -41,10 +41,12 @@
 // 32 words][odd chunks: 32 words]; all lanes of a warp are at chunks of one parity at any step, so they
 // still read 32 different words.  Each table buffer fills a 64 KB region of its own.
 //
-// Split K.  The rows of consumer warp c are the same in every K split of a row block.  Each warp stores its
-// partial rows, publishes them (fence + one atomic on the counter of (row block, c)) and is done unless it
-// was the last of the k_splits warps to arrive: that one adds the partial rows in split order
-// (deterministic), rounds and stores y.  No block-wide barrier and no waiting on other blocks.
+// Split K.  Every row of the launch owns one 64-bit word of the workspace.  A K split adds its partial row
+// sum to that word as a biased fixed-point number, together with an arrival count in the word's top bits,
+// with ONE atomic add per row; the add returns the word as it was, so the split that finds k_splits - 1
+// earlier arrivals knows the complete sum (what it got back + what it added), rounds it to fp16, stores y
+// and puts the word back to zero.  Integer addition is associative: the result does not depend on the order
+// of arrival, there is no fence, no second round trip to read partial rows, and no waiting on other blocks.
 //
 // The kernel is launched with programmatic stream serialisation: it lets its dependents start as soon as
 // it runs and waits for its own predecessor only before it touches x, the workspace or y; the packed
@@ -102,8 +104,7 @@ struct LutOne {
     const __half *z;       // per-row scales only: [u][r]
     const __half *x;
     __half *y;
-    float *partial;  // [k_splits][cols][N] when k_splits > 1
-    int *counters;   // [row_blocks][32] when k_splits > 1
+    unsigned long long *accum;  // [cols][N] split-K words (see splitk_encode), all zero between launches; k_splits > 1 only
     int N, K;        // N: rows of all operands together
     int row_blocks, k_splits;
     int test_flags;  // BCQ_PLAN_TEST_* (read by the test instantiations only)
@@ -112,7 +113,7 @@ struct LutOne {
 // row block belongs to exactly one operand (row blocks rb_first[o] .. rb_first[o + 1] - 1 split operand o's
 // row units evenly), so a block works on one operand exactly as it would in a launch of its own.
 struct LutMany {
-    LutOne one;      // x, workspace, sizes and decomposition; its tiles / alpha / z / y are not used
+    LutOne one;      // x, split-K words, sizes and decomposition; its tiles / alpha / z / y are not used
     const uint8_t *tiles[kLutMaxOperands];
     const __half *alpha[kLutMaxOperands];
     const __half *z[kLutMaxOperands];
@@ -328,6 +329,31 @@ __device__ __forceinline__ void build_pair(unsigned char *table, const f32x2 (&x
             *reinterpret_cast<uint32_t *>(dst + gray * 256 + 128) = *reinterpret_cast<const uint32_t *>(&odd);
         });
     }
+}
+
+// ---- split-K words -------------------------------------------------------------------------------
+// bits 63..57: arrivals; bits 56..50: arrivals whose partial sum was NaN; bits 49..0: sum over the arrivals of
+// (partial sum in units of 2^-26, clamped to +-(2^17 - 1)) + 2^43.  Every term of the low field is below 2^44,
+// so 64 arrivals stay below 2^50 and no field carries into the next.  fp32 partial sums of magnitude 2^-2
+// and more are represented exactly; the rest is rounded to a multiple of 2^-26, a quarter of the smallest
+// step of the fp16 result.  Partial sums beyond +-131071 (twice the fp16 range) saturate; an infinite one
+// saturates too and makes the result infinite unless the other splits cancel it.
+constexpr int kSplitFracBits = 26;
+constexpr long long kSplitBias = 1ll << 43;
+__device__ __forceinline__ unsigned long long splitk_encode(float v)
+{
+    if (v != v) return (1ull << 57) + (1ull << 50) + (unsigned long long)kSplitBias;
+    v = fminf(fmaxf(v, -131071.f), 131071.f);
+    const long long f = __float2ll_rn(v * float(1 << kSplitFracBits));   // exact product, |f| < 2^43
+    return (1ull << 57) + (unsigned long long)(f + kSplitBias);
+}
+__device__ __forceinline__ int splitk_arrivals(unsigned long long w) { return int(w >> 57); }
+// the fp16 result from a complete word: one rounding of the exact fixed-point sum
+__device__ __forceinline__ __half splitk_decode(unsigned long long w, int k_splits)
+{
+    if ((w >> 50) & 127) return __ushort_as_half((unsigned short)0x7fffu);   // a NaN partial sum
+    const long long s = (long long)(w & ((1ull << 50) - 1)) - (long long)k_splits * kSplitBias;
+    return __double2half(double(s) * (1.0 / double(1 << kSplitFracBits)));
 }
 
 __host__ __device__ inline const LutOne &lut_one(const LutOne &p) { return p; }
@@ -683,23 +709,26 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     }
     if (!alive) return;   // the block is giving up: y is undefined (bcq_poll_status reports it)
 
-    // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up; lanes 0..7 store y, or this K
-    // split's partial rows (two columns: those of column 1 follow column 0, N elements further on) ------
-    float *partial = p.k_splits > 1 ? p.partial + size_t(ks) * NB * p.N + row0 : nullptr;
+    // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up (all four end up with the sum).
+    // One K split: lanes 0..7 store y.  Several: lane 8 g + j adds the rows j of the warp's accumulator slots
+    // g and g + 4 to their split-K words; whoever completes a word stores that row of y and clears the word.
+    // (Two columns: the second column's words follow the first column's, N further on; its rows of y start
+    // after the operand's own rows.) ----------------------------------------------------------------------
+    const bool split = p.k_splits > 1;
+    unsigned long long *accum = split ? p.accum + row0 : nullptr;
     const size_t Nop = size_t(U) * kUnitRows;   // rows of this operand: its second column of y starts there
 #pragma unroll
     for (int a = 0; a < kUnitsPerWarp; ++a) {
         const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;   // the unit, counted inside the block
+        if (ul >= V) continue;                                  // (the same for the whole warp)
         float v = acc[a][0];
         if constexpr (!GROUPED) {
             // one scale per row: apply the row's alphas and offset to the sums over this block's K range
+            const int u = u0 + ul;
             v = 0.f;
-            if (ul < V) {
-                const int u = u0 + ul;
 #pragma unroll
-                for (int i = 0; i < Q; ++i) v = fmaf(__half2float(alpha[(size_t(u) * Q + i) * kUnitRows + jr]), acc[a][i % NACC], v);
-                v = fmaf(__half2float(zoff[size_t(u) * kUnitRows + jr]), xacc, v);
-            }
+            for (int i = 0; i < Q; ++i) v = fmaf(__half2float(alpha[(size_t(u) * Q + i) * kUnitRows + jr]), acc[a][i % NACC], v);
+            v = fmaf(__half2float(zoff[size_t(u) * kUnitRows + jr]), xacc, v);
         }
         v += __shfl_xor_sync(0xffffffffu, v, 8);
         v += __shfl_xor_sync(0xffffffffu, v, 16);
@@ -709,67 +738,27 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
             v1 += __shfl_xor_sync(0xffffffffu, v1, 8);
             v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
         }
-        if (lane < 8 && ul < V) {
-            const size_t n = size_t(u0 + ul) * kUnitRows + lane;   // row inside the operand
-            if (partial)
-                partial[n] = v;
-            else
+        const size_t n = size_t(u0 + ul) * kUnitRows + jr;   // row inside the operand
+        if (!split) {
+            if (lane < 8) {
                 y[n] = __float2half_rn(v);
+                if constexpr (NB == 2) y[Nop + n] = __float2half_rn(v1);
+            }
+        } else if ((a & 3) == g4) {
+            const unsigned long long mine = splitk_encode(v);
+            const unsigned long long before = atomicAdd(accum + n, mine);
+            if (splitk_arrivals(before) == p.k_splits - 1) {
+                y[n] = splitk_decode(before + mine, p.k_splits);
+                accum[n] = 0;
+            }
             if constexpr (NB == 2) {
-                if (partial)
-                    partial[size_t(p.N) + n] = v1;
-                else
-                    y[Nop + n] = __float2half_rn(v1);
+                const unsigned long long mine1 = splitk_encode(v1);
+                const unsigned long long before1 = atomicAdd(accum + size_t(p.N) + n, mine1);
+                if (splitk_arrivals(before1) == p.k_splits - 1) {
+                    y[Nop + n] = splitk_decode(before1 + mine1, p.k_splits);
+                    accum[size_t(p.N) + n] = 0;
+                }
             }
-        }
-    }
-
-    // ---- split K: the last warp to arrive for (row block, consumer warp) adds the partial rows ------
-    if (p.k_splits > 1 && kJ * cw < V) {
-        __syncwarp();                     // the lanes' partial rows are ordered before lane 0's fence
-        int last = 0;
-        int *counter = p.counters + rbi * 32 + cw;
-        if (lane == 0) {
-            __threadfence();              // cumulative: publishes the whole warp's rows
-            last = (atomicAdd(counter, 1) == p.k_splits - 1);
-            if (last) __threadfence();    // the other splits' rows are visible to what follows
-        }
-        last = __shfl_sync(0xffffffffu, last, 0);
-        if (last) {
-            __syncwarp();
-            // lane -> two rows per column: (accumulator slot lane >> 3, row lane & 7) and slot + 4; fixed
-            // summation order; the loads of 8 splits of all the lane's rows are issued together
-            constexpr int R = 2 * NB;
-            size_t n[R];   // row inside the operand (+ the operand's rows for the second column)
-            size_t at[R];  // the same row among all rows of the launch, per column: index into a split's partials
-            bool on[R];
-            float v[R];
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const int a = (lane >> 3) + 4 * (r & 1);
-                const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;
-                on[r] = ul < V;
-                const size_t row = size_t(u0 + (on[r] ? ul : 0)) * kUnitRows + (lane & 7);
-                n[r] = size_t(r >> 1) * Nop + row;
-                at[r] = size_t(r >> 1) * p.N + row0 + row;
-                v[r] = 0.f;
-            }
-            for (int k0 = 0; k0 < p.k_splits; k0 += 8) {
-                float part[R][8];
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        part[r][k] = (on[r] && k0 + k < p.k_splits) ? __ldcg(p.partial + size_t(k0 + k) * NB * p.N + at[r]) : 0.f;
-#pragma unroll
-                for (int r = 0; r < R; ++r)
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) v[r] += part[r][k];
-            }
-#pragma unroll
-            for (int r = 0; r < R; ++r)
-                if (on[r]) y[n[r]] = __float2half_rn(v[r]);
-            if (lane == 0) *counter = 0;
         }
     }
 }

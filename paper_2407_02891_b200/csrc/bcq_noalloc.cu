@@ -1,8 +1,8 @@
 // bcq_gemv_noalloc: the batch-1 product for callers that cannot obtain device memory.
 //
-// The split-K form of the lookup-table kernel needs scratch memory (per-split partial sums and
-// arrival counters).  Here that scratch is a fixed array that is part of the library image, so
-// the call neither takes a workspace nor allocates one.
+// The split-K form of the lookup-table kernel needs scratch memory (one 64-bit word per row that
+// gathers the K splits' partial sums and counts their arrivals).  Here that scratch is a fixed
+// array that is part of the library image, so the call neither takes a workspace nor allocates one.
 #include <mutex>
 
 #include "bcq_internal.cuh"
@@ -51,9 +51,9 @@ extern "C" int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, co
     void *scratch = nullptr;
     rc = scratch_address(&scratch);
     if (rc != BCQ_OK) return rc;
-    // The array keeps whatever the previous call left.  The kernel needs its arrival counters (the head
-    // of the scratch) to start at zero; the partial sums are fully overwritten before they are read.
-    const cudaError_t e = cudaMemsetAsync(scratch, 0, bcq::lut_counter_bytes(plan), static_cast<cudaStream_t>(stream));
+    // The array keeps whatever the previous call left (a completed product leaves its words zero, one that
+    // was cut short need not): the kernel needs every word it uses to start at zero.
+    const cudaError_t e = cudaMemsetAsync(scratch, 0, need, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return bcq::record_cuda_error(e);
     return bcq_gemv_plan(desc, &plan, packed_dev, alpha_dev, z_dev, x_dev, y_dev, scratch,
                          size_t(BCQ_NOALLOC_SCRATCH_BYTES), stream);

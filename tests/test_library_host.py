@@ -78,7 +78,7 @@ def test_null_and_misaligned_pointers_are_rejected_before_any_launch():
     dt = bq.desc(64, 1024, 3, 128, bq.LAYOUT_TILED)
     split = bq.Plan(1, 1, 2, 0)
     need = bq.workspace_bytes(dt, 1, split)
-    assert need == 256 + 2 * 64 * 4          # 32 counters per row block (rounded up to 256 bytes) + [2][64] fp32
+    assert need == 64 * 8                    # one 64-bit split-K word per row
     args = (ctypes.byref(dt), ctypes.byref(split), ok, ok, ok, ok, ok)
     assert L.bcq_gemv_plan(*args, None, 0, None) == bq.ERR_INVALID_ARG
     assert L.bcq_gemv_plan(*args, ok, need - 1, None) == bq.ERR_WORKSPACE_TOO_SMALL
@@ -134,8 +134,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     blocks = p.row_blocks * p.k_splits
     if U * W >= 148 * 8:
         assert blocks >= 0.7 * 148
-    counters = -(-p.row_blocks * 128 // 256) * 256          # lookup-table kernel: 32 counters per row block
-    assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else counters + p.k_splits * N * 4)
+    assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else N * 8)   # lookup-table kernel: a word per row
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
     for B in (2, 3):                                       # two or three columns: the lookup-table kernel on column pairs
@@ -148,7 +147,7 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
         assert -(-U // pb.row_blocks) <= 176 and -(-W // pb.k_splits) <= 32
         assert bq.workspace_bytes(d, B, pb) == (0 if pb.k_splits == 1 else 4096 * 4 + pb.k_splits * B * N * 4)
         # a lookup-table plan runs the columns two at a time: partial sums of two columns
-        assert bq.workspace_bytes(d, B, p) == (0 if p.k_splits == 1 else counters + p.k_splits * 2 * N * 4)
+        assert bq.workspace_bytes(d, B, p) == (0 if p.k_splits == 1 else 2 * N * 8)   # a word per row and column
     assert bq.workspace_bytes(d, 1, bq.plan_default(d, 4, 148)) == 0        # the small-batch kernel needs B >= 2
     assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
 
