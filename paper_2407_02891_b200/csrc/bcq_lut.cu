@@ -69,6 +69,9 @@ static void fill_common(LutOne &one, const bcq_desc &d, const bcq_plan &plan, co
     one.K = d.K;
     one.row_blocks = plan.row_blocks;
     one.k_splits = plan.k_splits;
+    const int U = d.N / kUnitRows, W = d.K / kWindow;
+    one.u_base = U / plan.row_blocks, one.u_rem = U % plan.row_blocks;   // (several operands: per operand, see launch_lut_multi)
+    one.w_base = W / plan.k_splits, one.w_rem = W % plan.k_splits;
     one.test_flags = plan.reserved;
 }
 
@@ -105,6 +108,8 @@ cudaError_t launch_lut_multi(const bcq_desc &d, const bcq_plan &plan, const LutO
         many.z[o] = reinterpret_cast<const __half *>(ops[o].z);
         many.y[o] = reinterpret_cast<__half *>(ops[o].y);
         many.U[o] = ops[o].N / kUnitRows;
+        many.u_base[o] = many.U[o] / ops[o].row_blocks;
+        many.u_rem[o] = many.U[o] % ops[o].row_blocks;
         many.row0[o] = rows;
         many.rb_first[o] = rb;
         rows += ops[o].N;

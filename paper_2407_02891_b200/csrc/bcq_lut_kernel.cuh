@@ -106,7 +106,11 @@ struct LutOne {
     __half *y;
     unsigned long long *accum;  // [cols][N] split-K words (see splitk_encode), all zero between launches; k_splits > 1 only
     int N, K;        // N: rows of all operands together
-    int row_blocks, k_splits;
+    int row_blocks, k_splits;   // the grid: blockIdx.x = row block, blockIdx.y = K split
+    // Even partitions, prepared by the host so that no block spends its first microsecond dividing: part r of a
+    // range cut into n parts starts at r * base + min(r, rem) and has base + (r < rem) items.
+    int u_base, u_rem;   // row units over row blocks (one operand)
+    int w_base, w_rem;   // windows over K splits
     int test_flags;  // BCQ_PLAN_TEST_* (read by the test instantiations only)
 };
 // Up to kLutMaxOperands matrices that share x, K, q and the scaling unit are multiplied in one launch: every
@@ -119,6 +123,7 @@ struct LutMany {
     const __half *z[kLutMaxOperands];
     __half *y[kLutMaxOperands];
     int U[kLutMaxOperands];       // row units of each operand
+    int u_base[kLutMaxOperands], u_rem[kLutMaxOperands];   // its row units over its row blocks
     int row0[kLutMaxOperands];    // first row of each operand among all rows of the launch
     int rb_first[kLutMaxOperands + 1];
     int count;
@@ -396,22 +401,21 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     constexpr int NACC = GROUPED ? 1 : Q;   // accumulators per unit and lane: the row's sum, or one per plane
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    const int rbi = blockIdx.x % p.row_blocks, ks = blockIdx.x / p.row_blocks;
-    int op = 0, rbl = rbi, rbn = p.row_blocks, U = p.N / kUnitRows, row0 = 0;
+    const int rbi = blockIdx.x, ks = blockIdx.y;
+    int op = 0, rbl = rbi, U = p.N / kUnitRows, row0 = 0, u_base = p.u_base, u_rem = p.u_rem;
     const uint8_t *tiles = p.tiles;
     const __half *alpha = p.alpha, *zoff = p.z;
     __half *y = p.y;
     if constexpr (MULTI) {   // the operand this row block belongs to
         while (op + 1 < pm.count && rbi >= pm.rb_first[op + 1]) ++op;
-        rbl = rbi - pm.rb_first[op], rbn = pm.rb_first[op + 1] - pm.rb_first[op];
-        U = pm.U[op], row0 = pm.row0[op];
+        rbl = rbi - pm.rb_first[op];
+        U = pm.U[op], row0 = pm.row0[op], u_base = pm.u_base[op], u_rem = pm.u_rem[op];
         tiles = pm.tiles[op], alpha = pm.alpha[op], zoff = pm.z[op], y = pm.y[op];
     }
-    const int W = p.K / kWindow;
-    const int u0 = int((long long)rbl * U / rbn), u1 = int((long long)(rbl + 1) * U / rbn);
-    const int w0 = int((long long)ks * W / p.k_splits), w1 = int((long long)(ks + 1) * W / p.k_splits);
-    const int V = u1 - u0;                       // row units of this block
-    const int nwin = w1 - w0;                    // windows of this block
+    const int u0 = rbl * u_base + min(rbl, u_rem);
+    const int w0 = ks * p.w_base + min(ks, p.w_rem);
+    const int V = u_base + (rbl < u_rem ? 1 : 0);        // row units of this block
+    const int nwin = p.w_base + (ks < p.w_rem ? 1 : 0);  // windows of this block
     const int njobs = (V + kJ - 1) / kJ;         // jobs per window
     constexpr int spin_limit = TEST ? kTestSpinLimit : kSpinLimit;
 
@@ -778,7 +782,7 @@ static cudaError_t launch_lut_inst(const typename LutParamsOf<MULTI>::type &prm,
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(lut_one(prm).row_blocks * lut_one(prm).k_splits);
+    cfg.gridDim = dim3(lut_one(prm).row_blocks, lut_one(prm).k_splits);
     cfg.blockDim = dim3(kLutThreads);
     cfg.dynamicSmemBytes = kLutSmemBytes;
     cfg.stream = st;
