@@ -715,15 +715,19 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
 
     // ---- a unit's row j is spread over the 4 lanes 8 g + j: add them up (all four end up with the sum).
     // One K split: lanes 0..7 store y.  Several: lane 8 g + j adds the rows j of the warp's accumulator slots
-    // g and g + 4 to their split-K words; whoever completes a word stores that row of y and clears the word.
+    // g and g + 4 to their split-K words (32 rows per atomic instruction); whoever completes a word stores
+    // that row of y and clears the word.
     // (Two columns: the second column's words follow the first column's, N further on; its rows of y start
     // after the operand's own rows.) ----------------------------------------------------------------------
     const bool split = p.k_splits > 1;
     unsigned long long *accum = split ? p.accum + row0 : nullptr;
     const size_t Nop = size_t(U) * kUnitRows;   // rows of this operand: its second column of y starts there
+    float tot[kUnitsPerWarp], tot1[NB == 2 ? kUnitsPerWarp : 1];
 #pragma unroll
     for (int a = 0; a < kUnitsPerWarp; ++a) {
         const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;   // the unit, counted inside the block
+        tot[a] = 0.f;
+        if constexpr (NB == 2) tot1[a] = 0.f;
         if (ul >= V) continue;                                  // (the same for the whole warp)
         float v = acc[a][0];
         if constexpr (!GROUPED) {
@@ -736,31 +740,42 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
         }
         v += __shfl_xor_sync(0xffffffffu, v, 8);
         v += __shfl_xor_sync(0xffffffffu, v, 16);
-        float v1 = 0.f;
+        tot[a] = v;
         if constexpr (NB == 2) {
-            v1 = acc1[a];
+            float v1 = acc1[a];
             v1 += __shfl_xor_sync(0xffffffffu, v1, 8);
             v1 += __shfl_xor_sync(0xffffffffu, v1, 16);
+            tot1[a] = v1;
         }
-        const size_t n = size_t(u0 + ul) * kUnitRows + jr;   // row inside the operand
-        if (!split) {
-            if (lane < 8) {
-                y[n] = __float2half_rn(v);
-                if constexpr (NB == 2) y[Nop + n] = __float2half_rn(v1);
-            }
-        } else if ((a & 3) == g4) {
-            const unsigned long long mine = splitk_encode(v);
-            const unsigned long long before = atomicAdd(accum + n, mine);
-            if (splitk_arrivals(before) == p.k_splits - 1) {
-                y[n] = splitk_decode(before + mine, p.k_splits);
-                accum[n] = 0;
-            }
-            if constexpr (NB == 2) {
-                const unsigned long long mine1 = splitk_encode(v1);
-                const unsigned long long before1 = atomicAdd(accum + size_t(p.N) + n, mine1);
-                if (splitk_arrivals(before1) == p.k_splits - 1) {
-                    y[Nop + n] = splitk_decode(before1 + mine1, p.k_splits);
-                    accum[size_t(p.N) + n] = 0;
+        if (!split && lane < 8) {
+            const size_t n = size_t(u0 + ul) * kUnitRows + jr;   // row inside the operand
+            y[n] = __float2half_rn(v);
+            if constexpr (NB == 2) y[Nop + n] = __float2half_rn(tot1[a]);
+        }
+    }
+    if (split) {
+        // two passes over the warp's accumulator slots, 32 rows each: lane 8 g + j takes row j of slot 4 h + g
+#pragma unroll
+        for (int h = 0; h < kUnitsPerWarp / 4; ++h) {
+            const int a = 4 * h + g4;
+            const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;
+            if (ul < V) {
+                const size_t n = size_t(u0 + ul) * kUnitRows + jr;
+                const float v = g4 == 0 ? tot[4 * h] : (g4 == 1 ? tot[4 * h + 1] : (g4 == 2 ? tot[4 * h + 2] : tot[4 * h + 3]));
+                const unsigned long long mine = splitk_encode(v);
+                const unsigned long long before = atomicAdd(accum + n, mine);
+                if (splitk_arrivals(before) == p.k_splits - 1) {
+                    y[n] = splitk_decode(before + mine, p.k_splits);
+                    accum[n] = 0;
+                }
+                if constexpr (NB == 2) {
+                    const float v1 = g4 == 0 ? tot1[4 * h] : (g4 == 1 ? tot1[4 * h + 1] : (g4 == 2 ? tot1[4 * h + 2] : tot1[4 * h + 3]));
+                    const unsigned long long mine1 = splitk_encode(v1);
+                    const unsigned long long before1 = atomicAdd(accum + size_t(p.N) + n, mine1);
+                    if (splitk_arrivals(before1) == p.k_splits - 1) {
+                        y[Nop + n] = splitk_decode(before1 + mine1, p.k_splits);
+                        accum[size_t(p.N) + n] = 0;
+                    }
                 }
             }
         }
