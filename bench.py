@@ -324,18 +324,24 @@ class Stack:
         return e0.elapsed_time(e1)
 
     def per_shape_us(self, reps=3):
-        """Mean device time per launch of each distinct shape, every launch on different weights."""
+        """Mean device time per launch of each distinct shape: all launches of the shape, every one on its own
+        weights, captured in a CUDA graph (plain launches from Python would time the host, not the device)."""
         torch = self.torch
         out = {}
         shapes = sorted({it[7] for it in self.items})
         for s in shapes:
             its = [it for it in self.items if it[7] == s]
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for it in its:
+                    self.launch_one(it)
+            g.replay()
+            torch.cuda.synchronize(self.device)
             best = None
             for _ in range(reps):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                for it in its:
-                    self.launch_one(it)
+                g.replay()
                 e1.record()
                 e1.synchronize()
                 t = e0.elapsed_time(e1) * 1e3 / len(its)

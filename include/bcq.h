@@ -75,7 +75,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 200
+#define BCQ_VERSION 210
 
 typedef enum bcq_status {
     BCQ_OK = 0,
