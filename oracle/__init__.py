@@ -198,3 +198,63 @@ def forward_planes(planes, alpha, z, x, group: int) -> np.ndarray:
                                     ctypes.c_int(q), ctypes.c_int(group), ctypes.c_int(B), _p(y))
     _check(rc, "forward_planes")
     return y
+
+
+# ---- the search over BCchoice and the re-explored scale (sections "Quantize Weight Twice" and
+# ---- "Re-explore Scale Factor") -------------------------------------------------------------------
+
+def set_partitions(n_bits: int, q: int):
+    """Every way of dealing the n step-1 bits into q non-empty planes (the BCchoice candidates of Eq. round
+    built as Eq. fuse_step2 builds them), each once, as bit_to_plane arrays: planes are numbered in the
+    order of their lowest bit, and the arrays come in lexicographic order."""
+    out = []
+
+    def grow(prefix, used):
+        if len(prefix) == n_bits:
+            if used == q:
+                out.append(np.array(prefix, np.uint8))
+            return
+        for p in range(min(used + 1, q)):
+            grow(prefix + [p], max(used, p + 1))
+
+    grow([], 0)
+    return out
+
+
+def reexplore_factors(n_bits: int, count: int) -> np.ndarray:
+    """`count` evenly spaced scale factors strictly inside the interval of Eq. reexplore, as multiples s of the
+    step-1 scale (Wmax - Wmin)/(2^n - 1):  s in ((2^n - 1)/(2^(n+1) - 1), (2^n - 1)/(2^(n-1) - 1))."""
+    lo = (2.0 ** n_bits - 1.0) / (2.0 ** (n_bits + 1) - 1.0)
+    hi = (2.0 ** n_bits - 1.0) / (2.0 ** (n_bits - 1) - 1.0)
+    return lo + (hi - lo) * (np.arange(count, dtype=np.float64) + 1.0) / (count + 1.0)
+
+
+def grid_search(W, X, group: int, n_bits: int, partitions, s_factors):
+    """Eq. gptqt step 2 searched as the section "Re-explore Scale Factor" says: for every scale factor (outer
+    loop) and every BCchoice (inner loop) quantise W by step 1 with that scale, round to the BCchoice, and
+    measure the output error on the calibration inputs,  sum_t || (S W_q + qbias - W) x_t ||^2  (fp64).
+    W fp16 [N, K]; X fp16 [T, K].  Returns (err_rows [S, P, N], err [S, P], (si, pi)) where (si, pi) is the
+    first candidate, in loop order, whose error is below all earlier ones."""
+    W = _c(W, np.float16)
+    X = _c(X, np.float16)
+    N, K = W.shape
+    G = 1 if group == 0 else K // group
+    glen = K // G
+    Wd, Xd = W.astype(np.float64), X.astype(np.float64)
+    err_rows = np.zeros((len(s_factors), len(partitions), N), np.float64)
+    for si, s in enumerate(s_factors):
+        w_int, S, qbias = quantize_rtn(W, group, n_bits, float(s))
+        Sd = np.repeat(S.astype(np.float64), glen, axis=1)
+        qd = np.repeat(qbias.astype(np.float64), glen, axis=1)
+        for pi, b2p in enumerate(partitions):
+            wq, _ = round_to_bcchoice(w_int, n_bits, b2p)
+            dW = Sd * wq.astype(np.float64) + qd - Wd           # dequantised minus original weights
+            E = dW @ Xd.T                                        # [N, T]: the error of every output
+            err_rows[si, pi] = (E * E).sum(axis=1)
+    err = err_rows.sum(axis=2)
+    best, best_err = (0, 0), np.inf
+    for si in range(len(s_factors)):
+        for pi in range(len(partitions)):
+            if err[si, pi] < best_err:
+                best, best_err = (si, pi), err[si, pi]
+    return err_rows, err, best
