@@ -326,6 +326,40 @@ int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, const uint16_
                      const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev, void *stream);
 
 /*
+ * The search of GPTQT's second step on calibration inputs (section "Quantize Weight Twice", Eq. gptqt step 2:
+ * the BCchoice of Eq. round is the one with the smallest output error; section "Re-explore Scale Factor",
+ * Eq. reexplore: so is the scale of step 1).  For every scale factor s (outer loop) and every candidate split
+ * p of the n_bits step-1 bits into desc->q planes (inner loop):
+ *     step 1 as in bcq_quantize_rtn with s_factor = s  ->  W_int, S, qbias per (row, scaling unit)
+ *     W_q = the integer of BCchoice p nearest to W_int (Eq. round; ties: the smaller)
+ *     err_rows[s][p][n] = sum_t ( sum_k (S W_q[n][k] + qbias - W[n][k]) X[t][k] )^2
+ *     err[s][p]         = sum_n err_rows[s][p][n]
+ * and best = (s, p) of the first candidate, in loop order, whose err is below all earlier ones.
+ * The contraction runs on the tensor cores with fp16 operands (the weight differences are rounded once to
+ * fp16) and fp32 accumulation; the error values agree with an fp64 evaluation to about 1e-3 relative, so
+ * candidates closer than that may swap places.  GPTQ's error compensation is not part of this call.
+ *   W [N][K] fp16 weights, X [T][K] fp16 calibration inputs (device, 16-byte aligned); T a multiple of 16,
+ *   16..256; K a multiple of 64; desc->group 0 or a multiple of 64; n_bits 1..6; desc->layout is ignored.
+ *   partitions_host [P][n_bits]: bit_to_plane arrays as in bcq_merge_linear (bcq_partition_get lists them all);
+ *   s_factors_host [n_scales] (bcq_reexplore_factors gives an even grid inside the interval of Eq. reexplore).
+ *   err_dev [n_scales][P] fp64; err_rows_dev [n_scales][P][N] fp32 or NULL; best_dev [2] int32.
+ *   workspace: bcq_grid_search_workspace(desc, T, n_bits, P, n_scales, err_rows_dev != NULL) bytes, 256-byte
+ *   aligned; holds W_int, S, qbias and a scratch operand of the current scale.  Asynchronous on `stream`.
+ */
+size_t bcq_grid_search_workspace(const bcq_desc *desc, int T, int n_bits, int P, int n_scales, int rows_given);
+int bcq_grid_search(const bcq_desc *desc, const uint16_t *W_dev, const uint16_t *X_dev, int T, int n_bits,
+                    const uint8_t *partitions_host, int P, const double *s_factors_host, int n_scales,
+                    double *err_dev, float *err_rows_dev, int32_t *best_dev, void *workspace_dev,
+                    size_t workspace_bytes, void *stream);
+/* Every split of n_bits step-1 bits into q non-empty planes (the candidates Eq. fuse_step2 can build), each
+ * once: planes numbered by their lowest bit, arrays in lexicographic order.  Host functions. */
+int bcq_partition_count(int n_bits, int q);                                      /* 0 when the arguments are invalid */
+int bcq_partition_get(int n_bits, int q, int index, uint8_t *bit_to_plane_out);  /* [n_bits] */
+/* `count` evenly spaced scale factors strictly inside the interval of Eq. reexplore, as multiples of the
+ * step-1 scale (Wmax - Wmin)/(2^n - 1): between (2^n - 1)/(2^(n+1) - 1) and (2^n - 1)/(2^(n-1) - 1). */
+int bcq_reexplore_factors(int n_bits, int count, double *s_factors_out);
+
+/*
  * Every wait inside the kernels (on an mbarrier fed by an asynchronous copy or by other warps)
  * is bounded.  If one ever runs out, the block stops waiting, lets its outstanding copies land,
  * returns without a fault, and records the event in a device status word; y is then undefined.

@@ -94,6 +94,11 @@ SIGNATURES = {
     "bcq_gemv_host": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_noalloc": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bcq_poll_status": (_i, []),
+    "bcq_grid_search_workspace": (_sz, [_dp, _i, _i, _i, _i, _i]),
+    "bcq_grid_search": (_i, [_dp, _vp, _vp, _i, _i, _vp, _i, _vp, _i, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_partition_count": (_i, [_i, _i]),
+    "bcq_partition_get": (_i, [_i, _i, _i, _vp]),
+    "bcq_reexplore_factors": (_i, [_i, _i, _vp]),
 }
 
 
@@ -337,3 +342,42 @@ def pack_layer(N, K, q, group, layout, codes, alpha, z) -> Layer:
     packed, a, zz = empty_operands(d, codes.device)
     pack(d, codes, alpha, z, packed, a, zz)
     return Layer(d, packed, a, zz)
+
+
+def partitions(n_bits: int, q: int):
+    """All bit_to_plane arrays of bcq_partition_get, as a uint8 numpy array [P, n_bits]."""
+    import numpy as np
+    P = lib().bcq_partition_count(n_bits, q)
+    out = np.zeros((P, n_bits), np.uint8)
+    for i in range(P):
+        _check(lib().bcq_partition_get(n_bits, q, i, out[i].ctypes.data_as(ctypes.c_void_p)), "bcq_partition_get")
+    return out
+
+
+def reexplore_factors(n_bits: int, count: int):
+    import numpy as np
+    out = np.zeros(count, np.float64)
+    _check(lib().bcq_reexplore_factors(n_bits, count, out.ctypes.data_as(ctypes.c_void_p)), "bcq_reexplore_factors")
+    return out
+
+
+def grid_search(N, K, q, group, W, X, n_bits, parts, s_factors, want_rows=True):
+    """bcq_grid_search on torch CUDA tensors W [N, K], X [T, K] (fp16); parts: uint8 numpy [P, n_bits]; s_factors:
+    float64 numpy.  Returns (err [S, P] float64 tensor, err_rows [S, P, N] float32 tensor or None, best [2] int32 tensor)."""
+    import numpy as np
+    _dev(W, X)
+    d = desc(N, K, q, group, LAYOUT_CANONICAL)
+    parts = np.ascontiguousarray(parts, np.uint8)
+    s_factors = np.ascontiguousarray(s_factors, np.float64)
+    P, S, T = parts.shape[0], s_factors.shape[0], X.shape[0]
+    nbytes = lib().bcq_grid_search_workspace(ctypes.byref(d), T, n_bits, P, S, 1 if want_rows else 0)
+    if nbytes == 0:
+        raise BcqError(ERR_INVALID_ARG, "bcq_grid_search_workspace")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    err = torch.empty((S, P), dtype=torch.float64, device=W.device)
+    rows = torch.empty((S, P, N), dtype=torch.float32, device=W.device) if want_rows else None
+    best = torch.zeros(2, dtype=torch.int32, device=W.device)
+    _check(lib().bcq_grid_search(ctypes.byref(d), _ptr(W), _ptr(X), T, n_bits, parts.ctypes.data_as(ctypes.c_void_p), P,
+                                 s_factors.ctypes.data_as(ctypes.c_void_p), S, _ptr(err), _ptr(rows), _ptr(best), _ptr(ws),
+                                 nbytes, _stream()), "bcq_grid_search")
+    return err, rows, best

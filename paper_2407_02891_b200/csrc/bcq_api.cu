@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <vector>
 
 #include "bcq_internal.cuh"
 
@@ -353,6 +354,89 @@ int merge_table(int q, int n_bits, const uint8_t *bit_to_plane, double (&weight)
     return BCQ_OK;
 }
 
+// lut[v] = the integer the planes of bit_to_plane reach that is nearest to the step-1 integer v (ties: the smaller)
+int nearest_reachable(int q, int n_bits, const uint8_t *bit_to_plane, float *lut /*[64]*/)
+{
+    double weight[4];
+    uint8_t code_of_int[256];
+    const int rc = merge_table(q, n_bits, bit_to_plane, weight, code_of_int);
+    if (rc != BCQ_OK) return rc;
+    for (int v = 0; v < 64; ++v) {
+        int reach = 0;
+        if (v < (1 << n_bits))
+            for (int i = 0; i < n_bits; ++i) reach |= ((code_of_int[v] >> bit_to_plane[i]) & 1) << i;
+        lut[v] = float(reach);
+    }
+    return BCQ_OK;
+}
+
+// bit_to_plane arrays of all splits of n bits into q non-empty planes: planes numbered by their lowest bit,
+// arrays in lexicographic order.  Returns the count; writes the index-th array when out is given.
+int enumerate_partitions(int n, int q, int index, uint8_t *out)
+{
+    uint8_t cur[8];
+    int count = 0;
+    // iterative depth-first walk over restricted-growth strings
+    int pos = 0, used[9];
+    used[0] = 0;
+    cur[0] = 0;
+    int next[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    while (pos >= 0) {
+        const int limit = used[pos] + 1 < q ? used[pos] + 1 : q;   // values 0 .. limit-1 are allowed here
+        if (next[pos] >= limit) {
+            --pos;
+            continue;
+        }
+        cur[pos] = uint8_t(next[pos]++);
+        const int u = cur[pos] + 1 > used[pos] ? cur[pos] + 1 : used[pos];
+        if (pos == n - 1) {
+            if (u == q) {
+                if (out && count == index)
+                    for (int i = 0; i < n; ++i) out[i] = cur[i];
+                ++count;
+            }
+        } else {
+            ++pos;
+            used[pos] = u;
+            next[pos] = 0;
+        }
+    }
+    return count;
+}
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct SearchLayout {
+    size_t lut, w_int, S, qbias, packed, alpha, z, err, err_rows, total;
+};
+SearchLayout search_layout(const bcq_desc &d, int P, int n_scales, bool own_rows)
+{
+    SearchLayout L;
+    const size_t G = size_t(n_groups(d));
+    size_t at = 0;
+    L.lut = at, at += round_up(size_t(P) * 64 * sizeof(float), 256);
+    L.w_int = at, at += round_up(size_t(d.N) * d.K, 256);
+    L.S = at, at += round_up(size_t(d.N) * G * 2, 256);
+    L.qbias = at, at += round_up(size_t(d.N) * G * 2, 256);
+    L.packed = at, at += round_up(size_t(d.q) * d.N * (d.K / 8), 256);
+    L.alpha = at, at += round_up(size_t(d.q) * d.N * G * 2, 256);
+    L.z = at, at += round_up(size_t(d.N) * G * 2, 256);
+    L.err = at, at += round_up(size_t(n_scales) * P * sizeof(double), 256);
+    L.err_rows = at, at += own_rows ? round_up(size_t(P) * d.N * sizeof(float), 256) : 0;
+    L.total = at;
+    return L;
+}
+
+int check_search(const bcq_desc *desc, int T, int n_bits, int P, int n_scales)
+{
+    const int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (n_bits < 1 || n_bits > 6 || desc->q > n_bits || P < 1 || P > 4096 || n_scales < 1 || n_scales > 4096) return BCQ_ERR_INVALID_ARG;
+    if (T < 16 || T > 256 || T % 16 != 0) return BCQ_ERR_INVALID_ARG;
+    if (desc->K % 64 != 0 || (desc->group != 0 && desc->group % 64 != 0)) return BCQ_ERR_UNSUPPORTED_SHAPE;
+    return BCQ_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -380,13 +464,15 @@ int bcq_poll_status(void)
 {
     int v = 0;
     int w = 0;
+    int u = 0;
     cudaError_t e = cudaDeviceSynchronize();   // kernels on non-blocking streams included
     if (e == cudaSuccess) e = lut_status_take(&v);
     if (e == cudaSuccess) e = mma_status_take(&w);
+    if (e == cudaSuccess) e = search_status_take(&u);
     if (e != cudaSuccess) return cuda_fail(e);
-    if (v != 0 || w != 0) {
-        snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: bounded wait %d ran out", v ? "lut_gemv_kernel" : "mma_gemm_kernel",
-                 v ? v : w);
+    if (v != 0 || w != 0 || u != 0) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: bounded wait %d ran out",
+                 v ? "lut_gemv_kernel" : (w ? "mma_gemm_kernel" : "search_error_kernel"), v ? v : (w ? w : u));
         return BCQ_ERR_TIMEOUT;
     }
     return BCQ_OK;
@@ -685,6 +771,89 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed, const uint16_t *alph
     rc = bcq_gemv(desc, packed, alpha, z, x_stage, y_direct ? y_direct : y_stage, ws, ws_bytes, stream);
     if (rc != BCQ_OK || y_direct) return rc;
     e = cudaMemcpyAsync(y_host, y_stage, size_t(desc->N) * 2, cudaMemcpyDeviceToHost, st);
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
+int bcq_partition_count(int n_bits, int q)
+{
+    if (n_bits < 1 || n_bits > 8 || q < 1 || q > 4 || q > n_bits) return 0;
+    return enumerate_partitions(n_bits, q, -1, nullptr);
+}
+
+int bcq_partition_get(int n_bits, int q, int index, uint8_t *bit_to_plane_out)
+{
+    if (!bit_to_plane_out || n_bits < 1 || n_bits > 8 || q < 1 || q > 4 || q > n_bits) return BCQ_ERR_INVALID_ARG;
+    if (index < 0 || index >= enumerate_partitions(n_bits, q, -1, nullptr)) return BCQ_ERR_INVALID_ARG;
+    enumerate_partitions(n_bits, q, index, bit_to_plane_out);
+    return BCQ_OK;
+}
+
+int bcq_reexplore_factors(int n_bits, int count, double *s_factors_out)
+{
+    if (!s_factors_out || n_bits < 2 || n_bits > 8 || count < 1) return BCQ_ERR_INVALID_ARG;
+    const double full = double((1u << n_bits) - 1u);
+    const double lo = full / double((1u << (n_bits + 1)) - 1u), hi = full / double((1u << (n_bits - 1)) - 1u);
+    for (int i = 0; i < count; ++i) s_factors_out[i] = lo + (hi - lo) * double(i + 1) / double(count + 1);
+    return BCQ_OK;
+}
+
+size_t bcq_grid_search_workspace(const bcq_desc *desc, int T, int n_bits, int P, int n_scales, int rows_given)
+{
+    bcq_desc d;
+    if (!desc) return 0;
+    d = *desc;
+    d.layout = BCQ_LAYOUT_CANONICAL;
+    if (check_search(&d, T, n_bits, P, n_scales) != BCQ_OK) return 0;
+    return search_layout(d, P, n_scales, rows_given == 0).total;
+}
+
+int bcq_grid_search(const bcq_desc *desc, const uint16_t *W, const uint16_t *X, int T, int n_bits, const uint8_t *partitions,
+                    int P, const double *s_factors, int n_scales, double *err, float *err_rows, int32_t *best, void *ws,
+                    size_t ws_bytes, void *stream)
+{
+    if (!desc) return BCQ_ERR_INVALID_ARG;
+    bcq_desc d = *desc;
+    d.layout = BCQ_LAYOUT_CANONICAL;
+    int rc = check_search(&d, T, n_bits, P, n_scales);
+    if (rc != BCQ_OK) return rc;
+    if (!W || !X || !partitions || !s_factors || !err || !best || !ws) return BCQ_ERR_INVALID_ARG;
+    if (!aligned(W, 16) || !aligned(X, 16) || !aligned(err, 8) || !aligned(err_rows, 4) || !aligned(best, 4) || !aligned(ws, 256))
+        return BCQ_ERR_MISALIGNED;
+    const SearchLayout L = search_layout(d, P, n_scales, err_rows == nullptr);
+    if (ws_bytes < L.total) return BCQ_ERR_WORKSPACE_TOO_SMALL;
+    for (int s = 0; s < n_scales; ++s)
+        if (!(s_factors[s] > 0.0) || !(s_factors[s] < 1e30)) return BCQ_ERR_INVALID_ARG;
+
+    std::vector<float> lut(size_t(P) * 64);
+    for (int c = 0; c < P; ++c) {
+        rc = nearest_reachable(d.q, n_bits, partitions + size_t(c) * n_bits, lut.data() + size_t(c) * 64);
+        if (rc != BCQ_OK) return rc;
+    }
+    double weight[4];
+    uint8_t code_of_int[256];
+    rc = merge_table(d.q, n_bits, partitions, weight, code_of_int);   // step 1 does not depend on the BCchoice: any will do
+    if (rc != BCQ_OK) return rc;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char *base = static_cast<unsigned char *>(ws);
+    float *lut_dev = reinterpret_cast<float *>(base + L.lut);
+    uint8_t *w_int = base + L.w_int;
+    uint16_t *S = reinterpret_cast<uint16_t *>(base + L.S), *qbias = reinterpret_cast<uint16_t *>(base + L.qbias);
+    double *err_all = reinterpret_cast<double *>(base + L.err);
+    // (pageable host memory: the copy has left the vector when the call returns)
+    cudaError_t e = cudaMemcpyAsync(lut_dev, lut.data(), lut.size() * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const View scratch = make_view(d, base + L.packed, reinterpret_cast<uint16_t *>(base + L.alpha), reinterpret_cast<uint16_t *>(base + L.z));
+    for (int s = 0; s < n_scales; ++s) {
+        e = launch_quantize_rtn(W, n_bits, s_factors[s], code_of_int, weight, S, qbias, w_int, scratch, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        float *rows = err_rows ? err_rows + size_t(s) * P * d.N : reinterpret_cast<float *>(base + L.err_rows);
+        e = launch_search_errors(W, w_int, S, qbias, X, d.N, d.K, d.group, T, n_bits, lut_dev, P, rows, err_all + size_t(s) * P, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    e = launch_search_argmin(err_all, n_scales * P, P, best, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaMemcpyAsync(err, err_all, size_t(n_scales) * P * sizeof(double), cudaMemcpyDeviceToDevice, st);
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
 

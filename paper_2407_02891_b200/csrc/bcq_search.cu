@@ -1,0 +1,367 @@
+// Output error of the candidates of the GPTQT search (Eq. gptqt step 2; Eq. reexplore) on tcgen05.
+//
+// For one re-explored scale (W_int, S, qbias of step 1 are given) and a set of BCchoice candidates p:
+//
+//     err[p][n] = sum_t ( sum_k ( S lut_p[W_int[n][k]] + qbias - W[n][k] ) X[t][k] )^2
+//
+// lut_p[v] = the integer of BCchoice p nearest to v (Eq. round).  The inner sum is a dense contraction
+// dW_p (N x K) times X^T (K x T): here the tensor cores are the right unit.  A block owns 128 rows of W
+// and up to four candidates; per 64-wide slice of K its threads form the four dW_p tiles (fp16, one fused
+// multiply-add and one rounding per element) straight into shared memory in the 128-byte-swizzled K-major
+// operand layout, X's slice is copied in beside them in the same layout, and one thread issues
+// tcgen05.mma (M = 128, N = T, K = 16, fp16 x fp16 -> fp32) into one accumulator per candidate in tensor
+// memory.  Two operand stages: the tensor cores work on one slice while the threads form the next; a
+// stage is handed back by tcgen05.commit on its mbarrier.  At the end every row's T outputs are read
+// back with tcgen05.ld, squared and summed.
+//
+// All waits are bounded; a wait that runs out sets a device status word (see search_status_take), the
+// block still frees its tensor memory and returns.
+#include "bcq_async.cuh"
+#include "bcq_internal.cuh"
+
+namespace bcq {
+
+constexpr int kSearchThreads = 256;
+constexpr int kSearchRows = 128;        // rows of W per block = M of the MMA
+constexpr int kSearchKTile = 64;        // weights along K per stage: 128 bytes of fp16, one swizzle row
+constexpr int kSearchMaxCand = 4;       // candidates (accumulators) per block
+constexpr int kSearchATile = kSearchRows * kSearchKTile * 2;   // 16 KB
+constexpr int kSearchMaxT = 256;
+constexpr int kSearchSpin = 1 << 22;
+
+static __device__ int g_search_status = 0;
+
+struct SearchParams {
+    const __half *W;        // [N][K]
+    const uint8_t *w_int;   // [N][K]
+    const __half *S;        // [N][G]
+    const __half *qbias;    // [N][G]
+    const __half *X;        // [T][K]
+    float *err_rows;        // [P][N] of this scale factor
+    int N, K, G, L;         // L = weights per scaling unit (K when one per row)
+    int T, P;
+    int cand_per_block;     // 1..4, so that cand_per_block * T <= 512 columns of tensor memory
+    int tmem_cols;          // power of two >= 32 covering cand_per_block * T
+    int lut_size;           // 2^n_bits <= 64
+    const float *lut;       // [P][64]: lut[p][v] = the integer of BCchoice p nearest to v
+};
+
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    // K-major operand, 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart
+    uint64_t d = 0;
+    d |= uint64_t((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= uint64_t(1) << 16;                        // leading byte offset (unused with a swizzled K-major tile)
+    d |= uint64_t(1024 >> 4) << 32;                // stride byte offset: 8 rows further on
+    d |= uint64_t(1) << 46;                        // descriptor version of this architecture
+    d |= uint64_t(2) << 61;                        // 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool search_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code)
+{
+    for (int it = 0; it < kSearchSpin; ++it) {
+        if (mbar_test_wait(bar, parity)) return true;
+        __nanosleep(64);
+        if ((it & 255) == 255 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicExch(&g_search_status, code);
+    return false;
+}
+
+// grid (row tiles of 128, groups of cand_per_block candidates); dynamic shared memory:
+// 2 stages x (cand_per_block x 16 KB of dW tiles + 32 KB for X), 1024-byte aligned.
+__global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const SearchParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ __align__(8) unsigned long long bars[3];   // stage 0 free, stage 1 free, all done
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    __shared__ float lut_s[kSearchMaxCand * 64];
+    __shared__ float part[2][kSearchMaxCand][kSearchRows];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cand0 = blockIdx.y * p.cand_per_block;
+    const int ncand = min(p.cand_per_block, p.P - cand0);
+    const int T = p.T;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t stage_bytes = uint32_t(p.cand_per_block) * kSearchATile + uint32_t(kSearchMaxT) * 128u;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    volatile int *abort_flag = &abort_s;
+
+    for (int i = tid; i < ncand * p.lut_size; i += kSearchThreads) {
+        const int c = i / p.lut_size, v = i % p.lut_size;
+        lut_s[c * 64 + v] = p.lut[size_t(cand0 + c) * 64 + v];
+    }
+    if (tid == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        mbar_init(bar0 + 16, 1);
+        abort_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {   // one warp allocates the accumulators' columns of tensor memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(uint32_t(p.tmem_cols)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_s;
+
+    // instruction descriptor: fp32 accumulate, fp16 A and B, both K-major, N = T, M = 128
+    const uint32_t idesc = (1u << 4) | (uint32_t(T >> 3) << 17) | (uint32_t(kSearchRows >> 4) << 24);
+
+    // this thread's part of a dW tile: row r of the block, 32 consecutive weights (4 pieces of 16 bytes)
+    const int r = tid >> 1, half = tid & 1;
+    const int n = blockIdx.x * kSearchRows + r;
+    const bool row_ok = n < p.N;
+    const __half *wrow = p.W + size_t(row_ok ? n : 0) * p.K + 32 * half;
+    const uint8_t *irow = p.w_int + size_t(row_ok ? n : 0) * p.K + 32 * half;
+    const uint32_t a_row_off = uint32_t(r) * 128u;
+    const int ktiles = p.K / kSearchKTile;
+
+    uint4 wreg[4], ireg[2];
+    auto load_tile = [&](int kt) {
+        const uint4 *wp = reinterpret_cast<const uint4 *>(wrow + size_t(kt) * kSearchKTile);
+        const uint4 *ip = reinterpret_cast<const uint4 *>(irow + size_t(kt) * kSearchKTile);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wreg[i] = row_ok ? __ldg(wp + i) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) ireg[i] = row_ok ? __ldg(ip + i) : make_uint4(0u, 0u, 0u, 0u);
+    };
+    load_tile(0);
+
+    bool alive = true;
+    for (int kt = 0; kt < ktiles && alive; ++kt) {
+        const int s = kt & 1;
+        const uint32_t st_base = base + uint32_t(s) * stage_bytes;
+        const uint32_t x_base = st_base + uint32_t(p.cand_per_block) * kSearchATile;
+        // the MMAs that read this stage two slices ago must be complete before it is overwritten
+        // (every thread takes the same decision: a wait that gives up must not split the block at a barrier)
+        if (kt >= 2 && !__syncthreads_and(search_wait(bar0 + 8 * s, uint32_t(((kt >> 1) - 1) & 1), abort_flag, 1) ? 1 : 0)) {
+            alive = false;
+            break;
+        }
+        // X's slice: T rows of 128 bytes, 16-byte pieces, swizzled like the dW tiles
+        for (int c = tid; c < T * 8; c += kSearchThreads) {
+            const int row = c >> 3, piece = c & 7;
+            const uint32_t dst = x_base + uint32_t(row) * 128u + uint32_t((piece ^ (row & 7)) << 4);
+            const __half *src = p.X + size_t(row) * p.K + size_t(kt) * kSearchKTile + piece * 8;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+
+        // this slice's weights are in registers; have the next slice's on their way
+        uint4 wcur[4], icur[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wcur[i] = wreg[i];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) icur[i] = ireg[i];
+        if (kt + 1 < ktiles) load_tile(kt + 1);
+
+        // scale and offset of (row, scaling unit): a slice of 64 lies inside one unit
+        float Sf = 0.f, qb = 0.f;
+        if (row_ok) {
+            const int g = (kt * kSearchKTile) / p.L;
+            Sf = __half2float(p.S[size_t(n) * p.G + g]);
+            qb = __half2float(p.qbias[size_t(n) * p.G + g]);
+        }
+        float rest[32];        // qbias - W
+        unsigned char wi[32];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&wcur[i]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 f = __half22float2(h2[j]);
+                rest[8 * i + 2 * j] = qb - f.x;
+                rest[8 * i + 2 * j + 1] = qb - f.y;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t w4[4] = {icur[i].x, icur[i].y, icur[i].z, icur[i].w};
+#pragma unroll
+            for (int j = 0; j < 16; ++j) wi[16 * i + j] = (unsigned char)((w4[j >> 2] >> (8 * (j & 3))) & 0xffu);
+        }
+        for (int c = 0; c < ncand; ++c) {
+            const float *lut = lut_s + c * 64;
+            const uint32_t a_base = st_base + uint32_t(c) * kSearchATile + a_row_off;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t packed[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int e = 8 * i + 2 * j;
+                    const float d0 = row_ok ? fmaf(Sf, lut[wi[e]], rest[e]) : 0.f;
+                    const float d1 = row_ok ? fmaf(Sf, lut[wi[e + 1]], rest[e + 1]) : 0.f;
+                    const __half2 h = __floats2half2_rn(d0, d1);
+                    packed[j] = *reinterpret_cast<const uint32_t *>(&h);
+                }
+                const int piece = 4 * half + i;
+                const uint32_t dst = a_base + uint32_t((piece ^ (r & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[0]), "r"(packed[1]), "r"(packed[2]), "r"(packed[3]) : "memory");
+            }
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tiles are read by the tensor cores' proxy
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t bdesc = smem_desc_sw128(x_base);
+            for (int c = 0; c < ncand; ++c) {
+                const uint64_t adesc = smem_desc_sw128(st_base + uint32_t(c) * kSearchATile);
+                const uint32_t d = tmem_base + uint32_t(c * T);
+#pragma unroll
+                for (int j = 0; j < kSearchKTile / 16; ++j)   // 16 weights = 32 bytes further along the row
+                    umma_f16(d, adesc + uint64_t(2 * j), bdesc + uint64_t(2 * j), idesc, (kt > 0 || j > 0) ? 1u : 0u);
+            }
+            umma_commit(bar0 + 8 * s);
+            if (kt == ktiles - 1) umma_commit(bar0 + 16);
+        }
+    }
+
+    // ---- the accumulators are complete: every row's squared outputs ------------------------------------
+    alive = __syncthreads_and((alive && search_wait(bar0 + 16, 0u, abort_flag, 2)) ? 1 : 0) != 0;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int quarter = warp & 3, colhalf = warp >> 2;   // a warp reads the 32 lanes of its quarter
+    if (alive) {
+        for (int c = 0; c < ncand; ++c) {
+            float sum = 0.f;
+            for (int ch = colhalf; ch < T / 16; ch += 2) {
+                uint32_t v[16];
+                const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(c * T + ch * 16);
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                      "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                    : "r"(taddr));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float e = __uint_as_float(v[j]);
+                    sum = fmaf(e, e, sum);
+                }
+            }
+            part[colhalf][c][quarter * 32 + lane] = sum;
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (alive && tid < kSearchRows) {
+        const int row = blockIdx.x * kSearchRows + tid;
+        if (row < p.N)
+            for (int c = 0; c < ncand; ++c) p.err_rows[size_t(cand0 + c) * p.N + row] = part[0][c][tid] + part[1][c][tid];
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(p.tmem_cols)) : "memory");
+    }
+}
+
+// err[c] = sum over rows of err_rows[c][.] in a fixed order (fp64), one block per candidate
+__global__ void __launch_bounds__(256) search_sum_kernel(const float *__restrict__ err_rows, int N, double *__restrict__ err)
+{
+    __shared__ double sh[256];
+    const float *src = err_rows + size_t(blockIdx.x) * N;
+    double s = 0.0;
+    for (int i = threadIdx.x; i < N; i += 256) s += double(src[i]);
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) err[blockIdx.x] = sh[0];
+}
+
+// the first candidate, in order, whose error is below all earlier ones
+__global__ void search_argmin_kernel(const double *__restrict__ err, int count, int P, int *__restrict__ best)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int at = 0;
+    double lowest = err[0];
+    for (int i = 1; i < count; ++i)
+        if (err[i] < lowest) lowest = err[i], at = i;
+    best[0] = at / P;
+    best[1] = at % P;
+}
+
+size_t search_smem_bytes(int cand_per_block) { return 2 * (size_t(cand_per_block) * kSearchATile + size_t(kSearchMaxT) * 128) + 1024; }
+
+int search_cand_per_block(int T)
+{
+    int c = 512 / T;
+    return c > kSearchMaxCand ? kSearchMaxCand : c;
+}
+
+cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias, const uint16_t *X,
+                                 int N, int K, int group, int T, int n_bits, const float *lut_dev /*[P][64]*/, int P,
+                                 float *err_rows /*[P][N]*/, double *err /*[P]*/, cudaStream_t st)
+{
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    SearchParams p = {};
+    p.W = reinterpret_cast<const __half *>(W), p.w_int = w_int;
+    p.S = reinterpret_cast<const __half *>(S), p.qbias = reinterpret_cast<const __half *>(qbias);
+    p.X = reinterpret_cast<const __half *>(X), p.err_rows = err_rows;
+    p.N = N, p.K = K, p.L = group == 0 ? K : group, p.G = K / p.L, p.T = T, p.P = P;
+    p.cand_per_block = search_cand_per_block(T);
+    int cols = 32;
+    while (cols < p.cand_per_block * T) cols *= 2;
+    p.tmem_cols = cols;
+    p.lut_size = 1 << n_bits;
+    p.lut = lut_dev;
+    const size_t smem = search_smem_bytes(p.cand_per_block);
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(search_error_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(search_smem_bytes(kSearchMaxCand)));
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    const unsigned row_tiles = unsigned((N + kSearchRows - 1) / kSearchRows);
+    const unsigned groups = unsigned((P + p.cand_per_block - 1) / p.cand_per_block);
+    search_error_kernel<<<dim3(row_tiles, groups), kSearchThreads, smem, st>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    search_sum_kernel<<<unsigned(P), 256, 0, st>>>(err_rows, N, err);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_search_argmin(const double *err, int count, int P, int *best, cudaStream_t st)
+{
+    search_argmin_kernel<<<1, 32, 0, st>>>(err, count, P, best);
+    return cudaGetLastError();
+}
+
+cudaError_t search_status_take(int *status)
+{
+    int v = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&v, g_search_status, sizeof(int));
+    if (e != cudaSuccess) return e;
+    if (v != 0) {
+        const int zero = 0;
+        e = cudaMemcpyToSymbol(g_search_status, &zero, sizeof(int));
+    }
+    *status = v;
+    return e;
+}
+
+}  // namespace bcq

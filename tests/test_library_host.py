@@ -185,3 +185,23 @@ def test_multi_row_blocks_are_shared_in_proportion():
         bq.multi_row_blocks(d, bq.Plan(1, 6, 7, 0), [8192, 2048])
     with pytest.raises(bq.BcqError):                                  # fewer row blocks than operands
         bq.multi_row_blocks(d, bq.Plan(1, 1, 7, 0), [8192, 2048])
+
+
+def test_search_host_helpers_agree_with_the_oracle():
+    """The enumeration of bit partitions and the scale-factor grid are host code: compared with the
+    oracle's own enumeration (written independently) without touching a GPU."""
+    import numpy as np
+    import oracle
+    for (n, q) in [(1, 1), (2, 1), (3, 2), (4, 3), (5, 3), (5, 2), (4, 4), (6, 4), (8, 2)]:
+        got = bq.partitions(n, q)
+        want = np.array(oracle.set_partitions(n, q))
+        assert got.shape == want.shape and (got == want).all()
+    assert bq.lib().bcq_partition_count(3, 4) == 0 and bq.lib().bcq_partition_count(9, 2) == 0
+    for n in (2, 3, 4, 5):
+        np.testing.assert_allclose(bq.reexplore_factors(n, 7), oracle.reexplore_factors(n, 7), rtol=1e-15)
+    d = bq.desc(256, 512, 3, 128)
+    L = bq.lib()
+    assert L.bcq_grid_search_workspace(ctypes.byref(d), 64, 4, 6, 3, 1) > 256 * 512
+    assert L.bcq_grid_search_workspace(ctypes.byref(d), 24, 4, 6, 3, 1) == 0      # T not a multiple of 16
+    assert L.bcq_grid_search_workspace(ctypes.byref(d), 64, 7, 6, 3, 1) == 0      # more than 6 step-1 bits
+    assert L.bcq_grid_search_workspace(ctypes.byref(bq.desc(256, 512, 3, 96)), 64, 4, 6, 3, 1) == 0
