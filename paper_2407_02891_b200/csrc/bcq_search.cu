@@ -21,7 +21,7 @@
 
 namespace bcq {
 
-constexpr int kSearchThreads = 256;
+constexpr int kSearchThreads = 512;      // 16 warps: forming the operand tiles is latency-bound with fewer
 constexpr int kSearchRows = 128;        // rows of W per block = M of the MMA
 constexpr int kSearchKTile = 64;        // weights along K per stage: 128 bytes of fp16, one swizzle row
 constexpr int kSearchMaxCand = 4;       // candidates (accumulators) per block
@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ float lut_s[kSearchMaxCand * 64];
-    __shared__ float part[2][kSearchMaxCand][kSearchRows];
+    __shared__ float part[4][kSearchMaxCand][kSearchRows];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cand0 = blockIdx.y * p.cand_per_block;
@@ -126,23 +126,23 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
     // instruction descriptor: fp32 accumulate, fp16 A and B, both K-major, N = T, M = 128
     const uint32_t idesc = (1u << 4) | (uint32_t(T >> 3) << 17) | (uint32_t(kSearchRows >> 4) << 24);
 
-    // this thread's part of a dW tile: row r of the block, 32 consecutive weights (4 pieces of 16 bytes)
-    const int r = tid >> 1, half = tid & 1;
+    // this thread's part of a dW tile: row r of the block, 16 consecutive weights (2 pieces of 16 bytes)
+    const int r = tid >> 2, quart = tid & 3;
     const int n = blockIdx.x * kSearchRows + r;
     const bool row_ok = n < p.N;
-    const __half *wrow = p.W + size_t(row_ok ? n : 0) * p.K + 32 * half;
-    const uint8_t *irow = p.w_int + size_t(row_ok ? n : 0) * p.K + 32 * half;
+    const __half *wrow = p.W + size_t(row_ok ? n : 0) * p.K + 16 * quart;
+    const uint8_t *irow = p.w_int + size_t(row_ok ? n : 0) * p.K + 16 * quart;
     const uint32_t a_row_off = uint32_t(r) * 128u;
+    const uint32_t lut_u32 = smem_u32(lut_s);
     const int ktiles = p.K / kSearchKTile;
 
-    uint4 wreg[4], ireg[2];
+    uint4 wreg[2], ireg;
     auto load_tile = [&](int kt) {
         const uint4 *wp = reinterpret_cast<const uint4 *>(wrow + size_t(kt) * kSearchKTile);
         const uint4 *ip = reinterpret_cast<const uint4 *>(irow + size_t(kt) * kSearchKTile);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) wreg[i] = row_ok ? __ldg(wp + i) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-        for (int i = 0; i < 2; ++i) ireg[i] = row_ok ? __ldg(ip + i) : make_uint4(0u, 0u, 0u, 0u);
+        wreg[0] = row_ok ? __ldg(wp) : make_uint4(0u, 0u, 0u, 0u);
+        wreg[1] = row_ok ? __ldg(wp + 1) : make_uint4(0u, 0u, 0u, 0u);
+        ireg = row_ok ? __ldg(ip) : make_uint4(0u, 0u, 0u, 0u);
     };
     load_tile(0);
 
@@ -167,11 +167,7 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
         asm volatile("cp.async.commit_group;" ::: "memory");
 
         // this slice's weights are in registers; have the next slice's on their way
-        uint4 wcur[4], icur[2];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) wcur[i] = wreg[i];
-#pragma unroll
-        for (int i = 0; i < 2; ++i) icur[i] = ireg[i];
+        const uint4 wcur0 = wreg[0], wcur1 = wreg[1], icur = ireg;
         if (kt + 1 < ktiles) load_tile(kt + 1);
 
         // scale and offset of (row, scaling unit): a slice of 64 lies inside one unit
@@ -181,43 +177,43 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
             Sf = __half2float(p.S[size_t(n) * p.G + g]);
             qb = __half2float(p.qbias[size_t(n) * p.G + g]);
         }
-        float rest[32];        // qbias - W
-        unsigned char wi[32];
+        float rest[16];        // qbias - W
+        uint32_t at[16];       // shared-memory address of the first candidate's table entry of W_int
+        {
+            const uint32_t w8[8] = {wcur0.x, wcur0.y, wcur0.z, wcur0.w, wcur1.x, wcur1.y, wcur1.z, wcur1.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const __half2 *h2 = reinterpret_cast<const __half2 *>(&wcur[i]);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float2 f = __half22float2(h2[j]);
-                rest[8 * i + 2 * j] = qb - f.x;
-                rest[8 * i + 2 * j + 1] = qb - f.y;
+            for (int j = 0; j < 8; ++j) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w8[j]));
+                rest[2 * j] = qb - f.x;
+                rest[2 * j + 1] = qb - f.y;
             }
+            const uint32_t i4[4] = {icur.x, icur.y, icur.z, icur.w};
+#pragma unroll
+            for (int j = 0; j < 16; ++j) at[j] = lut_u32 + (((i4[j >> 2] >> (8 * (j & 3))) & 0xffu) << 2);
         }
+        if (!row_ok) Sf = 0.f;   // rows beyond N: dW = 0 (rest is 0 there as well)
+        static_for<0, kSearchMaxCand>([&](auto C) {
+            constexpr int c = decltype(C)::value;
+            if (c < ncand) {
+                const uint32_t a_base = st_base + uint32_t(c) * kSearchATile + a_row_off;
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const uint32_t w4[4] = {icur[i].x, icur[i].y, icur[i].z, icur[i].w};
+                for (int i = 0; i < 2; ++i) {
+                    uint32_t packed[4];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) wi[16 * i + j] = (unsigned char)((w4[j >> 2] >> (8 * (j & 3))) & 0xffu);
-        }
-        for (int c = 0; c < ncand; ++c) {
-            const float *lut = lut_s + c * 64;
-            const uint32_t a_base = st_base + uint32_t(c) * kSearchATile + a_row_off;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t packed[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int e = 8 * i + 2 * j;
-                    const float d0 = row_ok ? fmaf(Sf, lut[wi[e]], rest[e]) : 0.f;
-                    const float d1 = row_ok ? fmaf(Sf, lut[wi[e + 1]], rest[e + 1]) : 0.f;
-                    const __half2 h = __floats2half2_rn(d0, d1);
-                    packed[j] = *reinterpret_cast<const uint32_t *>(&h);
+                    for (int j = 0; j < 4; ++j) {
+                        const int e = 8 * i + 2 * j;
+                        float l0, l1;
+                        asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l0) : "r"(at[e]), "n"(c * 256));
+                        asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l1) : "r"(at[e + 1]), "n"(c * 256));
+                        const __half2 h = __floats2half2_rn(fmaf(Sf, l0, rest[e]), fmaf(Sf, l1, rest[e + 1]));
+                        packed[j] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                    const int piece = 2 * quart + i;
+                    const uint32_t dst = a_base + uint32_t((piece ^ (r & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[0]), "r"(packed[1]), "r"(packed[2]), "r"(packed[3]) : "memory");
                 }
-                const int piece = 4 * half + i;
-                const uint32_t dst = a_base + uint32_t((piece ^ (r & 7)) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[0]), "r"(packed[1]), "r"(packed[2]), "r"(packed[3]) : "memory");
             }
-        }
+        });
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tiles are read by the tensor cores' proxy
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -240,11 +236,11 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
     // ---- the accumulators are complete: every row's squared outputs ------------------------------------
     alive = __syncthreads_and((alive && search_wait(bar0 + 16, 0u, abort_flag, 2)) ? 1 : 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int quarter = warp & 3, colhalf = warp >> 2;   // a warp reads the 32 lanes of its quarter
+    const int quarter = warp & 3, colpart = warp >> 2;   // a warp reads the 32 lanes of its quarter, every fourth piece of 16 columns
     if (alive) {
         for (int c = 0; c < ncand; ++c) {
             float sum = 0.f;
-            for (int ch = colhalf; ch < T / 16; ch += 2) {
+            for (int ch = colpart; ch < T / 16; ch += 4) {
                 uint32_t v[16];
                 const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(c * T + ch * 16);
                 asm volatile(
@@ -259,7 +255,7 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
                     sum = fmaf(e, e, sum);
                 }
             }
-            part[colhalf][c][quarter * 32 + lane] = sum;
+            part[colpart][c][quarter * 32 + lane] = sum;
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -267,7 +263,8 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
     if (alive && tid < kSearchRows) {
         const int row = blockIdx.x * kSearchRows + tid;
         if (row < p.N)
-            for (int c = 0; c < ncand; ++c) p.err_rows[size_t(cand0 + c) * p.N + row] = part[0][c][tid] + part[1][c][tid];
+            for (int c = 0; c < ncand; ++c)
+                p.err_rows[size_t(cand0 + c) * p.N + row] = (part[0][c][tid] + part[1][c][tid]) + (part[2][c][tid] + part[3][c][tid]);
     }
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
