@@ -463,6 +463,63 @@ def spawn_replicas(n: int) -> int:
     return subprocess.call(cmd)
 
 
+def run_search(args):
+    """--search: the search over BCchoice and the re-explored scale (bcq_grid_search) on one OPT-30B-shaped
+    projection; a second benchmark beside the per-token line, with its own roofline (tensor cores)."""
+    import torch
+    from paper_2407_02891_b200 import binding as bq
+
+    N = K = 7168
+    T, n_bits, q, group, n_scales = args.search_tokens, 5, 3, 128, 8
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    W = (0.05 * synth.normal("search/W", 0, N * K)).reshape(N, K).astype(np.float16)
+    X = synth.activations("search/X", T, K)
+    Wd, Xd = torch.from_numpy(W).to(device), torch.from_numpy(X).to(device)
+    parts, s = bq.partitions(n_bits, q), bq.reexplore_factors(n_bits, n_scales)
+    for _ in range(max(3, args.warmup)):
+        out = bq.grid_search(N, K, q, group, Wd, Xd, n_bits, parts, s)
+    torch.cuda.synchronize(device)
+    steps = min(args.steps, 20)
+    with ClockSampler(physical_gpu_index(0)) as clocks:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            out = bq.grid_search(N, K, q, group, Wd, Xd, n_bits, parts, s)
+        e1.record()
+        e1.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    flops = 2.0 * N * K * T * len(parts) * n_scales
+    peak = 1590.0
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak_kind = "fallback"
+    if os.path.exists(path):
+        with open(path) as f:
+            peak, peak_kind = float(json.load(f)["bf16_tflops"]), "measured (bf16 burst; fp16 runs at the same rate)"
+    # parity on sampled rows (rows are independent): the oracle on the same weights, inputs and candidates
+    import oracle
+    rows = np.unique(synth.u64("search/rows", 0, 24) % np.uint64(N)).astype(np.int64)
+    ref_rows, _, _ = oracle.grid_search(W[rows], X, group, n_bits, list(parts), s)
+    got = out[1].cpu().numpy().astype(np.float64)[:, :, rows]
+    rel = float(np.abs(got - ref_rows).max() / np.abs(ref_rows).max())
+    status = bq.lib().bcq_poll_status()
+    print(json.dumps({
+        "metric": "GPTQT search over BCchoice and scale factor, ms per layer", "value": ms, "unit": "ms", "n_gpus": 1,
+        "steps": steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 operands, f32 accumulate (tcgen05)", "data": "synthetic",
+        "config": {"workload": f"search_{N}x{K}_T{T}_n{n_bits}_q{q}_g{group}", "candidates": int(len(parts)),
+                   "scale_factors": n_scales, "tokens": T},
+        "clocks": clocks.summary(), "gpu_launches": steps * n_scales * 3 + steps,
+        "roofline": {"bound": "tensor", "achieved": round(flops / ms / 1e9, 1), "peak": peak, "unit": "TFLOP/s",
+                     "frac": round(flops / ms / 1e9 / peak, 4), "peak_kind": peak_kind, "traffic": None,
+                     "kernel": "search_error_kernel", "flops_per_step": flops},
+        "parity": {"max_rel_err": rel, "tol": 5e-3, "rows": int(len(rows)), "ok": bool(rel <= 5e-3 and status == 0),
+                   "what": "per-row errors of all candidates on sampled rows against the fp64 oracle"},
+        "best": [int(v) for v in out[2].cpu().numpy()]}))
+    if not (rel <= 5e-3 and status == 0):
+        sys.exit(1)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -478,10 +535,15 @@ def main():
                     help="stack the projections that share an activation (q/k/v, gate/up) into one product each; "
                          "not the default workload: a second number beside it")
     ap.add_argument("--layers", type=int, default=0, help="override the number of decoder layers (profiling)")
+    ap.add_argument("--search", action="store_true",
+                    help="time bcq_grid_search on a 7168 x 7168 projection instead of the per-token step")
+    ap.add_argument("--search-tokens", type=int, default=128, help="calibration tokens T of --search (16..256)")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: plain launches instead of a CUDA graph, warm-up as given, "
                          "no per-shape, e2e or CPU legs; the printed number is not a benchmark value")
     args = ap.parse_args()
+    if args.search:
+        return run_search(args)
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         sys.exit(spawn_replicas(args.gpus))

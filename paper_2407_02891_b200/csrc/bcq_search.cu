@@ -137,12 +137,18 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
     const int ktiles = p.K / kSearchKTile;
 
     uint4 wreg[2], ireg;
+    __half s_next = __float2half_rn(0.f), b_next = s_next;   // scale and offset of (row, scaling unit) of the slice on its way
     auto load_tile = [&](int kt) {
         const uint4 *wp = reinterpret_cast<const uint4 *>(wrow + size_t(kt) * kSearchKTile);
         const uint4 *ip = reinterpret_cast<const uint4 *>(irow + size_t(kt) * kSearchKTile);
         wreg[0] = row_ok ? __ldg(wp) : make_uint4(0u, 0u, 0u, 0u);
         wreg[1] = row_ok ? __ldg(wp + 1) : make_uint4(0u, 0u, 0u, 0u);
         ireg = row_ok ? __ldg(ip) : make_uint4(0u, 0u, 0u, 0u);
+        if (row_ok) {   // a slice of 64 lies inside one scaling unit
+            const int g = (kt * kSearchKTile) / p.L;
+            s_next = __ldg(p.S + size_t(n) * p.G + g);
+            b_next = __ldg(p.qbias + size_t(n) * p.G + g);
+        }
     };
     load_tile(0);
 
@@ -168,15 +174,10 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
 
         // this slice's weights are in registers; have the next slice's on their way
         const uint4 wcur0 = wreg[0], wcur1 = wreg[1], icur = ireg;
+        float Sf = __half2float(s_next);
+        const float qb = __half2float(b_next);
         if (kt + 1 < ktiles) load_tile(kt + 1);
 
-        // scale and offset of (row, scaling unit): a slice of 64 lies inside one unit
-        float Sf = 0.f, qb = 0.f;
-        if (row_ok) {
-            const int g = (kt * kSearchKTile) / p.L;
-            Sf = __half2float(p.S[size_t(n) * p.G + g]);
-            qb = __half2float(p.qbias[size_t(n) * p.G + g]);
-        }
         float rest[16];        // qbias - W
         uint32_t at[16];       // shared-memory address of the first candidate's table entry of W_int
         {
