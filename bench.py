@@ -190,18 +190,25 @@ class Stack:
         for (pname, N, K) in layer_shapes(w):
             if (N, K) not in distinct:
                 distinct.append((N, K))
-        # the activations of a token: one vector (B vectors) per distinct shape, side by side in ONE device
-        # buffer, so that the end-to-end leg can bring a token's activations in with a single copy
-        x_np = [synth.activations(f"{wname}/{N}x{K}", B, K).reshape(-1) for (N, K) in distinct]
+        # the activations of a token: one vector (B vectors) per distinct input width K (projections of equal K
+        # read the same vector, as q/k/v or gate/up do), side by side in ONE device buffer, so that the
+        # end-to-end leg can bring a token's activations in with a single copy
+        widths = []
+        for (_, K) in distinct:
+            if K not in widths:
+                widths.append(K)
+        x_np = [synth.activations(f"{wname}/K{K}", B, K).reshape(-1) for K in widths]
         self.x_host_all = torch.from_numpy(np.concatenate(x_np))
         self.x_all = self.x_host_all.to(device)
-        off = 0
-        for (N, K), xv in zip(distinct, x_np):
+        xk, off = {}, 0
+        for K, xv in zip(widths, x_np):
+            xk[K] = self.x_all[off:off + xv.size]            # 16-byte aligned: K is a multiple of 512
+            off += xv.size
+        for (N, K) in distinct:
             a, z = synth.scale_rows(f"{wname}/{N}x{K}", N, K, q, group)
             dt = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
             scales[(N, K)] = (torch.from_numpy(a).to(device), torch.from_numpy(z).to(device))
-            xs[(N, K)] = self.x_all[off:off + xv.size]       # 16-byte aligned: K is a multiple of 512
-            off += xv.size
+            xs[(N, K)] = xk[K]
             wss[(N, K)] = bq.new_workspace(dt, B, device=device)
         self.names = []       # generator names of every item, for the parity check
         for layer in range(w["layers"]):
@@ -367,7 +374,7 @@ class Stack:
             r = synth.u64(name + "/bench_rows", 0, rows_per_shape) % np.uint64(N)
             rows = np.unique(np.concatenate([r.astype(np.int64), [0, N - 1]]))
             a, z = synth.scale_rows(f"{self.wname}/{N}x{K}", N, K, q, group)
-            X = synth.activations(f"{self.wname}/{N}x{K}", self.B, K)
+            X = synth.activations(f"{self.wname}/K{K}", self.B, K)
             ref = oracle.forward_planes(synth.plane_rows(name, N, K, q, rows), a[:, rows], z[rows], X, group)
             err = float(np.abs(y[:, rows] - ref).max() / np.abs(ref).max()) if np.isfinite(y).all() else float("inf")
             per_shape[f"{N}x{K}"] = err
@@ -423,7 +430,7 @@ class OracleSample:
         for (pname, N, K) in layer_shapes(self.w):
             p = synth.planes(f"{wname}/L0/{pname}", N, K, q)
             a, z = synth.scale_rows(f"{wname}/{N}x{K}", N, K, q, group)
-            x = synth.activations(f"{wname}/{N}x{K}", 1, K)
+            x = synth.activations(f"{wname}/K{K}", 1, K)
             self.data.append((p, a, z, x))
         self.cores = oracle.num_threads()
 

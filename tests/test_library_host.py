@@ -137,10 +137,10 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
     assert bq.workspace_bytes(d, 1, p) == (0 if p.k_splits == 1 else N * 8)   # lookup-table kernel: a word per row
     # canonical descriptors and batches > 1 use the generic kernel
     assert bq.plan_default(bq.desc(N, K, 3, 128), 1, 148).kernel == 0
-    for B in (2, 3):                                       # two or three columns: the lookup-table kernel on column pairs
+    for B in (2, 3, 4):                                    # up to four columns: the lookup-table kernel on column pairs
         p2 = bq.plan_default(d, B, 148)
         assert (p2.kernel, p2.row_blocks, p2.k_splits) == (p.kernel, p.row_blocks, p.k_splits)
-    for B in (4, 8, 16):                                   # more: one pass of the tensor-core kernel
+    for B in (5, 8, 16):                                   # more: one pass of the tensor-core kernel
         pb = bq.plan_default(d, B, 148)
         assert pb.kernel == 2
         assert 1 <= pb.row_blocks <= U and 1 <= pb.k_splits <= W
@@ -148,7 +148,8 @@ def test_default_plan_is_valid_and_fills_the_gpu(N, K):
         assert bq.workspace_bytes(d, B, pb) == (0 if pb.k_splits == 1 else 4096 * 4 + pb.k_splits * B * N * 4)
         # a lookup-table plan runs the columns two at a time: partial sums of two columns
         assert bq.workspace_bytes(d, B, p) == (0 if p.k_splits == 1 else 2 * N * 8)   # a word per row and column
-    assert bq.workspace_bytes(d, 1, bq.plan_default(d, 4, 148)) == 0        # the small-batch kernel needs B >= 2
+    assert bq.workspace_bytes(d, 1, bq.plan_default(d, 8, 148)) == 0        # the small-batch kernel needs B >= 2
+    assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 4, 148).kernel == 2    # one scale per row: no column pairs
     assert bq.plan_default(bq.desc(N, K, 2, 0, bq.LAYOUT_TILED), 1, 148).kernel == 1     # one scale per row
 
 
