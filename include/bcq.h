@@ -294,6 +294,26 @@ int bcq_gemv_host(const bcq_desc *desc, const void *packed_dev, const uint16_t *
                   void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /*
+ * The product with what follows it in a decoder layer fused into its last step (the per-token decode of the
+ * paper's section "Setup" runs bias, activation and residual additions as steps of their own):
+ *     y = act(W x + bias) + residual
+ * evaluated in fp32 from the complete sum and rounded once to fp16.  bias_dev, residual_dev: [N] fp16 device
+ * arrays or NULL; residual_dev may be y_dev itself (every row is read before it is written, by the same
+ * thread).  activation: BCQ_ACT_NONE, BCQ_ACT_RELU, BCQ_ACT_GELU (x/2 (1 + erf(x/sqrt 2))), BCQ_ACT_SILU
+ * (x / (1 + exp(-x))).  Tiled layout only (the lookup-table kernel); otherwise as bcq_gemv.
+ */
+enum { BCQ_ACT_NONE = 0, BCQ_ACT_RELU = 1, BCQ_ACT_GELU = 2, BCQ_ACT_SILU = 3 };
+typedef struct bcq_epilogue {
+    const uint16_t *bias_dev;
+    const uint16_t *residual_dev;
+    int32_t activation;
+    int32_t reserved;   /* 0 */
+} bcq_epilogue;
+int bcq_gemv_fused(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
+                   const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev, const bcq_epilogue *epilogue,
+                   void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
  * bcq_gemv without a workspace argument and without any allocation.  (The paper has no
  * counterpart; this entry point exists for the library's users.)
  *

@@ -56,6 +56,15 @@ class Operand(ctypes.Structure):
                 ("y_dev", ctypes.c_void_p), ("N", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
+class Epilogue(ctypes.Structure):
+    """bcq_epilogue"""
+    _fields_ = [("bias_dev", ctypes.c_void_p), ("residual_dev", ctypes.c_void_p), ("activation", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+ACT_NONE, ACT_RELU, ACT_GELU, ACT_SILU = 0, 1, 2, 3
+
+
 class BcqError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
@@ -86,6 +95,7 @@ SIGNATURES = {
     "bcq_repack": (_i, [_dp, _vp, _vp, _vp, _dp, _vp, _vp, _vp, _vp]),
     "bcq_gemv": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_gemv_fused": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_multi": (_i, [_dp, _vp, _i, _vp, _vp, _sz, _vp]),
     "bcq_gemv_multi_plan": (_i, [_dp, _pp, _vp, _i, _vp, _vp, _sz, _vp]),
     "bcq_multi_row_blocks": (_i, [_dp, _pp, _vp, _i, _vp]),
@@ -231,6 +241,15 @@ def gemv(d: Desc, packed, alpha, z, x, y, workspace=None):
     wp, wn = _ws_args(workspace)
     _check(lib().bcq_gemv(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y), wp, wn,
                           _stream()), "bcq_gemv")
+
+
+def gemv_fused(d: Desc, packed, alpha, z, x, y, bias=None, residual=None, activation=ACT_NONE, workspace=None):
+    """y = act(W x + bias) + residual (bcq_gemv_fused)."""
+    _dev(packed, alpha, z, x, y, bias, residual)
+    wp, wn = _ws_args(workspace)
+    ep = Epilogue(None if bias is None else bias.data_ptr(), None if residual is None else residual.data_ptr(), activation, 0)
+    _check(lib().bcq_gemv_fused(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y), ctypes.byref(ep),
+                                wp, wn, _stream()), "bcq_gemv_fused")
 
 
 def gemv_plan(d: Desc, plan: Plan, packed, alpha, z, x, y, workspace=None):

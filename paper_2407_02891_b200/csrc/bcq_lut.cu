@@ -78,7 +78,8 @@ static void fill_common(LutOne &one, const bcq_desc &d, const bcq_plan &plan, co
 // cols = 1: y = W x.  cols = 2 (grouped scales only): x and y hold two columns, K and N elements apart.
 // A plan with test bits set runs the test instantiation (one column only).
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
-                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st, int cols)
+                            const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st, int cols,
+                            const bcq_epilogue *epilogue)
 {
     LutOne one = {};
     one.tiles = static_cast<const uint8_t *>(packed);
@@ -86,6 +87,12 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
     one.z = reinterpret_cast<const __half *>(z);
     one.y = reinterpret_cast<__half *>(y);
     fill_common(one, d, plan, x, workspace);
+    if (epilogue) {
+        if (cols != 1) return cudaErrorInvalidValue;
+        one.bias = reinterpret_cast<const __half *>(epilogue->bias_dev);
+        one.residual = reinterpret_cast<const __half *>(epilogue->residual_dev);
+        one.activation = epilogue->activation;
+    }
     return launch_lut_any(d.q, d.group != 0, cols, plan.reserved != 0, &one, nullptr, st);
 }
 

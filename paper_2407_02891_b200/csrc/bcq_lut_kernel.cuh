@@ -112,6 +112,10 @@ struct LutOne {
     int u_base, u_rem;   // row units over row blocks (one operand)
     int w_base, w_rem;   // windows over K splits
     int test_flags;  // BCQ_PLAN_TEST_* (read by the test instantiations only)
+    // what follows the product (one operand, one column): y = act(W x + bias) + residual, in fp32, rounded once
+    const __half *bias;      // [N] or null
+    const __half *residual;  // [N] or null
+    int activation;          // BCQ_ACT_*
 };
 // Up to kLutMaxOperands matrices that share x, K, q and the scaling unit are multiplied in one launch: every
 // row block belongs to exactly one operand (row blocks rb_first[o] .. rb_first[o + 1] - 1 split operand o's
@@ -359,6 +363,27 @@ __device__ __forceinline__ __half splitk_decode(unsigned long long w, int k_spli
     if ((w >> 50) & 127) return __ushort_as_half((unsigned short)0x7fffu);   // a NaN partial sum
     const long long s = (long long)(w & ((1ull << 50) - 1)) - (long long)k_splits * kSplitBias;
     return __double2half(double(s) * (1.0 / double(1 << kSplitFracBits)));
+}
+// the same sum as fp32 (for what follows the product)
+__device__ __forceinline__ float splitk_decode_f32(unsigned long long w, int k_splits)
+{
+    if ((w >> 50) & 127) return __int_as_float(0x7fffffff);
+    const long long s = (long long)(w & ((1ull << 50) - 1)) - (long long)k_splits * kSplitBias;
+    return float(double(s) * (1.0 / double(1 << kSplitFracBits)));
+}
+
+// y = act(v + bias) + residual for row n
+__device__ __forceinline__ __half lut_finish(float v, const LutOne &p, size_t n)
+{
+    if (p.bias) v += __half2float(p.bias[n]);
+    switch (p.activation) {
+        case BCQ_ACT_RELU: v = fmaxf(v, 0.f); break;
+        case BCQ_ACT_GELU: v = 0.5f * v * (1.f + erff(v * 0.70710678118654752f)); break;
+        case BCQ_ACT_SILU: v = v / (1.f + expf(-v)); break;
+        default: break;
+    }
+    if (p.residual) v += __half2float(p.residual[n]);
+    return __float2half_rn(v);
 }
 
 __host__ __device__ inline const LutOne &lut_one(const LutOne &p) { return p; }
@@ -720,6 +745,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     // (Two columns: the second column's words follow the first column's, N further on; its rows of y start
     // after the operand's own rows.) ----------------------------------------------------------------------
     const bool split = p.k_splits > 1;
+    bool finish = false;   // something follows the product (one operand, one column only)
+    if constexpr (NB == 1 && !MULTI) finish = p.bias != nullptr || p.residual != nullptr || p.activation != BCQ_ACT_NONE;
     unsigned long long *accum = split ? p.accum + row0 : nullptr;
     const size_t Nop = size_t(U) * kUnitRows;   // rows of this operand: its second column of y starts there
     float tot[kUnitsPerWarp], tot1[NB == 2 ? kUnitsPerWarp : 1];
@@ -749,7 +776,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
         }
         if (!split && lane < 8) {
             const size_t n = size_t(u0 + ul) * kUnitRows + jr;   // row inside the operand
-            y[n] = __float2half_rn(v);
+            y[n] = finish ? lut_finish(v, p, n) : __float2half_rn(v);
             if constexpr (NB == 2) y[Nop + n] = __float2half_rn(tot1[a]);
         }
     }
@@ -765,7 +792,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
                 const unsigned long long mine = splitk_encode(v);
                 const unsigned long long before = atomicAdd(accum + n, mine);
                 if (splitk_arrivals(before) == p.k_splits - 1) {
-                    y[n] = splitk_decode(before + mine, p.k_splits);
+                    y[n] = finish ? lut_finish(splitk_decode_f32(before + mine, p.k_splits), p, n) : splitk_decode(before + mine, p.k_splits);
                     accum[n] = 0;
                 }
                 if constexpr (NB == 2) {
