@@ -267,6 +267,29 @@ class Stack:
             layers = [bq.Layer(it[0], it[1], it[2], it[3]) for it in its]
             bq.gemv_multi(d, layers, its[0][4], [it[5] for it in its], ws_multi[(d.N, d.K)])
 
+    def time_dequant(self, steps):
+        """us per token of the ablation without lookup tables (bcq_gemv_dequant) on the same operands."""
+        torch, bq = self.torch, self.bq
+
+        def launch():
+            for (d, packed, a, z, x, y, ws, _) in self.items:
+                bq.gemv_dequant(d, packed, a, z, x, y)
+
+        launch()
+        torch.cuda.synchronize(self.device)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            launch()
+        g.replay()
+        torch.cuda.synchronize(self.device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            g.replay()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / steps
+
     def time_grouped(self, steps):
         """us per token with those projections launched together; None when nothing is grouped."""
         torch, bq = self.torch, self.bq
@@ -647,6 +670,17 @@ def main():
                        "parity_max_rel_err": None if gp is None else gp["max_rel_err"]}
             if gp is not None and not gp["ok"]:
                 parity = gp
+    ablation = None
+    if world == 1 and args.batch == 1 and not args.fuse:
+        us = stack.time_dequant(max(2, min(args.steps, 10)))
+        ap_ = stack.parity() if not args.no_parity else None      # the ablation wrote the same y tensors
+        ablation = {"value": us, "unit": UNIT, "ratio_to_value": round(us / (ms_per_step * 1e3), 2),
+                    "parity_max_rel_err": None if ap_ is None else ap_["max_rel_err"],
+                    "what": "the same token through bcq_gemv_dequant: every weight dequantised to fp16 and multiplied, no "
+                            "lookup tables, same operands and bytes; the paper quotes 1.24x for binary-coded weights over "
+                            "a 3-bit linear kernel on OPT-30B (RTX A5000): context, other hardware"}
+        if ap_ is not None and not ap_["ok"]:
+            parity = ap_
     e2e = None
     if not args.no_e2e:
         e_ms, h2d, d2h = stack.e2e_steps(max(3, min(args.steps, 50)))
@@ -688,6 +722,7 @@ def main():
         "e2e": e2e,
         "parity": parity,
         "grouped_projections": grouped,
+        "dequant_ablation": ablation,
     }
     if not args.no_cpu_baseline and args.batch == 1:
         smp = OracleSample(args.workload, w)

@@ -314,6 +314,16 @@ int bcq_gemv_fused(const bcq_desc *desc, const void *packed_dev, const uint16_t 
                    void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /*
+ * Ablation: the product of bcq_gemv computed without lookup tables.  Every weight is dequantised to fp16
+ * (Eq. bcw dequantisation + Eq. fuse_step3: w = sum_i alpha_i b_i + z, fp16 additions) and multiplied with its
+ * activation (fp32 accumulation), the way a kernel for linearly quantised weights works; operand, layout
+ * (tiled only) and bytes read are those of bcq_gemv.  Its time against bcq_gemv shows, on this GPU, the shape
+ * of the paper's speed claim for binary-coded weights (Tab. "The speed up of GPTQT").  No workspace.
+ */
+int bcq_gemv_dequant(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
+                     const uint16_t *z_dev, const uint16_t *x_dev, uint16_t *y_dev, void *stream);
+
+/*
  * bcq_gemv without a workspace argument and without any allocation.  (The paper has no
  * counterpart; this entry point exists for the library's users.)
  *

@@ -95,6 +95,7 @@ SIGNATURES = {
     "bcq_repack": (_i, [_dp, _vp, _vp, _vp, _dp, _vp, _vp, _vp, _vp]),
     "bcq_gemv": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_gemv_dequant": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bcq_gemv_fused": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_multi": (_i, [_dp, _vp, _i, _vp, _vp, _sz, _vp]),
     "bcq_gemv_multi_plan": (_i, [_dp, _pp, _vp, _i, _vp, _vp, _sz, _vp]),
@@ -241,6 +242,13 @@ def gemv(d: Desc, packed, alpha, z, x, y, workspace=None):
     wp, wn = _ws_args(workspace)
     _check(lib().bcq_gemv(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y), wp, wn,
                           _stream()), "bcq_gemv")
+
+
+def gemv_dequant(d: Desc, packed, alpha, z, x, y):
+    """The ablation without lookup tables (bcq_gemv_dequant)."""
+    _dev(packed, alpha, z, x, y)
+    _check(lib().bcq_gemv_dequant(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y), _stream()),
+           "bcq_gemv_dequant")
 
 
 def gemv_fused(d: Desc, packed, alpha, z, x, y, bias=None, residual=None, activation=ACT_NONE, workspace=None):

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbcq.so")
 SOURCES = ["bcq_api.cu", "bcq_pack.cu", "bcq_gemv.cu", "bcq_lut.cu", "bcq_lut_q1.cu", "bcq_lut_q2.cu", "bcq_lut_q3.cu",
-           "bcq_lut_q4.cu", "bcq_mma.cu", "bcq_quant.cu", "bcq_noalloc.cu", "bcq_search.cu"]
+           "bcq_lut_q4.cu", "bcq_mma.cu", "bcq_quant.cu", "bcq_noalloc.cu", "bcq_search.cu", "bcq_dequant.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -659,6 +659,22 @@ int bcq_gemv(const bcq_desc *desc, const void *packed, const uint16_t *alpha, co
     return run_gemv(desc, &plan, packed, alpha, z, x, y, ws, ws_bytes, stream);
 }
 
+int bcq_gemv_dequant(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z, const uint16_t *x,
+                     uint16_t *y, void *stream)
+{
+    int rc = check_desc(desc);
+    if (rc != BCQ_OK) return rc;
+    if (!lut_kernel_covers(desc)) return BCQ_ERR_INVALID_ARG;
+    if (!packed || !x || !y) return BCQ_ERR_INVALID_ARG;
+    if (interleaved(desc))
+        alpha = z = nullptr;
+    else if (!alpha || !z)
+        return BCQ_ERR_INVALID_ARG;
+    if (!aligned(packed, 16) || !aligned(alpha, 2) || !aligned(z, 2) || !aligned(x, 16) || !aligned(y, 2)) return BCQ_ERR_MISALIGNED;
+    const cudaError_t e = launch_dequant_gemv(*desc, packed, alpha, z, x, y, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
+}
+
 int bcq_gemv_fused(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z, const uint16_t *x,
                    uint16_t *y, const bcq_epilogue *epilogue, void *ws, size_t ws_bytes, void *stream)
 {

@@ -126,6 +126,10 @@ struct LutOperand {
 cudaError_t launch_lut_multi(const bcq_desc &d, const bcq_plan &plan, const LutOperand *ops, int count, const uint16_t *x,
                              void *workspace, cudaStream_t st);
 
+// the ablation without lookup tables (tiled layout): every weight dequantised to fp16 and multiplied
+cudaError_t launch_dequant_gemv(const bcq_desc &d, const void *packed, const uint16_t *alpha, const uint16_t *z,
+                                const uint16_t *x, uint16_t *y, cudaStream_t st);
+
 cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *X, uint16_t *Y, int B, void *workspace, cudaStream_t st);
 
