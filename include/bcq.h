@@ -314,6 +314,17 @@ int bcq_gemv_fused(const bcq_desc *desc, const void *packed_dev, const uint16_t 
                    void *workspace_dev, size_t workspace_bytes, void *stream);
 
 /*
+ * bcq_gemv with bfloat16 activations and outputs: x [K] and y [N] (and the epilogue's bias and residual, when an
+ * epilogue is given; NULL = none) are bfloat16 bit patterns; the packed operand and its fp16 scales are
+ * unchanged.  The sums of 8 activations in the lookup tables are still rounded to fp16, so eight activations of
+ * one sign must not add up beyond 65504; accumulation is fp32, the result is rounded once to bfloat16
+ * (2^-9 relative).  Tiled layout only.
+ */
+int bcq_gemv_bf16(const bcq_desc *desc, const void *packed_dev, const uint16_t *alpha_dev,
+                  const uint16_t *z_dev, const uint16_t *x_bf16_dev, uint16_t *y_bf16_dev,
+                  const bcq_epilogue *epilogue_or_null, void *workspace_dev, size_t workspace_bytes, void *stream);
+
+/*
  * Ablation: the product of bcq_gemv computed without lookup tables.  Every weight is dequantised to fp16
  * (Eq. bcw dequantisation + Eq. fuse_step3: w = sum_i alpha_i b_i + z, fp16 additions) and multiplied with its
  * activation (fp32 accumulation), the way a kernel for linearly quantised weights works; operand, layout

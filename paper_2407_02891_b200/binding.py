@@ -95,6 +95,7 @@ SIGNATURES = {
     "bcq_repack": (_i, [_dp, _vp, _vp, _vp, _dp, _vp, _vp, _vp, _vp]),
     "bcq_gemv": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_plan": (_i, [_dp, _pp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "bcq_gemv_bf16": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_dequant": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bcq_gemv_fused": (_i, [_dp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bcq_gemv_multi": (_i, [_dp, _vp, _i, _vp, _vp, _sz, _vp]),
@@ -242,6 +243,18 @@ def gemv(d: Desc, packed, alpha, z, x, y, workspace=None):
     wp, wn = _ws_args(workspace)
     _check(lib().bcq_gemv(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y), wp, wn,
                           _stream()), "bcq_gemv")
+
+
+def gemv_bf16(d: Desc, packed, alpha, z, x, y, bias=None, residual=None, activation=ACT_NONE, workspace=None):
+    """bcq_gemv_bf16: x, y (and bias, residual) are torch.bfloat16 tensors."""
+    _dev(packed, alpha, z, x, y, bias, residual)
+    wp, wn = _ws_args(workspace)
+    ep = None
+    if bias is not None or residual is not None or activation != ACT_NONE:
+        ep = ctypes.byref(Epilogue(None if bias is None else bias.data_ptr(), None if residual is None else residual.data_ptr(),
+                                   activation, 0))
+    _check(lib().bcq_gemv_bf16(ctypes.byref(d), _ptr(packed), _ptr(alpha), _ptr(z), _ptr(x), _ptr(y), ep, wp, wn, _stream()),
+           "bcq_gemv_bf16")
 
 
 def gemv_dequant(d: Desc, packed, alpha, z, x, y):

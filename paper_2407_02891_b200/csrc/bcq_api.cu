@@ -234,7 +234,7 @@ size_t plan_workspace(const bcq_desc *d, const bcq_plan *p, int B)
 // cols: 1, or 2 (lookup-table kernel with the scales in the tiles): x and y hold two columns
 int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, const uint16_t *alpha, const uint16_t *z,
              const uint16_t *x, uint16_t *y, void *ws, size_t ws_bytes, void *stream, int cols = 1,
-             const bcq_epilogue *epilogue = nullptr)
+             const bcq_epilogue *epilogue = nullptr, bool bf16 = false)
 {
     if (!packed || !x || !y) return BCQ_ERR_INVALID_ARG;
     if (interleaved(desc))
@@ -246,7 +246,7 @@ int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, con
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     if (plan->kernel == 0) {
-        if (epilogue) return BCQ_ERR_INVALID_ARG;   // the fused form exists in the lookup-table kernel only
+        if (epilogue || bf16) return BCQ_ERR_INVALID_ARG;   // the fused and bfloat16 forms exist in the lookup-table kernel only
         e = launch_generic(*desc, packed, alpha, z, x, y, 1, st);
     } else {
         const size_t need = plan_workspace(desc, plan, cols);
@@ -255,7 +255,7 @@ int run_gemv(const bcq_desc *desc, const bcq_plan *plan, const void *packed, con
             if (!aligned(ws, 16)) return BCQ_ERR_MISALIGNED;
             if (ws_bytes < need) return BCQ_ERR_WORKSPACE_TOO_SMALL;
         }
-        e = launch_lut_gemv(*desc, *plan, packed, alpha, z, x, y, need ? ws : nullptr, st, cols, epilogue);
+        e = launch_lut_gemv(*desc, *plan, packed, alpha, z, x, y, need ? ws : nullptr, st, cols, epilogue, bf16);
     }
     return e == cudaSuccess ? BCQ_OK : cuda_fail(e);
 }
@@ -657,6 +657,19 @@ int bcq_gemv(const bcq_desc *desc, const void *packed, const uint16_t *alpha, co
     int rc = bcq_plan_default(desc, 1, 0, &plan);
     if (rc != BCQ_OK) return rc;
     return run_gemv(desc, &plan, packed, alpha, z, x, y, ws, ws_bytes, stream);
+}
+
+int bcq_gemv_bf16(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z, const uint16_t *x,
+                  uint16_t *y, const bcq_epilogue *epilogue, void *ws, size_t ws_bytes, void *stream)
+{
+    bcq_plan plan;
+    int rc = bcq_plan_default(desc, 1, 0, &plan);
+    if (rc != BCQ_OK) return rc;
+    if (epilogue) {
+        if (epilogue->reserved != 0 || epilogue->activation < BCQ_ACT_NONE || epilogue->activation > BCQ_ACT_SILU) return BCQ_ERR_INVALID_ARG;
+        if (!aligned(epilogue->bias_dev, 2) || !aligned(epilogue->residual_dev, 2)) return BCQ_ERR_MISALIGNED;
+    }
+    return run_gemv(desc, &plan, packed, alpha, z, x, y, ws, ws_bytes, stream, 1, epilogue, true);
 }
 
 int bcq_gemv_dequant(const bcq_desc *desc, const void *packed, const uint16_t *alpha, const uint16_t *z, const uint16_t *x,

@@ -113,7 +113,7 @@ cudaError_t launch_generic(const bcq_desc &d, const void *packed, const uint16_t
                            const uint16_t *X, uint16_t *Y, int B, cudaStream_t st);
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st,
-                            int cols = 1, const bcq_epilogue *epilogue = nullptr);
+                            int cols = 1, const bcq_epilogue *epilogue = nullptr, bool bf16 = false);
 // Several operands that share x, K, q and the scaling unit, one launch: d.N = all their rows, the operands' row
 // blocks add up to plan.row_blocks.
 constexpr int kLutMaxOperands = 4;

@@ -79,7 +79,7 @@ static void fill_common(LutOne &one, const bcq_desc &d, const bcq_plan &plan, co
 // A plan with test bits set runs the test instantiation (one column only).
 cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void *packed, const uint16_t *alpha,
                             const uint16_t *z, const uint16_t *x, uint16_t *y, void *workspace, cudaStream_t st, int cols,
-                            const bcq_epilogue *epilogue)
+                            const bcq_epilogue *epilogue, bool bf16)
 {
     LutOne one = {};
     one.tiles = static_cast<const uint8_t *>(packed);
@@ -87,6 +87,8 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
     one.z = reinterpret_cast<const __half *>(z);
     one.y = reinterpret_cast<__half *>(y);
     fill_common(one, d, plan, x, workspace);
+    if (bf16 && cols != 1) return cudaErrorInvalidValue;
+    one.bf16 = bf16 ? 1 : 0;
     if (epilogue) {
         if (cols != 1) return cudaErrorInvalidValue;
         one.bias = reinterpret_cast<const __half *>(epilogue->bias_dev);

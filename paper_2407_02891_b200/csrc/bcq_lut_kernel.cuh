@@ -116,6 +116,7 @@ struct LutOne {
     const __half *bias;      // [N] or null
     const __half *residual;  // [N] or null
     int activation;          // BCQ_ACT_*
+    int bf16;                // x, y, bias and residual are bfloat16 instead of fp16 (one operand, one column)
 };
 // Up to kLutMaxOperands matrices that share x, K, q and the scaling unit are multiplied in one launch: every
 // row block belongs to exactly one operand (row blocks rb_first[o] .. rb_first[o + 1] - 1 split operand o's
@@ -221,16 +222,22 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
 // stored with one 64-bit store (16 quads = 128 contiguous bytes per entry: no bank conflicts).
 // `table` points at entry 0 of the buffer being built.  Loading (load_quad) and building are separate
 // so that a builder can have the next window's activations on their way while it waits for the buffer.
-__device__ __forceinline__ void load_quad(const __half *xw, int cq, f32x2 (&x01)[8], f32x2 (&x23)[8])
+// two 16-bit activations -> fp32 (exact): fp16, or bfloat16 (the upper half of an fp32)
+__device__ __forceinline__ float2 act_pair_to_f32(uint32_t raw, bool bf16)
+{
+    if (bf16) return make_float2(__uint_as_float(raw << 16), __uint_as_float(raw & 0xffff0000u));
+    return __half22float2(*reinterpret_cast<const __half2 *>(&raw));
+}
+__device__ __forceinline__ void load_quad(const __half *xw, int cq, f32x2 (&x01)[8], f32x2 (&x23)[8], bool bf16 = false)
 {
     float xf[4][8];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
         const uint4 raw = *reinterpret_cast<const uint4 *>(xw + 32 * cq + 8 * k);
-        const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+        const uint32_t r4[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const float2 f = __half22float2(h2[j]);
+            const float2 f = act_pair_to_f32(r4[j], bf16);
             xf[k][2 * j] = f.x;
             xf[k][2 * j + 1] = f.y;
         }
@@ -373,16 +380,27 @@ __device__ __forceinline__ float splitk_decode_f32(unsigned long long w, int k_s
 }
 
 // y = act(v + bias) + residual for row n
+__device__ __forceinline__ float lut_ld16(const __half *a, size_t n, bool bf16)
+{
+    const unsigned short raw = __half_as_ushort(a[n]);
+    return bf16 ? __uint_as_float(uint32_t(raw) << 16) : __half2float(__ushort_as_half(raw));
+}
 __device__ __forceinline__ __half lut_finish(float v, const LutOne &p, size_t n)
 {
-    if (p.bias) v += __half2float(p.bias[n]);
+    const bool bf16 = p.bf16 != 0;
+    if (p.bias) v += lut_ld16(p.bias, n, bf16);
     switch (p.activation) {
         case BCQ_ACT_RELU: v = fmaxf(v, 0.f); break;
         case BCQ_ACT_GELU: v = 0.5f * v * (1.f + erff(v * 0.70710678118654752f)); break;
         case BCQ_ACT_SILU: v = v / (1.f + expf(-v)); break;
         default: break;
     }
-    if (p.residual) v += __half2float(p.residual[n]);
+    if (p.residual) v += lut_ld16(p.residual, n, bf16);
+    if (bf16) {   // round to nearest even on the upper 16 bits; NaN stays NaN
+        const uint32_t u = __float_as_uint(v);
+        const uint32_t r = (v != v) ? 0x7fc0u : ((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+        return __ushort_as_half((unsigned short)r);
+    }
     return __float2half_rn(v);
 }
 
@@ -558,6 +576,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     // The weights above are constants; everything from here on (x, partial sums, counters, y) may
     // depend on the previous kernel in the stream: wait for it to be complete and visible.
     const __half *xblk = p.x + size_t(w0) * kWindow;   // this block's slice of x
+    bool in_bf16 = false;
+    if constexpr (NB == 1 && !MULTI) in_bf16 = p.bf16 != 0;
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- start-up: builders and consumers build the first window's table together -----------------
@@ -565,7 +585,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     if (bt < 512) {
         if constexpr (NB == 1) {
             f32x2 x01[8], x23[8];
-            load_quad(xblk, bt & 15, x01, x23);
+            load_quad(xblk, bt & 15, x01, x23, in_bf16);
             build_quad(tables, x01, x23, bt & 15, bt >> 4, 32);
         } else {
             f32x2 xa[8], xb[8];
@@ -585,7 +605,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
             const int b = wi & 1, use = wi >> 1;
             f32x2 x01[8], x23[8];   // one column: a chunk quad; two columns: a chunk pair of each
             if constexpr (NB == 1)
-                load_quad(xblk + wi * kWindow, bt & 15, x01, x23);   // in flight while waiting for the buffer
+                load_quad(xblk + wi * kWindow, bt & 15, x01, x23, in_bf16);   // in flight while waiting for the buffer
             else
                 load_pair(xblk + wi * kWindow, size_t(p.K), bt & 31, x01, x23);
             if (use > 0 && !lut_wait<true>(bar_tab_free + 8 * b, (use - 1) & 1, abort_flag, kWaitTableFree, spin_limit)) break;
@@ -746,7 +766,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     // after the operand's own rows.) ----------------------------------------------------------------------
     const bool split = p.k_splits > 1;
     bool finish = false;   // something follows the product (one operand, one column only)
-    if constexpr (NB == 1 && !MULTI) finish = p.bias != nullptr || p.residual != nullptr || p.activation != BCQ_ACT_NONE;
+    if constexpr (NB == 1 && !MULTI) finish = p.bias != nullptr || p.residual != nullptr || p.activation != BCQ_ACT_NONE || p.bf16 != 0;
     unsigned long long *accum = split ? p.accum + row0 : nullptr;
     const size_t Nop = size_t(U) * kUnitRows;   // rows of this operand: its second column of y starts there
     float tot[kUnitsPerWarp], tot1[NB == 2 ? kUnitsPerWarp : 1];

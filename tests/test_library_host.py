@@ -20,7 +20,7 @@ def built():
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "bcq.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(bcq_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(bcq_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
