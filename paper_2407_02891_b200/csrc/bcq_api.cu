@@ -88,8 +88,7 @@ int lut_max_units(const bcq_desc *d, int B)
 // decompositions; it does not predict time exactly.
 long long lut_cost(int U, int W, int rb, int ks, int sm, bool grouped)
 {
-    // (a split costs more with one scale per row: every split applies the row's scales to its sums)
-    const long long per_tile = 38, per_window = 250, table_build = 1200, split_fixed = 1500, per_split = grouped ? 40 : 100,
+    const long long per_tile = 38, per_window = 250, table_build = 1200, split_fixed = 1500, per_split = 40,
                     per_block = 20;
     const long long blocks = static_cast<long long>(rb) * ks;
     const long long waves = (blocks + sm - 1) / sm;

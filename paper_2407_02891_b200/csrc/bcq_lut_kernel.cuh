@@ -633,6 +633,18 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
         for (int i = 0; i < NACC; ++i) acc[t][i] = 0.f;
 #pragma unroll
     for (int t = 0; t < (NB == 2 ? kUnitsPerWarp : 1); ++t) acc1[t] = 0.f;
+    if constexpr (!GROUPED) {
+        // One scale per row: the rows' alphas and offsets are needed once, after the last window.  Ask for their
+        // lines now (constants, like the weights), so that the block's last step does not wait for them.
+        if (lane < 2 * kUnitsPerWarp) {
+            const int a = lane & (kUnitsPerWarp - 1);
+            const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;
+            if (ul < V) {
+                const __half *line = lane < kUnitsPerWarp ? alpha + size_t(u0 + ul) * Q * kUnitRows : zoff + size_t(u0 + ul) * kUnitRows;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
+            }
+        }
+    }
     bool alive = !*abort_flag;
     const unsigned char *ring = ring_ptr(cw);
     const uint32_t full0 = bar_full + 8 * kD * cw, empty0 = bar_empty + 8 * kD * cw;
