@@ -88,9 +88,10 @@ int lut_max_units(const bcq_desc *d, int B)
 // warps (about 2.2 us from the previous table, and not before the buffer it overwrites is free), so blocks
 // with short windows wait for tables; a K split costs little (one atomic per row).  It ranks decompositions;
 // it does not predict time exactly.
-double lut_cost(int U, int W, int rb, int ks, int sm, int cons, int tiles_per_job)
+double lut_cost(int U, int W, int rb, int ks, int sm, int cons, int tiles_per_job, int cols)
 {
-    const double per_tile = 38.0, table_build = 2200.0, split_fixed = 500.0, per_split = 10.0, round_weight = 0.3;
+    // (two columns: twice the table entries to build, 4 instead of 3 instructions per lookup)
+    const double per_tile = cols == 2 ? 50.0 : 38.0, table_build = 2200.0 * cols, split_fixed = 500.0, per_split = 10.0, round_weight = 0.3;
     const long long blocks = static_cast<long long>(rb) * ks;
     const long long waves = (blocks + sm - 1) / sm;
     const int wc = (W + ks - 1) / ks;
@@ -124,7 +125,8 @@ int plan_lut(const bcq_desc *d, int B, int sm, bcq_plan *out)
                 const int rb = k == 0 ? rb_min : (k * sm) / ks - j;
                 if (rb < rb_min || rb < 1 || rb > U || rb > kMaxRowBlocks) continue;
                 if (j > 0 && 10LL * rb * ks < 7LL * sm) continue;   // the fit covers plans down to 0.7 of the GPU
-                const double c = lut_cost(U, W, rb, ks, sm, cons, per_job);
+                double c = lut_cost(U, W, rb, ks, sm, cons, per_job, cols);
+                if (static_cast<long long>(rb) * ks > sm) c *= 1.25;   // (the fit saw single waves only: measured, a second wave costs more than its blocks)
                 if (best < 0 || c < best) {
                     best = c;
                     out->kernel = 1;
