@@ -48,19 +48,28 @@
  * Tiled layout (BCQ_LAYOUT_TILED): the same bytes and the same fp16 values, permuted so that
  * the batch-1 kernel fetches everything it needs for 8 rows x 512 weights with ONE contiguous
  * bulk copy, and so that the 32 lanes of a warp always look up 32 different shared-memory
- * banks.  It needs K % 512 == 0, N % 8 == 0 and group in {0, 128}.  With U = N/8 row units and
- * K/512 windows, `packed` is a sequence of tiles, tile (w, u) at byte (w*U + u) * T.  Inside a
- * tile, lane l = 8 g + j (g < 4, j < 8) stands for row 8u + j and the g-th group of 128 weights
- * of window w:
+ * banks.  It needs K % 512 == 0, N % 8 == 0 and group in {0, 128, 64, 32}.  With U = N/8 row units
+ * and K/512 windows, `packed` is a sequence of tiles, tile (w, u) at byte (w*U + u) * T.  Inside a
+ * tile, lane l = 8 g + j (g < 4, j < 8) stands for row 8u + j and the g-th segment of 128 weights
+ * of window w.  SUB = 128 / group is the number of scaling units in a segment (1 for group 128 and,
+ * for the walk below, for group 0):
  *   bytes [0, q*512)      planes as [i < q][lane < 32][s < 16]: byte s of lane l in plane i holds
- *                         plane i of the 8 weights
- *                         k = 512 w + 128 g + 8 ((s + 2 j) mod 16) .. + 7   (bit order as canonical)
- *   group 128, T = q*576 + 64: the tile continues with the lanes' scales,
- *     bytes [q*512, T)    fp16 [lane < 32][alpha_0 .. alpha_{q-1}, z]
- *                         <- alpha[i][8u + j][4w + g], z[8u + j][4w + g]
+ *                         plane i of the 8 weights  k = 512 w + 128 g + 8 c .. + 7  (bit order as
+ *                         canonical) of chunk c of the segment, where
+ *                           SUB = 1:     c = (s + 2 j) mod 16
+ *                           SUB = 2, 4:  the lane walks its segment unit by unit.  With C = 16/SUB chunks
+ *                                        and P = 8/SUB chunk pairs per unit, ph = s div C, t = s mod C:
+ *                                        unit  sg = (ph + j div P) mod SUB,
+ *                                        c = 2 (P sg + ((t div 2 + j) mod P)) + (t mod 2)
+ *   group != 0, T = q*512 + 64*SUB*(q+1): the tile continues with the lanes' scales,
+ *     bytes [q*512, T)    fp16 [lane < 32][ph < SUB][alpha_0 .. alpha_{q-1}, z]: the ph-th set is that of
+ *                         the unit the lane walks in phase ph,
+ *                         <- alpha[i][8u + j][(4w + g) SUB + sg], z[8u + j][(4w + g) SUB + sg]
  *     and the alpha / z arguments of every call are ignored for this layout (pass NULL);
  *   group 0 (one scale per row), T = q*512: alpha and z stay in arrays of their own,
  *     alpha [u][i][r], z [u][r].
+ * Groups of 64 and 32 run the lookup-table kernel one column at a time (no column pairs, no
+ * tensor-core kernel, no bcq_gemv_multi, no bcq_gemv_dequant).
  * bcq_packed_bytes gives the size of `packed` for the descriptor's layout (it includes the
  * scales exactly when they live in the tiles); bcq_alpha_elems and bcq_offset_elems give the
  * element counts of separate alpha / z arrays (the canonical counts).
@@ -121,7 +130,7 @@ typedef struct bcq_plan {
 enum { BCQ_PLAN_TEST_SHORT_WAITS = 1, BCQ_PLAN_TEST_WITHHOLD_TABLE = 2 };
 
 /* ---- sizes (pure host functions; 0 when the descriptor is invalid) -------------------- */
-size_t bcq_packed_bytes(const bcq_desc *desc);   /* q*N*K/8, plus 2*(q+1)*N*G when tiled with group 128 */
+size_t bcq_packed_bytes(const bcq_desc *desc);   /* q*N*K/8, plus 2*(q+1)*N*G when tiled with grouped scales */
 size_t bcq_alpha_elems(const bcq_desc *desc);    /* q * N * G                              */
 size_t bcq_offset_elems(const bcq_desc *desc);   /* N * G                                  */
 

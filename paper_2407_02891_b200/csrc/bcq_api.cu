@@ -36,7 +36,7 @@ int check_desc(const bcq_desc *d)
     if (d->group != 0 && (d->K % d->group != 0 || d->group % 32 != 0)) return BCQ_ERR_UNSUPPORTED_SHAPE;
     if (d->layout == BCQ_LAYOUT_TILED) {
         if (d->K % kWindow != 0 || d->N % kUnitRows != 0) return BCQ_ERR_UNSUPPORTED_SHAPE;
-        if (d->group != 0 && d->group != 128) return BCQ_ERR_UNSUPPORTED_SHAPE;
+        if (d->group != 0 && d->group != 128 && d->group != 64 && d->group != 32) return BCQ_ERR_UNSUPPORTED_SHAPE;
     }
     return BCQ_OK;
 }
@@ -61,7 +61,11 @@ int device_sm_count(int *out)
 // pass of the tensor-core kernel (measured on Llama-2-70B-shaped layers: 1.73 against 2.03 ms per 8 layers).
 constexpr int kSmallBatchMin = 4;
 constexpr int kSmallBatchMinPairs = 5;
-int small_batch_min(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group != 0 ? kSmallBatchMinPairs : kSmallBatchMin; }
+// column pairs and the tensor-core kernel exist for groups of 128 (and, the latter, one scale per row); groups of
+// 64 and 32 run the lookup-table kernel column by column
+bool pairs_ok(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d->group == 128; }
+bool mma_ok(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && (d->group == 128 || d->group == 0); }
+int small_batch_min(const bcq_desc *d) { return !mma_ok(d) ? 17 : (pairs_ok(d) ? kSmallBatchMinPairs : kSmallBatchMin); }
 
 bool lut_kernel_covers(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED; }   // group 128 or one scale per row
 
@@ -72,10 +76,10 @@ bool interleaved(const bcq_desc *d) { return d->layout == BCQ_LAYOUT_TILED && d-
 // scales in the tiles runs column pairs, and a last single column with the same plan).
 int lut_max_units(const bcq_desc *d, int B)
 {
-    const bool grouped = d->group != 0;
-    int cons = lut_consumer_warps(d->q, grouped, 1);
-    if (B >= 2 && interleaved(d)) {
-        const int c2 = lut_consumer_warps(d->q, grouped, 2);
+    const int sub = scale_subs(d->group);
+    int cons = lut_consumer_warps(d->q, sub, 1);
+    if (B >= 2 && pairs_ok(d)) {
+        const int c2 = lut_consumer_warps(d->q, sub, 2);
         if (c2 < cons) cons = c2;
     }
     return cons * kLutUnitsPerWarp;
@@ -116,8 +120,8 @@ int plan_lut(const bcq_desc *d, int B, int sm, bcq_plan *out)
     const int max_units = lut_max_units(d, B);
     const int rb_min = (U + max_units - 1) / max_units;
     double best = -1.0;
-    const int cols = (B >= 2 && interleaved(d)) ? 2 : 1;
-    const int cons = lut_consumer_warps(d->q, d->group != 0, cols), per_job = lut_tiles_per_job(d->q, d->group != 0, cols);
+    const int cols = (B >= 2 && pairs_ok(d)) ? 2 : 1;
+    const int cons = lut_consumer_warps(d->q, scale_subs(d->group), cols), per_job = lut_tiles_per_job(d->q, scale_subs(d->group), cols);
     for (int ks = (W + kMaxWindowsPerBlock - 1) / kMaxWindowsPerBlock; ks <= W && ks <= 64; ++ks) {
         // row blocks that fill whole waves of the GPU, or a little less than that, and the fewest possible
         for (int k = 0; k <= 16; ++k) {
@@ -224,7 +228,8 @@ int check_plan(const bcq_desc *d, const bcq_plan *p, int B)
     if (p->kernel == 0) return BCQ_OK;
     if ((p->kernel != 1 && p->kernel != 2) || !lut_kernel_covers(d)) return BCQ_ERR_INVALID_ARG;
     if (p->reserved & ~(BCQ_PLAN_TEST_SHORT_WAITS | BCQ_PLAN_TEST_WITHHOLD_TABLE)) return BCQ_ERR_INVALID_ARG;
-    if (p->kernel == 2 && B < 2) return BCQ_ERR_INVALID_ARG;
+    if (p->reserved != 0 && d->group != 0 && d->group != 128) return BCQ_ERR_INVALID_ARG;   // the test instantiations
+    if (p->kernel == 2 && (B < 2 || !mma_ok(d))) return BCQ_ERR_INVALID_ARG;
     const int U = d->N / kUnitRows, W = d->K / kWindow;
     const int max_units = p->kernel == 1 ? lut_max_units(d, B) : kMmaMaxUnitsPerBlock;
     if (p->row_blocks < 1 || p->row_blocks > U || p->row_blocks > kMaxRowBlocks) return BCQ_ERR_INVALID_ARG;
@@ -238,7 +243,7 @@ size_t plan_workspace(const bcq_desc *d, const bcq_plan *p, int B)
 {
     if (p->k_splits <= 1) return 0;
     // kernel 1 runs one column per launch, or two when the scales live in the tiles
-    if (p->kernel == 1) return lut_workspace_bytes(d->N, (B >= 2 && interleaved(d)) ? 2 : 1);
+    if (p->kernel == 1) return lut_workspace_bytes(d->N, (B >= 2 && pairs_ok(d)) ? 2 : 1);
     if (p->kernel == 2) return kCounterBytes + size_t(p->k_splits) * B * d->N * sizeof(float);
     return 0;
 }
@@ -315,6 +320,7 @@ int run_multi(const bcq_desc *desc, const bcq_plan *plan, const bcq_operand *ops
 {
     if (!ops || !x || count < 1 || count > kLutMaxOperands) return BCQ_ERR_INVALID_ARG;
     if (!lut_kernel_covers(desc) || plan->kernel != 1) return BCQ_ERR_INVALID_ARG;
+    if (count > 1 && desc->group != 0 && desc->group != 128) return BCQ_ERR_INVALID_ARG;   // several operands: groups of 128 or per row
     int32_t N[kLutMaxOperands], rb[kLutMaxOperands];
     for (int o = 0; o < count; ++o) N[o] = ops[o].N;
     int rc = share_row_blocks(desc, plan, N, count, rb);
@@ -689,7 +695,7 @@ int bcq_gemv_dequant(const bcq_desc *desc, const void *packed, const uint16_t *a
 {
     int rc = check_desc(desc);
     if (rc != BCQ_OK) return rc;
-    if (!lut_kernel_covers(desc)) return BCQ_ERR_INVALID_ARG;
+    if (!lut_kernel_covers(desc) || (desc->group != 0 && desc->group != 128)) return BCQ_ERR_INVALID_ARG;
     if (!packed || !x || !y) return BCQ_ERR_INVALID_ARG;
     if (interleaved(desc))
         alpha = z = nullptr;
@@ -777,7 +783,7 @@ int bcq_gemm_smallbatch_plan(const bcq_desc *desc, const bcq_plan *plan, const v
     if (plan->kernel == 1) {
         // The lookup-table kernel column by column -- or, with the scales in the tiles, two columns at a
         // time (tables that hold both columns' sums side by side: one pass over the weights per pair).
-        const int step = interleaved(desc) ? 2 : 1;
+        const int step = pairs_ok(desc) ? 2 : 1;
         for (int b = 0; b < B; b += step) {
             const int cols = (b + step <= B) ? step : 1;
             rc = run_gemv(desc, plan, packed, alpha, z, X + size_t(b) * desc->K, Y + size_t(b) * desc->N, ws, ws_bytes, stream,

@@ -26,23 +26,52 @@ constexpr size_t kCounterBytes = size_t(kMaxRowBlocks) * sizeof(int);   // small
 // one word, see bcq_lut_kernel.cuh); all zero between launches.
 inline size_t lut_workspace_bytes(int N, int cols) { return size_t(cols) * size_t(N) * sizeof(unsigned long long); }
 // consumer warps and tiles per copy of the instantiation for (q, scales per group?, columns per launch)
-int lut_consumer_warps(int q, bool grouped, int cols);
-int lut_tiles_per_job(int q, bool grouped, int cols);
+// (sub: scaling units per 128 weights -- 0 = one scale per row, 1, 2 or 4 = groups of 128, 64 or 32)
+int lut_consumer_warps(int q, int sub, int cols);
+int lut_tiles_per_job(int q, int sub, int cols);
+inline int scale_subs(int group) { return group == 0 ? 0 : 128 / group; }
 
 inline int n_groups(const bcq_desc &d) { return d.group == 0 ? 1 : d.K / d.group; }
 
 // ---- where the operands of one layer live (host and device) ---------------------------------
 //
 // Canonical: packed[i][n][k/8], alpha[i][n][g], z[n][g] in three arrays.
-// Tiled: tile (w, u) of `packed` covers window w (512 weights = 64 chunks of 8 = 4 groups of 128)
-// of row unit u (8 rows).  Lane l = 8 g + j of a warp owns row 8u + j and group g of the window:
-//   q*512 bytes of planes as [i < q][lane < 32][s < 16]; byte s of a lane in plane i is
-//   plane i of chunk 16 g + ((s + 2 j) mod 16): the 8 lanes of a group walk the group's 16 chunks
-//   skewed by two chunks per row, so that at every step the 32 lanes of a warp look up 32
-//   different chunk columns of the table (32 different shared-memory banks);
-//   group 128 only: followed, in the same tile, by the lanes' scales [lane < 32][alpha_0 .. alpha_{q-1}, z]
-//   (fp16) -- the tile is one contiguous piece of memory, fetched by one bulk copy;
+// Tiled: tile (w, u) of `packed` covers window w (512 weights = 64 chunks of 8 = 4 segments of 128)
+// of row unit u (8 rows).  Lane l = 8 g + j of a warp owns row 8u + j and segment g of the window:
+//   q*512 bytes of planes as [i < q][lane < 32][s < 16].  With groups of 128 (or one scale per row) byte s of a
+//   lane in plane i is plane i of chunk 16 g + ((s + 2 j) mod 16): the 8 lanes of a segment walk its 16 chunks
+//   skewed by two chunks per row, so that at every step the 32 lanes of a warp look up 32 different chunk
+//   columns of the table (32 different shared-memory banks).  With SUB = 2 or 4 scaling units per segment
+//   (groups of 64 or 32) a lane walks its segment unit by unit -- steps ph*(16/SUB) .. cover unit
+//   (ph + j / (8/SUB)) mod SUB, inside it the chunk pairs rotate by j -- which keeps the 32 columns distinct
+//   and a unit's chunks in consecutive steps (tile_step / tile_chunk below are the two directions);
+//   grouped scales: followed, in the same tile, by the lanes' scales [lane < 32][ph < SUB][alpha_0 ..
+//   alpha_{q-1}, z] (fp16), ph-th entry = the unit the lane walks in phase ph -- the tile is one contiguous
+//   piece of memory, fetched by one bulk copy;
 //   group 0 (per row): alpha [u][i][r] and z [u][r] stay in their own arrays.
+// chunk (0..15 inside the segment) that byte s of lane row j covers, and the inverse
+__host__ __device__ inline int tile_chunk(int sub, int j, int s)
+{
+    if (sub <= 1) return (s + 2 * j) & 15;
+    const int cps = 16 / sub, wps = 8 / sub;
+    const int ph = s / cps, t = s % cps;
+    const int sg = (ph + j / wps) % sub;
+    return 2 * (wps * sg + ((t >> 1) + j) % wps) + (t & 1);
+}
+__host__ __device__ inline int tile_step(int sub, int j, int cc)
+{
+    if (sub <= 1) return (cc - 2 * j) & 15;
+    const int cps = 16 / sub, wps = 8 / sub;
+    const int col = cc >> 1, sg = col / wps, cw = col % wps;
+    const int ph = (sg - j / wps + sub) % sub, th = (cw - j % wps + wps) % wps;
+    return ph * cps + 2 * th + (cc & 1);
+}
+// phase in which lane row j walks scaling unit sg of its segment
+__host__ __device__ inline int tile_phase(int sub, int j, int sg)
+{
+    if (sub <= 1) return 0;
+    return (sg - j / (8 / sub) + sub) % sub;
+}
 struct View {
     int layout, N, K, q, group;
     unsigned char *packed;
@@ -51,7 +80,8 @@ struct View {
 
     __host__ __device__ int G() const { return group == 0 ? 1 : K / group; }
     __host__ __device__ bool interleaved() const { return layout == BCQ_LAYOUT_TILED && group != 0; }
-    __host__ __device__ size_t tile_bytes() const { return size_t(q) * 512 + (interleaved() ? size_t(q) * 64 + 64 : 0); }
+    __host__ __device__ int subs() const { return group == 0 ? 0 : 128 / group; }   // scaling units per segment (tiled: group 32, 64, 128)
+    __host__ __device__ size_t tile_bytes() const { return size_t(q) * 512 + (interleaved() ? size_t(subs()) * (q + 1) * 64 : 0); }
     __host__ __device__ size_t tile_base(int w, int u) const { return (size_t(w) * (N / kUnitRows) + u) * tile_bytes(); }
 
     // the byte holding weights k = 8*kb .. 8*kb+7 of (plane i, row n)
@@ -60,7 +90,7 @@ struct View {
         if (layout == BCQ_LAYOUT_CANONICAL) return packed + (size_t(i) * N + n) * size_t(K / 8) + kb;
         const int w = kb / (kWindow / 8), c = kb % (kWindow / 8);
         const int g = c >> 4, u = n / kUnitRows, j = n % kUnitRows;
-        const int s = ((c & 15) - 2 * j) & 15;   // step at which lane 8g + j reaches chunk c
+        const int s = tile_step(subs(), j, c & 15);   // step at which lane 8g + j reaches chunk c
         const int lane = 8 * g + j;
         return packed + tile_base(w, u) + size_t(i) * 512 + size_t(lane) * 16 + s;
     }
@@ -74,16 +104,18 @@ struct View {
         if (layout == BCQ_LAYOUT_CANONICAL) return alpha + (size_t(i) * N + n) * G() + g;
         const int u = n / kUnitRows, r = n % kUnitRows;
         if (group == 0) return alpha + (size_t(u) * q + i) * kUnitRows + r;
-        const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
-        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + (gi * kUnitRows + r) * (q + 1) + i;
+        const int sub = subs(), per_window = kGroupsPerWindow * sub;
+        const int w = g / per_window, gi = (g % per_window) / sub, ph = tile_phase(sub, r, g % sub);
+        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + ((gi * kUnitRows + r) * sub + ph) * (q + 1) + i;
     }
     __host__ __device__ uint16_t *z_elem(int n, int g) const
     {
         if (layout == BCQ_LAYOUT_CANONICAL) return z + size_t(n) * G() + g;
         const int u = n / kUnitRows, r = n % kUnitRows;
         if (group == 0) return z + size_t(u) * kUnitRows + r;
-        const int w = g / kGroupsPerWindow, gi = g % kGroupsPerWindow;
-        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + (gi * kUnitRows + r) * (q + 1) + q;
+        const int sub = subs(), per_window = kGroupsPerWindow * sub;
+        const int w = g / per_window, gi = (g % per_window) / sub, ph = tile_phase(sub, r, g % sub);
+        return reinterpret_cast<uint16_t *>(packed + tile_base(w, u) + size_t(q) * 512) + ((gi * kUnitRows + r) * sub + ph) * (q + 1) + q;
     }
 };
 

@@ -4,59 +4,57 @@
 
 namespace bcq {
 
-cudaError_t launch_lut_q1(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
-cudaError_t launch_lut_q2(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
-cudaError_t launch_lut_q3(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
-cudaError_t launch_lut_q4(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t launch_lut_q1(int sub, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t launch_lut_q2(int sub, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t launch_lut_q3(int sub, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
+cudaError_t launch_lut_q4(int sub, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st);
 cudaError_t lut_status_take_q1(int *status);
 cudaError_t lut_status_take_q2(int *status);
 cudaError_t lut_status_take_q3(int *status);
 cudaError_t lut_status_take_q4(int *status);
 
-int lut_consumer_warps(int q, bool grouped, int cols)
+template <int Q>
+static void lut_geometry(int sub, int cols, int *cons, int *per_job)
 {
-    switch (q * 4 + (grouped ? 2 : 0) + (cols == 2 ? 1 : 0)) {
-        case 4: return LutCfg<1, false, 1>::kCons;
-        case 6: return LutCfg<1, true, 1>::kCons;
-        case 7: return LutCfg<1, true, 2>::kCons;
-        case 8: return LutCfg<2, false, 1>::kCons;
-        case 10: return LutCfg<2, true, 1>::kCons;
-        case 11: return LutCfg<2, true, 2>::kCons;
-        case 12: return LutCfg<3, false, 1>::kCons;
-        case 14: return LutCfg<3, true, 1>::kCons;
-        case 15: return LutCfg<3, true, 2>::kCons;
-        case 16: return LutCfg<4, false, 1>::kCons;
-        case 18: return LutCfg<4, true, 1>::kCons;
-        case 19: return LutCfg<4, true, 2>::kCons;
+    switch (sub * 4 + cols) {
+        case 1: *cons = LutCfg<Q, 0, 1>::kCons, *per_job = LutCfg<Q, 0, 1>::kJ; break;
+        case 5: *cons = LutCfg<Q, 1, 1>::kCons, *per_job = LutCfg<Q, 1, 1>::kJ; break;
+        case 6: *cons = LutCfg<Q, 1, 2>::kCons, *per_job = LutCfg<Q, 1, 2>::kJ; break;
+        case 9: *cons = LutCfg<Q, 2, 1>::kCons, *per_job = LutCfg<Q, 2, 1>::kJ; break;
+        case 17: *cons = LutCfg<Q, 4, 1>::kCons, *per_job = LutCfg<Q, 4, 1>::kJ; break;
+        default: *cons = 0, *per_job = 1; break;
     }
-    return 0;
 }
-int lut_tiles_per_job(int q, bool grouped, int cols)
+static void lut_geometry_any(int q, int sub, int cols, int *cons, int *per_job)
 {
-    switch (q * 4 + (grouped ? 2 : 0) + (cols == 2 ? 1 : 0)) {
-        case 4: return LutCfg<1, false, 1>::kJ;
-        case 6: return LutCfg<1, true, 1>::kJ;
-        case 7: return LutCfg<1, true, 2>::kJ;
-        case 8: return LutCfg<2, false, 1>::kJ;
-        case 10: return LutCfg<2, true, 1>::kJ;
-        case 11: return LutCfg<2, true, 2>::kJ;
-        case 12: return LutCfg<3, false, 1>::kJ;
-        case 14: return LutCfg<3, true, 1>::kJ;
-        case 15: return LutCfg<3, true, 2>::kJ;
-        case 16: return LutCfg<4, false, 1>::kJ;
-        case 18: return LutCfg<4, true, 1>::kJ;
-        case 19: return LutCfg<4, true, 2>::kJ;
+    *cons = 0, *per_job = 1;
+    switch (q) {
+        case 1: lut_geometry<1>(sub, cols, cons, per_job); break;
+        case 2: lut_geometry<2>(sub, cols, cons, per_job); break;
+        case 3: lut_geometry<3>(sub, cols, cons, per_job); break;
+        case 4: lut_geometry<4>(sub, cols, cons, per_job); break;
     }
-    return 1;
+}
+int lut_consumer_warps(int q, int sub, int cols)
+{
+    int cons, per_job;
+    lut_geometry_any(q, sub, cols, &cons, &per_job);
+    return cons;
+}
+int lut_tiles_per_job(int q, int sub, int cols)
+{
+    int cons, per_job;
+    lut_geometry_any(q, sub, cols, &cons, &per_job);
+    return per_job;
 }
 
-static cudaError_t launch_lut_any(int q, bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
+static cudaError_t launch_lut_any(int q, int sub, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
 {
     switch (q) {
-        case 1: return launch_lut_q1(grouped, cols, test, one, many, st);
-        case 2: return launch_lut_q2(grouped, cols, test, one, many, st);
-        case 3: return launch_lut_q3(grouped, cols, test, one, many, st);
-        case 4: return launch_lut_q4(grouped, cols, test, one, many, st);
+        case 1: return launch_lut_q1(sub, cols, test, one, many, st);
+        case 2: return launch_lut_q2(sub, cols, test, one, many, st);
+        case 3: return launch_lut_q3(sub, cols, test, one, many, st);
+        case 4: return launch_lut_q4(sub, cols, test, one, many, st);
     }
     return cudaErrorInvalidValue;
 }
@@ -95,7 +93,7 @@ cudaError_t launch_lut_gemv(const bcq_desc &d, const bcq_plan &plan, const void 
         one.residual = reinterpret_cast<const __half *>(epilogue->residual_dev);
         one.activation = epilogue->activation;
     }
-    return launch_lut_any(d.q, d.group != 0, cols, plan.reserved != 0, &one, nullptr, st);
+    return launch_lut_any(d.q, scale_subs(d.group), cols, plan.reserved != 0, &one, nullptr, st);
 }
 
 // Several operands that share x in one launch (batch 1); d.N is the sum of their rows and ops[o].row_blocks the
@@ -127,7 +125,7 @@ cudaError_t launch_lut_multi(const bcq_desc &d, const bcq_plan &plan, const LutO
     for (int o = count; o <= kLutMaxOperands; ++o) many.rb_first[o] = rb;
     many.count = count;
     fill_common(many.one, d, plan, x, workspace);
-    return launch_lut_any(d.q, d.group != 0, 1, false, nullptr, &many, st);
+    return launch_lut_any(d.q, scale_subs(d.group), 1, false, nullptr, &many, st);
 }
 
 // Read and clear the device status words of the kernels (one per translation unit that instantiates them).

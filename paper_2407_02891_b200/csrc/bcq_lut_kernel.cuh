@@ -74,9 +74,10 @@ static __device__ int g_lut_status = 0;  // 0, or the code of the wait that ran 
 // Geometry of one instantiation: tile bytes, tiles per job (kJ), slots per ring (kD), consumer warps.
 // The rings are cut from the two pieces of shared memory before and after the 64 KB-aligned tables; the
 // sizes below assume the usual 1 KB offset of a block's shared window (the kernel checks what it finds).
-template <int Q, bool GROUPED, int NB>
+// SUB: scaling units per 128 weights: 0 = one scale per row (no scales in the tiles), 1, 2, 4 = groups of 128, 64, 32.
+template <int Q, int SUB, int NB>
 struct LutCfg {
-    static constexpr int kTile = Q * 512 + (GROUPED ? Q * 64 + 64 : 0);
+    static constexpr int kTile = Q * 512 + SUB * (Q + 1) * 64;
     static constexpr int kTables = NB * 65536;
     static constexpr int kFront = 65536 - 1024;
     static constexpr int kBack = kLutSmemBytes - kFront - kTables - kFixedBytes;
@@ -431,13 +432,17 @@ __device__ __forceinline__ bool lut_wait(uint32_t bar, uint32_t parity, volatile
 // 64 KB region of its own.
 // MULTI: several operands (batch 1); TEST: the instantiation the library's tests use to see a wait run out
 // (short limits, and the builders keep a finished table to themselves when the plan asks for it).
-template <int Q, bool GROUPED, int NB, bool MULTI, bool TEST>
+template <int Q, int SUB, int NB, bool MULTI, bool TEST>
 __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename LutParamsOf<MULTI>::type pm)
 {
-    static_assert(NB == 1 || (NB == 2 && GROUPED), "two columns need the scales inside the tiles");
+    constexpr bool GROUPED = SUB > 0;
+    constexpr int kPhase = SUB > 1 ? 16 / SUB : 16;   // steps (chunks) a lane spends in one scaling unit of its segment
+    constexpr int kWordsPerUnit = SUB > 1 ? 8 / SUB : 8;
+    static_assert(SUB == 0 || SUB == 1 || SUB == 2 || SUB == 4, "scaling units per 128 weights");
+    static_assert(NB == 1 || (NB == 2 && SUB == 1), "two columns: groups of 128 only");
     static_assert(!MULTI || NB == 1, "several operands: batch 1");
     const LutOne &p = lut_one(pm);
-    using C = LutCfg<Q, GROUPED, NB>;
+    using C = LutCfg<Q, SUB, NB>;
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int kTile = C::kTile, kJ = C::kJ, kD = C::kD, kCons = C::kCons;
     constexpr int kSlotBytes = kJ * kTile;
@@ -660,10 +665,32 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
         // next one share the 4-byte column 8 g + ((h + j) mod 8); the odd chunk is its upper half.
         uint32_t off[8];
 #pragma unroll
-        for (int h = 0; h < 8; ++h) off[h] = tab0 + uint32_t(b * (NB == 1 ? 128 : 65536) + 4 * (8 * g4 + ((h + jr) & 7)));
+        for (int h = 0; h < 8; ++h) {
+            int col = (h + jr) & 7;
+            if constexpr (SUB > 1) {   // unit by unit: see tile_chunk() for the walk
+                const int ph = (2 * h) / kPhase, th = ((2 * h) % kPhase) >> 1;
+                col = kWordsPerUnit * ((ph + jr / kWordsPerUnit) % SUB) + (th + jr) % kWordsPerUnit;
+            }
+            off[h] = tab0 + uint32_t(b * (NB == 1 ? 128 : 65536) + 4 * (8 * g4 + col));
+        }
         // sum of x over this lane's group: the all-ones entries of the group's 16 chunks (two per lane)
         float xsum, xsum1 = 0.f;
-        if constexpr (NB == 1) {
+        [[maybe_unused]] float xs[SUB > 1 ? SUB : 1];   // SUB > 1: sum of x over the unit of every phase
+        if constexpr (SUB > 1) {
+#pragma unroll
+            for (int ph = 0; ph < SUB; ++ph) {
+                const int sg = (ph + jr / kWordsPerUnit) % SUB;
+                float acc_x = 0.f;
+#pragma unroll
+                for (int k = 0; k < kWordsPerUnit; ++k) {
+                    const uint32_t ones = lds_b32<255 * 256>(tab0 + uint32_t(b * 128 + 4 * (8 * g4 + kWordsPerUnit * sg + k)));
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&ones));
+                    acc_x += f.x + f.y;
+                }
+                xs[ph] = acc_x;
+            }
+            xsum = 0.f;
+        } else if constexpr (NB == 1) {
             const uint32_t ones = lds_b32<255 * 256>(off[0]);
             const float2 ones_f = __half22float2(*reinterpret_cast<const __half2 *>(&ones));
             xsum = ones_f.x + ones_f.y;
@@ -677,9 +704,11 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
             xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 2);
             xsum1 += __shfl_xor_sync(0xffffffffu, xsum1, 4);
         }
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
-        xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
+        if constexpr (SUB <= 1) {
+            xsum += __shfl_xor_sync(0xffffffffu, xsum, 1);
+            xsum += __shfl_xor_sync(0xffffffffu, xsum, 2);
+            xsum += __shfl_xor_sync(0xffffffffu, xsum, 4);
+        }
         xacc += xsum;
 
         static_for<0, C::kJobsPerWarp>([&](auto T) {
@@ -705,8 +734,13 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
                                 wbuf[4 * j + 2] = v.z;
                                 wbuf[4 * j + 3] = v.w;
                             }
-                            [[maybe_unused]] __half sc[Q + 1];   // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane
-                            if constexpr (GROUPED) {
+                            // alpha_0 .. alpha_{q-1}, z of (row, group) = this lane; SUB > 1: one set per phase
+                            [[maybe_unused]] __align__(8) __half sc[(SUB > 1 ? SUB : 1) * (Q + 1)];
+                            if constexpr (SUB > 1) {
+                                const uint32_t *sp = reinterpret_cast<const uint32_t *>(tile + Q * 512 + lane * (2 * SUB * (Q + 1)));
+#pragma unroll
+                                for (int k = 0; k < SUB * (Q + 1) / 2; ++k) reinterpret_cast<uint32_t *>(sc)[k] = sp[k];
+                            } else if constexpr (GROUPED) {
                                 const unsigned char *sp = tile + Q * 512 + lane * (2 * (Q + 1));
                                 if constexpr (Q == 3) {
                                     *reinterpret_cast<uint2 *>(sc) = *reinterpret_cast<const uint2 *>(sp);
@@ -722,6 +756,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
                                 if (lane == 0) mbar_arrive(empty0 + 8 * slot);
                             }
                             float sum[Q], sum1[NB == 2 ? Q : 1];
+                            [[maybe_unused]] float vsub = acc[a][0];   // SUB > 1: the row's sum, a scaling unit at a time
                             static_for<0, 16>([&](auto S) {
                                 constexpr int st = decltype(S)::value;
                                 static_for<0, Q>([&](auto I) {
@@ -729,8 +764,8 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
                                     constexpr int pb = i * 16 + st;
                                     const uint32_t addr = __byte_perm(wbuf[pb >> 2], off[st >> 1], 0x7604 | ((pb & 3) << 4));
                                     if constexpr (NB == 1) {
-                                        if constexpr (st == 0)
-                                            sum[i] = lut_first<0>(addr);
+                                        if constexpr (st % kPhase == 0)
+                                            sum[i] = lut_first<(st & 1) * 2>(addr);
                                         else
                                             lut_add<(st & 1) * 2>(sum[i], addr);
                                     } else {
@@ -740,8 +775,16 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
                                             lut_add2<(st & 1) * 128>(sum[i], sum1[i], addr);
                                     }
                                 });
+                                if constexpr (SUB > 1 && st % kPhase == kPhase - 1) {   // a scaling unit is complete
+                                    constexpr int ph = st / kPhase;
+                                    vsub = fmaf(__half2float(sc[ph * (Q + 1) + Q]), xs[ph], vsub);
+#pragma unroll
+                                    for (int i = 0; i < Q; ++i) vsub = fmaf(__half2float(sc[ph * (Q + 1) + i]), sum[i], vsub);
+                                }
                             });
-                            if constexpr (GROUPED) {
+                            if constexpr (SUB > 1) {
+                                acc[a][0] = vsub;
+                            } else if constexpr (GROUPED) {
                                 float v = fmaf(__half2float(sc[Q]), xsum, acc[a][0]);
 #pragma unroll
                                 for (int i = 0; i < Q; ++i) v = fmaf(__half2float(sc[i]), sum[i], v);
@@ -841,7 +884,7 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     }
 }
 
-template <int Q, bool GROUPED, int NB, bool MULTI, bool TEST>
+template <int Q, int SUB, int NB, bool MULTI, bool TEST>
 static cudaError_t launch_lut_inst(const typename LutParamsOf<MULTI>::type &prm, cudaStream_t st)
 {
     // The opt-in to more than 48 KB of dynamic shared memory is per function and per device:
@@ -851,7 +894,7 @@ static cudaError_t launch_lut_inst(const typename LutParamsOf<MULTI>::type &prm,
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(lut_gemv_kernel<Q, GROUPED, NB, MULTI, TEST>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
+        e = cudaFuncSetAttribute(lut_gemv_kernel<Q, SUB, NB, MULTI, TEST>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLutSmemBytes);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
@@ -865,7 +908,7 @@ static cudaError_t launch_lut_inst(const typename LutParamsOf<MULTI>::type &prm,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, GROUPED, NB, MULTI, TEST>, prm);
+    return cudaLaunchKernelEx(&cfg, lut_gemv_kernel<Q, SUB, NB, MULTI, TEST>, prm);
 }
 
 // Read and clear this translation unit's device status word.
@@ -885,18 +928,22 @@ static cudaError_t lut_status_take_here(int *status)
 // All instantiations for one number of planes: one column or two (grouped scales), one operand or several
 // (one column), and the test instantiation (one operand, one column).
 template <int Q>
-static cudaError_t launch_lut_for_q(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
+static cudaError_t launch_lut_for_q(int sub, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
 {
+    if (sub == 2 || sub == 4) {   // groups of 64 and 32: one operand, one column
+        if (many || cols != 1 || test) return cudaErrorInvalidValue;
+        return sub == 2 ? launch_lut_inst<Q, 2, 1, false, false>(*one, st) : launch_lut_inst<Q, 4, 1, false, false>(*one, st);
+    }
     if (many) {
         if (cols != 1 || test) return cudaErrorInvalidValue;
-        return grouped ? launch_lut_inst<Q, true, 1, true, false>(*many, st) : launch_lut_inst<Q, false, 1, true, false>(*many, st);
+        return sub ? launch_lut_inst<Q, 1, 1, true, false>(*many, st) : launch_lut_inst<Q, 0, 1, true, false>(*many, st);
     }
     if (cols == 2) {
-        if (!grouped || test) return cudaErrorInvalidValue;
-        return launch_lut_inst<Q, true, 2, false, false>(*one, st);
+        if (!sub || test) return cudaErrorInvalidValue;
+        return launch_lut_inst<Q, 1, 2, false, false>(*one, st);
     }
-    if (test) return grouped ? launch_lut_inst<Q, true, 1, false, true>(*one, st) : launch_lut_inst<Q, false, 1, false, true>(*one, st);
-    return grouped ? launch_lut_inst<Q, true, 1, false, false>(*one, st) : launch_lut_inst<Q, false, 1, false, false>(*one, st);
+    if (test) return sub ? launch_lut_inst<Q, 1, 1, false, true>(*one, st) : launch_lut_inst<Q, 0, 1, false, true>(*one, st);
+    return sub ? launch_lut_inst<Q, 1, 1, false, false>(*one, st) : launch_lut_inst<Q, 0, 1, false, false>(*one, st);
 }
 
 }  // namespace bcq

@@ -3,9 +3,9 @@
 
 namespace bcq {
 
-cudaError_t launch_lut_q3(bool grouped, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
+cudaError_t launch_lut_q3(int sub, int cols, bool test, const LutOne *one, const LutMany *many, cudaStream_t st)
 {
-    return launch_lut_for_q<3>(grouped, cols, test, one, many, st);
+    return launch_lut_for_q<3>(sub, cols, test, one, many, st);
 }
 cudaError_t lut_status_take_q3(int *status) { return lut_status_take_here(status); }
 

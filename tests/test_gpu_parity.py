@@ -50,7 +50,8 @@ def test_pack_canonical_bit_exact(N, K, q, group):
 
 
 @pytest.mark.parametrize("N,K,q,group", [(40, 1024, 3, 128), (24, 512, 2, 128), (8, 1536, 4, 128), (72, 512, 1, 0),
-                                         (296, 2048, 3, 128), (64, 1024, 2, 0)])
+                                         (296, 2048, 3, 128), (64, 1024, 2, 0), (40, 1024, 3, 64), (24, 512, 2, 32),
+                                         (8, 1536, 4, 32), (72, 512, 1, 64), (296, 2048, 3, 32), (64, 1024, 4, 64)])
 def test_pack_tiled_and_repack_bit_exact(N, K, q, group):
     p, codes, alpha, z, _ = make_layer(f"tile/{N}x{K}", N, K, q, group)
     canon = oracle.pack_canonical(codes, q)

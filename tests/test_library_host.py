@@ -47,11 +47,13 @@ def test_desc_validation_and_sizes():
     assert bq.packed_bytes(bq.desc(64, 1024, 2, 0, bq.LAYOUT_TILED)) == 2 * 64 * 1024 // 8
     assert bq.alpha_elems(d) == 3 * 7168 * 56 and bq.offset_elems(d) == 7168 * 56
     assert bq.offset_elems(bq.desc(16, 32, 3, 0)) == 16
+    for g in (64, 32):                                                           # smaller groups: more scales in the tiles
+        assert bq.packed_bytes(bq.desc(64, 1024, 3, g, bq.LAYOUT_TILED)) == 3 * 64 * 1024 // 8 + 2 * 4 * 64 * (1024 // g)
     bad = [(0, 32, 3, 32, 0, bq.ERR_INVALID_ARG), (16, 32, 0, 32, 0, bq.ERR_INVALID_ARG),
            (16, 32, 5, 32, 0, bq.ERR_INVALID_ARG), (16, 32, 3, 32, 7, bq.ERR_INVALID_ARG),
            (16, 40, 3, 0, 0, bq.ERR_UNSUPPORTED_SHAPE), (16, 96, 3, 64, 0, bq.ERR_UNSUPPORTED_SHAPE),
            (16, 96, 3, 48, 0, bq.ERR_UNSUPPORTED_SHAPE), (16, 256, 3, 128, 1, bq.ERR_UNSUPPORTED_SHAPE),
-           (12, 512, 3, 128, 1, bq.ERR_UNSUPPORTED_SHAPE), (16, 512, 3, 64, 1, bq.ERR_UNSUPPORTED_SHAPE)]
+           (12, 512, 3, 128, 1, bq.ERR_UNSUPPORTED_SHAPE), (16, 512, 3, 256, 1, bq.ERR_UNSUPPORTED_SHAPE)]
     for N, K, q, g, lay, want in bad:
         d = bq.desc(N, K, q, g, lay)
         assert bq.check_desc(d) == want, (N, K, q, g, lay)
