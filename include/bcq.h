@@ -84,7 +84,7 @@
 extern "C" {
 #endif
 
-#define BCQ_VERSION 210
+#define BCQ_VERSION 220
 
 typedef enum bcq_status {
     BCQ_OK = 0,

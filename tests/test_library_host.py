@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(L, n), n
     assert set(names) == set(bq.SIGNATURES), "binding and header disagree"
-    assert bq.lib().bcq_version() == 210
+    assert bq.lib().bcq_version() == 220
 
 
 def test_status_strings():
