@@ -49,7 +49,7 @@ def test_noalloc_matches_gemv_twice_in_a_row(N, K, q):
 
 
 def test_noalloc_refuses_products_beyond_its_scratch():
-    cand = [(262144, 4096), (65536, 32768), (32768, 65536), (131072, 16384), (262144, 16384)]
+    cand = [(393216, 16384), (524288, 32768), (262144, 4096), (65536, 32768), (32768, 65536), (131072, 16384), (262144, 16384)]   # 8 bytes of scratch per row
     for N, K in cand:
         d = bq.desc(N, K, 3, 128, bq.LAYOUT_TILED)
         if bq.workspace_bytes(d, 1) > bq.NOALLOC_SCRATCH_BYTES:
