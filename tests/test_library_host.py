@@ -209,3 +209,29 @@ def test_search_host_helpers_agree_with_the_oracle():
     assert L.bcq_grid_search_workspace(ctypes.byref(d), 24, 4, 6, 3, 1) == 0      # T not a multiple of 16
     assert L.bcq_grid_search_workspace(ctypes.byref(d), 64, 7, 6, 3, 1) == 0      # more than 6 step-1 bits
     assert L.bcq_grid_search_workspace(ctypes.byref(bq.desc(256, 512, 3, 96)), 64, 4, 6, 3, 1) == 0
+
+
+def test_default_plans_are_valid_for_every_layout_variant():
+    """Seeded sweep over shapes, plane counts, scaling units and batches: the planner's choice always passes
+    the library's own plan check (workspace query non-failing, limits respected).  Host logic only."""
+    import numpy as np
+    rng = np.random.default_rng(7)
+    for _ in range(300):
+        N = 8 * int(rng.integers(1, 6000))
+        K = 512 * int(rng.integers(1, 80))
+        q = int(rng.integers(1, 5))
+        group = int(rng.choice([0, 32, 64, 128]))
+        B = int(rng.choice([1, 2, 3, 4, 5, 8, 16]))
+        d = bq.desc(N, K, q, group, bq.LAYOUT_TILED)
+        assert bq.check_desc(d) == bq.OK
+        p = bq.plan_default(d, B, 148)
+        U, W = N // 8, K // 512
+        assert p.kernel in (1, 2) and 1 <= p.row_blocks <= U and 1 <= p.k_splits <= W
+        assert -(-W // p.k_splits) <= 32
+        if group in (32, 64):
+            assert p.kernel == 1                              # no tensor-core kernel for the small groups
+        need = bq.workspace_bytes(d, B, p)
+        assert (need == 0) == (p.k_splits == 1)
+        if p.kernel == 1:
+            cols = 2 if (group == 128 and B >= 2) else 1
+            assert need in (0, cols * N * 8)
