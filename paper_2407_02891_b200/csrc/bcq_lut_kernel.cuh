@@ -825,6 +825,19 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
     unsigned long long *accum = split ? p.accum + row0 : nullptr;
     const size_t Nop = size_t(U) * kUnitRows;   // rows of this operand: its second column of y starts there
     float tot[kUnitsPerWarp], tot1[NB == 2 ? kUnitsPerWarp : 1];
+    // one scale per row: all the rows' alphas and offsets are asked for together, before the first is used
+    // (one trip to L2 for the block's last step instead of one per unit)
+    [[maybe_unused]] __half row_scale[GROUPED ? 1 : kUnitsPerWarp][Q + 1];
+    if constexpr (!GROUPED) {
+#pragma unroll
+        for (int a = 0; a < kUnitsPerWarp; ++a) {
+            const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;
+            const int u = u0 + (ul < V ? ul : 0);
+#pragma unroll
+            for (int i = 0; i < Q; ++i) row_scale[a][i] = alpha[(size_t(u) * Q + i) * kUnitRows + jr];
+            row_scale[a][Q] = zoff[size_t(u) * kUnitRows + jr];
+        }
+    }
 #pragma unroll
     for (int a = 0; a < kUnitsPerWarp; ++a) {
         const int ul = kJ * (cw + kCons * (a / kJ)) + a % kJ;   // the unit, counted inside the block
@@ -833,12 +846,11 @@ __global__ void __launch_bounds__(kLutThreads, 1) lut_gemv_kernel(const typename
         if (ul >= V) continue;                                  // (the same for the whole warp)
         float v = acc[a][0];
         if constexpr (!GROUPED) {
-            // one scale per row: apply the row's alphas and offset to the sums over this block's K range
-            const int u = u0 + ul;
+            // apply the row's alphas and offset to the sums over this block's K range
             v = 0.f;
 #pragma unroll
-            for (int i = 0; i < Q; ++i) v = fmaf(__half2float(alpha[(size_t(u) * Q + i) * kUnitRows + jr]), acc[a][i % NACC], v);
-            v = fmaf(__half2float(zoff[size_t(u) * kUnitRows + jr]), xacc, v);
+            for (int i = 0; i < Q; ++i) v = fmaf(__half2float(row_scale[a][i]), acc[a][i % NACC], v);
+            v = fmaf(__half2float(row_scale[a][Q]), xacc, v);
         }
         v += __shfl_xor_sync(0xffffffffu, v, 8);
         v += __shfl_xor_sync(0xffffffffu, v, 16);
