@@ -8,10 +8,11 @@
 // dW_p (N x K) times X^T (K x T): here the tensor cores are the right unit.  A block owns 128 rows of W
 // and up to four candidates; per 64-wide slice of K its threads form the four dW_p tiles (fp16, one fused
 // multiply-add and one rounding per element) straight into shared memory in the 128-byte-swizzled K-major
-// operand layout, X's slice is copied in beside them in the same layout, and one thread issues
+// operand layout, X's slice is copied in beside them in the same layout, and a warp of its own issues
 // tcgen05.mma (M = 128, N = T, K = 16, fp16 x fp16 -> fp32) into one accumulator per candidate in tensor
-// memory.  Two operand stages: the tensor cores work on one slice while the threads form the next; a
-// stage is handed back by tcgen05.commit on its mbarrier.  At the end every row's T outputs are read
+// memory.  Two operand stages: the 16 forming warps publish a stage on its "full" mbarrier, the issuing warp
+// hands it back by tcgen05.commit on its "free" mbarrier, so the tensor cores work on one slice while the
+// next is formed (issuing 16 MMAs holds a thread for about a microsecond: a forming thread cannot do it).  At the end every row's T outputs are read
 // back with tcgen05.ld, squared and summed.
 //
 // All waits are bounded; a wait that runs out sets a device status word (see search_status_take), the
@@ -21,7 +22,8 @@
 
 namespace bcq {
 
-constexpr int kSearchThreads = 512;      // 16 warps: forming the operand tiles is latency-bound with fewer
+constexpr int kSearchThreads = 512;      // 16 warps form the operand tiles (latency-bound with fewer)
+constexpr int kSearchBlock = kSearchThreads + 32;   // + the warp that issues the MMAs
 constexpr int kSearchRows = 128;        // rows of W per block = M of the MMA
 constexpr int kSearchKTile = 64;        // weights along K per stage: 128 bytes of fp16, one swizzle row
 constexpr int kSearchMaxCand = 4;       // candidates (accumulators) per block
@@ -85,10 +87,25 @@ __device__ __forceinline__ bool search_wait(uint32_t bar, uint32_t parity, volat
 
 // grid (row tiles of 128, groups of cand_per_block candidates); dynamic shared memory:
 // 2 stages x (cand_per_block x 16 KB of dW tiles + 32 KB for X), 1024-byte aligned.
-__global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const SearchParams p)
+// all forming threads take the same decision (a wait that gives up must not split them at a barrier)
+__device__ __forceinline__ bool formers_all(bool ok)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "barrier.cta.red.and.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(ok ? 1u : 0u), "n"(kSearchThreads)
+        : "memory");
+    return out != 0;
+}
+
+__global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const SearchParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long bars[3];   // stage 0 free, stage 1 free, all done
+    __shared__ __align__(8) unsigned long long bars[5];   // stage 0 free, stage 1 free, all done, stage 0 full, stage 1 full
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ float lut_s[kSearchMaxCand * 64];
@@ -103,7 +120,7 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
     const uint32_t bar0 = smem_u32(&bars[0]);
     volatile int *abort_flag = &abort_s;
 
-    for (int i = tid; i < ncand * p.lut_size; i += kSearchThreads) {
+    for (int i = tid; i < ncand * p.lut_size; i += kSearchBlock) {
         const int c = i / p.lut_size, v = i % p.lut_size;
         lut_s[c * 64 + v] = p.lut[size_t(cand0 + c) * 64 + v];
     }
@@ -111,6 +128,8 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
         mbar_init(bar0, 1);
         mbar_init(bar0 + 8, 1);
         mbar_init(bar0 + 16, 1);
+        mbar_init(bar0 + 24, 1);
+        mbar_init(bar0 + 32, 1);
         abort_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -126,119 +145,133 @@ __global__ void __launch_bounds__(kSearchThreads, 1) search_error_kernel(const S
     // instruction descriptor: fp32 accumulate, fp16 A and B, both K-major, N = T, M = 128
     const uint32_t idesc = (1u << 4) | (uint32_t(T >> 3) << 17) | (uint32_t(kSearchRows >> 4) << 24);
 
-    // this thread's part of a dW tile: row r of the block, 16 consecutive weights (2 pieces of 16 bytes)
-    const int r = tid >> 2, quart = tid & 3;
-    const int n = blockIdx.x * kSearchRows + r;
-    const bool row_ok = n < p.N;
-    const __half *wrow = p.W + size_t(row_ok ? n : 0) * p.K + 16 * quart;
-    const uint8_t *irow = p.w_int + size_t(row_ok ? n : 0) * p.K + 16 * quart;
-    const uint32_t a_row_off = uint32_t(r) * 128u;
-    const uint32_t lut_u32 = smem_u32(lut_s);
     const int ktiles = p.K / kSearchKTile;
-
-    uint4 wreg[2], ireg;
-    __half s_next = __float2half_rn(0.f), b_next = s_next;   // scale and offset of (row, scaling unit) of the slice on its way
-    auto load_tile = [&](int kt) {
-        const uint4 *wp = reinterpret_cast<const uint4 *>(wrow + size_t(kt) * kSearchKTile);
-        const uint4 *ip = reinterpret_cast<const uint4 *>(irow + size_t(kt) * kSearchKTile);
-        wreg[0] = row_ok ? __ldg(wp) : make_uint4(0u, 0u, 0u, 0u);
-        wreg[1] = row_ok ? __ldg(wp + 1) : make_uint4(0u, 0u, 0u, 0u);
-        ireg = row_ok ? __ldg(ip) : make_uint4(0u, 0u, 0u, 0u);
-        if (row_ok) {   // a slice of 64 lies inside one scaling unit
-            const int g = (kt * kSearchKTile) / p.L;
-            s_next = __ldg(p.S + size_t(n) * p.G + g);
-            b_next = __ldg(p.qbias + size_t(n) * p.G + g);
-        }
-    };
-    load_tile(0);
-
     bool alive = true;
-    for (int kt = 0; kt < ktiles && alive; ++kt) {
-        const int s = kt & 1;
-        const uint32_t st_base = base + uint32_t(s) * stage_bytes;
-        const uint32_t x_base = st_base + uint32_t(p.cand_per_block) * kSearchATile;
-        // the MMAs that read this stage two slices ago must be complete before it is overwritten
-        // (every thread takes the same decision: a wait that gives up must not split the block at a barrier)
-        if (kt >= 2 && !__syncthreads_and(search_wait(bar0 + 8 * s, uint32_t(((kt >> 1) - 1) & 1), abort_flag, 1) ? 1 : 0)) {
-            alive = false;
-            break;
-        }
-        // X's slice: T rows of 128 bytes, 16-byte pieces, swizzled like the dW tiles
-        for (int c = tid; c < T * 8; c += kSearchThreads) {
-            const int row = c >> 3, piece = c & 7;
-            const uint32_t dst = x_base + uint32_t(row) * 128u + uint32_t((piece ^ (row & 7)) << 4);
-            const __half *src = p.X + size_t(row) * p.K + size_t(kt) * kSearchKTile + piece * 8;
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-
-        // this slice's weights are in registers; have the next slice's on their way
-        const uint4 wcur0 = wreg[0], wcur1 = wreg[1], icur = ireg;
-        float Sf = __half2float(s_next);
-        const float qb = __half2float(b_next);
-        if (kt + 1 < ktiles) load_tile(kt + 1);
-
-        float rest[16];        // qbias - W
-        uint32_t at[16];       // shared-memory address of the first candidate's table entry of W_int
-        {
-            const uint32_t w8[8] = {wcur0.x, wcur0.y, wcur0.z, wcur0.w, wcur1.x, wcur1.y, wcur1.z, wcur1.w};
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w8[j]));
-                rest[2 * j] = qb - f.x;
-                rest[2 * j + 1] = qb - f.y;
+    if (warp == kSearchThreads / 32) {
+        // ---- the issuing warp: per slice, wait until the stage is full, issue the slice's MMAs, hand the stage back ----
+        for (int kt = 0; kt < ktiles && alive; ++kt) {
+            const int s = kt & 1;
+            if (!search_wait(bar0 + 24 + 8 * s, uint32_t((kt >> 1) & 1), abort_flag, 3)) {
+                alive = false;
+                break;
             }
-            const uint32_t i4[4] = {icur.x, icur.y, icur.z, icur.w};
+            if (lane == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t st_base = base + uint32_t(s) * stage_bytes;
+                const uint64_t bdesc = smem_desc_sw128(st_base + uint32_t(p.cand_per_block) * kSearchATile);
+                for (int c = 0; c < ncand; ++c) {
+                    const uint64_t adesc = smem_desc_sw128(st_base + uint32_t(c) * kSearchATile);
+                    const uint32_t d = tmem_base + uint32_t(c * T);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) at[j] = lut_u32 + (((i4[j >> 2] >> (8 * (j & 3))) & 0xffu) << 2);
-        }
-        if (!row_ok) Sf = 0.f;   // rows beyond N: dW = 0 (rest is 0 there as well)
-        static_for<0, kSearchMaxCand>([&](auto C) {
-            constexpr int c = decltype(C)::value;
-            if (c < ncand) {
-                const uint32_t a_base = st_base + uint32_t(c) * kSearchATile + a_row_off;
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    uint32_t packed[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int e = 8 * i + 2 * j;
-                        float l0, l1;
-                        asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l0) : "r"(at[e]), "n"(c * 256));
-                        asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l1) : "r"(at[e + 1]), "n"(c * 256));
-                        const __half2 h = __floats2half2_rn(fmaf(Sf, l0, rest[e]), fmaf(Sf, l1, rest[e + 1]));
-                        packed[j] = *reinterpret_cast<const uint32_t *>(&h);
-                    }
-                    const int piece = 2 * quart + i;
-                    const uint32_t dst = a_base + uint32_t((piece ^ (r & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[0]), "r"(packed[1]), "r"(packed[2]), "r"(packed[3]) : "memory");
+                    for (int j = 0; j < kSearchKTile / 16; ++j)   // 16 weights = 32 bytes further along the row
+                        umma_f16(d, adesc + uint64_t(2 * j), bdesc + uint64_t(2 * j), idesc, (kt > 0 || j > 0) ? 1u : 0u);
                 }
+                umma_commit(bar0 + 8 * s);
+                if (kt == ktiles - 1) umma_commit(bar0 + 16);
             }
-        });
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tiles are read by the tensor cores' proxy
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        if (tid == 0) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint64_t bdesc = smem_desc_sw128(x_base);
-            for (int c = 0; c < ncand; ++c) {
-                const uint64_t adesc = smem_desc_sw128(st_base + uint32_t(c) * kSearchATile);
-                const uint32_t d = tmem_base + uint32_t(c * T);
-#pragma unroll
-                for (int j = 0; j < kSearchKTile / 16; ++j)   // 16 weights = 32 bytes further along the row
-                    umma_f16(d, adesc + uint64_t(2 * j), bdesc + uint64_t(2 * j), idesc, (kt > 0 || j > 0) ? 1u : 0u);
-            }
-            umma_commit(bar0 + 8 * s);
-            if (kt == ktiles - 1) umma_commit(bar0 + 16);
+            __syncwarp();
         }
+    } else {
+        // this thread's part of a dW tile: row r of the block, 16 consecutive weights (2 pieces of 16 bytes)
+        const int r = tid >> 2, quart = tid & 3;
+        const int n = blockIdx.x * kSearchRows + r;
+        const bool row_ok = n < p.N;
+        const __half *wrow = p.W + size_t(row_ok ? n : 0) * p.K + 16 * quart;
+        const uint8_t *irow = p.w_int + size_t(row_ok ? n : 0) * p.K + 16 * quart;
+        const uint32_t a_row_off = uint32_t(r) * 128u;
+        const uint32_t lut_u32 = smem_u32(lut_s);
+
+        uint4 wreg[2], ireg;
+        __half s_next = __float2half_rn(0.f), b_next = s_next;   // scale and offset of (row, scaling unit) of the slice on its way
+        auto load_tile = [&](int kt) {
+            const uint4 *wp = reinterpret_cast<const uint4 *>(wrow + size_t(kt) * kSearchKTile);
+            const uint4 *ip = reinterpret_cast<const uint4 *>(irow + size_t(kt) * kSearchKTile);
+            wreg[0] = row_ok ? __ldg(wp) : make_uint4(0u, 0u, 0u, 0u);
+            wreg[1] = row_ok ? __ldg(wp + 1) : make_uint4(0u, 0u, 0u, 0u);
+            ireg = row_ok ? __ldg(ip) : make_uint4(0u, 0u, 0u, 0u);
+            if (row_ok) {   // a slice of 64 lies inside one scaling unit
+                const int g = (kt * kSearchKTile) / p.L;
+                s_next = __ldg(p.S + size_t(n) * p.G + g);
+                b_next = __ldg(p.qbias + size_t(n) * p.G + g);
+            }
+        };
+        load_tile(0);
+
+        for (int kt = 0; kt < ktiles && alive; ++kt) {
+            const int s = kt & 1;
+            const uint32_t st_base = base + uint32_t(s) * stage_bytes;
+            const uint32_t x_base = st_base + uint32_t(p.cand_per_block) * kSearchATile;
+            // the MMAs that read this stage two slices ago must be complete before it is overwritten
+            // (every thread takes the same decision: a wait that gives up must not split the block at a barrier)
+            if (kt >= 2 && !formers_all(search_wait(bar0 + 8 * s, uint32_t(((kt >> 1) - 1) & 1), abort_flag, 1))) {
+                alive = false;
+                break;
+            }
+            // X's slice: T rows of 128 bytes, 16-byte pieces, swizzled like the dW tiles
+            for (int c = tid; c < T * 8; c += kSearchThreads) {
+                const int row = c >> 3, piece = c & 7;
+                const uint32_t dst = x_base + uint32_t(row) * 128u + uint32_t((piece ^ (row & 7)) << 4);
+                const __half *src = p.X + size_t(row) * p.K + size_t(kt) * kSearchKTile + piece * 8;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+
+            // this slice's weights are in registers; have the next slice's on their way
+            const uint4 wcur0 = wreg[0], wcur1 = wreg[1], icur = ireg;
+            float Sf = __half2float(s_next);
+            const float qb = __half2float(b_next);
+            if (kt + 1 < ktiles) load_tile(kt + 1);
+
+            float rest[16];        // qbias - W
+            uint32_t at[16];       // shared-memory address of the first candidate's table entry of W_int
+            {
+                const uint32_t w8[8] = {wcur0.x, wcur0.y, wcur0.z, wcur0.w, wcur1.x, wcur1.y, wcur1.z, wcur1.w};
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w8[j]));
+                    rest[2 * j] = qb - f.x;
+                    rest[2 * j + 1] = qb - f.y;
+                }
+                const uint32_t i4[4] = {icur.x, icur.y, icur.z, icur.w};
+    #pragma unroll
+                for (int j = 0; j < 16; ++j) at[j] = lut_u32 + (((i4[j >> 2] >> (8 * (j & 3))) & 0xffu) << 2);
+            }
+            if (!row_ok) Sf = 0.f;   // rows beyond N: dW = 0 (rest is 0 there as well)
+            static_for<0, kSearchMaxCand>([&](auto C) {
+                constexpr int c = decltype(C)::value;
+                if (c < ncand) {
+                    const uint32_t a_base = st_base + uint32_t(c) * kSearchATile + a_row_off;
+    #pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        uint32_t packed[4];
+    #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int e = 8 * i + 2 * j;
+                            float l0, l1;
+                            asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l0) : "r"(at[e]), "n"(c * 256));
+                            asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l1) : "r"(at[e + 1]), "n"(c * 256));
+                            const __half2 h = __floats2half2_rn(fmaf(Sf, l0, rest[e]), fmaf(Sf, l1, rest[e + 1]));
+                            packed[j] = *reinterpret_cast<const uint32_t *>(&h);
+                        }
+                        const int piece = 2 * quart + i;
+                        const uint32_t dst = a_base + uint32_t((piece ^ (r & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[0]), "r"(packed[1]), "r"(packed[2]), "r"(packed[3]) : "memory");
+                    }
+                }
+            });
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tiles are read by the tensor cores' proxy
+            named_barrier(1, kSearchThreads);                 // every forming thread's part of the stage is written and fenced
+            if (tid == 0) mbar_arrive(bar0 + 24 + 8 * s);     // the stage is full
+        }
+
     }
 
     // ---- the accumulators are complete: every row's squared outputs ------------------------------------
     alive = __syncthreads_and((alive && search_wait(bar0 + 16, 0u, abort_flag, 2)) ? 1 : 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int quarter = warp & 3, colpart = warp >> 2;   // a warp reads the 32 lanes of its quarter, every fourth piece of 16 columns
-    if (alive) {
+    if (alive && warp < kSearchThreads / 32) {
         for (int c = 0; c < ncand; ++c) {
             float sum = 0.f;
             for (int ch = colpart; ch < T / 16; ch += 4) {
@@ -336,7 +369,7 @@ cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const 
     }
     const unsigned row_tiles = unsigned((N + kSearchRows - 1) / kSearchRows);
     const unsigned groups = unsigned((P + p.cand_per_block - 1) / p.cand_per_block);
-    search_error_kernel<<<dim3(row_tiles, groups), kSearchThreads, smem, st>>>(p);
+    search_error_kernel<<<dim3(row_tiles, groups), kSearchBlock, smem, st>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     search_sum_kernel<<<unsigned(P), 256, 0, st>>>(err_rows, N, err);
