@@ -17,6 +17,8 @@
 //
 // All waits are bounded; a wait that runs out sets a device status word (see search_status_take), the
 // block still frees its tensor memory and returns.
+#include <cuda.h>   // CUtensorMap and its enumerations (types only: the encoder is taken from the runtime)
+
 #include "bcq_async.cuh"
 #include "bcq_internal.cuh"
 
@@ -29,6 +31,8 @@ constexpr int kSearchKTile = 64;        // weights along K per stage: 128 bytes 
 constexpr int kSearchMaxCand = 4;       // candidates (accumulators) per block
 constexpr int kSearchATile = kSearchRows * kSearchKTile * 2;   // 16 KB
 constexpr int kSearchMaxT = 256;
+constexpr int kSearchWTile = kSearchRows * kSearchKTile * 2;   // a slice of W: 16 KB
+constexpr int kSearchITile = kSearchRows * kSearchKTile;       // a slice of W_int: 8 KB
 constexpr int kSearchSpin = 1 << 22;
 
 static __device__ int g_search_status = 0;
@@ -102,10 +106,30 @@ __device__ __forceinline__ bool formers_all(bool ok)
     return out != 0;
 }
 
-__global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const SearchParams p)
+// one box of a tiled tensor map into shared memory, completion counted in bytes on an mbarrier (x: the
+// innermost coordinate in elements, a multiple of 64 here: 64- or 128-byte aligned)
+__device__ __forceinline__ void tma_box_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+                 "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+// a copy this block has started must have landed before the block's shared memory is given up
+__device__ __forceinline__ void search_drain(uint32_t bar, uint32_t parity)
+{
+    for (int it = 0; it < kSearchSpin; ++it) {
+        if (mbar_test_wait(bar, parity)) return;
+        __nanosleep(64);
+    }
+}
+
+__global__ void __launch_bounds__(kSearchBlock, 1)
+    search_error_kernel(const SearchParams p, const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
+                        const __grid_constant__ CUtensorMap imap)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long bars[5];   // stage 0 free, stage 1 free, all done, stage 0 full, stage 1 full
+    // stage 0 free, stage 1 free, all done, stage 0/1 full, X of stage 0/1 landed, W and W_int of stage 0/1 landed
+    __shared__ __align__(8) unsigned long long bars[9];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ float lut_s[kSearchMaxCand * 64];
@@ -116,7 +140,8 @@ __global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const Sea
     const int ncand = min(p.cand_per_block, p.P - cand0);
     const int T = p.T;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t stage_bytes = uint32_t(p.cand_per_block) * kSearchATile + uint32_t(kSearchMaxT) * 128u;
+    const uint32_t a_bytes = uint32_t(p.cand_per_block) * kSearchATile, x_bytes = (uint32_t(T) * 128u + 1023u) & ~1023u;
+    const uint32_t stage_bytes = a_bytes + x_bytes + kSearchWTile + kSearchITile;   // dW tiles | X | W | W_int
     const uint32_t bar0 = smem_u32(&bars[0]);
     volatile int *abort_flag = &abort_s;
 
@@ -130,6 +155,7 @@ __global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const Sea
         mbar_init(bar0 + 16, 1);
         mbar_init(bar0 + 24, 1);
         mbar_init(bar0 + 32, 1);
+        for (int i = 5; i < 9; ++i) mbar_init(bar0 + 8 * i, 1);
         abort_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -151,14 +177,15 @@ __global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const Sea
         // ---- the issuing warp: per slice, wait until the stage is full, issue the slice's MMAs, hand the stage back ----
         for (int kt = 0; kt < ktiles && alive; ++kt) {
             const int s = kt & 1;
-            if (!search_wait(bar0 + 24 + 8 * s, uint32_t((kt >> 1) & 1), abort_flag, 3)) {
+            if (!search_wait(bar0 + 24 + 8 * s, uint32_t((kt >> 1) & 1), abort_flag, 3) ||
+                !search_wait(bar0 + 40 + 8 * s, uint32_t((kt >> 1) & 1), abort_flag, 4)) {
                 alive = false;
                 break;
             }
             if (lane == 0) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t st_base = base + uint32_t(s) * stage_bytes;
-                const uint64_t bdesc = smem_desc_sw128(st_base + uint32_t(p.cand_per_block) * kSearchATile);
+                const uint64_t bdesc = smem_desc_sw128(st_base + a_bytes);
                 for (int c = 0; c < ncand; ++c) {
                     const uint64_t adesc = smem_desc_sw128(st_base + uint32_t(c) * kSearchATile);
                     const uint32_t d = tmem_base + uint32_t(c * T);
@@ -174,53 +201,71 @@ __global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const Sea
     } else {
         // this thread's part of a dW tile: row r of the block, 16 consecutive weights (2 pieces of 16 bytes)
         const int r = tid >> 2, quart = tid & 3;
-        const int n = blockIdx.x * kSearchRows + r;
+        const int row0 = blockIdx.x * kSearchRows;
+        const int n = row0 + r;
         const bool row_ok = n < p.N;
-        const __half *wrow = p.W + size_t(row_ok ? n : 0) * p.K + 16 * quart;
-        const uint8_t *irow = p.w_int + size_t(row_ok ? n : 0) * p.K + 16 * quart;
         const uint32_t a_row_off = uint32_t(r) * 128u;
         const uint32_t lut_u32 = smem_u32(lut_s);
+        // W's slice lands with the 128-byte swizzle (16-byte piece ^ row & 7: a warp's loads then spread over
+        // all banks), W_int's as it is
+        const uint32_t w_off0 = a_bytes + x_bytes + uint32_t(r) * 128u + uint32_t(((2 * quart) ^ (r & 7)) << 4);
+        const uint32_t w_off1 = a_bytes + x_bytes + uint32_t(r) * 128u + uint32_t(((2 * quart + 1) ^ (r & 7)) << 4);
+        const uint32_t i_off = a_bytes + x_bytes + kSearchWTile + uint32_t(r) * 64u + uint32_t(quart << 4);
 
-        uint4 wreg[2], ireg;
-        __half s_next = __float2half_rn(0.f), b_next = s_next;   // scale and offset of (row, scaling unit) of the slice on its way
-        auto load_tile = [&](int kt) {
-            const uint4 *wp = reinterpret_cast<const uint4 *>(wrow + size_t(kt) * kSearchKTile);
-            const uint4 *ip = reinterpret_cast<const uint4 *>(irow + size_t(kt) * kSearchKTile);
-            wreg[0] = row_ok ? __ldg(wp) : make_uint4(0u, 0u, 0u, 0u);
-            wreg[1] = row_ok ? __ldg(wp + 1) : make_uint4(0u, 0u, 0u, 0u);
-            ireg = row_ok ? __ldg(ip) : make_uint4(0u, 0u, 0u, 0u);
-            if (row_ok) {   // a slice of 64 lies inside one scaling unit
-                const int g = (kt * kSearchKTile) / p.L;
-                s_next = __ldg(p.S + size_t(n) * p.G + g);
-                b_next = __ldg(p.qbias + size_t(n) * p.G + g);
-            }
-        };
-        load_tile(0);
+        // scale and offset of (row, scaling unit): loaded one slice before the unit starts (rows beyond N keep 0)
+        const int slices_per_unit = p.L / kSearchKTile;
+        const __half *srow = p.S + size_t(row_ok ? n : 0) * p.G, *brow = p.qbias + size_t(row_ok ? n : 0) * p.G;
+        __half s_next = __float2half_rn(0.f), b_next = s_next;
+        if (row_ok) s_next = __ldg(srow), b_next = __ldg(brow);
+        float Sf = 0.f, qb = 0.f;
+        int unit = 0, left = 0;   // slices left in the current scaling unit
+
+        // slices of X, W and W_int travel by tensor-map copies that one thread starts: W and W_int one slice ahead
+        // of their use, X as soon as the tensor cores have let go of the stage
+        int x_started = -1, w_started = -1;
+        if (tid == 0) {
+            mbar_expect_tx(bar0 + 56, kSearchWTile + kSearchITile);
+            tma_box_2d(base + a_bytes + x_bytes, &wmap, 0, row0, bar0 + 56);
+            tma_box_2d(base + a_bytes + x_bytes + kSearchWTile, &imap, 0, row0, bar0 + 56);
+            w_started = 0;
+        }
 
         for (int kt = 0; kt < ktiles && alive; ++kt) {
             const int s = kt & 1;
             const uint32_t st_base = base + uint32_t(s) * stage_bytes;
-            const uint32_t x_base = st_base + uint32_t(p.cand_per_block) * kSearchATile;
-            // the MMAs that read this stage two slices ago must be complete before it is overwritten
-            // (every thread takes the same decision: a wait that gives up must not split the block at a barrier)
-            if (kt >= 2 && !formers_all(search_wait(bar0 + 8 * s, uint32_t(((kt >> 1) - 1) & 1), abort_flag, 1))) {
+            // the MMAs that read this stage two slices ago must be complete before it is overwritten, and this slice
+            // of W must have landed (every thread takes the same decision: a wait that gives up must not split the
+            // block at a barrier)
+            bool ok = kt < 2 || search_wait(bar0 + 8 * s, uint32_t(((kt >> 1) - 1) & 1), abort_flag, 1);
+            ok = ok && search_wait(bar0 + 56 + 8 * s, uint32_t((kt >> 1) & 1), abort_flag, 5);
+            if (!formers_all(ok)) {
                 alive = false;
                 break;
             }
-            // X's slice: T rows of 128 bytes, 16-byte pieces, swizzled like the dW tiles
-            for (int c = tid; c < T * 8; c += kSearchThreads) {
-                const int row = c >> 3, piece = c & 7;
-                const uint32_t dst = x_base + uint32_t(row) * 128u + uint32_t((piece ^ (row & 7)) << 4);
-                const __half *src = p.X + size_t(row) * p.K + size_t(kt) * kSearchKTile + piece * 8;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            if (tid == 0) {
+                mbar_expect_tx(bar0 + 40 + 8 * s, uint32_t(T) * 128u);
+                tma_box_2d(st_base + a_bytes, &xmap, kt * kSearchKTile, 0, bar0 + 40 + 8 * s);
+                x_started = kt;
+                if (kt + 1 < ktiles) {   // the other stage's W was last read one slice ago, before that slice's barrier
+                    const uint32_t other = base + uint32_t(s ^ 1) * stage_bytes + a_bytes + x_bytes;
+                    mbar_expect_tx(bar0 + 56 + 8 * (s ^ 1), kSearchWTile + kSearchITile);
+                    tma_box_2d(other, &wmap, (kt + 1) * kSearchKTile, row0, bar0 + 56 + 8 * (s ^ 1));
+                    tma_box_2d(other + kSearchWTile, &imap, (kt + 1) * kSearchKTile, row0, bar0 + 56 + 8 * (s ^ 1));
+                    w_started = kt + 1;
+                }
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
 
-            // this slice's weights are in registers; have the next slice's on their way
-            const uint4 wcur0 = wreg[0], wcur1 = wreg[1], icur = ireg;
-            float Sf = __half2float(s_next);
-            const float qb = __half2float(b_next);
-            if (kt + 1 < ktiles) load_tile(kt + 1);
+            uint4 wcur0, wcur1, icur;
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(wcur0.x), "=r"(wcur0.y), "=r"(wcur0.z), "=r"(wcur0.w) : "r"(st_base + w_off0));
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(wcur1.x), "=r"(wcur1.y), "=r"(wcur1.z), "=r"(wcur1.w) : "r"(st_base + w_off1));
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(icur.x), "=r"(icur.y), "=r"(icur.z), "=r"(icur.w) : "r"(st_base + i_off));
+            if (left == 0) {
+                Sf = __half2float(s_next), qb = __half2float(b_next);
+                left = slices_per_unit;
+                ++unit;
+                if (row_ok && unit < p.G) s_next = __ldg(srow + unit), b_next = __ldg(brow + unit);
+            }
+            --left;
 
             float rest[16];        // qbias - W
             uint32_t at[16];       // shared-memory address of the first candidate's table entry of W_int
@@ -236,7 +281,7 @@ __global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const Sea
     #pragma unroll
                 for (int j = 0; j < 16; ++j) at[j] = lut_u32 + (((i4[j >> 2] >> (8 * (j & 3))) & 0xffu) << 2);
             }
-            if (!row_ok) Sf = 0.f;   // rows beyond N: dW = 0 (rest is 0 there as well)
+            // (rows beyond N: the copies filled zeros and the scale and offset are 0, so dW = 0)
             static_for<0, kSearchMaxCand>([&](auto C) {
                 constexpr int c = decltype(C)::value;
                 if (c < ncand) {
@@ -259,10 +304,13 @@ __global__ void __launch_bounds__(kSearchBlock, 1) search_error_kernel(const Sea
                     }
                 }
             });
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tiles are read by the tensor cores' proxy
             named_barrier(1, kSearchThreads);                 // every forming thread's part of the stage is written and fenced
             if (tid == 0) mbar_arrive(bar0 + 24 + 8 * s);     // the stage is full
+        }
+        if (tid == 0 && !alive) {   // giving up: the copies that were started still land in this block's shared memory
+            for (int j = x_started; j >= 0 && j > x_started - 2; --j) search_drain(bar0 + 40 + 8 * (j & 1), uint32_t((j >> 1) & 1));
+            for (int j = w_started; j >= 0 && j > w_started - 2; --j) search_drain(bar0 + 56 + 8 * (j & 1), uint32_t((j >> 1) & 1));
         }
 
     }
@@ -334,12 +382,44 @@ __global__ void search_argmin_kernel(const double *__restrict__ err, int count, 
     best[1] = at % P;
 }
 
-size_t search_smem_bytes(int cand_per_block) { return 2 * (size_t(cand_per_block) * kSearchATile + size_t(kSearchMaxT) * 128) + 1024; }
-
 int search_cand_per_block(int T)
 {
     int c = 512 / T;
     return c > kSearchMaxCand ? kSearchMaxCand : c;
+}
+
+// two stages of (dW tiles | X | W | W_int), each part a multiple of 1024 bytes, + room to align the first
+size_t search_smem_bytes(int T)
+{
+    const size_t x_bytes = (size_t(T) * 128 + 1023) / 1024 * 1024;
+    return 2 * (size_t(search_cand_per_block(T)) * kSearchATile + x_bytes + kSearchWTile + kSearchITile) + 1024;
+}
+
+// Tensor map of a row-major matrix [rows][cols] for boxes of 64 columns x box_rows rows.  The encoder is a
+// driver function; the runtime hands out its address, so the library links against the runtime only.
+static cudaError_t search_tensor_map(CUtensorMap *map, const void *ptr, bool bytes, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                                     bool swizzle)
+{
+    using Encode = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static Encode encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
+        const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &found);
+        if (e != cudaSuccess) return e;
+        if (found != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        encode = reinterpret_cast<Encode>(fn);
+    }
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * (bytes ? 1u : 2u)};
+    const cuuint32_t box[2] = {uint32_t(kSearchKTile), box_rows};
+    const cuuint32_t steps[2] = {1u, 1u};
+    const CUresult r = encode(map, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(ptr), dims,
+                              strides, box, steps, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias, const uint16_t *X,
@@ -361,15 +441,22 @@ cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const 
     p.tmem_cols = cols;
     p.lut_size = 1 << n_bits;
     p.lut = lut_dev;
-    const size_t smem = search_smem_bytes(p.cand_per_block);
+    const size_t smem = search_smem_bytes(T);
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(search_error_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(search_smem_bytes(kSearchMaxCand)));
+        size_t most = 0;
+        for (int t = 16; t <= kSearchMaxT; t += 16) most = search_smem_bytes(t) > most ? search_smem_bytes(t) : most;
+        e = cudaFuncSetAttribute(search_error_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(most));
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
+    // the slices of X (all T rows), W and W_int (the block's 128 rows; rows beyond N read as zeros)
+    CUtensorMap xmap, wmap, imap;
+    if ((e = search_tensor_map(&xmap, X, false, uint64_t(T), uint64_t(K), uint32_t(T), true)) != cudaSuccess) return e;
+    if ((e = search_tensor_map(&wmap, W, false, uint64_t(N), uint64_t(K), uint32_t(kSearchRows), true)) != cudaSuccess) return e;
+    if ((e = search_tensor_map(&imap, w_int, true, uint64_t(N), uint64_t(K), uint32_t(kSearchRows), false)) != cudaSuccess) return e;
     const unsigned row_tiles = unsigned((N + kSearchRows - 1) / kSearchRows);
     const unsigned groups = unsigned((P + p.cand_per_block - 1) / p.cand_per_block);
-    search_error_kernel<<<dim3(row_tiles, groups), kSearchBlock, smem, st>>>(p);
+    search_error_kernel<<<dim3(row_tiles, groups), kSearchBlock, smem, st>>>(p, xmap, wmap, imap);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     search_sum_kernel<<<unsigned(P), 256, 0, st>>>(err_rows, N, err);
