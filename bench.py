@@ -539,7 +539,7 @@ def run_search(args):
         "vs_baseline": None, "dtype": "f16 operands, f32 accumulate (tcgen05)", "data": "synthetic",
         "config": {"workload": f"search_{N}x{K}_T{T}_n{n_bits}_q{q}_g{group}", "candidates": int(len(parts)),
                    "scale_factors": n_scales, "tokens": T},
-        "clocks": clocks.summary(), "gpu_launches": steps * n_scales * 3 + steps,
+        "clocks": clocks.summary(), "gpu_launches": steps * (n_scales + 2 * ((n_scales + 7) // 8) + 1),   # quantiser per factor; errors and sums per 8 factors; argmin
         "roofline": {"bound": "tensor", "achieved": round(flops / ms / 1e9, 1), "peak": peak, "unit": "TFLOP/s",
                      "frac": round(flops / ms / 1e9 / peak, 4), "peak_kind": peak_kind, "traffic": None,
                      "kernel": "search_error_kernel", "flops_per_step": flops},

@@ -431,23 +431,30 @@ int enumerate_partitions(int n, int q, int index, uint8_t *out)
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Scale factors are searched several per launch (a launch of 128-row blocks x groups of candidates alone leaves the
+// last wave of blocks partly empty): step 1's outputs of kSearchScalesPerLaunch factors sit side by side.
+constexpr int kSearchScalesPerLaunch = 8;
 struct SearchLayout {
     size_t lut, w_int, S, qbias, packed, alpha, z, err, err_rows, total;
+    size_t w_int_each, S_each;   // bytes of one scale factor's W_int; of its S (and of its qbias)
+    int together;                // scale factors per launch
 };
 SearchLayout search_layout(const bcq_desc &d, int P, int n_scales, bool own_rows)
 {
     SearchLayout L;
     const size_t G = size_t(n_groups(d));
+    L.together = n_scales < kSearchScalesPerLaunch ? n_scales : kSearchScalesPerLaunch;
+    L.w_int_each = size_t(d.N) * d.K, L.S_each = round_up(size_t(d.N) * G * 2, 256);
     size_t at = 0;
     L.lut = at, at += round_up(size_t(P) * 64 * sizeof(float), 256);
-    L.w_int = at, at += round_up(size_t(d.N) * d.K, 256);
-    L.S = at, at += round_up(size_t(d.N) * G * 2, 256);
-    L.qbias = at, at += round_up(size_t(d.N) * G * 2, 256);
+    L.w_int = at, at += round_up(L.w_int_each * L.together, 256);
+    L.S = at, at += L.S_each * L.together;
+    L.qbias = at, at += L.S_each * L.together;
     L.packed = at, at += round_up(size_t(d.q) * d.N * (d.K / 8), 256);
     L.alpha = at, at += round_up(size_t(d.q) * d.N * G * 2, 256);
     L.z = at, at += round_up(size_t(d.N) * G * 2, 256);
     L.err = at, at += round_up(size_t(n_scales) * P * sizeof(double), 256);
-    L.err_rows = at, at += own_rows ? round_up(size_t(P) * d.N * sizeof(float), 256) : 0;
+    L.err_rows = at, at += own_rows ? round_up(size_t(L.together) * P * d.N * sizeof(float), 256) : 0;
     L.total = at;
     return L;
 }
@@ -910,11 +917,16 @@ int bcq_grid_search(const bcq_desc *desc, const uint16_t *W, const uint16_t *X, 
     cudaError_t e = cudaMemcpyAsync(lut_dev, lut.data(), lut.size() * sizeof(float), cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return cuda_fail(e);
     const View scratch = make_view(d, base + L.packed, reinterpret_cast<uint16_t *>(base + L.alpha), reinterpret_cast<uint16_t *>(base + L.z));
-    for (int s = 0; s < n_scales; ++s) {
-        e = launch_quantize_rtn(W, n_bits, s_factors[s], code_of_int, weight, S, qbias, w_int, scratch, st);
-        if (e != cudaSuccess) return cuda_fail(e);
-        float *rows = err_rows ? err_rows + size_t(s) * P * d.N : reinterpret_cast<float *>(base + L.err_rows);
-        e = launch_search_errors(W, w_int, S, qbias, X, d.N, d.K, d.group, T, n_bits, lut_dev, P, rows, err_all + size_t(s) * P, st);
+    for (int s0 = 0; s0 < n_scales; s0 += L.together) {
+        const int count = n_scales - s0 < L.together ? n_scales - s0 : L.together;
+        for (int i = 0; i < count; ++i) {
+            e = launch_quantize_rtn(W, n_bits, s_factors[s0 + i], code_of_int, weight, S + i * (L.S_each / 2), qbias + i * (L.S_each / 2),
+                                    w_int + i * L.w_int_each, scratch, st);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+        float *rows = err_rows ? err_rows + size_t(s0) * P * d.N : reinterpret_cast<float *>(base + L.err_rows);
+        e = launch_search_errors(W, w_int, S, qbias, L.S_each / 2, X, d.N, d.K, d.group, T, n_bits, lut_dev, P, count, rows,
+                                 err_all + size_t(s0) * P, st);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     e = launch_search_argmin(err_all, n_scales * P, P, best, st);

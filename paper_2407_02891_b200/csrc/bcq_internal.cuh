@@ -168,11 +168,12 @@ cudaError_t launch_mma_gemm(const bcq_desc &d, const bcq_plan &plan, const void 
 int record_cuda_error(cudaError_t e);   // text for bcq_last_cuda_error(); returns BCQ_ERR_CUDA
 
 // The search of section "Quantize Weight Twice" / "Re-explore Scale Factor": output errors of P candidates for
-// one scale factor (err_rows [P][N] per row, err [P] summed in a fixed order), and the first minimum of `count`
-// errors laid out [.][P].
-cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias, const uint16_t *X,
-                                 int N, int K, int group, int T, int n_bits, const float *lut_dev /*[P][64]*/, int P,
-                                 float *err_rows, double *err, cudaStream_t st);
+// `scales` scale factors in one launch (step 1's outputs of the factors side by side: w_int [scales][N][K], S and
+// qbias `scale_stride` elements apart; err_rows [scales][P][N] per row, err [scales][P] summed in a fixed order),
+// and the first minimum of `count` errors laid out [.][P].
+cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias, size_t scale_stride,
+                                 const uint16_t *X, int N, int K, int group, int T, int n_bits, const float *lut_dev /*[P][64]*/, int P,
+                                 int scales, float *err_rows, double *err, cudaStream_t st);
 cudaError_t launch_search_argmin(const double *err, int count, int P, int *best, cudaStream_t st);
 cudaError_t search_status_take(int *status);
 

@@ -8,12 +8,13 @@
 // dW_p (N x K) times X^T (K x T): here the tensor cores are the right unit.  A block owns 128 rows of W
 // and up to four candidates; per 64-wide slice of K its threads form the four dW_p tiles (fp16, one fused
 // multiply-add and one rounding per element) straight into shared memory in the 128-byte-swizzled K-major
-// operand layout, X's slice is copied in beside them in the same layout, and a warp of its own issues
-// tcgen05.mma (M = 128, N = T, K = 16, fp16 x fp16 -> fp32) into one accumulator per candidate in tensor
-// memory.  Two operand stages: the 16 forming warps publish a stage on its "full" mbarrier, the issuing warp
-// hands it back by tcgen05.commit on its "free" mbarrier, so the tensor cores work on one slice while the
-// next is formed (issuing 16 MMAs holds a thread for about a microsecond: a forming thread cannot do it).  At the end every row's T outputs are read
-// back with tcgen05.ld, squared and summed.
+// operand layout, and a warp of its own issues tcgen05.mma (M = 128, N = T, K = 16, fp16 x fp16 -> fp32) into
+// one accumulator per candidate in tensor memory.  The slices of X (same layout), W and W_int arrive by tensor-map
+// copies that one thread starts: thousands of 16-byte loads per slice would hold the forming warps at the load
+// queue.  Two operand stages: the 16 forming warps publish a stage on its "full" mbarrier, the issuing warp hands it
+// back by tcgen05.commit on its "free" mbarrier, so the tensor cores work on one slice while the next is formed
+// (issuing 16 MMAs holds a thread for about a microsecond: a forming thread cannot do it).  At the end every row's
+// T outputs are read back with tcgen05.ld, squared and summed.  Several scale factors share a launch (grid z).
 //
 // All waits are bounded; a wait that runs out sets a device status word (see search_status_take), the
 // block still frees its tensor memory and returns.
@@ -40,10 +41,11 @@ static __device__ int g_search_status = 0;
 struct SearchParams {
     const __half *W;        // [N][K]
     const uint8_t *w_int;   // [N][K]
-    const __half *S;        // [N][G]
-    const __half *qbias;    // [N][G]
+    const __half *S;        // [N][G] per scale factor, scale_stride elements apart
+    const __half *qbias;    // [N][G], likewise
+    size_t scale_stride;
     const __half *X;        // [T][K]
-    float *err_rows;        // [P][N] of this scale factor
+    float *err_rows;        // [scale factor][P][N]
     int N, K, G, L;         // L = weights per scaling unit (K when one per row)
     int T, P;
     int cand_per_block;     // 1..4, so that cand_per_block * T <= 512 columns of tensor memory
@@ -89,7 +91,7 @@ __device__ __forceinline__ bool search_wait(uint32_t bar, uint32_t parity, volat
     return false;
 }
 
-// grid (row tiles of 128, groups of cand_per_block candidates); dynamic shared memory:
+// grid (row tiles of 128, groups of cand_per_block candidates, scale factors); dynamic shared memory:
 // 2 stages x (cand_per_block x 16 KB of dW tiles + 32 KB for X), 1024-byte aligned.
 // all forming threads take the same decision (a wait that gives up must not split them at a barrier)
 __device__ __forceinline__ bool formers_all(bool ok)
@@ -214,7 +216,9 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
 
         // scale and offset of (row, scaling unit): loaded one slice before the unit starts (rows beyond N keep 0)
         const int slices_per_unit = p.L / kSearchKTile;
-        const __half *srow = p.S + size_t(row_ok ? n : 0) * p.G, *brow = p.qbias + size_t(row_ok ? n : 0) * p.G;
+        const size_t s_at = size_t(blockIdx.z) * p.scale_stride + size_t(row_ok ? n : 0) * p.G;
+        const __half *srow = p.S + s_at, *brow = p.qbias + s_at;
+        const int irow0 = int(blockIdx.z) * p.N + row0;   // W_int of the scale factors: one matrix of gridDim.z * N rows
         __half s_next = __float2half_rn(0.f), b_next = s_next;
         if (row_ok) s_next = __ldg(srow), b_next = __ldg(brow);
         float Sf = 0.f, qb = 0.f;
@@ -226,7 +230,7 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
         if (tid == 0) {
             mbar_expect_tx(bar0 + 56, kSearchWTile + kSearchITile);
             tma_box_2d(base + a_bytes + x_bytes, &wmap, 0, row0, bar0 + 56);
-            tma_box_2d(base + a_bytes + x_bytes + kSearchWTile, &imap, 0, row0, bar0 + 56);
+            tma_box_2d(base + a_bytes + x_bytes + kSearchWTile, &imap, 0, irow0, bar0 + 56);
             w_started = 0;
         }
 
@@ -250,7 +254,7 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
                     const uint32_t other = base + uint32_t(s ^ 1) * stage_bytes + a_bytes + x_bytes;
                     mbar_expect_tx(bar0 + 56 + 8 * (s ^ 1), kSearchWTile + kSearchITile);
                     tma_box_2d(other, &wmap, (kt + 1) * kSearchKTile, row0, bar0 + 56 + 8 * (s ^ 1));
-                    tma_box_2d(other + kSearchWTile, &imap, (kt + 1) * kSearchKTile, row0, bar0 + 56 + 8 * (s ^ 1));
+                    tma_box_2d(other + kSearchWTile, &imap, (kt + 1) * kSearchKTile, irow0, bar0 + 56 + 8 * (s ^ 1));
                     w_started = kt + 1;
                 }
             }
@@ -281,7 +285,8 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
     #pragma unroll
                 for (int j = 0; j < 16; ++j) at[j] = lut_u32 + (((i4[j >> 2] >> (8 * (j & 3))) & 0xffu) << 2);
             }
-            // (rows beyond N: the copies filled zeros and the scale and offset are 0, so dW = 0)
+            // (rows beyond N: W reads as zeros and the scale and offset are 0, so dW = 0 whatever W_int holds there --
+            // zeros, or the next scale factor's first rows)
             static_for<0, kSearchMaxCand>([&](auto C) {
                 constexpr int c = decltype(C)::value;
                 if (c < ncand) {
@@ -346,7 +351,7 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
         const int row = blockIdx.x * kSearchRows + tid;
         if (row < p.N)
             for (int c = 0; c < ncand; ++c)
-                p.err_rows[size_t(cand0 + c) * p.N + row] = (part[0][c][tid] + part[1][c][tid]) + (part[2][c][tid] + part[3][c][tid]);
+                p.err_rows[(size_t(blockIdx.z) * p.P + size_t(cand0 + c)) * p.N + row] = (part[0][c][tid] + part[1][c][tid]) + (part[2][c][tid] + part[3][c][tid]);
     }
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -422,9 +427,9 @@ static cudaError_t search_tensor_map(CUtensorMap *map, const void *ptr, bool byt
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias, const uint16_t *X,
-                                 int N, int K, int group, int T, int n_bits, const float *lut_dev /*[P][64]*/, int P,
-                                 float *err_rows /*[P][N]*/, double *err /*[P]*/, cudaStream_t st)
+cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const uint16_t *S, const uint16_t *qbias, size_t scale_stride,
+                                 const uint16_t *X, int N, int K, int group, int T, int n_bits, const float *lut_dev /*[P][64]*/, int P,
+                                 int scales, float *err_rows /*[scales][P][N]*/, double *err /*[scales][P]*/, cudaStream_t st)
 {
     static bool configured[64] = {};
     int dev = 0;
@@ -432,7 +437,7 @@ cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const 
     if (e != cudaSuccess) return e;
     SearchParams p = {};
     p.W = reinterpret_cast<const __half *>(W), p.w_int = w_int;
-    p.S = reinterpret_cast<const __half *>(S), p.qbias = reinterpret_cast<const __half *>(qbias);
+    p.S = reinterpret_cast<const __half *>(S), p.qbias = reinterpret_cast<const __half *>(qbias), p.scale_stride = scale_stride;
     p.X = reinterpret_cast<const __half *>(X), p.err_rows = err_rows;
     p.N = N, p.K = K, p.L = group == 0 ? K : group, p.G = K / p.L, p.T = T, p.P = P;
     p.cand_per_block = search_cand_per_block(T);
@@ -449,17 +454,18 @@ cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const 
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    // the slices of X (all T rows), W and W_int (the block's 128 rows; rows beyond N read as zeros)
+    // the slices of X (all T rows), W (the block's 128 rows; rows beyond N read as zeros) and W_int (the scale
+    // factors' matrices as one of scales * N rows)
     CUtensorMap xmap, wmap, imap;
     if ((e = search_tensor_map(&xmap, X, false, uint64_t(T), uint64_t(K), uint32_t(T), true)) != cudaSuccess) return e;
     if ((e = search_tensor_map(&wmap, W, false, uint64_t(N), uint64_t(K), uint32_t(kSearchRows), true)) != cudaSuccess) return e;
-    if ((e = search_tensor_map(&imap, w_int, true, uint64_t(N), uint64_t(K), uint32_t(kSearchRows), false)) != cudaSuccess) return e;
+    if ((e = search_tensor_map(&imap, w_int, true, uint64_t(scales) * uint64_t(N), uint64_t(K), uint32_t(kSearchRows), false)) != cudaSuccess) return e;
     const unsigned row_tiles = unsigned((N + kSearchRows - 1) / kSearchRows);
     const unsigned groups = unsigned((P + p.cand_per_block - 1) / p.cand_per_block);
-    search_error_kernel<<<dim3(row_tiles, groups), kSearchBlock, smem, st>>>(p, xmap, wmap, imap);
+    search_error_kernel<<<dim3(row_tiles, groups, unsigned(scales)), kSearchBlock, smem, st>>>(p, xmap, wmap, imap);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    search_sum_kernel<<<unsigned(P), 256, 0, st>>>(err_rows, N, err);
+    search_sum_kernel<<<unsigned(P) * unsigned(scales), 256, 0, st>>>(err_rows, N, err);
     return cudaGetLastError();
 }
 

@@ -54,6 +54,7 @@ def _check(N, K, T, q, group, n_bits, n_scales, name):
     (136, 576, 48, 3, 0, 5, 1),        # 25 candidates, K = 9 slices, T = 48
     (128, 128, 64, 1, 128, 2, 3),      # one plane
     (128, 256, 32, 4, 128, 6, 1),      # six step-1 bits into four planes: 65 candidates, tables of 64 entries
+    (200, 256, 32, 2, 128, 3, 11),     # more scale factors than one launch takes (8 + 3), ragged row tiles between them
 ])
 def test_grid_search_matches_the_oracle(N, K, T, q, group, n_bits, n_scales):
     _check(N, K, T, q, group, n_bits, n_scales, f"search/{N}x{K}x{T}")
