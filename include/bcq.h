@@ -394,7 +394,8 @@ int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, const uint16_
  *   s_factors_host [n_scales] (bcq_reexplore_factors gives an even grid inside the interval of Eq. reexplore).
  *   err_dev [n_scales][P] fp64; err_rows_dev [n_scales][P][N] fp32 or NULL; best_dev [2] int32.
  *   workspace: bcq_grid_search_workspace(desc, T, n_bits, P, n_scales, err_rows_dev != NULL) bytes, 256-byte
- *   aligned; holds W_int, S, qbias and a scratch operand of the current scale.  Asynchronous on `stream`.
+ *   aligned; holds W_int, S and qbias of up to 8 scale factors (searched together in one launch: N * K bytes
+ *   each) and a scratch operand.  Asynchronous on `stream`.
  */
 size_t bcq_grid_search_workspace(const bcq_desc *desc, int T, int n_bits, int P, int n_scales, int rows_given);
 int bcq_grid_search(const bcq_desc *desc, const uint16_t *W_dev, const uint16_t *X_dev, int T, int n_bits,
