@@ -97,3 +97,24 @@ def test_grid_search_exact_candidate_has_zero_error():
     e = err.cpu().numpy()
     assert e[1, 2] == 0.0 and tuple(best.cpu().numpy()) == (1, 2)
     assert (np.delete(e[1], 2) > 0).all()
+
+
+@pytest.mark.parametrize("T", [128, 256])
+def test_grid_search_fullsize_sampled_rows(T):
+    # the configuration bench.py --search times (7168 x 7168, 25 candidates x 8 scale factors in one launch): rows
+    # are independent, so the oracle recomputes a seeded sample of them
+    N = K = 7168
+    W, X = _inputs("search/full", N, K, T)
+    parts, s = bq.partitions(5, 3), bq.reexplore_factors(5, 8)
+    err, rows_out, best = bq.grid_search(N, K, 3, 128, torch.from_numpy(W).to(DEV), torch.from_numpy(X).to(DEV), 5, parts, s)
+    torch.cuda.synchronize()
+    assert bq.lib().bcq_poll_status() == bq.OK
+    rows = np.unique(synth.u64("search/full/rows", 0, 12) % np.uint64(N)).astype(np.int64)
+    rows = np.concatenate([rows, [0, N - 1]])
+    ref_rows, _, _ = oracle.grid_search(W[rows], X, 128, 5, list(parts), s)
+    got = rows_out.cpu().numpy().astype(np.float64)
+    assert np.abs(got[:, :, rows] - ref_rows).max() <= RTOL * np.abs(ref_rows).max()
+    e = err.cpu().numpy()
+    np.testing.assert_allclose(e, got.sum(axis=2), rtol=1e-5)
+    si, pi = (int(v) for v in best.cpu().numpy())
+    assert e[si, pi] == e.min()
