@@ -87,7 +87,8 @@ struct LutCfg {
     static constexpr int kJ = kChoice == 0 ? 2 : 1;
     static constexpr int kD = kChoice == 0 ? 2 : (kChoice == 1 ? 3 : 2);
     static constexpr int kCons = rings(kJ, kD) < kLutConsumersMax ? rings(kJ, kD) : kLutConsumersMax;
-    static constexpr int kProducers = kJ == 1 ? 2 : 1;   // one warp starts about 18 copies per microsecond
+    // one warp starts about 18 copies per microsecond: enough for jobs of two 1792-byte tiles, not for smaller ones
+    static constexpr int kProducers = (kJ == 1 || Q <= 2) ? 2 : 1;
     static constexpr int kFirstCons = kProducers + kBuilderWarps;
     static constexpr int kWorking = kBuilderWarps + kCons;   // warps that take part after the producers split off
     static constexpr int kJobsPerWarp = kUnitsPerWarp / kJ;
