@@ -385,8 +385,9 @@ int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, const uint16_
  *     err_rows[s][p][n] = sum_t ( sum_k (S W_q[n][k] + qbias - W[n][k]) X[t][k] )^2
  *     err[s][p]         = sum_n err_rows[s][p][n]
  * and best = (s, p) of the first candidate, in loop order, whose err is below all earlier ones.
- * The contraction runs on the tensor cores with fp16 operands (the weight differences are rounded once to
- * fp16) and fp32 accumulation; the error values agree with an fp64 evaluation to about 1e-3 relative, so
+ * The contraction runs on the tensor cores with fp16 operands (a weight difference is formed as
+ * S (W_q - W_int) + r, r = S W_int + qbias - W computed in fp32 and rounded to fp16, by one fp16 fused
+ * multiply-add) and fp32 accumulation; the error values agree with an fp64 evaluation to about 1e-3 relative, so
  * candidates closer than that may swap places.  GPTQ's error compensation is not part of this call.
  *   W [N][K] fp16 weights, X [T][K] fp16 calibration inputs (device, 16-byte aligned); T a multiple of 16,
  *   16..256; K a multiple of 64; desc->group 0 or a multiple of 64; n_bits 1..6; desc->layout is ignored.

@@ -6,8 +6,10 @@
 //
 // lut_p[v] = the integer of BCchoice p nearest to v (Eq. round).  The inner sum is a dense contraction
 // dW_p (N x K) times X^T (K x T): here the tensor cores are the right unit.  A block owns 128 rows of W
-// and up to four candidates; per 64-wide slice of K its threads form the four dW_p tiles (fp16, one fused
-// multiply-add and one rounding per element) straight into shared memory in the 128-byte-swizzled K-major
+// and up to four candidates; per 64-wide slice of K its threads form the four dW_p tiles in fp16 (dW_p = S step_p[v] + r:
+// step_p[v] = lut_p[v] - v, one shared-memory word per element holds it for all four candidates; r = S v + qbias - W, the
+// residual of step 1, fp32 and rounded to fp16 once; one fp16 fused multiply-add per pair of elements and candidate)
+// straight into shared memory in the 128-byte-swizzled K-major
 // operand layout, and a warp of its own issues tcgen05.mma (M = 128, N = T, K = 16, fp16 x fp16 -> fp32) into
 // one accumulator per candidate in tensor memory.  The slices of X (same layout), W and W_int arrive by tensor-map
 // copies that one thread starts: thousands of 16-byte loads per slice would hold the forming warps at the load
@@ -134,7 +136,9 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
     __shared__ __align__(8) unsigned long long bars[9];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    __shared__ float lut_s[kSearchMaxCand * 64];
+    // per value v of W_int one word: byte c = 128 + lut_c[v] - v, the step from v to the nearest integer of the block's
+    // candidate c (between -63 and 63).  One lookup per operand element serves the four candidates.
+    __shared__ uint32_t step_s[64];
     __shared__ float part[4][kSearchMaxCand][kSearchRows];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -147,9 +151,13 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
     const uint32_t bar0 = smem_u32(&bars[0]);
     volatile int *abort_flag = &abort_s;
 
-    for (int i = tid; i < ncand * p.lut_size; i += kSearchBlock) {
-        const int c = i / p.lut_size, v = i % p.lut_size;
-        lut_s[c * 64 + v] = p.lut[size_t(cand0 + c) * 64 + v];
+    for (int v = tid; v < p.lut_size; v += kSearchBlock) {
+        uint32_t word = 0x80808080u;   // candidates the block does not have: step 0
+        for (int c = 0; c < ncand; ++c) {
+            const int step = int(p.lut[size_t(cand0 + c) * 64 + v]) - v;   // the table holds integers
+            word = (word & ~(0xffu << (8 * c))) | (uint32_t(128 + step) << (8 * c));
+        }
+        step_s[v] = word;
     }
     if (tid == 0) {
         mbar_init(bar0, 1);
@@ -207,7 +215,7 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
         const int n = row0 + r;
         const bool row_ok = n < p.N;
         const uint32_t a_row_off = uint32_t(r) * 128u;
-        const uint32_t lut_u32 = smem_u32(lut_s);
+        const uint32_t step_u32 = smem_u32(step_s);
         // W's slice lands with the 128-byte swizzle (16-byte piece ^ row & 7: a warp's loads then spread over
         // all banks), W_int's as it is
         const uint32_t w_off0 = a_bytes + x_bytes + uint32_t(r) * 128u + uint32_t(((2 * quart) ^ (r & 7)) << 4);
@@ -222,6 +230,7 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
         __half s_next = __float2half_rn(0.f), b_next = s_next;
         if (row_ok) s_next = __ldg(srow), b_next = __ldg(brow);
         float Sf = 0.f, qb = 0.f;
+        __half Sh = s_next;
         int unit = 0, left = 0;   // slices left in the current scaling unit
 
         // slices of X, W and W_int travel by tensor-map copies that one thread starts: W and W_int one slice ahead
@@ -264,51 +273,66 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
             asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(wcur1.x), "=r"(wcur1.y), "=r"(wcur1.z), "=r"(wcur1.w) : "r"(st_base + w_off1));
             asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(icur.x), "=r"(icur.y), "=r"(icur.z), "=r"(icur.w) : "r"(st_base + i_off));
             if (left == 0) {
-                Sf = __half2float(s_next), qb = __half2float(b_next);
+                Sh = s_next, Sf = __half2float(s_next), qb = __half2float(b_next);
                 left = slices_per_unit;
                 ++unit;
                 if (row_ok && unit < p.G) s_next = __ldg(srow + unit), b_next = __ldg(brow + unit);
             }
             --left;
 
-            float rest[16];        // qbias - W
-            uint32_t at[16];       // shared-memory address of the first candidate's table entry of W_int
+            // dW_p = S lut_p[v] + qbias - W = S (lut_p[v] - v) + r with r = S v + qbias - W, the residual of step 1.
+            // r: one fp32 fused multiply-add, rounded to fp16 once for all candidates.  Per candidate the step comes
+            // out of the lookup's byte as the fp16 number 1024 + byte (bit pattern 0x6400 | byte), minus 1152; one
+            // fp16 fused multiply-add on a pair of weights then is the operand as it is stored (rounded once).
+            uint32_t resid[8];     // r of weights (2 j, 2 j + 1), fp16 pairs
+            uint32_t at[16];       // shared-memory address of the word of W_int's value
             {
                 const uint32_t w8[8] = {wcur0.x, wcur0.y, wcur0.z, wcur0.w, wcur1.x, wcur1.y, wcur1.z, wcur1.w};
+                const uint32_t i4[4] = {icur.x, icur.y, icur.z, icur.w};
     #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w8[j]));
-                    rest[2 * j] = qb - f.x;
-                    rest[2 * j + 1] = qb - f.y;
+                    // a byte below the bit pattern of 2^23 is the float 2^23 + v
+                    const float v0 = __uint_as_float(__byte_perm(i4[j >> 1], 0x4B000000u, 0x7440u + uint32_t(2 * (j & 1)))) - 8388608.f;
+                    const float v1 = __uint_as_float(__byte_perm(i4[j >> 1], 0x4B000000u, 0x7441u + uint32_t(2 * (j & 1)))) - 8388608.f;
+                    const __half2 h = __floats2half2_rn(fmaf(Sf, v0, qb - f.x), fmaf(Sf, v1, qb - f.y));
+                    resid[j] = *reinterpret_cast<const uint32_t *>(&h);
                 }
-                const uint32_t i4[4] = {icur.x, icur.y, icur.z, icur.w};
     #pragma unroll
-                for (int j = 0; j < 16; ++j) at[j] = lut_u32 + (((i4[j >> 2] >> (8 * (j & 3))) & 0xffu) << 2);
+                for (int j = 0; j < 16; ++j) at[j] = step_u32 + (((i4[j >> 2] >> (8 * (j & 3))) & 0xffu) << 2);
             }
+            const __half2 S2 = __half2half2(Sh);
+            const __half2 bias2 = __half2half2(__float2half_rn(-1152.f));
             // (rows beyond N: W reads as zeros and the scale and offset are 0, so dW = 0 whatever W_int holds there --
             // zeros, or the next scale factor's first rows)
-            static_for<0, kSearchMaxCand>([&](auto C) {
-                constexpr int c = decltype(C)::value;
-                if (c < ncand) {
-                    const uint32_t a_base = st_base + uint32_t(c) * kSearchATile + a_row_off;
     #pragma unroll
-                    for (int i = 0; i < 2; ++i) {
+            for (int i = 0; i < 2; ++i) {
+                uint32_t e[8];   // the words of weights 8 i .. 8 i + 7
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(e[j]) : "r"(at[8 * i + j]));
+                uint32_t pair01[4], pair23[4];   // bytes: candidates (0, 1) resp. (2, 3) of weights (2 j, 2 j + 1)
+    #pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    pair01[j] = __byte_perm(e[2 * j], e[2 * j + 1], 0x5140u);
+                    pair23[j] = __byte_perm(e[2 * j], e[2 * j + 1], 0x7362u);
+                }
+                const int piece = 2 * quart + i;
+                const uint32_t dst = st_base + a_row_off + uint32_t((piece ^ (r & 7)) << 4);
+                static_for<0, kSearchMaxCand>([&](auto C) {
+                    constexpr int c = decltype(C)::value;
+                    if (c < ncand) {
                         uint32_t packed[4];
     #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const int e = 8 * i + 2 * j;
-                            float l0, l1;
-                            asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l0) : "r"(at[e]), "n"(c * 256));
-                            asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(l1) : "r"(at[e + 1]), "n"(c * 256));
-                            const __half2 h = __floats2half2_rn(fmaf(Sf, l0, rest[e]), fmaf(Sf, l1, rest[e + 1]));
+                            const uint32_t raw = __byte_perm(c < 2 ? pair01[j] : pair23[j], 0x64646464u, (c & 1) ? 0x4342u : 0x4140u);
+                            const __half2 step = __hadd2(*reinterpret_cast<const __half2 *>(&raw), bias2);
+                            const __half2 h = __hfma2(S2, step, *reinterpret_cast<const __half2 *>(&resid[4 * i + j]));
                             packed[j] = *reinterpret_cast<const uint32_t *>(&h);
                         }
-                        const int piece = 2 * quart + i;
-                        const uint32_t dst = a_base + uint32_t((piece ^ (r & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(packed[0]), "r"(packed[1]), "r"(packed[2]), "r"(packed[3]) : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + uint32_t(c) * kSearchATile), "r"(packed[0]), "r"(packed[1]), "r"(packed[2]), "r"(packed[3]) : "memory");
                     }
-                }
-            });
+                });
+            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tiles are read by the tensor cores' proxy
             named_barrier(1, kSearchThreads);                 // every forming thread's part of the stage is written and fenced
             if (tid == 0) mbar_arrive(bar0 + 24 + 8 * s);     // the stage is full
