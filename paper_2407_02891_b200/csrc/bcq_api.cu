@@ -921,7 +921,7 @@ int bcq_grid_search(const bcq_desc *desc, const uint16_t *W, const uint16_t *X, 
         const int count = n_scales - s0 < L.together ? n_scales - s0 : L.together;
         for (int i = 0; i < count; ++i) {
             e = launch_quantize_rtn(W, n_bits, s_factors[s0 + i], code_of_int, weight, S + i * (L.S_each / 2), qbias + i * (L.S_each / 2),
-                                    w_int + i * L.w_int_each, scratch, st);
+                                    w_int + i * L.w_int_each, scratch, st, false);   // the search needs no packed operand
             if (e != cudaSuccess) return cuda_fail(e);
         }
         float *rows = err_rows ? err_rows + size_t(s0) * P * d.N : reinterpret_cast<float *>(base + L.err_rows);

@@ -136,7 +136,7 @@ cudaError_t launch_merge(const bcq_desc &d, const uint8_t *w_int, const uint16_t
                          uint8_t *codes, uint16_t *alpha, uint16_t *z, cudaStream_t st);
 cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, const uint8_t *code_of_int /*[256]*/,
                                 const double *plane_weight /*[q]*/, uint16_t *S, uint16_t *qbias, uint8_t *w_int,
-                                const View &dst, cudaStream_t st);
+                                const View &dst, cudaStream_t st, bool pack = true);   // pack = false: S, qbias, w_int only
 cudaError_t launch_pack(const uint8_t *codes, const View &dst, cudaStream_t st);
 cudaError_t launch_permute_planes(const View &src, const View &dst, cudaStream_t st);
 cudaError_t launch_permute_scales(const View &src, const View &dst, cudaStream_t st);

@@ -76,6 +76,8 @@ __device__ __forceinline__ void load_spread_table(const QuantTable &tab, uint32_
 // is further from a rounding boundary than its own error bound; the few weights that are not (and
 // exact ties) take the fp64 division.  Same integers, a fraction of the fp64 work.  Rounding t: adding
 // 1.5 * 2^23 leaves the nearest integer in the low mantissa bits (valid below 2^22; larger t clamp).
+// PACK = false (the search over scale factors wants the integers only): no codes, no plane bytes.
+template <bool PACK>
 __device__ __forceinline__ void encode_chunk(const uint4 raw, __half s_h, __half b_h, const QuantTable &tab,
                                              const uint32_t *lut, uint8_t *__restrict__ w_int, const View &dst, int n, int kb)
 {
@@ -105,15 +107,17 @@ __device__ __forceinline__ void encode_chunk(const uint4 raw, __half s_h, __half
                 r = int(fmin(fmax(r64, 0.0), tab.top));
             }
         }
-        spread |= lut[r] << j;
+        if (PACK) spread |= lut[r] << j;
         if (j < 4)
             ints_lo |= uint32_t(r) << (8 * j);
         else
             ints_hi |= uint32_t(r) << (8 * (j - 4));
     }
-    unsigned char *out = dst.plane_byte(0, n, kb);
-    const size_t stride = dst.plane_stride();
-    for (int i = 0; i < dst.q; ++i) out[i * stride] = uint8_t(spread >> (8 * i));
+    if (PACK) {
+        unsigned char *out = dst.plane_byte(0, n, kb);
+        const size_t stride = dst.plane_stride();
+        for (int i = 0; i < dst.q; ++i) out[i * stride] = uint8_t(spread >> (8 * i));
+    }
     if (w_int) *reinterpret_cast<uint2 *>(w_int + size_t(n) * dst.K + size_t(kb) * 8) = make_uint2(ints_lo, ints_hi);
 }
 
@@ -135,6 +139,7 @@ __device__ __forceinline__ void range_to_scale(float lo, float hi, const QuantTa
 
 // Any group length: one thread per (row, chunk), S and qbias from the range kernel.  Block (x, y) covers
 // rows kQuantRows x .. + kQuantRows - 1 and chunks 256 y .. + 255.
+template <bool PACK>
 __global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restrict__ W, const __half *__restrict__ S,
                                                          const __half *__restrict__ qbias, int L, QuantTable tab,
                                                          uint8_t *__restrict__ w_int, const View dst)
@@ -146,13 +151,14 @@ __global__ void __launch_bounds__(256) rtn_encode_kernel(const __half *__restric
     const int G = dst.K / L, g = (kb * 8) / L;
     for (int n = blockIdx.x * kQuantRows; n < min(dst.N, (blockIdx.x + 1) * kQuantRows); ++n) {
         const uint4 raw = *reinterpret_cast<const uint4 *>(W + size_t(n) * dst.K + size_t(kb) * 8);
-        encode_chunk(raw, S[size_t(n) * G + g], qbias[size_t(n) * G + g], tab, lut, w_int, dst, n, kb);
+        encode_chunk<PACK>(raw, S[size_t(n) * G + g], qbias[size_t(n) * G + g], tab, lut, w_int, dst, n, kb);
     }
     __threadfence();   // operands visible device-wide before the block counts as finished (products fetch them early)
 }
 
 // Groups of 128: everything in one pass.  A group is 16 chunks = 16 consecutive lanes, each holding
 // its chunk in registers: range by shuffles, S and qbias by the group's first lane, then the encoding.
+template <bool PACK>
 __global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restrict__ W, QuantTable tab,
                                                            __half *__restrict__ S, __half *__restrict__ qbias,
                                                            uint8_t *__restrict__ w_int, const View dst)
@@ -196,7 +202,7 @@ __global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restr
         const unsigned got = __shfl_sync(0xffffffffu, pair, (threadIdx.x & 31) & 16);
         s_h = __ushort_as_half(uint16_t(got & 0xffffu));
         b_h = __ushort_as_half(uint16_t(got >> 16));
-        if (in && sub <= dst.q) {
+        if (PACK && in && sub <= dst.q) {
             const double mult = sub < dst.q ? tab.plane_weight[sub & 3] : tab.centre;
             const double add = sub < dst.q ? 0.0 : double(__half2float(b_h));
             const uint16_t v = __half_as_ushort(__double2half(double(__half2float(s_h)) * mult + add));   // exact, rounded once
@@ -205,7 +211,7 @@ __global__ void __launch_bounds__(256) rtn_fused128_kernel(const __half *__restr
             else
                 *dst.z_elem(n, g) = v;
         }
-        if (in) encode_chunk(raw, s_h, b_h, tab, lut, w_int, dst, n, kb);
+        if (in) encode_chunk<PACK>(raw, s_h, b_h, tab, lut, w_int, dst, n, kb);
     }
     __threadfence();   // operands visible device-wide before the block counts as finished (products fetch them early)
 }
@@ -223,7 +229,7 @@ __global__ void __launch_bounds__(256) rtn_scales_kernel(const __half *__restric
 
 cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, const uint8_t *code_of_int /*[256]*/,
                                 const double *plane_weight /*[q]*/, uint16_t *S, uint16_t *qbias, uint8_t *w_int,
-                                const View &dst, cudaStream_t st)
+                                const View &dst, cudaStream_t st, bool pack)
 {
     QuantTable tab;
     for (int t = 0; t < 256; ++t) tab.code_of_int[t] = code_of_int[t];
@@ -237,15 +243,21 @@ cudaError_t launch_quantize_rtn(const uint16_t *W, int n_bits, double s_factor, 
     __half *s = reinterpret_cast<__half *>(S), *b = reinterpret_cast<__half *>(qbias);
     const dim3 grid(unsigned((dst.N + kQuantRows - 1) / kQuantRows), unsigned((dst.K / 8 + 255) / 256));   // kQuantRows rows per block
     if (L == 128) {
-        rtn_fused128_kernel<<<grid, 256, 0, st>>>(w, tab, s, b, w_int, dst);
+        if (pack)
+            rtn_fused128_kernel<true><<<grid, 256, 0, st>>>(w, tab, s, b, w_int, dst);
+        else
+            rtn_fused128_kernel<false><<<grid, 256, 0, st>>>(w, tab, s, b, w_int, dst);
         return cudaGetLastError();
     }
     rtn_range_kernel<<<unsigned((units + 7) / 8), 256, 0, st>>>(w, dst.N, dst.K, L, tab, s, b);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    rtn_encode_kernel<<<grid, 256, 0, st>>>(w, s, b, L, tab, w_int, dst);
+    if (pack)
+        rtn_encode_kernel<true><<<grid, 256, 0, st>>>(w, s, b, L, tab, w_int, dst);
+    else
+        rtn_encode_kernel<false><<<grid, 256, 0, st>>>(w, s, b, L, tab, w_int, dst);
     e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || !pack) return e;
     rtn_scales_kernel<<<unsigned((units + 255) / 256), 256, 0, st>>>(s, b, tab, dst);
     return cudaGetLastError();
 }
