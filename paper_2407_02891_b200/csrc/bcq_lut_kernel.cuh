@@ -82,10 +82,12 @@ struct LutCfg {
     static constexpr int kFront = 65536 - 1024;
     static constexpr int kBack = kLutSmemBytes - kFront - kTables - kFixedBytes;
     static constexpr int rings(int j, int d) { return kFront / (j * d * kTile) + kBack / (j * d * kTile); }
-    // preference: two tiles per copy and two slots; then one tile per copy with three or two slots
-    static constexpr int kChoice = rings(2, 2) >= kLutConsumersMax ? 0 : (rings(1, 3) >= kLutConsumersMax ? 1 : 2);
-    static constexpr int kJ = kChoice == 0 ? 2 : 1;
-    static constexpr int kD = kChoice == 0 ? 2 : (kChoice == 1 ? 3 : 2);
+    // preference: two tiles per copy with three slots (small tiles: a warp is through a job before the copy for the
+    // slot after the next has crossed HBM), else with two slots; then one tile per copy with three or two slots
+    static constexpr int kChoice =
+        rings(2, 3) >= kLutConsumersMax ? 0 : (rings(2, 2) >= kLutConsumersMax ? 1 : (rings(1, 3) >= kLutConsumersMax ? 2 : 3));
+    static constexpr int kJ = kChoice <= 1 ? 2 : 1;
+    static constexpr int kD = (kChoice == 0 || kChoice == 2) ? 3 : 2;
     static constexpr int kCons = rings(kJ, kD) < kLutConsumersMax ? rings(kJ, kD) : kLutConsumersMax;
     // one warp starts about 18 copies per microsecond: enough for jobs of two 1792-byte tiles, not for smaller ones
     static constexpr int kProducers = (kJ == 1 || Q <= 2) ? 2 : 1;
