@@ -93,8 +93,6 @@ __device__ __forceinline__ bool search_wait(uint32_t bar, uint32_t parity, volat
     return false;
 }
 
-// grid (row tiles of 128, groups of cand_per_block candidates, scale factors); dynamic shared memory:
-// 2 stages x (cand_per_block x 16 KB of dW tiles + 32 KB for X), 1024-byte aligned.
 // all forming threads take the same decision (a wait that gives up must not split them at a barrier)
 __device__ __forceinline__ bool formers_all(bool ok)
 {
@@ -127,6 +125,9 @@ __device__ __forceinline__ void search_drain(uint32_t bar, uint32_t parity)
     }
 }
 
+// grid (row tiles of 128, groups of cand_per_block candidates, scale factors); dynamic shared memory: 2 stages x
+// (cand_per_block x 16 KB of dW tiles | X's slice, T x 128 bytes rounded up to 1 KB | W's slice 16 KB | W_int's 8 KB),
+// 1024-byte aligned.
 __global__ void __launch_bounds__(kSearchBlock, 1)
     search_error_kernel(const SearchParams p, const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap wmap,
                         const __grid_constant__ CUtensorMap imap)
