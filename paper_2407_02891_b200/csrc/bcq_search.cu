@@ -293,9 +293,8 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
     #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w8[j]));
-                    // a byte below the bit pattern of 2^23 is the float 2^23 + v
-                    const float v0 = __uint_as_float(__byte_perm(i4[j >> 1], 0x4B000000u, 0x7440u + uint32_t(2 * (j & 1)))) - 8388608.f;
-                    const float v1 = __uint_as_float(__byte_perm(i4[j >> 1], 0x4B000000u, 0x7441u + uint32_t(2 * (j & 1)))) - 8388608.f;
+                    const float v0 = float((i4[j >> 1] >> (16 * (j & 1))) & 0xffu);
+                    const float v1 = float((i4[j >> 1] >> (16 * (j & 1) + 8)) & 0xffu);
                     const __half2 h = __floats2half2_rn(fmaf(Sf, v0, qb - f.x), fmaf(Sf, v1, qb - f.y));
                     resid[j] = *reinterpret_cast<const uint32_t *>(&h);
                 }
