@@ -390,8 +390,8 @@ int bcq_gemv_noalloc(const bcq_desc *desc, const void *packed_dev, const uint16_
  * multiply-add) and fp32 accumulation; the error values agree with an fp64 evaluation to about 1e-3 relative, so
  * candidates closer than that may swap places.  GPTQ's error compensation is not part of this call.
  *   W [N][K] fp16 weights, X [T][K] fp16 calibration inputs (device, 16-byte aligned); T a multiple of 16,
- *   16..256 (the error is a sum over tokens: for more tokens call once per piece of X, add up the err arrays
- *   and take the minimum yourself); K a multiple of 64; desc->group 0 or a multiple of 64; n_bits 1..6; desc->layout is ignored.
+ *   16..65536 (the error is a sum over tokens: more than 256 tokens run as pieces of at most 256, one launch
+ *   each, on the same stream); K a multiple of 64; desc->group 0 or a multiple of 64; n_bits 1..6; desc->layout is ignored.
  *   partitions_host [P][n_bits]: bit_to_plane arrays as in bcq_merge_linear (bcq_partition_get lists them all);
  *   s_factors_host [n_scales] (bcq_reexplore_factors gives an even grid inside the interval of Eq. reexplore).
  *   err_dev [n_scales][P] fp64; err_rows_dev [n_scales][P][N] fp32 or NULL; best_dev [2] int32.

@@ -464,7 +464,7 @@ int check_search(const bcq_desc *desc, int T, int n_bits, int P, int n_scales)
     const int rc = check_desc(desc);
     if (rc != BCQ_OK) return rc;
     if (n_bits < 1 || n_bits > 6 || desc->q > n_bits || P < 1 || P > 4096 || n_scales < 1 || n_scales > 4096) return BCQ_ERR_INVALID_ARG;
-    if (T < 16 || T > 256 || T % 16 != 0) return BCQ_ERR_INVALID_ARG;
+    if (T < 16 || T > 65536 || T % 16 != 0) return BCQ_ERR_INVALID_ARG;
     if (desc->K % 64 != 0 || (desc->group != 0 && desc->group % 64 != 0)) return BCQ_ERR_UNSUPPORTED_SHAPE;
     return BCQ_OK;
 }

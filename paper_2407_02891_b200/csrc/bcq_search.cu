@@ -49,7 +49,8 @@ struct SearchParams {
     const __half *X;        // [T][K]
     float *err_rows;        // [scale factor][P][N]
     int N, K, G, L;         // L = weights per scaling unit (K when one per row)
-    int T, P;
+    int T, P;               // T: tokens of this launch (a piece of at most 256 of the call's)
+    int accumulate;         // add to err_rows instead of writing it (every piece but the first)
     int cand_per_block;     // 1..4, so that cand_per_block * T <= 512 columns of tensor memory
     int tmem_cols;          // power of two >= 32 covering cand_per_block * T
     int lut_size;           // 2^n_bits <= 64
@@ -374,8 +375,11 @@ __global__ void __launch_bounds__(kSearchBlock, 1)
     if (alive && tid < kSearchRows) {
         const int row = blockIdx.x * kSearchRows + tid;
         if (row < p.N)
-            for (int c = 0; c < ncand; ++c)
-                p.err_rows[(size_t(blockIdx.z) * p.P + size_t(cand0 + c)) * p.N + row] = (part[0][c][tid] + part[1][c][tid]) + (part[2][c][tid] + part[3][c][tid]);
+            for (int c = 0; c < ncand; ++c) {
+                float *out = p.err_rows + (size_t(blockIdx.z) * p.P + size_t(cand0 + c)) * p.N + row;
+                const float sum = (part[0][c][tid] + part[1][c][tid]) + (part[2][c][tid] + part[3][c][tid]);
+                *out = p.accumulate ? *out + sum : sum;   // pieces of tokens run one after the other on the stream
+            }
     }
     if (warp == 0) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -463,14 +467,9 @@ cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const 
     p.W = reinterpret_cast<const __half *>(W), p.w_int = w_int;
     p.S = reinterpret_cast<const __half *>(S), p.qbias = reinterpret_cast<const __half *>(qbias), p.scale_stride = scale_stride;
     p.X = reinterpret_cast<const __half *>(X), p.err_rows = err_rows;
-    p.N = N, p.K = K, p.L = group == 0 ? K : group, p.G = K / p.L, p.T = T, p.P = P;
-    p.cand_per_block = search_cand_per_block(T);
-    int cols = 32;
-    while (cols < p.cand_per_block * T) cols *= 2;
-    p.tmem_cols = cols;
+    p.N = N, p.K = K, p.L = group == 0 ? K : group, p.G = K / p.L, p.P = P;
     p.lut_size = 1 << n_bits;
     p.lut = lut_dev;
-    const size_t smem = search_smem_bytes(T);
     if (dev < 0 || dev >= 64 || !configured[dev]) {
         size_t most = 0;
         for (int t = 16; t <= kSearchMaxT; t += 16) most = search_smem_bytes(t) > most ? search_smem_bytes(t) : most;
@@ -478,17 +477,29 @@ cudaError_t launch_search_errors(const uint16_t *W, const uint8_t *w_int, const 
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    // the slices of X (all T rows), W (the block's 128 rows; rows beyond N read as zeros) and W_int (the scale
-    // factors' matrices as one of scales * N rows)
+    // the slices of W (the block's 128 rows; rows beyond N read as zeros) and W_int (the scale factors' matrices as one
+    // of scales * N rows)
     CUtensorMap xmap, wmap, imap;
-    if ((e = search_tensor_map(&xmap, X, false, uint64_t(T), uint64_t(K), uint32_t(T), true)) != cudaSuccess) return e;
     if ((e = search_tensor_map(&wmap, W, false, uint64_t(N), uint64_t(K), uint32_t(kSearchRows), true)) != cudaSuccess) return e;
     if ((e = search_tensor_map(&imap, w_int, true, uint64_t(scales) * uint64_t(N), uint64_t(K), uint32_t(kSearchRows), false)) != cudaSuccess) return e;
     const unsigned row_tiles = unsigned((N + kSearchRows - 1) / kSearchRows);
-    const unsigned groups = unsigned((P + p.cand_per_block - 1) / p.cand_per_block);
-    search_error_kernel<<<dim3(row_tiles, groups, unsigned(scales)), kSearchBlock, smem, st>>>(p, xmap, wmap, imap);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    // the error is a sum over tokens: pieces of at most 256 tokens, one launch each, the later ones adding to err_rows
+    // (pieces of about equal size, multiples of 16)
+    const int pieces = (T + kSearchMaxT - 1) / kSearchMaxT, piece = ((T + pieces - 1) / pieces + 15) / 16 * 16;
+    for (int t0 = 0; t0 < T; t0 += piece) {
+        const int Tp = T - t0 < piece ? T - t0 : piece;
+        p.X = reinterpret_cast<const __half *>(X) + size_t(t0) * K;
+        p.T = Tp, p.accumulate = t0 > 0 ? 1 : 0;
+        p.cand_per_block = search_cand_per_block(Tp);
+        int cols = 32;
+        while (cols < p.cand_per_block * Tp) cols *= 2;
+        p.tmem_cols = cols;
+        if ((e = search_tensor_map(&xmap, p.X, false, uint64_t(Tp), uint64_t(K), uint32_t(Tp), true)) != cudaSuccess) return e;   // all rows of the piece
+        const unsigned groups = unsigned((P + p.cand_per_block - 1) / p.cand_per_block);
+        search_error_kernel<<<dim3(row_tiles, groups, unsigned(scales)), kSearchBlock, search_smem_bytes(Tp), st>>>(p, xmap, wmap, imap);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     search_sum_kernel<<<unsigned(P) * unsigned(scales), 256, 0, st>>>(err_rows, N, err);
     return cudaGetLastError();
 }

@@ -49,12 +49,14 @@ def _check(N, K, T, q, group, n_bits, n_scales, name):
     (256, 512, 64, 3, 128, 4, 3),      # two row tiles, six candidates in two groups of four
     (128, 256, 16, 2, 0, 3, 2),        # the smallest T, one scale per row
     (200, 512, 128, 3, 128, 4, 2),     # a ragged last row tile
-    (384, 1024, 256, 3, 128, 4, 2),    # the largest T: two candidates per block
+    (384, 1024, 256, 3, 128, 4, 2),    # the most tokens one launch takes: two candidates per block
     (256, 512, 32, 2, 64, 5, 2),       # 15 candidates, scaling units of 64
     (136, 576, 48, 3, 0, 5, 1),        # 25 candidates, K = 9 slices, T = 48
     (128, 128, 64, 1, 128, 2, 3),      # one plane
     (128, 256, 32, 4, 128, 6, 1),      # six step-1 bits into four planes: 65 candidates, tables of 64 entries
     (200, 256, 32, 2, 128, 3, 11),     # more scale factors than one launch takes (8 + 3), ragged row tiles between them
+    (256, 256, 528, 3, 128, 4, 2),     # more tokens than one launch takes: three pieces of 176
+    (128, 512, 272, 2, 0, 4, 9),       # two pieces of 144 and 128 tokens, two launches of scale factors
 ])
 def test_grid_search_matches_the_oracle(N, K, T, q, group, n_bits, n_scales):
     _check(N, K, T, q, group, n_bits, n_scales, f"search/{N}x{K}x{T}")
