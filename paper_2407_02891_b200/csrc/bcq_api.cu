@@ -95,7 +95,8 @@ int lut_max_units(const bcq_desc *d, int B)
 double lut_cost(int U, int W, int rb, int ks, int sm, int cons, int tiles_per_job, int cols)
 {
     // (two columns: twice the table entries to build, 4 instead of 3 instructions per lookup)
-    const double per_tile = cols == 2 ? 50.0 : 38.0, table_build = 2200.0 * cols, split_fixed = 500.0, per_split = 10.0, round_weight = 0.3;
+    const double per_tile = cols == 2 ? 50.0 : 38.0, table_build = 2200.0 * cols, split_fixed = 500.0, per_split = 10.0, round_weight = 0.3,
+                 per_reuse = 100.0;   // measured on the long-K shapes (56 and 72 windows): fewer, longer windows per block lose
     const long long blocks = static_cast<long long>(rb) * ks;
     const long long waves = (blocks + sm - 1) / sm;
     const int wc = (W + ks - 1) / ks;
@@ -111,7 +112,8 @@ double lut_cost(int U, int W, int rb, int ks, int sm, int cons, int tiles_per_jo
         ready = (ready > end_prev ? ready : end_prev) + table_build;   // the table after this one reuses the buffer of the window before
         end_prev = start + window;
     }
-    return double(waves) * (end_prev + (ks > 1 ? split_fixed + per_split * ks : 0.0));
+    const int reuses = wc > 2 ? wc - 2 : 0;   // tables built into a buffer that consumers have to hand back first
+    return double(waves) * (end_prev + per_reuse * reuses + (ks > 1 ? split_fixed + per_split * ks : 0.0));
 }
 
 int plan_lut(const bcq_desc *d, int B, int sm, bcq_plan *out)
